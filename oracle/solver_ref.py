@@ -1,0 +1,212 @@
+"""Wave-quantized analytical selector: reference implementation (CPU oracle, test infrastructure).
+
+This file is test infrastructure: only the tests, the smoke check and the benchmark's
+CPU-baseline leg may import it.  It shares no code with the library's host solver.
+
+It follows the paper's Section III step by step, in the paper's order and notation:
+  Eq. 1   R(C) = ceil(C / o_comm)
+  Eq. 3   P(C) = o_comp * (G - R(C))
+  Eq. 5   W_comp = g * (sum_e ceil(M_e / T_M)) * ceil(ceil(N/L) / T_N)
+  Eq. 6   V_comp(C) = ceil(W_comp / P(C))
+  Eq. 7   W_comm = ceil(ceil(M/D) / T_M^comm) * ceil(ceil(N/L) / T_N^comm)   (per split and rank)
+  Eq. 8   V_comm(C) = ceil(W_comm / C)
+  Eq. 9   A_s(C) = ceil((s+1) * W_comp / P(C))
+  Eq. 10  q(C) = rho * V_comm(C)
+  Eq. 11  F_s = max(A_s, F_{s-1}) + q,  F_{-1} = 0
+  Eq. 12  T(C) = F_{L-1}
+  Eq. 13-15  rho = rho_ref * (K_ref/K) * (T_M,ref*T_N,ref / (T_M*T_N)) * (D/D_ref)
+  Algorithm 1  loop over C = 1..C_max, arg min T(C)
+  tie breaker  Delta_comp(C) = V_comp(C) * P(C) - W_comp, smaller wins
+
+Readings where the paper is silent (each is listed in the design notes):
+  * ties left after Delta_comp go to the smaller C: the winner is the lexicographic
+    minimum of (T, Delta_comp, C);
+  * candidates with P(C) <= 0 are not in the legal set (Section II-C: the legal set keeps
+    positive compute capacity);
+  * "the same wave-quantized T(C)" needs exact equality, so rho is quantised once to
+    fixed point, rho_q = floor(rho * 2^20 + 1/2), and A_s, q, F_s are carried as integers
+    scaled by 2^20;
+  * one GPU that emulates all D destination ranks serves every rank's tokens with the same
+    C communication CTAs, so the communication work it sees per split is the sum over the
+    ranks of Eq. 7 (w_comm_gpu below); Eq. 7 itself is w_comm_rank.
+
+All arithmetic is python int / Fraction: no rounding anywhere except the stated
+quantisation of rho.
+"""
+
+from __future__ import annotations
+
+from fractions import Fraction
+
+RHO_SHIFT = 20
+RHO_ONE = 1 << RHO_SHIFT
+
+
+def ceil_div(a: int, b: int) -> int:
+    return -(-a // b)
+
+
+# ----------------------------------------------------------------------------- work terms
+
+def w_comp(tiles, g: int, N: int, L: int, T_N: int) -> int:
+    """Eq. 5.  `tiles[e]` = ceil(M_e / T_M) (the routed-tile counts, Eq. 16 reduces them)."""
+    return g * sum(int(t) for t in tiles) * ceil_div(ceil_div(N, L), T_N)
+
+
+def w_comm_rank(M: int, D: int, N: int, L: int, T_Mc: int, T_Nc: int) -> int:
+    """Eq. 7: communication tiles per split and rank (a rank owns about ceil(M/D) tokens)."""
+    return ceil_div(ceil_div(M, D), T_Mc) * ceil_div(ceil_div(N, L), T_Nc)
+
+
+def owned_tokens(M: int, D: int, d: int) -> int:
+    """Tokens owned by rank d when ranks own contiguous blocks of ceil(M/D) tokens."""
+    blk = ceil_div(M, D)
+    return max(0, min(blk, M - d * blk))
+
+
+def w_comm_gpu(M: int, D: int, N: int, L: int, T_Mc: int, T_Nc: int) -> int:
+    """Communication tiles per split seen by one GPU that emulates all D ranks: the sum
+    over the ranks of Eq. 7 evaluated on the tokens each rank really owns."""
+    n_col = ceil_div(ceil_div(N, L), T_Nc)
+    return sum(ceil_div(owned_tokens(M, D, d), T_Mc) for d in range(D)) * n_col
+
+
+# ----------------------------------------------------------------------------- rho
+
+def rho_reference(t_comm_us: float, n_splits: int, t_comp_us: float, n_waves: int) -> float:
+    """Eq. 13: (time of one communication wave) / (time of one compute wave)."""
+    return (t_comm_us / n_splits) / (t_comp_us / n_waves)
+
+
+def rho_scaled(rho_ref: float, K_ref: int, T_M_ref: int, T_N_ref: int, D_ref: int,
+               K: int, T_M: int, T_N: int, D: int) -> float:
+    """Eq. 14, evaluated as one product over one product (all factors but rho_ref are
+    small integers, so the two products are exact in double precision)."""
+    num = float(K_ref * T_M_ref * T_N_ref * D)
+    den = float(K * T_M * T_N * D_ref)
+    return rho_ref * num / den
+
+
+def quantise_rho(rho: float) -> int:
+    """rho_q = floor(rho * 2^20 + 1/2) (rho * 2^20 is exact: a power-of-two scaling)."""
+    x = rho * float(RHO_ONE) + 0.5
+    return int(x // 1)
+
+
+# ----------------------------------------------------------------------------- the model
+
+def reservation(C: int, o_comm: int) -> int:
+    return ceil_div(C, o_comm)                       # Eq. 1
+
+
+def compute_capacity(C: int, G: int, o_comp: int, o_comm: int) -> int:
+    return o_comp * (G - reservation(C, o_comm))     # Eq. 3
+
+
+def makespan(C: int, Wc: int, Wm: int, L: int, G: int, o_comp: int, o_comm: int, rho):
+    """T(C) of Eq. 12 with rho any exact number type (int, Fraction).  Returns
+    (T, Delta_comp, R, P, [A_s], V_comm) or None when P(C) <= 0."""
+    R = reservation(C, o_comm)
+    P = o_comp * (G - R)
+    if P <= 0:
+        return None
+    A = [ceil_div((s + 1) * Wc, P) for s in range(L)]    # Eq. 9
+    V_comm = ceil_div(Wm, C)                              # Eq. 8
+    q = rho * V_comm                                      # Eq. 10
+    F = 0
+    for s in range(L):                                    # Eq. 11
+        F = max(A[s], F) + q
+    V_comp = ceil_div(Wc, P)                              # Eq. 6
+    delta = V_comp * P - Wc                               # tie breaker
+    return F, delta, R, P, A, V_comm
+
+
+def select(Wc: int, Wm: int, L: int, G: int, o_comp: int, o_comm: int, C_max: int, rho_q: int,
+           force_comm_ctas: int = 0, selector_off: bool = False, default_C: int = 3) -> dict:
+    """Algorithm 1 in fixed point.  T_q is T(C) * 2^20 with rho replaced by rho_q / 2^20.
+
+    Precedence (Section III-E): an explicit user value of C wins over everything; with the
+    selector switched off the fixed default is used.  Either must be a legal C."""
+    def evaluate(C):
+        R = reservation(C, o_comm)
+        P = o_comp * (G - R)
+        if P <= 0:
+            return None
+        V_comm = ceil_div(Wm, C)
+        q = rho_q * V_comm
+        F = 0
+        for s in range(L):
+            A_s = ceil_div((s + 1) * Wc, P)
+            F = max(A_s * RHO_ONE, F) + q
+        V_comp = ceil_div(Wc, P)
+        return dict(comm_ctas=C, R=R, P=P, T_q=F, delta=V_comp * P - Wc,
+                    W_comp=Wc, W_comm=Wm)
+
+    if force_comm_ctas > 0 or selector_off:
+        C = force_comm_ctas if force_comm_ctas > 0 else default_C
+        if C < 1:
+            raise ValueError("C must be at least 1")
+        r = evaluate(C)
+        if r is None:
+            raise ValueError("requested C leaves no compute capacity")
+        return r
+    best = None
+    for C in range(1, C_max + 1):
+        r = evaluate(C)
+        if r is None:
+            continue
+        key = (r["T_q"], r["delta"], r["comm_ctas"])
+        if best is None or key < (best["T_q"], best["delta"], best["comm_ctas"]):
+            best = r
+    if best is None:
+        raise ValueError("no legal C")
+    return best
+
+
+def curve(Wc: int, Wm: int, L: int, G: int, o_comp: int, o_comm: int, C_max: int, rho) -> dict:
+    """{C: (T, Delta_comp)} for every legal C, rho exact (Fraction or int)."""
+    out = {}
+    for C in range(1, C_max + 1):
+        m = makespan(C, Wc, Wm, L, G, o_comp, o_comm, rho)
+        if m is not None:
+            out[C] = (m[0], m[1])
+    return out
+
+
+# ----------------------------------------------------------------------------- simulator
+
+def simulate(C: int, Wc: int, Wm: int, L: int, P: int, rho: Fraction) -> dict:
+    """Tiny discrete-event simulation of the pipeline the model describes (Section III-C):
+      * P compute CTAs; CTA b takes global tiles b, b+P, b+2P, ... of the split-major
+        sequence (L splits of Wc tiles each); every tile takes one time unit;
+      * split s is published when its last tile has finished;
+      * C communication CTAs serve the splits in order; for one split, CTA c takes
+        communication tiles c, c+C, ...; every communication tile takes rho time units and
+        the CTAs move to the next split together (a split is served in waves);
+      * service of split s starts when it is published and split s-1 has been served.
+    Returns the publication times and the finish times, computed event by event (no
+    closed form is used)."""
+    rho = Fraction(rho)
+    # compute side: per-CTA clocks
+    clock = [Fraction(0)] * P
+    tile_end = [None] * (L * Wc)
+    for i in range(L * Wc):
+        b = i % P
+        clock[b] = clock[b] + 1
+        tile_end[i] = clock[b]
+    publish = []
+    for s in range(L):
+        seg = tile_end[s * Wc:(s + 1) * Wc]
+        publish.append(max(seg) if seg else Fraction(0))
+    # communication side
+    finish = []
+    prev = Fraction(0)
+    for s in range(L):
+        start = max(publish[s], prev)
+        worker = [start] * C
+        for j in range(Wm):
+            c = j % C
+            worker[c] = worker[c] + rho
+        prev = max(worker) if Wm > 0 else start
+        finish.append(prev)
+    return dict(publish=publish, finish=finish, T=finish[-1] if finish else Fraction(0))

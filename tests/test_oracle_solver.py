@@ -1,0 +1,171 @@
+"""Pins for the selector reference: the arithmetic the paper prints, hand-worked examples,
+closed forms, the discrete-event simulator and brute-force properties."""
+
+import os
+import random
+from fractions import Fraction
+
+import pytest
+
+from oracle import solver_ref as sr
+
+
+def _parse_golden(path):
+    ex, Ts, deltas, picks = {}, {}, {}, {}
+    for line in open(path):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        kind, name, *rest = line.split()
+        if kind == "example":
+            ex[name] = {k: (Fraction(v) if k == "rho" else int(v)) for k, v in (p.split("=") for p in rest)}
+        elif kind == "T":
+            Ts[name] = {int(k): Fraction(v) for k, v in (p.split("=") for p in rest)}
+        elif kind == "delta":
+            deltas[name] = {int(k): int(v) for k, v in (p.split("=") for p in rest)}
+        elif kind == "pick":
+            picks[name] = tuple(int(v) for v in rest)
+    return ex, Ts, deltas, picks
+
+
+def test_rho_reference_printed_arithmetic():
+    # Eq. 13: the paper prints (400.19/2)/(497.36/25) ~ 10.05
+    rho = sr.rho_reference(400.19, 2, 497.36, 25)
+    assert abs(rho - 10.05) < 0.01
+    assert abs(rho - 10.0579) < 1e-3
+
+
+def test_a100_reduction():
+    # Eq. 2 and Eq. 4: o_comm = 1 -> R(C) = C ; o_comp = 2 -> P(C) = 2 (G - C) with G = 108
+    for C in range(1, 17):
+        assert sr.reservation(C, 1) == C
+        assert sr.compute_capacity(C, 108, 2, 1) == 2 * (108 - C)
+    assert sr.reservation(5, 2) == 3 and sr.reservation(6, 2) == 3 and sr.reservation(7, 4) == 2
+
+
+def test_work_terms_of_the_examples():
+    # Ex.A: 64 experts x ceil(384/128) = 192 m-tiles; split width 1024 -> 8 n-tiles; g = 1
+    assert sr.w_comp([3] * 64, 1, 2048, 2, 128) == 1536
+    assert sr.w_comm_rank(4096, 4, 2048, 2, 128, 1024) == 8
+    # Ex.B: 32 x ceil(1024/128) = 256 m-tiles; N = 1024, L = 1 -> 8 n-tiles
+    assert sr.w_comp([8] * 32, 1, 1024, 1, 128) == 2048
+    assert sr.w_comm_rank(4096, 4, 1024, 1, 128, 1024) == 8
+    # Ex.C: 1024 m-tiles, g = 2, H = 2048, L = 2, T_N = 256 -> 4 n-tiles
+    assert sr.w_comp([16] * 64, 2, 2048, 2, 256) == 8192
+    # all ranks on one GPU: 2 ranks x ceil(8192/128) x 1 = 128 tiles; per rank 64
+    assert sr.w_comm_rank(16384, 2, 2048, 2, 128, 1024) == 64
+    assert sr.w_comm_gpu(16384, 2, 2048, 2, 128, 1024) == 128
+    # ragged ownership: T = 5, D = 4 -> blocks 2, 2, 1, 0
+    assert [sr.owned_tokens(5, 4, d) for d in range(4)] == [2, 2, 1, 0]
+    assert sr.w_comm_gpu(5, 4, 64, 1, 2, 64) == 1 + 1 + 1 + 0
+    # ceilings on a width that is no multiple of the tile: N = 1536, L = 1, T_Nc = 1024 -> 2
+    assert sr.w_comm_rank(4096, 2, 1536, 1, 128, 1024) == 16 * 2
+
+
+def test_rho_scaling_eq14():
+    # same configuration as the reference -> rho_ref ; K halves -> doubles ; tile doubles -> halves
+    assert sr.rho_scaled(10.05, 352, 128, 128, 4, 352, 128, 128, 4) == 10.05
+    assert sr.rho_scaled(10.05, 352, 128, 128, 4, 176, 128, 128, 4) == pytest.approx(20.10)
+    assert sr.rho_scaled(10.05, 352, 128, 128, 4, 352, 128, 256, 4) == pytest.approx(5.025)
+    assert sr.rho_scaled(10.05, 352, 128, 128, 4, 352, 128, 128, 2) == pytest.approx(5.025)
+    assert sr.rho_scaled(10.05, 352, 128, 128, 4, 128, 128, 128, 4) == pytest.approx(27.6375)
+    assert sr.quantise_rho(3.0) == 3145728 and sr.quantise_rho(2.5) == 2621440
+
+
+@pytest.mark.parametrize("name", ["A", "B", "C", "D"])
+def test_hand_worked_examples(golden_dir, name):
+    ex, Ts, deltas, picks = _parse_golden(os.path.join(golden_dir, "selector_worked_examples.txt"))
+    p = ex[name]
+    cur = sr.curve(p["W_comp"], p["W_comm"], p["L"], p["G"], p["o_comp"], p["o_comm"], p["C_max"], p["rho"])
+    for C, T in Ts[name].items():
+        assert cur[C][0] == T, (name, C, cur[C][0], T)
+    for C, d in deltas[name].items():
+        assert cur[C][1] == d, (name, C)
+    # fixed-point selection (rho of every example is exactly representable only for C and D;
+    # A and B are quantised, which must not move the pick)
+    rho_q = sr.quantise_rho(float(p["rho"]))
+    sel = sr.select(p["W_comp"], p["W_comm"], p["L"], p["G"], p["o_comp"], p["o_comm"], p["C_max"], rho_q)
+    assert (sel["comm_ctas"], sel["R"], sel["P"]) == picks[name]
+    if name in ("C", "D"):
+        assert Fraction(sel["T_q"], sr.RHO_ONE) == cur[sel["comm_ctas"]][0]
+
+
+def _rand_case(rng):
+    G = rng.choice([8, 20, 108, 148])
+    o_comp = rng.choice([1, 2])
+    o_comm = rng.choice([1, 2, 4])
+    L = rng.choice([1, 2, 4, 8])
+    Wc = rng.randint(0, 3000)
+    Wm = rng.randint(1, 300)
+    C_max = rng.randint(1, G * o_comm + 3)
+    rho = Fraction(rng.randint(1, 400), rng.choice([1, 2, 4, 8, 16]))
+    return G, o_comp, o_comm, L, Wc, Wm, C_max, rho
+
+
+def test_closed_forms():
+    rng = random.Random(1)
+    n_cb = n_pb = 0
+    for _ in range(3000):
+        G, o_comp, o_comm, L, Wc, Wm, C_max, rho = _rand_case(rng)
+        for C in range(1, C_max + 1):
+            m = sr.makespan(C, Wc, Wm, L, G, o_comp, o_comm, rho)
+            P = o_comp * (G - -(-C // o_comm))
+            if P <= 0:
+                assert m is None
+                continue
+            T, delta, R, P2, A, V = m
+            assert P2 == P and 0 <= delta < P
+            q = rho * -(-Wm // C)
+            if L == 1:
+                assert T == -(-Wc // P) + q
+            gaps = [A[s] - A[s - 1] for s in range(1, L)]
+            if all(q >= g for g in gaps):            # communication-bound: a queue forms after A_0
+                assert T == A[0] + L * q
+                n_cb += 1
+            if all(q <= g for g in gaps):            # compute-bound: every split waits for compute
+                assert T == A[L - 1] + q
+                n_pb += 1
+            # bounds that hold always
+            assert T >= A[L - 1] + q and T >= A[0] + L * q
+    assert n_cb > 100 and n_pb > 100
+
+
+def test_simulator_reproduces_recurrence():
+    rng = random.Random(2)
+    for _ in range(300):
+        G = rng.choice([4, 6, 10])
+        o_comp = rng.choice([1, 2])
+        L = rng.choice([1, 2, 3, 4])
+        Wc = rng.randint(1, 60)
+        Wm = rng.randint(1, 12)
+        rho = Fraction(rng.randint(1, 40), rng.choice([1, 2, 4]))
+        for C in range(1, G):
+            m = sr.makespan(C, Wc, Wm, L, G, o_comp, 1, rho)
+            T, delta, R, P, A, V = m
+            sim = sr.simulate(C, Wc, Wm, L, P, rho)
+            assert sim["publish"] == A
+            assert sim["T"] == T
+
+
+def test_select_is_the_lexicographic_minimum_and_overrides():
+    rng = random.Random(3)
+    for _ in range(500):
+        G, o_comp, o_comm, L, Wc, Wm, C_max, rho = _rand_case(rng)
+        rho_q = sr.quantise_rho(float(rho))
+        cur = sr.curve(Wc, Wm, L, G, o_comp, o_comm, C_max, Fraction(rho_q, sr.RHO_ONE))
+        if not cur:
+            with pytest.raises(ValueError):
+                sr.select(Wc, Wm, L, G, o_comp, o_comm, C_max, rho_q)
+            continue
+        sel = sr.select(Wc, Wm, L, G, o_comp, o_comm, C_max, rho_q)
+        best = min((T, d, C) for C, (T, d) in cur.items())
+        assert sel["comm_ctas"] == best[2]
+        assert Fraction(sel["T_q"], sr.RHO_ONE) == best[0] and sel["delta"] == best[1]
+        # an explicit C wins; selector off -> the fixed default
+        C_f = rng.choice(list(cur))
+        f = sr.select(Wc, Wm, L, G, o_comp, o_comm, C_max, rho_q, force_comm_ctas=C_f, selector_off=True, default_C=1)
+        assert f["comm_ctas"] == C_f and Fraction(f["T_q"], sr.RHO_ONE) == cur[C_f][0]
+        d = sr.select(Wc, Wm, L, G, o_comp, o_comm, C_max, rho_q, selector_off=True, default_C=min(cur))
+        assert d["comm_ctas"] == min(cur)
+    with pytest.raises(ValueError):
+        sr.select(10, 10, 1, 4, 1, 1, 16, sr.RHO_ONE, force_comm_ctas=4)   # P = 0
