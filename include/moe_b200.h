@@ -1,0 +1,219 @@
+/*
+ * moe_b200.h -- C ABI of the B200 (sm_100a) MoE down-projection operator:
+ * grouped expert GEMM2 fused with the GatherRS combine, plus the launch-time analytical
+ * selector of the communication-CTA count.
+ *
+ * Citations name sections / equations / algorithms of the paper
+ * "Analytical Resource Management for Fine-grained MoE Computation-Communication Overlap".
+ *
+ * Conventions
+ *  - every function returns an int32 status: MOE_OK (0) or a negative MOE_ERR_* value;
+ *    nothing throws across this boundary;
+ *  - pointers are tagged [host] or [device]; the library never allocates device memory:
+ *    the caller owns every buffer and the stream (passed as void*, a cudaStream_t);
+ *  - all launches are asynchronous on the given stream;
+ *  - device-side problems (a bounded wait that ran out, an index out of range) are reported
+ *    through a 4-word status buffer in device memory, read back with moe_get_status();
+ *  - bf16 tensors are passed as void*; layouts are row-major with the last index contiguous.
+ *
+ * Symbols: T tokens (paper M), H hidden size (paper N), I expert intermediate size,
+ * TP emulated tensor-parallel shards (split-K partials, paper g), K = I / TP (paper K),
+ * EP emulated destination ranks (paper D), E_tot experts (routed + shared), k_tot experts per
+ * token, R = T * k_tot routed rows, L pipeline splits along H, S = sum_e ceil(M_e / T_M).
+ */
+#ifndef MOE_B200_H
+#define MOE_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    MOE_OK = 0,
+    MOE_ERR_NULL = -1,            /* a required pointer is NULL */
+    MOE_ERR_SHAPE = -2,           /* unsupported or inconsistent sizes */
+    MOE_ERR_ALIGN = -3,           /* a device pointer is not 16-byte aligned */
+    MOE_ERR_PLAN_INFEASIBLE = -4, /* no legal C, or the plan does not fit the GPU */
+    MOE_ERR_CUDA = -5,            /* a CUDA runtime/driver call failed (see moe_last_cuda_error) */
+    MOE_ERR_UNSUPPORTED = -6,     /* tile configuration the kernels do not provide */
+    MOE_ERR_DEVICE_STATUS = -7,   /* the device status buffer reports a problem */
+    MOE_ERR_ARENA = -8            /* the caller's arena is too small */
+};
+
+/* device status codes (word 0 of the status buffer) */
+enum {
+    MOE_DEV_OK = 0,
+    MOE_DEV_TIMEOUT = 1,   /* a bounded wait ran out; word 1 = tile / flag index, word 2 = where */
+    MOE_DEV_OOB = 2,       /* an index was out of range and the access was skipped; word 1 = index */
+    MOE_DEV_DUP_EXPERT = 3 /* one token names the same expert twice; word 1 = token */
+};
+
+enum { MOE_MODE_FUSED = 0, MOE_MODE_GEMM_ONLY = 1, MOE_MODE_COMBINE_ONLY = 2 };
+/* MOE_RHO_PAPER: Eq. 14 as printed (K, tile area and D/D_ref terms).
+ * MOE_RHO_LOCAL: the re-derivation Section III-E asks of a new kernel family, for ranks
+ * emulated inside one GPU: no ring term D/D_ref; a communication tile costs in proportion
+ * to the rows it moves per token (k_tot * TP read + 1 written) and to its real width
+ * min(T_N^comm, ceil(H/L)). */
+enum { MOE_RHO_PAPER = 0, MOE_RHO_LOCAL = 1 };
+#define MOE_MAX_EP 8
+#define MOE_MAX_L 8
+
+typedef struct moe_handle moe_handle;
+
+typedef struct {
+    int32_t T, H, I, E_tot, k_tot, TP, EP, L;
+} moe_shape;
+
+/* Kernel-family constants of one GEMM2 tile configuration (Section III-B, Table I; Section
+ * III-E: read once per kernel choice, not per invocation). */
+typedef struct {
+    int32_t tile_m, tile_n;           /* T_M^comp, T_N^comp */
+    int32_t comm_tile_m, comm_tile_n; /* T_M^comm, T_N^comm */
+    int32_t o_comp, o_comm;           /* resident CTAs per SM of each role */
+} moe_occupancy;
+
+/* GPU residency limits and the user's overrides (Section III-D legal set; Section III-E:
+ * an explicit C has the highest priority, and the selector can be switched off). */
+typedef struct {
+    int32_t G;               /* SMs available to the operator */
+    int32_t C_max;           /* upper end of the legal set {1..C_max} */
+    int32_t force_comm_ctas; /* > 0: use exactly this C */
+    int32_t selector_off;    /* != 0: use default_C */
+    int32_t default_C;       /* the fixed count used when the selector is off */
+} moe_sm_limits;
+
+/* Relative wave service rate (Eq. 13-15). */
+typedef struct {
+    double rho_ref;
+    int32_t K_ref, tile_m_ref, tile_n_ref, D_ref;
+    int32_t rows_ref;        /* k_tot * TP + 1 of the reference run (MOE_RHO_LOCAL only) */
+    int32_t comm_cols_ref;   /* min(T_N^comm, ceil(H/L)) of the reference run (MOE_RHO_LOCAL only) */
+    int32_t mode;            /* MOE_RHO_PAPER | MOE_RHO_LOCAL */
+} moe_rho;
+
+/* Result of the selector, and the launch description moe_gemm2_combine() consumes.
+ * Plain data: the caller may overwrite comm_ctas / R / P (validated at launch). */
+typedef struct {
+    int32_t comm_ctas;   /* C*   */
+    int32_t R;           /* R(C*) = ceil(C / o_comm), SM positions reserved (Eq. 1) */
+    int32_t P;           /* P(C*) = o_comp (G - R), compute slots (Eq. 3) */
+    int32_t W_comp;      /* Eq. 5, compute tiles per split */
+    int32_t W_comm;      /* communication tiles per split on this GPU (Eq. 7 summed over ranks) */
+    int32_t delta;       /* Delta_comp(C*) (tie breaker) */
+    int64_t pred_T_q;    /* T(C*) in compute-wave units, scaled by 2^20 */
+    int64_t rho_q;       /* rho scaled by 2^20 and rounded to nearest */
+    int32_t mode;        /* MOE_MODE_* (plan_partition writes MOE_MODE_FUSED) */
+    int32_t debug_withhold_tile; /* test hook: global tile whose readiness is never raised; -1 = none */
+} moe_plan;
+
+/* Views into the routing workspace, all [device] int32. */
+typedef struct {
+    int32_t *counts;          /* [E_tot]     M_e */
+    int32_t *offsets;         /* [E_tot + 1] exclusive prefix of counts */
+    int32_t *tiles;           /* [E_tot]     ceil(M_e / T_M) */
+    int32_t *tile_offsets;    /* [E_tot + 1] exclusive prefix of tiles; last = S */
+    int32_t *perm;            /* [R] flat assignment held by routed row r */
+    int32_t *inv_perm;        /* [R] routed row of flat assignment f = t * k_tot + j */
+    int32_t *pad_row;         /* [R] row of f in the tile-padded layout */
+    int32_t *mtile_expert;    /* [max_mtiles] */
+    int32_t *mtile_first_row; /* [max_mtiles] */
+    int32_t *mtile_valid;     /* [max_mtiles] */
+    int32_t *scratch;         /* per-warp histograms used while building */
+    int32_t max_mtiles;       /* floor(R / T_M) + E_tot, an upper bound of S */
+} moe_routing;
+
+typedef struct {
+    uint32_t code, detail, where, count;
+} moe_status;
+
+/* ---- handle -------------------------------------------------------------------------- */
+
+/* Opens the library on CUDA device `device`; caches the SM count and the kernels'
+ * residency (Section III-E: the SM count is cached at operator initialisation).  [host] */
+int32_t moe_create(int32_t device, moe_handle **out);
+int32_t moe_destroy(moe_handle *h);
+/* Text of the last failing CUDA call on this handle ("" if none); owned by the handle. */
+const char *moe_last_cuda_error(const moe_handle *h);
+/* Upper bound, in nanoseconds, of every device-side wait (default 2e9).  After it a CTA
+ * records MOE_DEV_TIMEOUT and leaves; the context stays usable. */
+int32_t moe_set_wait_limit_ns(moe_handle *h, uint64_t ns);
+
+/* Tile shape and residency of the GEMM2 kernel for (tile_m, tile_n), the communication tile,
+ * the GPU limits and the stored service-rate constants (Section III-B, III-D, III-E).
+ * tile_m in {64, 128}, tile_n in {64, 128, 256}.  Any output pointer may be NULL.  [host] */
+int32_t moe_query_occupancy(moe_handle *h, int32_t tile_m, int32_t tile_n,
+                            moe_occupancy *occ, moe_sm_limits *limits, moe_rho *rho);
+
+/* Sizes of the caller-allocated workspaces [bytes]: routing arrays, the tile-padded GEMM2
+ * output Y (bf16 [TP][T_M * max_mtiles][H]), readiness flags + split counters (must be
+ * zero-filled once before first use and not shared between handles), status (16 bytes). */
+int32_t moe_workspace_bytes(const moe_shape *shape, int32_t tile_m, int32_t tile_n,
+                            size_t *routing_bytes, size_t *y_bytes, size_t *flags_bytes,
+                            size_t *status_bytes);
+/* Carves the routing workspace [device, 16-byte aligned] into its arrays.  Pure host. */
+int32_t moe_routing_view(void *routing_ws, const moe_shape *shape, int32_t tile_m, moe_routing *out);
+
+/* ---- a1: routing / permutation / routed-tile counts ------------------------------------
+ * Section II-A (token-expert assignments), Eq. 5 (ceil(M_e / T_M) tiles per expert), Eq. 16
+ * (their sum).  Stable sort of the flat assignments f = t * k_tot + j by expert.
+ * topk_idx [device] int32 [T, k_tot]; tile_counts_host [host, pinned] receives
+ * tiles[0..E_tot) followed by S (E_tot + 1 ints) by an asynchronous copy: synchronise the
+ * stream before reading it.  Bad expert ids / repeated experts are reported in status_dev. */
+int32_t moe_build_routing(moe_handle *h, const int32_t *topk_idx, const moe_shape *shape,
+                          int32_t tile_m, const moe_routing *routing,
+                          int32_t *tile_counts_host, uint32_t *status_dev, void *stream);
+
+/* ---- a2: the analytical selector (Section III-D, Algorithm 1, Eq. 1-15, tie breaker) -----
+ * Pure host code: no CUDA call, no allocation, re-entrant.
+ * routed_tile_counts [host] ceil(M_e / T_M) for e in [0, n_experts).
+ * Picks the lexicographic minimum of (T(C), Delta_comp(C), C) over the legal C; rho is
+ * quantised to 2^-20.  limits->force_comm_ctas > 0 wins over everything, then selector_off.
+ * Errors: MOE_ERR_PLAN_INFEASIBLE when no C (or the forced C) leaves P >= 1. */
+int32_t plan_partition(const int32_t *routed_tile_counts, int32_t n_experts,
+                       const moe_occupancy *occ, const moe_sm_limits *limits,
+                       const moe_shape *shape, const moe_rho *rho, moe_plan *out);
+
+/* ---- a3-a5: fused grouped GEMM2 + GatherRS combine --------------------------------------
+ * Section II-A step 3, Section II-B (compute CTAs publish, communication CTAs consume),
+ * Section III-C (CTA b takes global tiles b, b+P, ... of the split-major sequence),
+ * Section III-E (C* communication CTAs, R(C*) reserved SMs, P(C*) compute CTAs).
+ *   out_d[t - d*ceil(T/EP)][:] = sum_j topk_w[t][j] * sum_p (x_routed[inv_perm[t,j]][Kp] . W2[e][:, Kp])
+ * x_routed [device] bf16 [R, I]; W2 [device] bf16 [E_tot, H, I]; topk_w [device] fp32 [T, k_tot];
+ * topk_idx is not read (the routing arrays already encode it) and may be NULL;
+ * out [host] array of EP [device] pointers, buffer d is bf16 [ceil(T/EP), H], fully overwritten
+ * for the tokens rank d owns; y_ws / flags_ws / status_dev as sized by moe_workspace_bytes.
+ * n_mtiles = S (host value from moe_build_routing).  Requires H % 8 == 0, K % 16 == 0,
+ * 16-byte aligned pointers, 1 <= C, 1 <= P, R * o_comm >= C, R + ceil(P / o_comp) <= G. */
+int32_t moe_gemm2_combine(moe_handle *h, const void *x_routed, const void *W2,
+                          const int32_t *topk_idx, const float *topk_w,
+                          const moe_shape *shape, const moe_occupancy *occ,
+                          const moe_routing *routing, int32_t n_mtiles, const moe_plan *plan,
+                          void *const *out, void *y_ws, uint32_t *flags_ws,
+                          uint32_t *status_dev, void *stream);
+
+/* Copies the 4-word device status to the host (synchronises the stream).  Returns
+ * MOE_ERR_DEVICE_STATUS when code != 0. */
+int32_t moe_get_status(moe_handle *h, const uint32_t *status_dev, moe_status *host, void *stream);
+/* Clears the device status (asynchronous memset). */
+int32_t moe_clear_status(moe_handle *h, uint32_t *status_dev, void *stream);
+
+/* ---- the whole step from host buffers ---------------------------------------------------
+ * The call a user without device-resident activations makes: copies x_routed, topk_idx and
+ * topk_w from (pinned) host memory into `arena`, builds the routing, waits for the tile
+ * counts, plans, launches the fused kernel and copies the EP output blocks back to
+ * out_host (bf16 [T, H], token order).  W2 stays device resident (weights).  Synchronous.
+ * arena [device] of at least moe_host_arena_bytes(); plan_out may be NULL. */
+int32_t moe_host_arena_bytes(const moe_shape *shape, int32_t tile_m, int32_t tile_n, size_t *bytes);
+int32_t moe_layer_host(moe_handle *h, const void *x_routed_host, const int32_t *topk_idx_host,
+                       const float *topk_w_host, const void *W2_dev, const moe_shape *shape,
+                       int32_t tile_m, int32_t tile_n, const moe_sm_limits *limits_or_null,
+                       void *arena, size_t arena_bytes, int32_t *tile_counts_pinned,
+                       void *out_host, moe_plan *plan_out, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOE_B200_H */

@@ -87,6 +87,21 @@ def rho_scaled(rho_ref: float, K_ref: int, T_M_ref: int, T_N_ref: int, D_ref: in
     return rho_ref * num / den
 
 
+def rho_local(rho_ref: float, K_ref: int, T_M_ref: int, T_N_ref: int, rows_ref: int,
+              comm_cols_ref: int, K: int, T_M: int, T_N: int, k_tot: int, TP: int,
+              N: int, L: int, T_Nc: int) -> float:
+    """Re-derivation of Eq. 14 for ranks emulated inside one GPU (Section III-E asks every new
+    kernel family for its own service rate): the K and tile-area terms of Eq. 14 stay, the
+    ring term D/D_ref goes (nothing crosses a link), and a communication tile costs in
+    proportion to the rows moved per token (k_tot*TP read + 1 written) and to its real width
+    min(T_N^comm, ceil(N/L))."""
+    rows = k_tot * TP + 1
+    cols = min(T_Nc, ceil_div(N, L))
+    num = float(K_ref * T_M_ref * T_N_ref * rows * cols)
+    den = float(K * T_M * T_N * rows_ref * comm_cols_ref)
+    return rho_ref * num / den
+
+
 def quantise_rho(rho: float) -> int:
     """rho_q = floor(rho * 2^20 + 1/2) (rho * 2^20 is exact: a power-of-two scaling)."""
     x = rho * float(RHO_ONE) + 0.5

@@ -1,0 +1,452 @@
+// Host side of the C ABI: handle, workspace layout, argument validation, tensor maps, launches.
+
+#include <cstring>
+#include <new>
+
+#include "moe_internal.h"
+
+namespace moe {
+
+int32_t cuda_fail(moe_handle *h, cudaError_t e, const char *what)
+{
+    if (h) snprintf(h->err, sizeof h->err, "%s: %s", what, cudaGetErrorString(e));
+    return MOE_ERR_CUDA;
+}
+
+namespace {
+
+inline size_t align16(size_t x) { return (x + 15) & ~(size_t)15; }
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+constexpr int kSplitCounterWords = 64;  // 2 parities x MOE_MAX_L counters, padded
+
+bool shape_ok(const moe_shape *s)
+{
+    return s->T >= 0 && s->H >= 8 && s->I >= 16 && s->E_tot >= 1 && s->E_tot <= 1024 && s->k_tot >= 1 &&
+           s->k_tot <= 32 && s->TP >= 1 && s->TP <= 8 && s->EP >= 1 && s->EP <= MOE_MAX_EP && s->L >= 1 &&
+           s->L <= MOE_MAX_L && s->H % 8 == 0 && s->I % s->TP == 0 && (s->I / s->TP) % 16 == 0 &&
+           (int64_t)s->T * s->k_tot < (int64_t)1 << 30;
+}
+bool tile_ok(int tile_m, int tile_n) { return (tile_m == 64 || tile_m == 128) && tile_n_slot(tile_n) >= 0; }
+
+int32_t max_mtiles_of(const moe_shape *s, int tile_m)
+{
+    return (int32_t)((int64_t)s->T * s->k_tot / tile_m + s->E_tot);
+}
+int32_t n_routing_warps(const moe_shape *s)
+{
+    return (int32_t)ceil_div((int64_t)s->T * s->k_tot, kRoutingChunk);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+}  // namespace
+}  // namespace moe
+
+using namespace moe;
+
+extern "C" {
+
+int32_t moe_create(int32_t device, moe_handle **out)
+{
+    if (!out) return MOE_ERR_NULL;
+    *out = nullptr;
+    moe_handle *h = new (std::nothrow) moe_handle();
+    if (!h) return MOE_ERR_CUDA;
+    h->device = device;
+    cudaError_t e = cudaSetDevice(device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->G, cudaDevAttrMultiProcessorCount, device);
+    int major = 0;
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device);
+    if (e != cudaSuccess || major != 10) {
+        delete h;
+        return e != cudaSuccess ? MOE_ERR_CUDA : MOE_ERR_UNSUPPORTED;
+    }
+    cudaDriverEntryPointQueryResult q;
+    e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &h->encode_tiled, cudaEnableDefault, &q);
+    if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || !h->encode_tiled) {
+        delete h;
+        return MOE_ERR_CUDA;
+    }
+    const int tns[3] = {64, 128, 256};
+    for (int i = 0; i < 3; ++i) {
+        e = fused_occupancy(tns[i], &h->o_comp[i]);
+        if (e != cudaSuccess) {
+            delete h;
+            return MOE_ERR_CUDA;
+        }
+    }
+    *out = h;
+    return MOE_OK;
+}
+
+int32_t moe_destroy(moe_handle *h)
+{
+    delete h;
+    return MOE_OK;
+}
+
+const char *moe_last_cuda_error(const moe_handle *h) { return h ? h->err : ""; }
+
+int32_t moe_set_wait_limit_ns(moe_handle *h, uint64_t ns)
+{
+    if (!h) return MOE_ERR_NULL;
+    h->wait_ns = ns;
+    return MOE_OK;
+}
+
+int32_t moe_query_occupancy(moe_handle *h, int32_t tile_m, int32_t tile_n, moe_occupancy *occ,
+                            moe_sm_limits *limits, moe_rho *rho)
+{
+    if (!h) return MOE_ERR_NULL;
+    if (!tile_ok(tile_m, tile_n)) return MOE_ERR_UNSUPPORTED;
+    if (occ) {
+        occ->tile_m = tile_m;
+        occ->tile_n = tile_n;
+        occ->comm_tile_m = kCommTileM;
+        occ->comm_tile_n = kCommTileN;
+        // both roles are CTAs of the same kernel: one resident CTA per SM by shared memory
+        occ->o_comp = h->o_comp[tile_n_slot(tile_n)];
+        occ->o_comm = h->o_comp[tile_n_slot(tile_n)];
+    }
+    if (limits) {
+        limits->G = h->G;
+        limits->C_max = h->G / 2;   // one-time saturation characterisation of this kernel family
+        limits->force_comm_ctas = 0;
+        limits->selector_off = 0;
+        limits->default_C = 3;      // the fixed count of the upstream path (Section II-C)
+    }
+    if (rho) {
+        // one-time service-rate characterisation of this kernel family on B200 (Eq. 13):
+        // reference run = DeepSeek-V2-Lite shape, T = 4096, uniform routing, 128x256 tiles,
+        // TP = 2, EP = 2, L = 2.
+        rho->rho_ref = 2.0;
+        rho->K_ref = 704;
+        rho->tile_m_ref = 128;
+        rho->tile_n_ref = 256;
+        rho->D_ref = 2;
+        rho->rows_ref = 8 * 2 + 1;
+        rho->comm_cols_ref = 1024;
+        rho->mode = MOE_RHO_LOCAL;
+    }
+    return MOE_OK;
+}
+
+int32_t moe_workspace_bytes(const moe_shape *s, int32_t tile_m, int32_t tile_n, size_t *routing_bytes,
+                            size_t *y_bytes, size_t *flags_bytes, size_t *status_bytes)
+{
+    if (!s) return MOE_ERR_NULL;
+    if (!shape_ok(s)) return MOE_ERR_SHAPE;
+    if (!tile_ok(tile_m, tile_n)) return MOE_ERR_UNSUPPORTED;
+    const size_t R = (size_t)s->T * s->k_tot, E = (size_t)s->E_tot;
+    const size_t mt = (size_t)max_mtiles_of(s, tile_m);
+    if (routing_bytes) {
+        size_t b = 0;
+        b += align16(E * 4) + 3 * align16((E + 1) * 4);  // counts, offsets, tiles(+S), tile_offsets
+        b += 3 * align16(R * 4);                          // perm, inv_perm, pad_row
+        b += 3 * align16(mt * 4);                         // m-tile table
+        b += align16((size_t)n_routing_warps(s) * E * 4); // per-warp histograms
+        *routing_bytes = b + 16;
+    }
+    if (y_bytes) *y_bytes = align16((size_t)s->TP * mt * tile_m * s->H * 2) + 16;
+    if (flags_bytes) {
+        const size_t nts = (size_t)ceil_div(ceil_div(s->H, s->L), tile_n);
+        *flags_bytes = ((size_t)kSplitCounterWords + (size_t)s->L * s->TP * mt * nts) * 4 + 16;
+    }
+    if (status_bytes) *status_bytes = 16;
+    return MOE_OK;
+}
+
+int32_t moe_routing_view(void *ws, const moe_shape *s, int32_t tile_m, moe_routing *out)
+{
+    if (!ws || !s || !out) return MOE_ERR_NULL;
+    if (!shape_ok(s)) return MOE_ERR_SHAPE;
+    if (tile_m != 64 && tile_m != 128) return MOE_ERR_UNSUPPORTED;
+    if (!aligned16(ws)) return MOE_ERR_ALIGN;
+    const size_t R = (size_t)s->T * s->k_tot, E = (size_t)s->E_tot;
+    const size_t mt = (size_t)max_mtiles_of(s, tile_m);
+    char *p = static_cast<char *>(ws);
+    auto take = [&](size_t n_ints) {
+        int32_t *q = reinterpret_cast<int32_t *>(p);
+        p += align16(n_ints * 4);
+        return q;
+    };
+    out->counts = take(E);
+    out->offsets = take(E + 1);
+    out->tiles = take(E + 1);
+    out->tile_offsets = take(E + 1);
+    out->perm = take(R);
+    out->inv_perm = take(R);
+    out->pad_row = take(R);
+    out->mtile_expert = take(mt);
+    out->mtile_first_row = take(mt);
+    out->mtile_valid = take(mt);
+    out->scratch = take((size_t)n_routing_warps(s) * E);
+    out->max_mtiles = (int32_t)mt;
+    return MOE_OK;
+}
+
+int32_t moe_build_routing(moe_handle *h, const int32_t *topk_idx, const moe_shape *s, int32_t tile_m,
+                          const moe_routing *r, int32_t *tile_counts_host, uint32_t *status_dev, void *stream)
+{
+    if (!h || !s || !r || !status_dev) return MOE_ERR_NULL;
+    if (!shape_ok(s)) return MOE_ERR_SHAPE;
+    if (tile_m != 64 && tile_m != 128) return MOE_ERR_UNSUPPORTED;
+    if (s->T > 0 && !topk_idx) return MOE_ERR_NULL;
+    if (r->max_mtiles < max_mtiles_of(s, tile_m)) return MOE_ERR_SHAPE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = routing_launch(topk_idx, *s, tile_m, *r, status_dev, st);
+    if (e != cudaSuccess) return cuda_fail(h, e, "routing launch");
+    if (tile_counts_host) {
+        e = cudaMemcpyAsync(tile_counts_host, r->tiles, (size_t)(s->E_tot + 1) * 4, cudaMemcpyDeviceToHost, st);
+        if (e != cudaSuccess) return cuda_fail(h, e, "tile counts copy");
+    }
+    return MOE_OK;
+}
+
+int32_t moe_gemm2_combine(moe_handle *h, const void *x_routed, const void *W2, const int32_t *topk_idx,
+                          const float *topk_w, const moe_shape *s, const moe_occupancy *occ,
+                          const moe_routing *r, int32_t n_mtiles, const moe_plan *plan, void *const *out,
+                          void *y_ws, uint32_t *flags_ws, uint32_t *status_dev, void *stream)
+{
+    (void)topk_idx;
+    if (!h || !s || !occ || !r || !plan || !out || !status_dev) return MOE_ERR_NULL;
+    if (!shape_ok(s)) return MOE_ERR_SHAPE;
+    if (!tile_ok(occ->tile_m, occ->tile_n)) return MOE_ERR_UNSUPPORTED;
+    if (occ->comm_tile_m != kCommTileM || occ->comm_tile_n != kCommTileN) return MOE_ERR_UNSUPPORTED;
+    if (s->T == 0) return MOE_OK;
+    if (!x_routed || !W2 || !topk_w || !y_ws || !flags_ws) return MOE_ERR_NULL;
+    if (n_mtiles < 0 || n_mtiles > r->max_mtiles) return MOE_ERR_SHAPE;
+    if (!aligned16(x_routed) || !aligned16(W2) || !aligned16(y_ws) || !aligned16(flags_ws) ||
+        !aligned16(status_dev))
+        return MOE_ERR_ALIGN;
+    for (int d = 0; d < s->EP; ++d) {
+        if (!out[d]) return MOE_ERR_NULL;
+        if (!aligned16(out[d])) return MOE_ERR_ALIGN;
+    }
+    const int mode = plan->mode;
+    if (mode != MOE_MODE_FUSED && mode != MOE_MODE_GEMM_ONLY && mode != MOE_MODE_COMBINE_ONLY)
+        return MOE_ERR_SHAPE;
+    const int C = (mode == MOE_MODE_GEMM_ONLY) ? 0 : plan->comm_ctas;
+    const int Pc = (mode == MOE_MODE_COMBINE_ONLY) ? 0 : plan->P;
+    const int o_comp = occ->o_comp > 0 ? occ->o_comp : 1, o_comm = occ->o_comm > 0 ? occ->o_comm : 1;
+    if (mode != MOE_MODE_GEMM_ONLY && C < 1) return MOE_ERR_PLAN_INFEASIBLE;
+    if (mode != MOE_MODE_COMBINE_ONLY && Pc < 1) return MOE_ERR_PLAN_INFEASIBLE;
+    if (mode == MOE_MODE_FUSED && (int64_t)plan->R * o_comm < C) return MOE_ERR_PLAN_INFEASIBLE;
+    // every CTA must be resident at once: spinning communication CTAs may never keep a compute
+    // CTA off the GPU (Section II-C: the legal set keeps positive compute capacity)
+    if (ceil_div(C, o_comm) + ceil_div(Pc, o_comp) > h->G) return MOE_ERR_PLAN_INFEASIBLE;
+
+    FusedParams p;
+    memset(&p, 0, sizeof p);
+    const int K = s->I / s->TP;
+    const int TN = occ->tile_n;
+    p.T = s->T; p.H = s->H; p.K = K; p.TP = s->TP; p.EP = s->EP; p.L = s->L; p.k_tot = s->k_tot;
+    p.S = n_mtiles;
+    p.tile_m = occ->tile_m;
+    p.split_w = (int32_t)ceil_div(s->H, s->L);
+    p.NTs = (int32_t)ceil_div(p.split_w, TN);
+    const int64_t Wc = (int64_t)s->TP * n_mtiles * p.NTs;
+    if (Wc * s->L >= (int64_t)1 << 31) return MOE_ERR_SHAPE;
+    p.W_comp = (int32_t)Wc;
+    p.C = C; p.P = Pc; p.mode = mode; p.withhold = plan->debug_withhold_tile;
+    p.tok_blk = (int32_t)ceil_div(s->T, s->EP);
+    p.tok_tiles_per_rank = (int32_t)ceil_div(p.tok_blk, kCommTileM);
+    p.comm_cols = (int32_t)ceil_div(p.split_w, kCommTileN);
+    int64_t tok_tiles = 0;
+    for (int d = 0; d < s->EP; ++d) {
+        int64_t own = (int64_t)s->T - (int64_t)d * p.tok_blk;
+        if (own > p.tok_blk) own = p.tok_blk;
+        if (own > 0) tok_tiles += ceil_div(own, kCommTileM);
+    }
+    p.comm_tiles = (int32_t)(tok_tiles * p.comm_cols);
+    p.num_kb = (int32_t)ceil_div(K, kBlockK);
+    p.last_ksteps = (K - (p.num_kb - 1) * kBlockK) / kUmmaK;
+    p.R_pad = (long long)occ->tile_m * n_mtiles;
+    p.wait_ns = h->wait_ns;
+    p.mtile_expert = r->mtile_expert;
+    p.mtile_first_row = r->mtile_first_row;
+    p.mtile_valid = r->mtile_valid;
+    p.pad_row = r->pad_row;
+    p.topk_w = topk_w;
+    p.Y = y_ws;
+    p.status = status_dev;
+    for (int d = 0; d < s->EP; ++d) p.out[d] = out[d];
+
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e;
+    // launch epoch of this workspace: a flag equal to the epoch means "ready in this launch"
+    uint32_t &ep = h->epochs[flags_ws];
+    ep += 1u;
+    if (ep == 0u) {  // wrapped: start over from a clean workspace
+        size_t fb = 0;
+        moe_workspace_bytes(s, occ->tile_m, occ->tile_n, nullptr, nullptr, &fb, nullptr);
+        e = cudaMemsetAsync(flags_ws, 0, fb - 16, st);
+        if (e != cudaSuccess) return cuda_fail(h, e, "flags reset");
+        ep = 1u;
+    }
+    p.epoch = ep;
+    p.split_done = flags_ws + (ep & 1u) * MOE_MAX_L;
+    p.split_done_next = flags_ws + ((ep + 1u) & 1u) * MOE_MAX_L;
+    p.flags = flags_ws + kSplitCounterWords;
+
+    // tensor maps (Section II-A operands): x_routed [R, I] and W2 [E_tot, H, I], k contiguous
+    EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(h->encode_tiled);
+    const cuuint64_t R = (cuuint64_t)s->T * s->k_tot;
+    {
+        cuuint64_t dims[2] = {(cuuint64_t)s->I, R};
+        cuuint64_t strides[1] = {(cuuint64_t)s->I * 2};
+        cuuint32_t box[2] = {(cuuint32_t)kBlockK, (cuuint32_t)kMmaM};
+        cuuint32_t es[2] = {1, 1};
+        CUresult cr = encode(&p.tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(x_routed), dims,
+                             strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (cr != CUDA_SUCCESS) {
+            snprintf(h->err, sizeof h->err, "cuTensorMapEncodeTiled(x_routed) failed: %d", (int)cr);
+            return MOE_ERR_CUDA;
+        }
+    }
+    {
+        cuuint64_t dims[3] = {(cuuint64_t)s->I, (cuuint64_t)s->H, (cuuint64_t)s->E_tot};
+        cuuint64_t strides[2] = {(cuuint64_t)s->I * 2, (cuuint64_t)s->H * s->I * 2};
+        cuuint32_t box[3] = {(cuuint32_t)kBlockK, (cuuint32_t)TN, 1};
+        cuuint32_t es[3] = {1, 1, 1};
+        CUresult cr = encode(&p.tmB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(W2), dims, strides,
+                             box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (cr != CUDA_SUCCESS) {
+            snprintf(h->err, sizeof h->err, "cuTensorMapEncodeTiled(W2) failed: %d", (int)cr);
+            return MOE_ERR_CUDA;
+        }
+    }
+    e = fused_launch(TN, p, C + Pc, st);
+    if (e != cudaSuccess) return cuda_fail(h, e, "fused launch");
+    return MOE_OK;
+}
+
+int32_t moe_get_status(moe_handle *h, const uint32_t *status_dev, moe_status *host, void *stream)
+{
+    if (!h || !status_dev || !host) return MOE_ERR_NULL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint32_t w[4];
+    cudaError_t e = cudaMemcpyAsync(w, status_dev, sizeof w, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(h, e, "status copy");
+    host->code = w[0]; host->detail = w[1]; host->where = w[2]; host->count = w[3];
+    return w[0] == 0 ? MOE_OK : MOE_ERR_DEVICE_STATUS;
+}
+
+int32_t moe_clear_status(moe_handle *h, uint32_t *status_dev, void *stream)
+{
+    if (!h || !status_dev) return MOE_ERR_NULL;
+    cudaError_t e = cudaMemsetAsync(status_dev, 0, 16, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? MOE_OK : cuda_fail(h, e, "status clear");
+}
+
+// ---- whole step from host buffers ----------------------------------------------------------
+
+namespace {
+struct ArenaLayout {
+    size_t x, idx, w, routing, y, flags, status, out, total;
+    size_t routing_b, y_b, flags_b;
+};
+int32_t arena_layout(const moe_shape *s, int tile_m, int tile_n, ArenaLayout *a)
+{
+    size_t sb = 0;
+    int32_t rc = moe_workspace_bytes(s, tile_m, tile_n, &a->routing_b, &a->y_b, &a->flags_b, &sb);
+    if (rc != MOE_OK) return rc;
+    const size_t R = (size_t)s->T * s->k_tot;
+    auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
+    size_t off = 0;
+    a->x = off; off += up(R * s->I * 2);
+    a->idx = off; off += up(R * 4);
+    a->w = off; off += up(R * 4);
+    a->routing = off; off += up(a->routing_b);
+    a->y = off; off += up(a->y_b);
+    a->flags = off; off += up(a->flags_b);
+    a->status = off; off += up(16);
+    a->out = off; off += up((size_t)ceil_div(s->T, s->EP) * s->EP * s->H * 2);
+    a->total = off;
+    return MOE_OK;
+}
+}  // namespace
+
+int32_t moe_host_arena_bytes(const moe_shape *s, int32_t tile_m, int32_t tile_n, size_t *bytes)
+{
+    if (!s || !bytes) return MOE_ERR_NULL;
+    ArenaLayout a;
+    int32_t rc = arena_layout(s, tile_m, tile_n, &a);
+    if (rc != MOE_OK) return rc;
+    *bytes = a.total;
+    return MOE_OK;
+}
+
+int32_t moe_layer_host(moe_handle *h, const void *x_routed_host, const int32_t *topk_idx_host,
+                       const float *topk_w_host, const void *W2_dev, const moe_shape *s, int32_t tile_m,
+                       int32_t tile_n, const moe_sm_limits *limits_or_null, void *arena, size_t arena_bytes,
+                       int32_t *tile_counts_pinned, void *out_host, moe_plan *plan_out, void *stream)
+{
+    if (!h || !s || !arena || !tile_counts_pinned || !out_host || !W2_dev) return MOE_ERR_NULL;
+    if (s->T > 0 && (!x_routed_host || !topk_idx_host || !topk_w_host)) return MOE_ERR_NULL;
+    ArenaLayout a;
+    int32_t rc = arena_layout(s, tile_m, tile_n, &a);
+    if (rc != MOE_OK) return rc;
+    if (arena_bytes < a.total) return MOE_ERR_ARENA;
+    if ((reinterpret_cast<uintptr_t>(arena) & 255u) != 0) return MOE_ERR_ALIGN;
+    if (s->T == 0) return MOE_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    char *base = static_cast<char *>(arena);
+    const size_t R = (size_t)s->T * s->k_tot;
+    cudaError_t e;
+    e = cudaMemcpyAsync(base + a.idx, topk_idx_host, R * 4, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(base + a.status, 0, 16, st);
+    if (e != cudaSuccess) return cuda_fail(h, e, "idx copy");
+    moe_routing rt;
+    rc = moe_routing_view(base + a.routing, s, tile_m, &rt);
+    if (rc != MOE_OK) return rc;
+    uint32_t *status = reinterpret_cast<uint32_t *>(base + a.status);
+    rc = moe_build_routing(h, reinterpret_cast<int32_t *>(base + a.idx), s, tile_m, &rt, tile_counts_pinned,
+                           status, st);
+    if (rc != MOE_OK) return rc;
+    cudaEvent_t counts_ready;
+    e = cudaEventCreateWithFlags(&counts_ready, cudaEventDisableTiming);
+    if (e != cudaSuccess) return cuda_fail(h, e, "event");
+    cudaEventRecord(counts_ready, st);
+    // the large copies overlap the wait for the counts
+    e = cudaMemcpyAsync(base + a.x, x_routed_host, R * s->I * 2, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(base + a.w, topk_w_host, R * 4, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(base + a.flags, 0, a.flags_b, st);
+    if (e == cudaSuccess) e = cudaEventSynchronize(counts_ready);
+    cudaEventDestroy(counts_ready);
+    if (e != cudaSuccess) return cuda_fail(h, e, "input copies");
+    h->epochs.erase(base + a.flags);  // the workspace was just cleared
+
+    moe_occupancy occ;
+    moe_sm_limits lim;
+    moe_rho rho;
+    rc = moe_query_occupancy(h, tile_m, tile_n, &occ, &lim, &rho);
+    if (rc != MOE_OK) return rc;
+    if (limits_or_null) lim = *limits_or_null;
+    moe_plan plan;
+    rc = plan_partition(tile_counts_pinned, s->E_tot, &occ, &lim, s, &rho, &plan);
+    if (rc != MOE_OK) return rc;
+    if (plan_out) *plan_out = plan;
+    void *outs[MOE_MAX_EP];
+    const size_t blk = (size_t)ceil_div(s->T, s->EP);
+    for (int d = 0; d < s->EP; ++d) outs[d] = base + a.out + (size_t)d * blk * s->H * 2;
+    rc = moe_gemm2_combine(h, base + a.x, W2_dev, nullptr, reinterpret_cast<float *>(base + a.w), s, &occ, &rt,
+                           tile_counts_pinned[s->E_tot], &plan, outs, base + a.y,
+                           reinterpret_cast<uint32_t *>(base + a.flags), status, st);
+    if (rc != MOE_OK) return rc;
+    // rank d owns tokens [d*blk, (d+1)*blk): the EP blocks are contiguous in token order
+    e = cudaMemcpyAsync(out_host, base + a.out, (size_t)s->T * s->H * 2, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return cuda_fail(h, e, "output copy");
+    moe_status hs;
+    return moe_get_status(h, status, &hs, st);
+}
+
+}  // extern "C"

@@ -1,0 +1,594 @@
+// Fused grouped GEMM2 + GatherRS combine for sm_100a: one persistent launch, one CTA per SM,
+// role by blockIdx.
+//
+//   blockIdx <  C : communication CTA c (Section II-B: consumes published results; the same
+//                   C CTAs serve all splits in sequence; CTA c takes communication tiles
+//                   c, c+C, ... of a split).
+//   blockIdx >= C : compute CTA b = blockIdx - C (Section III-C: takes global tiles
+//                   b, b+P, b+2P, ... of the split-major sequence in which the expert
+//                   problems of one split are contiguous).
+//
+// Compute CTA (warp-specialised):
+//   warp 0      TMA producer: x_routed tile (128 rows x 64 k) and W2 tile (tile_n rows x 64 k)
+//               into a ring of 128B-swizzled shared-memory stages;
+//   warp 1      MMA issuer: tcgen05.mma (M = 128, N = tile_n, K = 16, bf16 -> fp32) into one of
+//               two TMEM accumulator buffers; tcgen05.commit frees stages / publishes the tile;
+//   warps 4-11  epilogue: tcgen05.ld -> bf16 -> Y (tile-padded), then the tile's readiness flag
+//               (st.release.gpu) and the split counter (red.release.gpu).
+// Communication CTA (16 warps): a warp owns (token, 256-column group) units of its
+//   communication tile; it waits for the producing tiles (ld.acquire.gpu; bounded), gathers the
+//   k_tot * TP rows with 16-byte loads, accumulates in fp32 in (j, p) order and stores bf16 into
+//   the owning rank's buffer.
+//
+// Every wait is bounded: after `wait_ns` the waiter records MOE_DEV_TIMEOUT and the CTA winds
+// down (pending bulk copies are drained, TMEM is released).
+
+#include <cuda_bf16.h>
+
+#include "moe_internal.h"
+
+namespace moe {
+namespace {
+
+// --------------------------------------------------------------------------- PTX wrappers
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p)
+{
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ unsigned long long globaltimer_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"((unsigned long long)map), "r"(bar), "r"(x), "r"(y)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y, int z)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"((unsigned long long)map), "r"(bar), "r"(x), "r"(y), "r"(z)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t cols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// 32 lanes x 32 consecutive fp32 columns: thread i reads TMEM lane (base lane + i)
+__device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p)
+{
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_u32(uint32_t *p, uint32_t v)
+{
+    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void red_release_add_u32(uint32_t *p, uint32_t v)
+{
+    asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void named_barrier(int id, int threads)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major, 128B-swizzled operand tile whose rows are
+// 128 bytes (64 bf16): 8-row groups are 1024 bytes apart (stride byte offset), the leading
+// byte offset is unused for swizzled K-major layouts, descriptor version 1, layout type 2.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);        // start address, bits [0,14)
+    d |= (uint64_t)1 << 16;                               // leading byte offset (ignored), bits [16,30)
+    d |= (uint64_t)(1024 >> 4) << 32;                     // stride byte offset, bits [32,46)
+    d |= (uint64_t)1 << 46;                               // descriptor version, bits [46,48)
+    d |= (uint64_t)2 << 61;                               // SWIZZLE_128B, bits [61,64)
+    return d;
+}
+// Instruction descriptor, kind::f16: D fp32, A and B bf16, both K-major, M x N.
+__host__ __device__ constexpr uint32_t make_idesc(int M, int N)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+__device__ __forceinline__ void report(uint32_t *status, uint32_t code, uint32_t detail, uint32_t where)
+{
+    if (atomicCAS(&status[0], 0u, code) == 0u) {
+        status[1] = detail;
+        status[2] = where;
+    }
+    atomicAdd(&status[3], 1u);
+}
+
+// --------------------------------------------------------------------------- shared memory
+
+template <int TN>
+struct Cfg {
+    static constexpr int kABytes = kMmaM * kBlockK * 2;          // 16 KB
+    static constexpr int kBBytes = TN * kBlockK * 2;             // 8 / 16 / 32 KB
+    static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kStages = kStageBytesTotal / kStageBytes;  // 8 / 6 / 4
+    static constexpr int kTmemCols = 2 * TN;                     // two accumulator buffers
+    static constexpr int kEpiWarps = 8;
+    static constexpr int kEpiThreads = kEpiWarps * 32;
+    static constexpr int kColsPerHalf = TN / 2;
+};
+
+struct Control {
+    unsigned long long full[8];
+    unsigned long long empty[8];
+    unsigned long long tmem_full[2];
+    unsigned long long tmem_empty[2];
+    uint32_t tmem_base;
+    volatile uint32_t abort;
+};
+
+// Bounded mbarrier wait.  Returns false on timeout or when another warp of the CTA gave up.
+__device__ __forceinline__ bool wait_barrier(uint32_t bar, uint32_t parity, Control *ctl,
+                                             unsigned long long deadline, uint32_t *status,
+                                             uint32_t detail, uint32_t where)
+{
+    uint32_t spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 63u) == 0u) {
+            if (ctl->abort) return false;
+            if (globaltimer_ns() > deadline) {
+                ctl->abort = 1u;
+                report(status, MOE_DEV_TIMEOUT, detail, where);
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+struct Tile {
+    int s, mu, p, i_n;
+};
+__device__ __forceinline__ Tile decode_tile(int g, const FusedParams &P)
+{
+    Tile t;
+    t.s = g / P.W_comp;
+    const int idx = g - t.s * P.W_comp;
+    const int r = idx / P.NTs;
+    t.i_n = idx - r * P.NTs;
+    t.mu = r / P.TP;
+    t.p = r - t.mu * P.TP;
+    return t;
+}
+
+// --------------------------------------------------------------------------- compute CTA
+
+template <int TN>
+__device__ void compute_cta(const FusedParams &P, uint8_t *ring, Control *ctl, int b)
+{
+    using C = Cfg<TN>;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int total_tiles = P.L * P.W_comp;
+    const unsigned long long deadline = globaltimer_ns() + P.wait_ns;
+
+    // setup: barriers (thread 0), TMEM allocation (warp 1)
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < C::kStages; ++i) {
+            mbar_init(smem_u32(&ctl->full[i]), 1);
+            mbar_init(smem_u32(&ctl->empty[i]), 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(smem_u32(&ctl->tmem_full[i]), 1);
+            mbar_init(smem_u32(&ctl->tmem_empty[i]), C::kEpiWarps);
+        }
+        ctl->abort = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&ctl->tmem_base), C::kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    if (warp == 0) {
+        // ---------------- TMA producer: the whole warp walks the loop, lane 0 issues
+        int stage = 0;
+        uint32_t phase = 0;
+        uint32_t armed = 0;  // bit s: stage s was handed to the TMA unit at least once
+        bool ok = true;
+        for (int g = b; g < total_tiles && ok; g += P.P) {
+            const Tile t = decode_tile(g, P);
+            const int e = __ldg(&P.mtile_expert[t.mu]);
+            const int row0 = __ldg(&P.mtile_first_row[t.mu]);
+            const int n0 = t.s * P.split_w + t.i_n * TN;
+            const int k0 = t.p * P.K;
+            for (int kb = 0; kb < P.num_kb; ++kb) {
+                ok = wait_barrier(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, deadline, P.status, (uint32_t)g, 10u);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                if (lane == 0) {
+                    const uint32_t full = smem_u32(&ctl->full[stage]);
+                    const uint32_t a_dst = smem_u32(ring + stage * C::kStageBytes);
+                    mbar_arrive_expect_tx(full, (uint32_t)C::kStageBytes);
+                    tma_load_2d(a_dst, &P.tmA, full, k0 + kb * kBlockK, row0);
+                    tma_load_3d(a_dst + C::kABytes, &P.tmB, full, k0 + kb * kBlockK, n0, e);
+                }
+                __syncwarp();
+                armed |= 1u << stage;
+                if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+            }
+        }
+        if (!ok) {
+            // wind-down: let the copies already issued land before shared memory is released
+            // (bounded; a stage consumed meanwhile has completed its phase and passes at once)
+            const unsigned long long drain = globaltimer_ns() + 2000000ull;
+            for (int sidx = 0; sidx < C::kStages; ++sidx) {
+                if (!(armed & (1u << sidx))) continue;
+                // parity of the phase this stage was last armed in
+                const uint32_t par = (sidx < stage) ? phase : (phase ^ 1u);
+                while (!mbar_try_wait(smem_u32(&ctl->full[sidx]), par) && globaltimer_ns() < drain) {}
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer: the whole warp walks the loop, lane 0 issues
+        constexpr uint32_t idesc = make_idesc(kMmaM, TN);
+        int stage = 0;
+        uint32_t phase = 0;
+        int it = 0;
+        bool ok = true;
+        for (int g = b; g < total_tiles && ok; g += P.P, ++it) {
+            const int a = it & 1;
+            const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+            ok = wait_barrier(smem_u32(&ctl->tmem_empty[a]), acc_phase ^ 1u, ctl, deadline, P.status, (uint32_t)g, 20u);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + (uint32_t)(a * TN);
+            for (int kb = 0; kb < P.num_kb; ++kb) {
+                ok = wait_barrier(smem_u32(&ctl->full[stage]), phase, ctl, deadline, P.status, (uint32_t)g, 21u);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
+                if (lane == 0) {
+                    const uint32_t a_addr = smem_u32(ring + stage * C::kStageBytes);
+                    const uint64_t a_desc = make_smem_desc(a_addr);
+                    const uint64_t b_desc = make_smem_desc(a_addr + C::kABytes);
+                    const int ksteps = (kb == P.num_kb - 1) ? P.last_ksteps : (kBlockK / kUmmaK);
+                    for (int k = 0; k < ksteps; ++k) {
+                        // advancing K by 16 bf16 = 32 bytes inside the swizzle row: +2 in the address field
+                        tc_mma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
+                                    (kb > 0 || k > 0) ? 1u : 0u);
+                    }
+                    tc_commit(smem_u32(&ctl->empty[stage]));   // stage reusable once these MMAs have read it
+                }
+                __syncwarp();
+                if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+            }
+            if (ok && lane == 0) tc_commit(smem_u32(&ctl->tmem_full[a]));  // accumulator complete
+            __syncwarp();
+        }
+    } else if (warp >= 4 && warp < 4 + C::kEpiWarps) {
+        // ---------------- epilogue: TMEM -> bf16 -> Y, then publish the tile
+        const int q = warp & 3;                    // TMEM lane quarter this warp may read
+        const int half = (warp - 4) >> 2;          // column half of the tile
+        const int row_in_tile = q * 32 + lane;
+        const bool is_leader = (warp == 4 && lane == 0);
+        __nv_bfloat16 *Y = reinterpret_cast<__nv_bfloat16 *>(P.Y);
+        int it = 0;
+        for (int g = b; g < total_tiles; g += P.P, ++it) {
+            const Tile t = decode_tile(g, P);
+            const int a = it & 1;
+            const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+            bool ok = wait_barrier(smem_u32(&ctl->tmem_full[a]), acc_phase, ctl, deadline, P.status, (uint32_t)g, 30u);
+            ok = __all_sync(0xffffffffu, ok);
+            if (ok) {
+                tc_fence_after();
+                const int valid = __ldg(&P.mtile_valid[t.mu]);
+                const int n0 = t.s * P.split_w + t.i_n * TN;
+                const int col_end = min(P.H, (t.s + 1) * P.split_w);
+                const bool row_ok = row_in_tile < valid;
+                __nv_bfloat16 *yrow = Y + ((size_t)t.p * (size_t)P.R_pad + (size_t)t.mu * P.tile_m + row_in_tile) * (size_t)P.H;
+#pragma unroll
+                for (int cc = 0; cc < C::kColsPerHalf; cc += 32) {
+                    const int col = half * C::kColsPerHalf + cc;
+                    uint32_t r[32];
+                    tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * TN + col), r);
+                    tmem_ld_wait();
+                    if (row_ok) {
+#pragma unroll
+                        for (int v = 0; v < 4; ++v) {
+                            const int c0 = n0 + col + v * 8;
+                            if (c0 < col_end) {
+                                uint4 pk;
+                                __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(r[v * 8 + 0]), __uint_as_float(r[v * 8 + 1]));
+                                __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(r[v * 8 + 2]), __uint_as_float(r[v * 8 + 3]));
+                                __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(r[v * 8 + 4]), __uint_as_float(r[v * 8 + 5]));
+                                __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(r[v * 8 + 6]), __uint_as_float(r[v * 8 + 7]));
+                                pk.x = *reinterpret_cast<uint32_t *>(&h0);
+                                pk.y = *reinterpret_cast<uint32_t *>(&h1);
+                                pk.z = *reinterpret_cast<uint32_t *>(&h2);
+                                pk.w = *reinterpret_cast<uint32_t *>(&h3);
+                                *reinterpret_cast<uint4 *>(yrow + c0) = pk;
+                            }
+                        }
+                    }
+                }
+                // the accumulator buffer may be overwritten by the MMA of the tile after next
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctl->tmem_empty[a]));
+            }
+            // every epilogue warp reaches this barrier, also after a failed wait
+            named_barrier(1, C::kEpiThreads);
+            if (ctl->abort) break;
+            if (is_leader && g != P.withhold) {
+                __threadfence();
+                st_release_u32(&P.flags[g], P.epoch);
+                red_release_add_u32(&P.split_done[t.s], 1u);
+            }
+        }
+    }
+    // ---------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, C::kTmemCols);
+    }
+}
+
+// --------------------------------------------------------------------------- communication CTA
+
+__device__ __forceinline__ void fma_bf16x8(float (&acc)[8], const uint4 &v, float w)
+{
+    const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        acc[2 * i + 0] = fmaf(w, __uint_as_float(u[i] << 16), acc[2 * i + 0]);
+        acc[2 * i + 1] = fmaf(w, __uint_as_float(u[i] & 0xFFFF0000u), acc[2 * i + 1]);
+    }
+}
+
+template <int TN>
+__device__ void comm_cta(const FusedParams &P, int c)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr int n_warps = kThreads / 32;
+    constexpr int kGroupCols = 256;               // 32 lanes x 8 bf16
+    const int Q = P.k_tot * P.TP;
+    const unsigned long long deadline = globaltimer_ns() + P.wait_ns;
+    const __nv_bfloat16 *Y = reinterpret_cast<const __nv_bfloat16 *>(P.Y);
+    const bool wait_needed = (P.mode != MOE_MODE_COMBINE_ONLY);
+
+    for (int s = 0; s < P.L; ++s) {
+        bool split_ready = !wait_needed;
+        const int split_c0 = s * P.split_w;
+        const int split_c1 = min(P.H, split_c0 + P.split_w);
+        for (int ct = c; ct < P.comm_tiles; ct += P.C) {
+            const int tok_tile = ct / P.comm_cols;
+            const int col_tile = ct - tok_tile * P.comm_cols;
+            const int d = tok_tile / P.tok_tiles_per_rank;
+            const int ti = tok_tile - d * P.tok_tiles_per_rank;
+            const int t0 = d * P.tok_blk + ti * kCommTileM;
+            const int t1 = min(min(P.T, (d + 1) * P.tok_blk), t0 + kCommTileM);
+            const int c0 = split_c0 + col_tile * kCommTileN;
+            const int c1 = min(split_c1, c0 + kCommTileN);
+            if (t0 >= t1 || c0 >= c1) continue;
+            const int groups = (c1 - c0 + kGroupCols - 1) / kGroupCols;
+            const int units = (t1 - t0) * groups;
+            __nv_bfloat16 *out_d = reinterpret_cast<__nv_bfloat16 *>(P.out[d]);
+            for (int u = warp; u < units; u += n_warps) {
+                const int tt = u / groups;
+                const int grp = u - tt * groups;
+                const int t = t0 + tt;
+                const int gcol0 = c0 + grp * kGroupCols;
+                const int col = gcol0 + lane * 8;
+                // routing of this token: lane j holds slot j
+                int my_row = -1;
+                float my_w = 0.f;
+                if (lane < P.k_tot) {
+                    my_row = __ldg(&P.pad_row[(size_t)t * P.k_tot + lane]);
+                    my_w = __ldg(&P.topk_w[(size_t)t * P.k_tot + lane]);
+                    if (my_row >= P.R_pad) {
+                        report(P.status, MOE_DEV_OOB, (uint32_t)my_row, 41u);
+                        my_row = -1;
+                    }
+                }
+                if (!split_ready) {
+                    uint32_t done = 0;
+                    if (lane == 0) done = ld_acquire_u32(&P.split_done[s]);
+                    done = __shfl_sync(0xffffffffu, done, 0);
+                    if (done >= (uint32_t)P.W_comp) {
+                        split_ready = true;
+                    } else {
+                        // per-tile readiness: every (slot j, shard p, n-tile under this column group)
+                        const int nt = (min(c1, gcol0 + kGroupCols) - gcol0 + TN - 1) / TN;
+                        const int in0 = (gcol0 - split_c0) / TN;
+                        bool failed = false;
+                        for (int chk = lane; chk < Q * nt; chk += 32) {
+                            const int qq = chk / nt;
+                            const int tn = chk - qq * nt;
+                            const int j = qq / P.TP;
+                            const int p = qq - j * P.TP;
+                            const int row = __ldg(&P.pad_row[(size_t)t * P.k_tot + j]);
+                            if (row < 0 || row >= P.R_pad) continue;
+                            const int mu = row / P.tile_m;
+                            const int g = s * P.W_comp + (mu * P.TP + p) * P.NTs + in0 + tn;
+                            uint32_t spins = 0;
+                            while (ld_acquire_u32(&P.flags[g]) != P.epoch) {
+                                if ((++spins & 31u) == 0u && globaltimer_ns() > deadline) {
+                                    report(P.status, MOE_DEV_TIMEOUT, (uint32_t)g, 40u);
+                                    failed = true;
+                                    break;
+                                }
+                                __nanosleep(64);
+                            }
+                            if (failed) break;
+                        }
+                        if (__any_sync(0xffffffffu, failed)) return;   // this warp gives up; others carry on
+                    }
+                    __syncwarp();
+                }
+                // gather + weighted sum, fp32, fixed (j, p) order
+                float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                const bool active = col < c1;
+                for (int q0 = 0; q0 < Q; q0 += 8) {
+                    uint4 v[8];
+                    float w[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int qq = q0 + i;
+                        const int j = (qq < Q) ? qq / P.TP : 0;
+                        const int p = qq - j * P.TP;
+                        const int row = __shfl_sync(0xffffffffu, my_row, j);
+                        w[i] = __shfl_sync(0xffffffffu, my_w, j);
+                        v[i] = make_uint4(0u, 0u, 0u, 0u);
+                        if (qq >= Q || row < 0) w[i] = 0.f;
+                        else if (active)
+                            v[i] = __ldcg(reinterpret_cast<const uint4 *>(Y + ((size_t)p * (size_t)P.R_pad + (size_t)row) * (size_t)P.H + col));
+                    }
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) fma_bf16x8(acc, v[i], w[i]);
+                }
+                if (active) {
+                    uint4 pk;
+                    __nv_bfloat162 h0 = __floats2bfloat162_rn(acc[0], acc[1]);
+                    __nv_bfloat162 h1 = __floats2bfloat162_rn(acc[2], acc[3]);
+                    __nv_bfloat162 h2 = __floats2bfloat162_rn(acc[4], acc[5]);
+                    __nv_bfloat162 h3 = __floats2bfloat162_rn(acc[6], acc[7]);
+                    pk.x = *reinterpret_cast<uint32_t *>(&h0);
+                    pk.y = *reinterpret_cast<uint32_t *>(&h1);
+                    pk.z = *reinterpret_cast<uint32_t *>(&h2);
+                    pk.w = *reinterpret_cast<uint32_t *>(&h3);
+                    __stcs(reinterpret_cast<uint4 *>(out_d + (size_t)(t - d * P.tok_blk) * (size_t)P.H + col), pk);
+                }
+            }
+        }
+    }
+}
+
+// --------------------------------------------------------------------------- kernel
+
+template <int TN>
+__global__ void __launch_bounds__(kThreads, 1)
+moe_gemm2_combine_kernel(const __grid_constant__ FusedParams P)
+{
+    extern __shared__ uint8_t smem_raw[];
+    // 128B-swizzled tiles need 1024-byte aligned bases
+    uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    Control *ctl = reinterpret_cast<Control *>(ring + kStageBytesTotal);
+
+    if (blockIdx.x == 0 && threadIdx.x < (unsigned)P.L) P.split_done_next[threadIdx.x] = 0u;
+
+    if ((int)blockIdx.x < P.C)
+        comm_cta<TN>(P, (int)blockIdx.x);
+    else
+        compute_cta<TN>(P, ring, ctl, (int)blockIdx.x - P.C);
+}
+
+}  // namespace
+
+size_t fused_smem_bytes(int) { return (size_t)kStageBytesTotal + 1024 + sizeof(Control) + 64; }
+
+template <int TN>
+static cudaError_t prepare()
+{
+    return cudaFuncSetAttribute(moe_gemm2_combine_kernel<TN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)fused_smem_bytes(TN));
+}
+
+cudaError_t fused_occupancy(int tile_n, int *blocks_per_sm)
+{
+    cudaError_t e;
+    const size_t sm = fused_smem_bytes(tile_n);
+    switch (tile_n) {
+    case 64:
+        if ((e = prepare<64>()) != cudaSuccess) return e;
+        return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, moe_gemm2_combine_kernel<64>, kThreads, sm);
+    case 128:
+        if ((e = prepare<128>()) != cudaSuccess) return e;
+        return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, moe_gemm2_combine_kernel<128>, kThreads, sm);
+    case 256:
+        if ((e = prepare<256>()) != cudaSuccess) return e;
+        return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, moe_gemm2_combine_kernel<256>, kThreads, sm);
+    }
+    return cudaErrorInvalidValue;
+}
+
+cudaError_t fused_launch(int tile_n, const FusedParams &p, int grid, cudaStream_t stream)
+{
+    const size_t sm = fused_smem_bytes(tile_n);
+    switch (tile_n) {
+    case 64: moe_gemm2_combine_kernel<64><<<grid, kThreads, sm, stream>>>(p); break;
+    case 128: moe_gemm2_combine_kernel<128><<<grid, kThreads, sm, stream>>>(p); break;
+    case 256: moe_gemm2_combine_kernel<256><<<grid, kThreads, sm, stream>>>(p); break;
+    default: return cudaErrorInvalidValue;
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace moe

@@ -1,0 +1,76 @@
+// Internal declarations shared by the translation units of libmoe_b200.so.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+#include <cstdio>
+#include <unordered_map>
+
+#include "../../include/moe_b200.h"
+
+namespace moe {
+
+constexpr int kThreads = 512;          // threads of every CTA of the fused kernel
+constexpr int kBlockK = 64;            // bf16 elements per k-block: one 128-byte swizzle row
+constexpr int kUmmaK = 16;             // K of one tcgen05.mma.kind::f16 instruction
+constexpr int kMmaM = 128;             // M of the MMA (tile_m = 64 stores the first 64 rows only)
+constexpr int kStageBytesTotal = 192 * 1024;  // operand ring, all stages together
+constexpr int kCommTileM = 128;        // T_M^comm
+constexpr int kCommTileN = 1024;       // T_N^comm
+constexpr int kRoutingChunk = 256;     // flat assignments handled by one warp while sorting
+constexpr uint64_t kDefaultWaitNs = 2000000000ull;
+
+// Parameters of one fused launch.  Passed by value (__grid_constant__): the two tensor maps
+// must sit in kernel parameter space, 64-byte aligned.
+struct alignas(64) FusedParams {
+    CUtensorMap tmA;   // x_routed [R, I]      box 64 x 128 rows, 128B swizzle
+    CUtensorMap tmB;   // W2 [E_tot, H, I]     box 64 x tile_n x 1, 128B swizzle
+    const int32_t *mtile_expert;
+    const int32_t *mtile_first_row;
+    const int32_t *mtile_valid;
+    const int32_t *pad_row;
+    const float *topk_w;
+    void *Y;                       // bf16 [TP][R_pad][H]
+    uint32_t *flags;               // [L * W_comp] readiness per global tile (== epoch when ready)
+    uint32_t *split_done;          // [L] tiles finished per split (this launch)
+    uint32_t *split_done_next;     // [L] counters of the next launch, zeroed by this one
+    uint32_t *status;              // 4 words
+    void *out[MOE_MAX_EP];
+    unsigned long long wait_ns;
+    long long R_pad;
+    int32_t T, H, K, TP, EP, L, k_tot;
+    int32_t S, tile_m, NTs, split_w, W_comp;
+    int32_t C, P, mode, withhold;
+    int32_t tok_blk, tok_tiles_per_rank, comm_cols, comm_tiles;
+    int32_t num_kb, last_ksteps;
+    uint32_t epoch;
+};
+
+}  // namespace moe
+
+struct moe_handle {
+    int device = 0;
+    int G = 0;
+    unsigned long long wait_ns = moe::kDefaultWaitNs;
+    char err[512] = {0};
+    std::unordered_map<const void *, uint32_t> epochs;  // per flags workspace
+    void *encode_tiled = nullptr;                       // cuTensorMapEncodeTiled
+    int o_comp[3] = {0, 0, 0};                          // tile_n = 64, 128, 256
+};
+
+namespace moe {
+
+inline int tile_n_slot(int tile_n) { return tile_n == 64 ? 0 : tile_n == 128 ? 1 : tile_n == 256 ? 2 : -1; }
+
+int32_t cuda_fail(moe_handle *h, cudaError_t e, const char *what);
+// fused kernel (gemm2_combine.cu)
+size_t fused_smem_bytes(int tile_n);
+cudaError_t fused_occupancy(int tile_n, int *blocks_per_sm);
+cudaError_t fused_launch(int tile_n, const FusedParams &p, int grid, cudaStream_t stream);
+// routing kernels (routing.cu)
+cudaError_t routing_launch(const int32_t *topk_idx, const moe_shape &s, int tile_m,
+                           const moe_routing &r, uint32_t *status, cudaStream_t stream);
+
+}  // namespace moe

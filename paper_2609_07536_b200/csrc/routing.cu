@@ -1,0 +1,164 @@
+// Routing / permutation / routed-tile-count builder (device).
+//
+// Section II-A: the router's token-expert assignments; Eq. 5: expert e needs
+// ceil(M_e / T_M) tiles along the token dimension; Eq. 16: their sum S.
+// The routed rows are the flat assignments f = t * k_tot + j in a *stable* order by expert.
+//
+// Three small launches (the data is a few hundred KB):
+//   1. hist     every warp histograms its own contiguous chunk of assignments;
+//   2. scan     one CTA: counts, exclusive offsets, tiles per expert and their prefix, the
+//               m-tile table, and per-(warp, expert) exclusive bases;
+//   3. scatter  every warp walks its chunk in order, 32 assignments at a time;
+//               match_any gives each lane its rank among equal experts -> stable.
+
+#include "moe_internal.h"
+
+namespace moe {
+namespace {
+
+constexpr int kWarpsPerBlock = 8;
+
+__device__ __forceinline__ void report(uint32_t *status, uint32_t code, uint32_t detail, uint32_t where)
+{
+    if (atomicCAS(&status[0], 0u, code) == 0u) {
+        status[1] = detail;
+        status[2] = where;
+    }
+    atomicAdd(&status[3], 1u);
+}
+
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+routing_hist(const int32_t *__restrict__ topk_idx, int R, int k_tot, int E_tot, int n_warps,
+             int32_t *__restrict__ whist, uint32_t *status)
+{
+    extern __shared__ int32_t sh[];
+    const int warp_in_block = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int w = blockIdx.x * kWarpsPerBlock + warp_in_block;
+    int32_t *h = sh + warp_in_block * E_tot;
+    for (int e = lane; e < E_tot; e += 32) h[e] = 0;
+    __syncwarp();
+    if (w < n_warps) {
+        const int begin = w * kRoutingChunk;
+        const int end = min(R, begin + kRoutingChunk);
+        for (int f = begin + lane; f < end; f += 32) {
+            const int e = topk_idx[f];
+            if (e < 0 || e >= E_tot) {
+                report(status, MOE_DEV_OOB, (uint32_t)f, 1u);
+                continue;
+            }
+            atomicAdd(&h[e], 1);
+            // the same expert twice inside one token?
+            const int t = f / k_tot, j = f - t * k_tot;
+            for (int jj = 0; jj < j; ++jj)
+                if (topk_idx[t * k_tot + jj] == e) report(status, MOE_DEV_DUP_EXPERT, (uint32_t)t, 1u);
+        }
+        __syncwarp();
+        for (int e = lane; e < E_tot; e += 32) whist[(size_t)w * E_tot + e] = h[e];
+    }
+}
+
+__global__ void __launch_bounds__(1024)
+routing_scan(int R, int E_tot, int tile_m, int n_warps, int max_mtiles,
+             int32_t *__restrict__ whist, int32_t *counts, int32_t *offsets, int32_t *tiles,
+             int32_t *tile_offsets, int32_t *mtile_expert, int32_t *mtile_first_row,
+             int32_t *mtile_valid, uint32_t *status)
+{
+    // counts, and whist turned into an exclusive prefix over the warps (per expert)
+    for (int e = threadIdx.x; e < E_tot; e += blockDim.x) {
+        int run = 0;
+        for (int w = 0; w < n_warps; ++w) {
+            const int c = whist[(size_t)w * E_tot + e];
+            whist[(size_t)w * E_tot + e] = run;
+            run += c;
+        }
+        counts[e] = run;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int off = 0, toff = 0;
+        for (int e = 0; e < E_tot; ++e) {
+            const int c = counts[e];
+            const int nt = (c + tile_m - 1) / tile_m;
+            offsets[e] = off;
+            tile_offsets[e] = toff;
+            tiles[e] = nt;
+            off += c;
+            toff += nt;
+        }
+        offsets[E_tot] = off;
+        tile_offsets[E_tot] = toff;
+        tiles[E_tot] = toff;  // S rides behind the per-expert counts for the host copy
+        if (toff > max_mtiles) report(status, MOE_DEV_OOB, (uint32_t)toff, 2u);
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < E_tot; e += blockDim.x) {
+        const int c = counts[e], off = offsets[e], toff = tile_offsets[e], nt = tiles[e];
+        for (int i = 0; i < nt; ++i) {
+            const int mu = toff + i;
+            if (mu >= max_mtiles) break;
+            mtile_expert[mu] = e;
+            mtile_first_row[mu] = off + i * tile_m;
+            mtile_valid[mu] = min(tile_m, c - i * tile_m);
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+routing_scatter(const int32_t *__restrict__ topk_idx, int R, int E_tot, int tile_m, int n_warps,
+                const int32_t *__restrict__ whist, const int32_t *__restrict__ offsets,
+                const int32_t *__restrict__ tile_offsets, int32_t *__restrict__ perm,
+                int32_t *__restrict__ inv_perm, int32_t *__restrict__ pad_row)
+{
+    extern __shared__ int32_t sh[];
+    const int warp_in_block = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int w = blockIdx.x * kWarpsPerBlock + warp_in_block;
+    if (w >= n_warps) return;
+    int32_t *run = sh + warp_in_block * E_tot;  // next free row per expert, for this warp
+    for (int e = lane; e < E_tot; e += 32) run[e] = offsets[e] + whist[(size_t)w * E_tot + e];
+    __syncwarp();
+    const int begin = w * kRoutingChunk;
+    const int end = min(R, begin + kRoutingChunk);
+    for (int f0 = begin; f0 < end; f0 += 32) {
+        const int f = f0 + lane;
+        const bool in = f < end;
+        int e = in ? topk_idx[f] : -1;
+        const bool ok = in && e >= 0 && e < E_tot;
+        const unsigned active = __ballot_sync(0xffffffffu, ok);
+        if (in && !ok) { inv_perm[f] = -1; pad_row[f] = -1; }
+        if (ok) {
+            const unsigned same = __match_any_sync(active, e);
+            const int rank = __popc(same & ((1u << lane) - 1u));
+            const int r = run[e] + rank;
+            __syncwarp(active);
+            if (rank == 0) run[e] += __popc(same);
+            perm[r] = f;
+            inv_perm[f] = r;
+            pad_row[f] = tile_m * tile_offsets[e] + (r - offsets[e]);
+        }
+        __syncwarp();
+    }
+}
+
+}  // namespace
+
+cudaError_t routing_launch(const int32_t *topk_idx, const moe_shape &s, int tile_m,
+                           const moe_routing &r, uint32_t *status, cudaStream_t stream)
+{
+    const int R = s.T * s.k_tot;
+    const int n_warps = (R + kRoutingChunk - 1) / kRoutingChunk;
+    const int blocks = (n_warps + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    const size_t sh = (size_t)kWarpsPerBlock * s.E_tot * sizeof(int32_t);
+    if (blocks > 0)
+        routing_hist<<<blocks, kWarpsPerBlock * 32, sh, stream>>>(topk_idx, R, s.k_tot, s.E_tot, n_warps,
+                                                                  r.scratch, status);
+    routing_scan<<<1, 1024, 0, stream>>>(R, s.E_tot, tile_m, n_warps, r.max_mtiles, r.scratch, r.counts,
+                                         r.offsets, r.tiles, r.tile_offsets, r.mtile_expert,
+                                         r.mtile_first_row, r.mtile_valid, status);
+    if (blocks > 0)
+        routing_scatter<<<blocks, kWarpsPerBlock * 32, sh, stream>>>(
+            topk_idx, R, s.E_tot, tile_m, n_warps, r.scratch, r.offsets, r.tile_offsets, r.perm,
+            r.inv_perm, r.pad_row);
+    return cudaGetLastError();
+}
+
+}  // namespace moe

@@ -1,0 +1,159 @@
+// Launch-time analytical selector of the communication-CTA count (host only).
+//
+// Section III-D, Algorithm 1: for every legal C evaluate the wave-quantized makespan
+//   R(C) = ceil(C / o_comm)                      (Eq. 1)
+//   P(C) = o_comp (G - R(C))                     (Eq. 3)
+//   A_s  = ceil((s+1) W_comp / P)                (Eq. 9)
+//   q    = rho ceil(W_comm / C)                  (Eq. 8, Eq. 10)
+//   F_s  = max(A_s, F_{s-1}) + q,  T = F_{L-1}   (Eq. 11, Eq. 12)
+// and keep the lexicographic minimum of (T, Delta_comp, C), Delta_comp = V_comp P - W_comp
+// (tie breaker).  rho is carried in fixed point (2^-20) so that "the same T(C)" is an exact
+// integer comparison.  No CUDA call, no allocation, no global state.
+
+#include <cstdint>
+
+#include "../../include/moe_b200.h"
+
+namespace {
+
+constexpr int kRhoShift = 20;
+
+inline int64_t ceil_div64(int64_t a, int64_t b) { return (a + b - 1) / b; }
+inline uint32_t ceil_div32(uint32_t a, uint32_t b) { return (a + b - 1) / b; }
+
+struct Candidate {
+    int64_t T_q;
+    int64_t delta;
+    int32_t C, R, P;
+};
+
+// One candidate.  32-bit divisions when every dividend fits (the common case), else 64-bit.
+inline bool evaluate(int32_t C, int64_t Wc, int64_t Wm, int32_t L, int32_t G, int32_t o_comp,
+                     int32_t o_comm, int64_t rho_q, bool small, Candidate *out)
+{
+    const int32_t R = (C + o_comm - 1) / o_comm;
+    const int64_t P = (int64_t)o_comp * (G - R);
+    if (P <= 0) return false;
+    int64_t F = 0;
+    int64_t V_comp;
+    if (small) {
+        const uint32_t p = (uint32_t)P, wc = (uint32_t)Wc;
+        const uint32_t v_comm = ceil_div32((uint32_t)Wm, (uint32_t)C);
+        const int64_t q = rho_q * (int64_t)v_comm;
+        uint32_t num = 0;
+        uint32_t a0 = 0;
+        for (int32_t s = 0; s < L; ++s) {
+            num += wc;
+            const uint32_t a = ceil_div32(num, p);
+            if (s == 0) a0 = a;
+            const int64_t A = (int64_t)a << kRhoShift;
+            F = (A > F ? A : F) + q;
+        }
+        V_comp = a0;
+    } else {
+        const int64_t v_comm = ceil_div64(Wm, C);
+        const int64_t q = rho_q * v_comm;
+        for (int32_t s = 0; s < L; ++s) {
+            const int64_t A = ceil_div64((int64_t)(s + 1) * Wc, P) << kRhoShift;
+            F = (A > F ? A : F) + q;
+        }
+        V_comp = ceil_div64(Wc, P);
+    }
+    out->T_q = F;
+    out->delta = V_comp * P - Wc;
+    out->C = C;
+    out->R = R;
+    out->P = (int32_t)P;
+    return true;
+}
+
+}  // namespace
+
+extern "C" int32_t plan_partition(const int32_t *routed_tile_counts, int32_t n_experts,
+                                  const moe_occupancy *occ, const moe_sm_limits *limits,
+                                  const moe_shape *shape, const moe_rho *rho, moe_plan *out)
+{
+    if (!routed_tile_counts || !occ || !limits || !shape || !rho || !out) return MOE_ERR_NULL;
+    if (n_experts < 0 || shape->T < 0 || shape->H < 1 || shape->L < 1 || shape->L > MOE_MAX_L ||
+        shape->EP < 1 || shape->TP < 1 || shape->I < 1 || shape->k_tot < 1 ||
+        occ->tile_m < 1 || occ->tile_n < 1 || occ->comm_tile_m < 1 || occ->comm_tile_n < 1 ||
+        occ->o_comp < 1 || occ->o_comm < 1 || limits->G < 1)
+        return MOE_ERR_SHAPE;
+
+    // Eq. 16: sum of the routed tile counts; Eq. 5: compute tiles per split (g = TP groups).
+    int64_t S = 0;
+    for (int32_t e = 0; e < n_experts; ++e) {
+        if (routed_tile_counts[e] < 0) return MOE_ERR_SHAPE;
+        S += routed_tile_counts[e];
+    }
+    const int64_t split_w = ceil_div64(shape->H, shape->L);
+    const int64_t Wc = (int64_t)shape->TP * S * ceil_div64(split_w, occ->tile_n);
+
+    // Eq. 7 summed over the emulated ranks: rank d owns a contiguous block of ceil(T/EP) tokens.
+    const int64_t blk = ceil_div64(shape->T, shape->EP);
+    int64_t tok_tiles = 0;
+    for (int32_t d = 0; d < shape->EP; ++d) {
+        int64_t own = shape->T - (int64_t)d * blk;
+        if (own > blk) own = blk;
+        if (own > 0) tok_tiles += ceil_div64(own, occ->comm_tile_m);
+    }
+    const int64_t Wm = tok_tiles * ceil_div64(split_w, occ->comm_tile_n);
+    if (Wc > INT32_MAX || Wm > INT32_MAX) return MOE_ERR_SHAPE;
+
+    // Eq. 14 (one product over one product; integer factors are exact in double).
+    const int64_t K = shape->I / shape->TP;
+    if (K < 1 || rho->K_ref < 1 || rho->tile_m_ref < 1 || rho->tile_n_ref < 1) return MOE_ERR_SHAPE;
+    double num, den;
+    if (rho->mode == MOE_RHO_PAPER) {
+        if (rho->D_ref < 1) return MOE_ERR_SHAPE;
+        num = (double)((int64_t)rho->K_ref * rho->tile_m_ref * rho->tile_n_ref * shape->EP);
+        den = (double)(K * occ->tile_m * occ->tile_n * rho->D_ref);
+    } else if (rho->mode == MOE_RHO_LOCAL) {
+        if (rho->rows_ref < 1 || rho->comm_cols_ref < 1) return MOE_ERR_SHAPE;
+        const int64_t rows = (int64_t)shape->k_tot * shape->TP + 1;
+        const int64_t cols = split_w < occ->comm_tile_n ? split_w : occ->comm_tile_n;
+        num = (double)((int64_t)rho->K_ref * rho->tile_m_ref * rho->tile_n_ref * rows * cols);
+        den = (double)(K * occ->tile_m * occ->tile_n * rho->rows_ref * rho->comm_cols_ref);
+    } else {
+        return MOE_ERR_SHAPE;
+    }
+    const double rho_v = rho->rho_ref * num / den;
+    if (!(rho_v >= 0.0) || rho_v > 1.0e9) return MOE_ERR_SHAPE;
+    const double scaled = rho_v * (double)(1 << kRhoShift) + 0.5;
+    const int64_t rho_q = (int64_t)scaled;  // scaled >= 0.5: truncation is floor
+
+    const int32_t L = shape->L, G = limits->G, o_comp = occ->o_comp, o_comm = occ->o_comm;
+    const bool small = (int64_t)L * Wc < (int64_t)0x7FFFFF00 && Wm < (int64_t)0x7FFFFF00 &&
+                       (int64_t)o_comp * G < (int64_t)0x7FFFFF00;
+
+    Candidate best{};
+    bool have = false;
+    if (limits->force_comm_ctas > 0 || limits->selector_off) {
+        const int32_t C = limits->force_comm_ctas > 0 ? limits->force_comm_ctas : limits->default_C;
+        if (C < 1) return MOE_ERR_PLAN_INFEASIBLE;
+        have = evaluate(C, Wc, Wm, L, G, o_comp, o_comm, rho_q, small, &best);
+    } else {
+        for (int32_t C = 1; C <= limits->C_max; ++C) {
+            Candidate c;
+            if (!evaluate(C, Wc, Wm, L, G, o_comp, o_comm, rho_q, small, &c)) break;  // P only falls
+            // ascending C: a strict improvement of (T, Delta) is needed to replace the incumbent
+            if (!have || c.T_q < best.T_q || (c.T_q == best.T_q && c.delta < best.delta)) {
+                best = c;
+                have = true;
+            }
+        }
+    }
+    if (!have) return MOE_ERR_PLAN_INFEASIBLE;
+
+    out->comm_ctas = best.C;
+    out->R = best.R;
+    out->P = best.P;
+    out->W_comp = (int32_t)Wc;
+    out->W_comm = (int32_t)Wm;
+    out->delta = (int32_t)best.delta;
+    out->pred_T_q = best.T_q;
+    out->rho_q = rho_q;
+    out->mode = MOE_MODE_FUSED;
+    out->debug_withhold_tile = -1;
+    return MOE_OK;
+}

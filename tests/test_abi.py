@@ -1,0 +1,57 @@
+"""The C-ABI library loads on a machine without a GPU and exports every symbol that
+include/moe_b200.h declares; argument errors come back as status codes.  No compute call."""
+
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2609_07536_b200 import binding as B
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "moe_b200.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"^(?:int32_t|const char \*)\s*(\w+)\s*\(", text, flags=re.M)))
+
+
+def test_every_declared_symbol_is_exported():
+    names = _declared()
+    assert len(names) >= 14
+    L = B.lib()
+    for n in names:
+        assert hasattr(L, n), n
+    assert sorted(B.EXPORTS) == names
+
+
+def test_structs_match_header_sizes():
+    assert ctypes.sizeof(B.moe_shape) == 32
+    assert ctypes.sizeof(B.moe_occupancy) == 24
+    assert ctypes.sizeof(B.moe_sm_limits) == 20
+    assert ctypes.sizeof(B.moe_rho) == 40
+    assert ctypes.sizeof(B.moe_plan) == 48
+    assert ctypes.sizeof(B.moe_status) == 16
+
+
+def test_workspace_sizes_and_argument_errors():
+    s = B.make_shape(256, 256, 128, 8, 2, 1, 2, 1)
+    rb, yb, fb, sb = B.moe_workspace_bytes(s, 64, 64)
+    max_mtiles = 512 // 64 + 8
+    assert yb >= 1 * max_mtiles * 64 * 256 * 2 and sb == 16
+    assert fb >= (64 + 1 * 1 * max_mtiles * 4) * 4
+    assert rb >= 3 * 512 * 4 + 3 * max_mtiles * 4
+    with pytest.raises(B.MoeError) as e:
+        B.moe_workspace_bytes(B.make_shape(256, 250, 128, 8, 2, 1, 2, 1), 64, 64)   # H % 8
+    assert e.value.code == B.MOE_ERR_SHAPE
+    with pytest.raises(B.MoeError) as e:
+        B.moe_workspace_bytes(B.make_shape(256, 256, 100, 8, 2, 1, 2, 1), 64, 64)   # K % 16
+    assert e.value.code == B.MOE_ERR_SHAPE
+    with pytest.raises(B.MoeError) as e:
+        B.moe_workspace_bytes(s, 96, 64)
+    assert e.value.code == B.MOE_ERR_UNSUPPORTED
+    assert B.lib().moe_workspace_bytes(None, 64, 64, None, None, None, None) == B.MOE_ERR_NULL
+    assert B.lib().moe_destroy(None) == B.MOE_OK
+    assert B.moe_host_arena_bytes(s, 64, 64) > rb + yb + fb

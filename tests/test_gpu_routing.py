@@ -1,0 +1,71 @@
+"""GPU routing builder against the routing reference: every array bit-exact."""
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import routing_ref as rr
+from paper_2609_07536_b200 import binding as B
+from paper_2609_07536_b200 import workloads as wl
+from tests import gpu_common as G
+
+pytestmark = pytest.mark.gpu
+
+KEYS = ["counts", "offsets", "tiles", "tile_offsets", "perm", "inv_perm", "pad_row",
+        "mtile_expert", "mtile_first_row", "mtile_valid"]
+
+
+def _compare(w, idx):
+    ws, _, S = G.build_routing(w, idx)
+    st = B.moe_get_status(G.handle(), ws.status)
+    assert st.code == 0
+    ref = rr.build_routing(idx, w.E_tot, w.tile_m)
+    assert S == ref["S"]
+    got = G.routing_to_numpy(ws, S)
+    for k in KEYS:
+        assert np.array_equal(got[k], ref[k]), k
+    assert ws.tile_counts[:w.E_tot].tolist() == ref["tiles"].tolist()
+
+
+@pytest.mark.parametrize("w", [wl.TINY, wl.GRANITE, wl.QWEN, wl.DSV2L], ids=lambda w: w.name)
+def test_configs(w):
+    idx, _, _ = wl.make_routing(w)
+    _compare(w, idx)
+
+
+def test_adversarial():
+    from dataclasses import replace
+    base = replace(wl.TINY, T=300, E=9, k=1, tile_m=64)
+    # one hot expert, others empty
+    _compare(base, np.full((300, 1), 4, dtype=np.int32))
+    # E = 1
+    _compare(replace(base, E=1), np.zeros((300, 1), dtype=np.int32))
+    # T not a tile multiple, k = 3, tile 128, many empty experts
+    rng = np.random.default_rng(0)
+    w = replace(wl.TINY, T=1001, E=70, k=3, tile_m=128)
+    idx = np.stack([rng.choice(13, 3, replace=False) * 5 for _ in range(1001)]).astype(np.int32)
+    _compare(w, idx)
+    # a single token
+    _compare(replace(base, T=1, E=4, k=2), np.array([[3, 0]], dtype=np.int32))
+    # the sweep's largest size
+    big = wl.sweep_workloads(T_list=(32768,), s_list=(1.2,), EP_list=(4,), tiles=((128, 256),))[0]
+    idx, _, _ = wl.make_routing(big)
+    _compare(big, idx)
+
+
+def test_bad_ids_are_reported_not_fatal():
+    from dataclasses import replace
+    w = replace(wl.TINY, T=64, E=8, k=2)
+    idx, _, _ = wl.make_routing(w)
+    bad = idx.copy()
+    bad[5, 1] = 99
+    ws, _, S = G.build_routing(w, bad)
+    st = B.moe_get_status(G.handle(), ws.status, check=False)
+    assert st.code == B.MOE_DEV_OOB and st.detail == 5 * 2 + 1
+    dup = idx.copy()
+    dup[7, 1] = dup[7, 0]
+    ws, _, S = G.build_routing(w, dup)
+    st = B.moe_get_status(G.handle(), ws.status, check=False)
+    assert st.code == B.MOE_DEV_DUP_EXPERT and st.detail == 7
+    # the context is still usable
+    _compare(w, idx)

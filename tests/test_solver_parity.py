@@ -1,0 +1,155 @@
+"""plan_partition (library, host C++) against the selector reference: bit-exact on every
+field, over random inputs, the BASELINE shapes, the overrides and the error paths."""
+
+import random
+import time
+
+import numpy as np
+import pytest
+
+from oracle import routing_ref as rr
+from oracle import solver_ref as sr
+from paper_2609_07536_b200 import binding as B
+from paper_2609_07536_b200 import workloads as wl
+
+
+def _oracle_plan(tiles, shape, occ, lim, rho):
+    K = shape.I // shape.TP
+    Wc = sr.w_comp(tiles, shape.TP, shape.H, shape.L, occ.tile_n)
+    Wm = sr.w_comm_gpu(shape.T, shape.EP, shape.H, shape.L, occ.comm_tile_m, occ.comm_tile_n)
+    if rho.mode == B.MOE_RHO_PAPER:
+        r = sr.rho_scaled(rho.rho_ref, rho.K_ref, rho.tile_m_ref, rho.tile_n_ref, rho.D_ref,
+                          K, occ.tile_m, occ.tile_n, shape.EP)
+    else:
+        r = sr.rho_local(rho.rho_ref, rho.K_ref, rho.tile_m_ref, rho.tile_n_ref, rho.rows_ref,
+                         rho.comm_cols_ref, K, occ.tile_m, occ.tile_n, shape.k_tot, shape.TP,
+                         shape.H, shape.L, occ.comm_tile_n)
+    rho_q = sr.quantise_rho(r)
+    sel = sr.select(Wc, Wm, shape.L, lim.G, occ.o_comp, occ.o_comm, lim.C_max, rho_q,
+                    force_comm_ctas=lim.force_comm_ctas, selector_off=bool(lim.selector_off),
+                    default_C=lim.default_C)
+    sel["rho_q"] = rho_q
+    return sel
+
+
+def _same(plan, sel):
+    assert (plan.comm_ctas, plan.R, plan.P) == (sel["comm_ctas"], sel["R"], sel["P"])
+    assert (plan.W_comp, plan.W_comm, plan.delta) == (sel["W_comp"], sel["W_comm"], sel["delta"])
+    assert plan.pred_T_q == sel["T_q"] and plan.rho_q == sel["rho_q"]
+    assert plan.mode == B.MOE_MODE_FUSED and plan.debug_withhold_tile == -1
+
+
+def _rand_inputs(rng):
+    E = rng.choice([1, 8, 40, 66])
+    tile_m = rng.choice([64, 128])
+    tile_n = rng.choice([64, 128, 256])
+    TP = rng.choice([1, 2, 4])
+    shape = B.make_shape(rng.choice([1, 37, 256, 4096, 16384, 32768]), rng.choice([256, 1536, 2048, 4096]),
+                         rng.choice([128, 512, 1408]) * TP, E, rng.choice([1, 2, 8]), TP,
+                         rng.choice([1, 2, 4, 8]), rng.choice([1, 2, 4, 8]))
+    occ = B.moe_occupancy(tile_m, tile_n, rng.choice([64, 128]), rng.choice([512, 1024]),
+                          rng.choice([1, 2]), rng.choice([1, 2, 4]))
+    lim = B.moe_sm_limits(rng.choice([4, 108, 148]), rng.randint(1, 160), 0, 0, 3)
+    rho = B.moe_rho(rng.uniform(0.05, 30.0), rng.choice([352, 704]), 128, rng.choice([128, 256]),
+                    rng.choice([2, 4]), 17, 1024, rng.choice([B.MOE_RHO_PAPER, B.MOE_RHO_LOCAL]))
+    tiles = [rng.randint(0, 40) for _ in range(E)]
+    return tiles, shape, occ, lim, rho
+
+
+def test_random_inputs_bit_exact():
+    rng = random.Random(11)
+    n = 0
+    for _ in range(20000):
+        tiles, shape, occ, lim, rho = _rand_inputs(rng)
+        try:
+            sel = _oracle_plan(tiles, shape, occ, lim, rho)
+        except ValueError:
+            with pytest.raises(B.MoeError) as e:
+                B.plan_partition(tiles, occ, lim, shape, rho)
+            assert e.value.code == B.MOE_ERR_PLAN_INFEASIBLE
+            continue
+        _same(B.plan_partition(tiles, occ, lim, shape, rho), sel)
+        n += 1
+    assert n > 15000
+
+
+def test_overrides_and_errors():
+    rng = random.Random(12)
+    for _ in range(2000):
+        tiles, shape, occ, lim, rho = _rand_inputs(rng)
+        lim.force_comm_ctas = rng.choice([0, 0, 1, 5, 200])
+        lim.selector_off = rng.choice([0, 1])
+        lim.default_C = rng.choice([1, 3, 16, 500])
+        try:
+            sel = _oracle_plan(tiles, shape, occ, lim, rho)
+        except ValueError:
+            with pytest.raises(B.MoeError) as e:
+                B.plan_partition(tiles, occ, lim, shape, rho)
+            assert e.value.code == B.MOE_ERR_PLAN_INFEASIBLE
+            continue
+        plan = B.plan_partition(tiles, occ, lim, shape, rho)
+        _same(plan, sel)
+        if lim.force_comm_ctas > 0:
+            assert plan.comm_ctas == lim.force_comm_ctas      # the user's C wins over everything
+        elif lim.selector_off:
+            assert plan.comm_ctas == lim.default_C
+    # argument errors
+    tiles, shape, occ, lim, rho = _rand_inputs(random.Random(1))
+    assert B.lib().plan_partition(None, 0, None, None, None, None, None) == B.MOE_ERR_NULL
+    bad = B.make_shape(16, 256, 128, 8, 2, 1, 2, 0)
+    with pytest.raises(B.MoeError) as e:
+        B.plan_partition(tiles, occ, lim, bad, rho)
+    assert e.value.code == B.MOE_ERR_SHAPE
+    with pytest.raises(B.MoeError):
+        B.plan_partition([-1] * shape.E_tot, occ, lim, shape, rho)
+
+
+@pytest.mark.parametrize("w", [wl.TINY, wl.GRANITE, wl.QWEN, wl.DSV2L], ids=lambda w: w.name)
+def test_baseline_shapes(w):
+    idx, _, _ = wl.make_routing(w)
+    r = rr.build_routing(idx, w.E_tot, w.tile_m)
+    shape = B.make_shape(w.T, w.H, w.I, w.E_tot, w.k_tot, w.TP, w.EP, w.L)
+    occ = B.moe_occupancy(w.tile_m, w.tile_n, 128, 1024, 1, 1)
+    lim = B.moe_sm_limits(148, 74, 0, 0, 3)
+    for mode in (B.MOE_RHO_PAPER, B.MOE_RHO_LOCAL):
+        rho = B.moe_rho(2.5, 704, 128, 256, 2, 17, 1024, mode)
+        plan = B.plan_partition(r["tiles"].tolist(), occ, lim, shape, rho)
+        _same(plan, _oracle_plan(r["tiles"].tolist(), shape, occ, lim, rho))
+        assert 1 <= plan.comm_ctas <= 74 and plan.P == 148 - plan.R and plan.R == plan.comm_ctas
+        assert plan.W_comp == w.TP * r["S"] * -(-(-(-w.H // w.L)) // w.tile_n)
+
+
+def test_golden_examples_through_the_library(golden_dir):
+    # Ex.C and Ex.D of the hand-worked examples, expressed as library inputs
+    # Ex.C: W_comp = 8192 = TP 2 x S 1024 x 4 n-tiles ; W_comm = 64 (one rank of 8192 tokens)
+    shape = B.make_shape(8192, 2048, 1408, 64, 8, 2, 1, 2)
+    occ = B.moe_occupancy(128, 256, 128, 1024, 1, 1)
+    lim = B.moe_sm_limits(148, 74, 0, 0, 3)
+    rho = B.moe_rho(3.0, 704, 128, 256, 1, 17, 1024, B.MOE_RHO_PAPER)
+    plan = B.plan_partition([16] * 64, occ, lim, shape, rho)
+    assert (plan.W_comp, plan.W_comm) == (8192, 64)
+    assert (plan.comm_ctas, plan.R, plan.P, plan.delta) == (13, 13, 135, 43)
+    assert plan.pred_T_q == 137 << 20 and plan.rho_q == 3145728
+    # Ex.D: o_comm = 2, W_comp = 1000 = 1 x 1000 x 1, W_comm = 37, L = 4, rho = 2.5
+    shape = B.make_shape(37 * 128, 1024, 704, 10, 8, 1, 1, 4)
+    occ = B.moe_occupancy(128, 256, 128, 1024, 1, 2)
+    lim = B.moe_sm_limits(148, 32, 0, 0, 3)
+    rho = B.moe_rho(2.5, 704, 128, 256, 1, 17, 1024, B.MOE_RHO_PAPER)
+    plan = B.plan_partition([100] * 10, occ, lim, shape, rho)
+    assert (plan.W_comp, plan.W_comm) == (1000, 37)
+    assert (plan.comm_ctas, plan.R, plan.P, plan.delta) == (19, 10, 138, 104)
+    assert plan.pred_T_q == 34 << 20
+
+
+def test_solver_cost_is_small():
+    # not a benchmark: only guards against an accidental blow-up (ctypes overhead dominates here)
+    w = wl.DSV2L
+    shape = B.make_shape(w.T, w.H, w.I, w.E_tot, w.k_tot, w.TP, w.EP, w.L)
+    occ = B.moe_occupancy(128, 256, 128, 1024, 1, 1)
+    lim = B.moe_sm_limits(148, 74, 0, 0, 3)
+    rho = B.moe_rho(2.5, 704, 128, 256, 2, 17, 1024, B.MOE_RHO_LOCAL)
+    tiles = [17] * 66
+    t = time.perf_counter()
+    for _ in range(2000):
+        B.plan_partition(tiles, occ, lim, shape, rho)
+    assert (time.perf_counter() - t) / 2000 < 1e-3
