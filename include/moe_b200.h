@@ -113,7 +113,7 @@ typedef struct {
 typedef struct {
     int32_t *counts;          /* [E_tot]     M_e */
     int32_t *offsets;         /* [E_tot + 1] exclusive prefix of counts */
-    int32_t *tiles;           /* [E_tot]     ceil(M_e / T_M) */
+    int32_t *tiles;           /* [E_tot + 1] ceil(M_e / T_M), then S */
     int32_t *tile_offsets;    /* [E_tot + 1] exclusive prefix of tiles; last = S */
     int32_t *perm;            /* [R] flat assignment held by routed row r */
     int32_t *inv_perm;        /* [R] routed row of flat assignment f = t * k_tot + j */
@@ -138,7 +138,8 @@ int32_t moe_destroy(moe_handle *h);
 /* Text of the last failing CUDA call on this handle ("" if none); owned by the handle. */
 const char *moe_last_cuda_error(const moe_handle *h);
 /* Upper bound, in nanoseconds, of every device-side wait (default 2e9).  After it a CTA
- * records MOE_DEV_TIMEOUT and leaves; the context stays usable. */
+ * records MOE_DEV_TIMEOUT and leaves; the context stays usable.  The limit is counted from
+ * the start of each CTA, so it bounds the whole launch as well. */
 int32_t moe_set_wait_limit_ns(moe_handle *h, uint64_t ns);
 
 /* Tile shape and residency of the GEMM2 kernel for (tile_m, tile_n), the communication tile,
@@ -175,6 +176,14 @@ int32_t moe_build_routing(moe_handle *h, const int32_t *topk_idx, const moe_shap
 int32_t plan_partition(const int32_t *routed_tile_counts, int32_t n_experts,
                        const moe_occupancy *occ, const moe_sm_limits *limits,
                        const moe_shape *shape, const moe_rho *rho, moe_plan *out);
+
+/* Mean cost [ns] of one plan_partition() call over `iters` calls rotating through n_sets
+ * routed-count vectors (n_sets x n_experts ints, back to back).  The paper reports the
+ * selector's standalone overhead (Section IV-B); this measures ours the same way.  [host] */
+int32_t moe_time_plan_partition(const int32_t *routed_tile_counts, int32_t n_sets, int32_t n_experts,
+                                const moe_occupancy *occ, const moe_sm_limits *limits,
+                                const moe_shape *shape, const moe_rho *rho, int64_t iters,
+                                double *mean_ns, int64_t *checksum);
 
 /* ---- a3-a5: fused grouped GEMM2 + GatherRS combine --------------------------------------
  * Section II-A step 3, Section II-B (compute CTAs publish, communication CTAs consume),

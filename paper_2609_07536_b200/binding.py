@@ -26,7 +26,7 @@ MOE_MAX_EP, MOE_MAX_L = 8, 8
 EXPORTS = [
     "moe_create", "moe_destroy", "moe_last_cuda_error", "moe_set_wait_limit_ns",
     "moe_query_occupancy", "moe_workspace_bytes", "moe_routing_view", "moe_build_routing",
-    "plan_partition", "moe_gemm2_combine", "moe_get_status", "moe_clear_status",
+    "plan_partition", "moe_time_plan_partition", "moe_gemm2_combine", "moe_get_status", "moe_clear_status",
     "moe_host_arena_bytes", "moe_layer_host",
 ]
 
@@ -94,6 +94,9 @@ def lib():
         L.moe_build_routing.argtypes = [vp, vp, P(moe_shape), i32, P(moe_routing), vp, vp, vp]
         L.plan_partition.argtypes = [P(i32), i32, P(moe_occupancy), P(moe_sm_limits), P(moe_shape),
                                      P(moe_rho), P(moe_plan)]
+        L.moe_time_plan_partition.argtypes = [P(i32), i32, i32, P(moe_occupancy), P(moe_sm_limits),
+                                              P(moe_shape), P(moe_rho), C.c_int64, P(C.c_double),
+                                              P(C.c_int64)]
         L.moe_gemm2_combine.argtypes = [vp, vp, vp, vp, vp, P(moe_shape), P(moe_occupancy), P(moe_routing),
                                         i32, P(moe_plan), P(vp), vp, vp, vp, vp]
         L.moe_get_status.argtypes = [vp, vp, P(moe_status), vp]
@@ -184,6 +187,18 @@ def plan_partition(routed_tile_counts, occ, limits, shape, rho) -> moe_plan:
     _check(lib().plan_partition(arr, n, C.byref(occ), C.byref(limits), C.byref(shape), C.byref(rho),
                                 C.byref(plan)), "plan_partition")
     return plan
+
+
+def moe_time_plan_partition(count_sets, occ, limits, shape, rho, iters: int) -> float:
+    """count_sets: list of equally long routed-count vectors.  Returns mean ns per call."""
+    n_sets, n = len(count_sets), len(count_sets[0])
+    flat = [int(v) for s in count_sets for v in s]
+    arr = (C.c_int32 * len(flat))(*flat)
+    mean, chk = C.c_double(), C.c_int64()
+    _check(lib().moe_time_plan_partition(arr, n_sets, n, C.byref(occ), C.byref(limits), C.byref(shape),
+                                         C.byref(rho), iters, C.byref(mean), C.byref(chk)),
+           "moe_time_plan_partition")
+    return mean.value
 
 
 def moe_gemm2_combine(h, x_routed, W2, topk_idx, topk_w, shape, occ, routing, n_mtiles, plan, out,

@@ -10,6 +10,7 @@
 // (tie breaker).  rho is carried in fixed point (2^-20) so that "the same T(C)" is an exact
 // integer comparison.  No CUDA call, no allocation, no global state.
 
+#include <chrono>
 #include <cstdint>
 
 #include "../../include/moe_b200.h"
@@ -156,4 +157,32 @@ extern "C" int32_t plan_partition(const int32_t *routed_tile_counts, int32_t n_e
     out->mode = MOE_MODE_FUSED;
     out->debug_withhold_tile = -1;
     return MOE_OK;
+}
+
+// Mean cost of one plan_partition() call in nanoseconds (steady_clock), over `iters` calls that
+// rotate through `n_sets` routed-count vectors laid out back to back.  Measurement aid for the
+// solver-overhead figure of Section IV-B; returns the sum of the chosen C values through
+// `checksum` so that the calls cannot be optimised away.
+extern "C" int32_t moe_time_plan_partition(const int32_t *routed_tile_counts, int32_t n_sets,
+                                           int32_t n_experts, const moe_occupancy *occ,
+                                           const moe_sm_limits *limits, const moe_shape *shape,
+                                           const moe_rho *rho, int64_t iters, double *mean_ns,
+                                           int64_t *checksum)
+{
+    if (!routed_tile_counts || !mean_ns || n_sets < 1 || iters < 1) return MOE_ERR_NULL;
+    moe_plan plan;
+    int64_t sum = 0;
+    int32_t rc = MOE_OK;
+    const auto t0 = std::chrono::steady_clock::now();
+    int32_t set = 0;
+    for (int64_t i = 0; i < iters; ++i) {
+        rc = plan_partition(routed_tile_counts + (size_t)set * n_experts, n_experts, occ, limits, shape, rho, &plan);
+        if (rc != MOE_OK) break;
+        sum += plan.comm_ctas;
+        if (++set == n_sets) set = 0;
+    }
+    const auto t1 = std::chrono::steady_clock::now();
+    *mean_ns = std::chrono::duration<double, std::nano>(t1 - t0).count() / (double)iters;
+    if (checksum) *checksum = sum;
+    return rc;
 }

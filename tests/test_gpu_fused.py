@@ -1,0 +1,267 @@
+"""Fused GEMM2 + combine (CUDA, through the C ABI) against the CPU oracle.
+
+Tolerance (bf16 inputs, fp32 accumulation, bf16 intermediate and output):
+    max |err| <= 1e-2 * rms(ref) + 1e-3
+Integer work (routing) is compared bit-exactly in test_gpu_routing.py.  Where several results
+are correct (summation order) the tolerance applies; what must be unique is checked as such:
+the GPU result is bitwise identical for every C, every P and from run to run.
+"""
+
+from dataclasses import replace
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import gemm2_combine_ref as ref
+from oracle import routing_ref as rr
+from paper_2609_07536_b200 import binding as B
+from paper_2609_07536_b200 import workloads as wl
+from tests import gpu_common as G
+
+pytestmark = pytest.mark.gpu
+
+
+def _oracle_tokens(w, idx, wt, x, W2, tokens=None):
+    r = rr.build_routing(idx, w.E_tot, w.tile_m)
+    return ref.gemm2_combine(wl.bf16_bits(x), wl.bf16_bits(W2), idx, wt, r["inv_perm"], tokens=tokens), r
+
+
+def _gather_tokens(outs, T, EP, tokens):
+    blk = -(-T // EP)
+    return np.stack([outs[t // blk][t % blk] for t in tokens])
+
+
+def _stratified_tokens(w, idx, r, n_random, seed=0):
+    """first/last tokens of each rank block, tokens sitting in partial m-tiles, tokens of the
+    hottest and the coldest expert, and a random rest."""
+    rng = np.random.default_rng(seed)
+    T, k_tot = idx.shape
+    blk = -(-T // w.EP)
+    toks = set()
+    for d in range(w.EP):
+        lo, hi = min(T, d * blk), min(T, (d + 1) * blk)
+        toks.update(range(lo, min(hi, lo + 3)))
+        toks.update(range(max(lo, hi - 3), hi))
+    partial = np.nonzero(r["mtile_valid"] < w.tile_m)[0][:8]
+    for mu in partial:
+        row = r["mtile_first_row"][mu] + r["mtile_valid"][mu] - 1
+        toks.add(int(r["perm"][row]) // k_tot)
+    counts = r["counts"].copy()
+    hot = int(np.argmax(counts))
+    cold = int(np.argmin(np.where(counts > 0, counts, counts.max() + 1)))
+    for e in (hot, cold):
+        rows = range(r["offsets"][e], min(r["offsets"][e + 1], r["offsets"][e] + 4))
+        toks.update(int(r["perm"][row]) // k_tot for row in rows)
+    toks.update(int(t) for t in rng.choice(T, size=min(T, n_random), replace=False))
+    return np.array(sorted(toks), dtype=np.int32)
+
+
+def _check_against_oracle(w, n_random=None, **run_kw):
+    idx, wt, _ = wl.make_routing(w)
+    x, W2 = wl.make_data(w)
+    outs, plan, ws, S, st = G.run_layer(w, idx, wt, x, W2, **run_kw)
+    assert st.code == 0
+    if n_random is None:
+        expect, r = _oracle_tokens(w, idx, wt, x, W2)
+        tokens = np.arange(w.T)
+    else:
+        r = rr.build_routing(idx, w.E_tot, w.tile_m)
+        tokens = _stratified_tokens(w, idx, r, n_random)
+        expect, _ = _oracle_tokens(w, idx, wt, x, W2, tokens=tokens)
+    got = _gather_tokens(outs, w.T, w.EP, tokens) if len(tokens) else np.zeros((0, w.H), np.float32)
+    assert not np.isnan(got).any()
+    tol = G.tolerance(expect)
+    err = float(np.max(np.abs(got - expect))) if got.size else 0.0
+    assert err <= tol, (w.name, err, tol)
+    # nothing but the owned rows is written: untouched tail rows of a short last block stay NaN
+    return outs, plan
+
+
+def test_tiny_config_all_tokens():
+    outs, plan = _check_against_oracle(wl.TINY)
+    assert plan.comm_ctas >= 1 and plan.P >= 1
+
+
+def test_granite_config_all_tokens():
+    _check_against_oracle(wl.GRANITE)
+
+
+def test_qwen_config_sampled():
+    _check_against_oracle(wl.QWEN, n_random=384)
+
+
+def test_dsv2lite_config_sampled_in_bench_configuration():
+    # the launch configuration bench.py times: analytical plan, 128x256 tiles, L = 2
+    _check_against_oracle(wl.DSV2L, n_random=160)
+
+
+@pytest.mark.parametrize("kw", [
+    dict(T=1, E=4, k=2, H=64, I=64, tile_m=64, tile_n=64),                 # a single token
+    dict(T=333, E=12, k=3, H=264, I=80, tile_m=64, tile_n=64, EP=4),       # ragged everything; K = 80
+    dict(T=777, E=5, k=2, H=1536, I=512, TP=2, EP=3, tile_m=128, tile_n=256, L=4),  # split 384: partial n-tile
+    dict(T=513, E=3, k=1, H=2048, I=352 * 4, TP=4, EP=2, tile_m=128, tile_n=128, L=2),  # K = 352: partial k-block
+    dict(T=1030, E=70, k=2, H=512, I=256, TP=2, EP=8, tile_m=128, tile_n=128, L=8),  # empty experts, L = 8
+    dict(T=200, E=6, k=2, n_shared=2, H=256, I=128, TP=1, EP=1, tile_m=128, tile_n=64, L=2),  # shared experts
+], ids=lambda kw: "-".join(f"{k}{v}" for k, v in kw.items()))
+def test_edge_shapes(kw):
+    base = dict(name="edge", routing_seed=3, data_seed=4, TP=1, EP=1, L=1)
+    base.update(kw)
+    w = replace(wl.TINY, **base)
+    _check_against_oracle(w)
+
+
+def test_one_hot_expert_and_forced_counts():
+    w = replace(wl.TINY, name="hot", T=900, E=8, k=1, H=512, I=256, TP=2, EP=2, tile_m=128, tile_n=256)
+    idx = np.full((w.T, 1), 5, dtype=np.int32)
+    wt = np.ones((w.T, 1), dtype=np.float32)
+    x, W2 = wl.make_data(w)
+    expect, _ = _oracle_tokens(w, idx, wt, x, W2)
+    for C in (1, 3, 40, 147):
+        outs, plan, ws, S, st = G.run_layer(w, idx, wt, x, W2, force_C=C)
+        assert plan.comm_ctas == C and plan.P == 148 - C and st.code == 0
+        got = np.concatenate([o[:len(G.tokens_of_rank(w.T, w.EP, d))] for d, o in enumerate(outs)])
+        assert np.max(np.abs(got - expect)) <= G.tolerance(expect)
+
+
+def test_bitwise_identical_across_C_P_and_runs():
+    w = replace(wl.GRANITE, name="det", T=1536)
+    idx, wt, _ = wl.make_routing(w)
+    x, W2 = wl.make_data(w)
+    base = None
+    for C, P in [(0, None), (1, None), (2, None), (7, None), (33, None), (74, None), (147, None), (5, 9), (5, 1)]:
+        for rep in range(2):
+            outs, plan, ws, S, st = G.run_layer(w, idx, wt, x, W2, force_C=C, P_override=P)
+            assert st.code == 0
+            bits = [torch.from_numpy(o).bfloat16().view(torch.int16).numpy() for o in outs]
+            if base is None:
+                base = bits
+            for a, b in zip(base, bits):
+                assert np.array_equal(a, b), (C, P, rep)
+
+
+def test_ep_concat_invariance_and_tp_within_tolerance():
+    w = replace(wl.QWEN, name="ep", T=1200, E=16)
+    idx, wt, _ = wl.make_routing(w)
+    x, W2 = wl.make_data(w)
+    cat = {}
+    for EP in (1, 2, 4):
+        we = replace(w, EP=EP)
+        outs, *_ = G.run_layer(we, idx, wt, x, W2)
+        cat[EP] = np.concatenate([o[:len(G.tokens_of_rank(w.T, EP, d))] for d, o in enumerate(outs)])
+    assert np.array_equal(cat[1], cat[2]) and np.array_equal(cat[1], cat[4])
+    expect, _ = _oracle_tokens(w, idx, wt, x, W2)
+    for TP in (1, 2, 4):
+        wt_ = replace(w, TP=TP)   # K = 1408, 704, 352
+        outs, *_ = G.run_layer(wt_, idx, wt, x, W2)
+        got = np.concatenate([o[:len(G.tokens_of_rank(w.T, w.EP, d))] for d, o in enumerate(outs)])
+        assert np.max(np.abs(got - expect)) <= G.tolerance(expect), TP
+
+
+def test_identity_weights_make_the_combine_exact():
+    # W2_e = identity (I = H), small integer activations, power-of-two weights: every partial
+    # sum is exactly representable in bf16, so the GPU output must equal the gather exactly
+    w = replace(wl.TINY, name="ident", T=300, E=6, k=2, H=128, I=128, TP=1, EP=2, tile_m=64, tile_n=64)
+    rng = np.random.default_rng(1)
+    idx = np.stack([rng.permutation(w.E)[:2] for _ in range(w.T)]).astype(np.int32)
+    wt = np.tile(np.array([0.5, 0.25], dtype=np.float32), (w.T, 1))
+    xv = rng.integers(-8, 9, (w.R, w.I)).astype(np.float32)
+    x = torch.from_numpy(xv).bfloat16()
+    W2 = torch.eye(w.H).repeat(w.E, 1, 1).bfloat16()
+    outs, plan, ws, S, st = G.run_layer(w, idx, wt, x, W2)
+    r = rr.build_routing(idx, w.E_tot, w.tile_m)
+    inv = r["inv_perm"].reshape(w.T, 2)
+    expect = 0.5 * xv[inv[:, 0]] + 0.25 * xv[inv[:, 1]]
+    got = np.concatenate([o[:len(G.tokens_of_rank(w.T, w.EP, d))] for d, o in enumerate(outs)])
+    assert np.array_equal(got, expect)
+
+
+def test_gemm_only_then_combine_only_equals_fused():
+    w = replace(wl.GRANITE, name="modes", T=1024)
+    idx, wt, _ = wl.make_routing(w)
+    x, W2 = wl.make_data(w)
+    fused, plan, ws, S, st = G.run_layer(w, idx, wt, x, W2)
+    fused = [o.copy() for o in fused]
+    G.run_layer(w, idx, wt, x, W2, mode=B.MOE_MODE_GEMM_ONLY, ws=ws)
+    two, *_ = G.run_layer(w, idx, wt, x, W2, mode=B.MOE_MODE_COMBINE_ONLY, ws=ws)
+    for a, b in zip(fused, two):
+        assert np.array_equal(a, b, equal_nan=True)
+
+
+def test_bounded_wait_reports_a_timeout_and_the_context_survives():
+    h = G.handle()
+    w = replace(wl.TINY, name="withhold", T=512, E=4, k=2, H=256, I=128, TP=1, EP=1, tile_m=128, tile_n=128)
+    idx, wt, _ = wl.make_routing(w)
+    x, W2 = wl.make_data(w)
+    B.moe_set_wait_limit_ns(h, 20_000_000)            # 20 ms
+    try:
+        # tile 0 = (split 0, m-tile 0, shard 0, n-tile 0) is computed but its readiness is never raised
+        outs, plan, ws, S, st = G.run_layer(w, idx, wt, x, W2, force_C=2, withhold=0, check_status=False)
+        assert st.code == B.MOE_DEV_TIMEOUT and st.detail == 0 and st.where == 40
+        # tokens that do not depend on the withheld tile are still correct
+        r = rr.build_routing(idx, w.E_tot, w.tile_m)
+        dep = set(int(r["perm"][row]) // w.k_tot for row in range(r["mtile_first_row"][0], r["mtile_first_row"][0] + r["mtile_valid"][0]))
+        free = np.array([t for t in range(w.T) if t not in dep], dtype=np.int32)
+        expect, _ = _oracle_tokens(w, idx, wt, x, W2, tokens=free)
+        got = outs[0][free]
+        done = ~np.isnan(got).any(axis=1)            # a warp that gave up leaves its later rows unwritten
+        assert done.sum() > 0
+        assert np.max(np.abs(got[done] - expect[done])) <= G.tolerance(expect)
+    finally:
+        B.moe_set_wait_limit_ns(h, 2_000_000_000)
+    # the same workspace and context keep working
+    outs, plan, ws, S, st = G.run_layer(w, idx, wt, x, W2, ws=ws)
+    assert st.code == 0
+    expect, _ = _oracle_tokens(w, idx, wt, x, W2)
+    assert np.max(np.abs(outs[0][:w.T] - expect)) <= G.tolerance(expect)
+
+
+def test_argument_validation():
+    h = G.handle()
+    w = wl.TINY
+    idx, wt, _ = wl.make_routing(w)
+    x, W2 = wl.make_data(w)
+    outs, plan, ws, S, st = G.run_layer(w, idx, wt, x, W2)
+    shape = G.shape_of(w)
+    occ, lim, rho = B.moe_query_occupancy(h, w.tile_m, w.tile_n)
+    xd, Wd, wd = x.cuda(), W2.cuda(), torch.from_numpy(wt).cuda()
+    args = lambda p, xx=xd: (h, xx, Wd, None, wd, shape, occ, ws.routing, S, p, ws.out, ws.y_ws, ws.flags_ws, ws.status)
+    bad = B.moe_plan.from_buffer_copy(plan); bad.comm_ctas = 0
+    with pytest.raises(B.MoeError) as e:
+        B.moe_gemm2_combine(*args(bad))
+    assert e.value.code == B.MOE_ERR_PLAN_INFEASIBLE
+    bad = B.moe_plan.from_buffer_copy(plan); bad.P = 148          # C + P > G
+    with pytest.raises(B.MoeError) as e:
+        B.moe_gemm2_combine(*args(bad))
+    assert e.value.code == B.MOE_ERR_PLAN_INFEASIBLE
+    bad = B.moe_plan.from_buffer_copy(plan); bad.R = 0            # reservation too small for C
+    with pytest.raises(B.MoeError) as e:
+        B.moe_gemm2_combine(*args(bad))
+    assert e.value.code == B.MOE_ERR_PLAN_INFEASIBLE
+    with pytest.raises(B.MoeError) as e:
+        B.moe_gemm2_combine(*args(plan, xd.data_ptr() + 2))   # misaligned
+    assert e.value.code == B.MOE_ERR_ALIGN
+    with pytest.raises(B.MoeError) as e:
+        B.moe_gemm2_combine(h, None, Wd, None, wd, shape, occ, ws.routing, S, plan, ws.out, ws.y_ws, ws.flags_ws, ws.status)
+    assert e.value.code == B.MOE_ERR_NULL
+
+
+def test_host_buffer_entry_point_matches_device_path():
+    h = G.handle()
+    w = replace(wl.GRANITE, name="host", T=1000)
+    idx, wt, _ = wl.make_routing(w)
+    x, W2 = wl.make_data(w)
+    dev, plan, ws, S, st = G.run_layer(w, idx, wt, x, W2)
+    shape = G.shape_of(w)
+    nbytes = B.moe_host_arena_bytes(shape, w.tile_m, w.tile_n)
+    arena = torch.empty(nbytes + 256, dtype=torch.uint8, device="cuda")
+    off = (-arena.data_ptr()) % 256
+    xh = x.pin_memory(); ih = torch.from_numpy(idx).pin_memory(); wh = torch.from_numpy(wt).pin_memory()
+    counts = torch.zeros(w.E_tot + 1, dtype=torch.int32).pin_memory()
+    out_h = torch.empty((w.T, w.H), dtype=torch.bfloat16).pin_memory()
+    p2 = B.moe_layer_host(h, xh, ih, wh, W2.cuda(), shape, w.tile_m, w.tile_n, None,
+                          arena.data_ptr() + off, nbytes, counts, out_h)
+    assert (p2.comm_ctas, p2.P) == (plan.comm_ctas, plan.P)
+    got = out_h.float().numpy()
+    cat = np.concatenate([o[:len(G.tokens_of_rank(w.T, w.EP, d))] for d, o in enumerate(dev)])
+    assert np.array_equal(got, cat)
