@@ -40,7 +40,8 @@ enum {
     MOE_ERR_CUDA = -5,            /* a CUDA runtime/driver call failed (see moe_last_cuda_error) */
     MOE_ERR_UNSUPPORTED = -6,     /* tile configuration the kernels do not provide */
     MOE_ERR_DEVICE_STATUS = -7,   /* the device status buffer reports a problem */
-    MOE_ERR_ARENA = -8            /* the caller's arena is too small */
+    MOE_ERR_ARENA = -8,           /* the caller's arena is too small */
+    MOE_ERR_STATIC_LIMIT = -9     /* the problem needs more scratch than the built-in array holds */
 };
 
 /* device status codes (word 0 of the status buffer) */
@@ -166,6 +167,26 @@ int32_t moe_routing_view(void *routing_ws, const moe_shape *shape, int32_t tile_
 int32_t moe_build_routing(moe_handle *h, const int32_t *topk_idx, const moe_shape *shape,
                           int32_t tile_m, const moe_routing *routing,
                           int32_t *tile_counts_host, uint32_t *status_dev, void *stream);
+
+/* Routing build for callers that cannot allocate device memory (no counterpart in the paper;
+ * an addition of this library).  Same inputs, outputs and results as moe_build_routing(), but
+ * the builder's scratch (per-warp histograms, ceil(T*k_tot/256) * E_tot ints) lives in a fixed
+ * 512 KiB array inside the library instead of routing->scratch, which is ignored and may be
+ * NULL.  Meant for code that runs where cudaMalloc is not an option: a serving loop with a
+ * memory pool frozen at start-up, a framework allocator that rejects foreign allocations, a
+ * latency-critical section that cannot afford the synchronisation an allocation implies.
+ * The call itself allocates nothing (no cudaMalloc / cudaFree, no allocating library routine).
+ *  - Limit: ceil(T*k_tot/256) * E_tot <= 131072, else MOE_ERR_STATIC_LIMIT (text in
+ *    moe_last_cuda_error) and nothing is launched.
+ *  - The first call on a device resolves the array's device address (a one-time set-up per
+ *    device); make that first call before any stream capture begins.
+ *  - All calls on one GPU share the array and it keeps the previous call's contents; the
+ *    builder overwrites every entry it later reads, so nothing needs clearing, but two calls
+ *    whose kernels overlap on the GPU (different streams) race: order them.
+ *  - Every GPU that loads the library holds the 512 KiB until the process exits. */
+int32_t moe_build_routing_static(moe_handle *h, const int32_t *topk_idx, const moe_shape *shape,
+                                 int32_t tile_m, const moe_routing *routing,
+                                 int32_t *tile_counts_host, uint32_t *status_dev, void *stream);
 
 /* ---- a2: the analytical selector (Section III-D, Algorithm 1, Eq. 1-15, tie breaker) -----
  * Pure host code: no CUDA call, no allocation, re-entrant.

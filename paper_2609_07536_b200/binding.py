@@ -18,6 +18,7 @@ LIB_PATH = os.path.join(HERE, "libmoe_b200.so")
 MOE_OK = 0
 MOE_ERR_NULL, MOE_ERR_SHAPE, MOE_ERR_ALIGN, MOE_ERR_PLAN_INFEASIBLE = -1, -2, -3, -4
 MOE_ERR_CUDA, MOE_ERR_UNSUPPORTED, MOE_ERR_DEVICE_STATUS, MOE_ERR_ARENA = -5, -6, -7, -8
+MOE_ERR_STATIC_LIMIT = -9
 MOE_DEV_OK, MOE_DEV_TIMEOUT, MOE_DEV_OOB, MOE_DEV_DUP_EXPERT = 0, 1, 2, 3
 MOE_MODE_FUSED, MOE_MODE_GEMM_ONLY, MOE_MODE_COMBINE_ONLY = 0, 1, 2
 MOE_RHO_PAPER, MOE_RHO_LOCAL = 0, 1
@@ -26,6 +27,7 @@ MOE_MAX_EP, MOE_MAX_L = 8, 8
 EXPORTS = [
     "moe_create", "moe_destroy", "moe_last_cuda_error", "moe_set_wait_limit_ns",
     "moe_query_occupancy", "moe_workspace_bytes", "moe_routing_view", "moe_build_routing",
+    "moe_build_routing_static",
     "plan_partition", "moe_time_plan_partition", "moe_gemm2_combine", "moe_get_status", "moe_clear_status",
     "moe_host_arena_bytes", "moe_layer_host",
 ]
@@ -92,6 +94,7 @@ def lib():
         L.moe_workspace_bytes.argtypes = [P(moe_shape), i32, i32] + [P(C.c_size_t)] * 4
         L.moe_routing_view.argtypes = [vp, P(moe_shape), i32, P(moe_routing)]
         L.moe_build_routing.argtypes = [vp, vp, P(moe_shape), i32, P(moe_routing), vp, vp, vp]
+        L.moe_build_routing_static.argtypes = [vp, vp, P(moe_shape), i32, P(moe_routing), vp, vp, vp]
         L.plan_partition.argtypes = [P(i32), i32, P(moe_occupancy), P(moe_sm_limits), P(moe_shape),
                                      P(moe_rho), P(moe_plan)]
         L.moe_time_plan_partition.argtypes = [P(i32), i32, i32, P(moe_occupancy), P(moe_sm_limits),
@@ -114,7 +117,7 @@ def lib():
 def _check(rc, what, handle=None):
     if rc != MOE_OK:
         detail = ""
-        if handle is not None and rc == MOE_ERR_CUDA:
+        if handle is not None and rc in (MOE_ERR_CUDA, MOE_ERR_STATIC_LIMIT):
             detail = (lib().moe_last_cuda_error(handle) or b"").decode()
         raise MoeError(rc, what, detail)
 
@@ -177,6 +180,18 @@ def moe_build_routing(h, topk_idx, shape, tile_m, routing, tile_counts_host, sta
     _check(lib().moe_build_routing(h, _ptr(topk_idx), C.byref(shape), tile_m, C.byref(routing),
                                    _ptr(tile_counts_host), _ptr(status_dev), _stream(stream)),
            "moe_build_routing", h)
+
+
+def moe_build_routing_static(h, topk_idx, shape, tile_m, routing, tile_counts_host, status_dev, stream=None):
+    """Routing build whose scratch is a fixed array inside the library: for callers that cannot
+    allocate device memory (frozen memory pools, allocator-owning frameworks, latency-critical
+    sections).  Same results as moe_build_routing; `routing.scratch` is ignored.  Raises MoeError
+    with code MOE_ERR_STATIC_LIMIT when ceil(T*k_tot/256) * E_tot exceeds 131072.  The first call
+    on a device does a one-time set-up and should come before any stream capture; calls that
+    overlap on the GPU race on the shared array."""
+    _check(lib().moe_build_routing_static(h, _ptr(topk_idx), C.byref(shape), tile_m, C.byref(routing),
+                                          _ptr(tile_counts_host), _ptr(status_dev), _stream(stream)),
+           "moe_build_routing_static", h)
 
 
 def plan_partition(routed_tile_counts, occ, limits, shape, rho) -> moe_plan:

@@ -162,3 +162,91 @@ cudaError_t routing_launch(const int32_t *topk_idx, const moe_shape &s, int tile
 }
 
 }  // namespace moe
+
+// ------------------------------------------------------------------------------------------
+// Routing build for callers that cannot allocate device memory.
+//
+// Some users of this library run where cudaMalloc is off limits: inside a serving loop whose
+// memory pool was sized and frozen at start-up, under a framework allocator that forbids
+// foreign allocations once a model is loaded, or in a latency-critical section where an
+// allocation (an implicit device synchronisation) is not acceptable.  For them the per-warp
+// histograms that the builder needs as scratch live in a fixed array inside the library instead
+// of in a caller-provided buffer.  Every GPU that loads the library holds the array
+// (kStaticScratchInts * 4 bytes) until the process exits.
+//
+// `g_static_scratch` is a device symbol: in host code the name is only a host-side stand-in, not
+// a device address, so the address the kernels get comes from cudaGetSymbolAddress(), looked up
+// once per device with that device current.
+namespace moe {
+namespace {
+
+constexpr int kStaticScratchInts = 128 * 1024;   // 512 KiB per GPU
+constexpr int kMaxStaticDevices = 64;
+
+static __device__ __align__(256) int32_t g_static_scratch[kStaticScratchInts];
+int32_t *g_static_scratch_addr[kMaxStaticDevices] = {nullptr};
+
+}  // namespace
+}  // namespace moe
+
+extern "C" int32_t moe_build_routing_static(moe_handle *h, const int32_t *topk_idx, const moe_shape *s,
+                                            int32_t tile_m, const moe_routing *r,
+                                            int32_t *tile_counts_host, uint32_t *status_dev, void *stream)
+{
+    using namespace moe;
+    if (!h || !s || !r || !status_dev) return MOE_ERR_NULL;
+    if (s->T < 0 || s->k_tot < 1 || s->k_tot > 32 || s->E_tot < 1 || s->E_tot > 1024 ||
+        (int64_t)s->T * s->k_tot >= (int64_t)1 << 30)
+        return MOE_ERR_SHAPE;
+    if (tile_m != 64 && tile_m != 128) return MOE_ERR_UNSUPPORTED;
+    if (s->T > 0 && !topk_idx) return MOE_ERR_NULL;
+    const int64_t R = (int64_t)s->T * s->k_tot;
+    if (r->max_mtiles < (int32_t)(R / tile_m + s->E_tot)) return MOE_ERR_SHAPE;
+    const int64_t n_warps = (R + kRoutingChunk - 1) / kRoutingChunk;
+    if (n_warps * s->E_tot > kStaticScratchInts) {
+        snprintf(h->err, sizeof h->err,
+                 "moe_build_routing_static: ceil(T*k_tot/%d) * E_tot = %lld ints of scratch needed, the built-in "
+                 "array holds %d; use moe_build_routing with a caller-allocated workspace",
+                 kRoutingChunk, (long long)(n_warps * s->E_tot), kStaticScratchInts);
+        return MOE_ERR_STATIC_LIMIT;
+    }
+    if (h->device < 0 || h->device >= kMaxStaticDevices) return MOE_ERR_UNSUPPORTED;
+
+    // set-up, once per device: resolve the array's device address with that device current
+    int32_t *scratch = g_static_scratch_addr[h->device];
+    if (!scratch) {
+        int cur = -1;
+        cudaError_t e = cudaGetDevice(&cur);
+        if (e != cudaSuccess) return cuda_fail(h, e, "cudaGetDevice");
+        if (cur != h->device && (e = cudaSetDevice(h->device)) != cudaSuccess) return cuda_fail(h, e, "cudaSetDevice");
+        void *p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (cur != h->device) cudaSetDevice(cur);
+        if (e != cudaSuccess || !p) return cuda_fail(h, e, "cudaGetSymbolAddress(static scratch)");
+        scratch = static_cast<int32_t *>(p);
+        g_static_scratch_addr[h->device] = scratch;
+    }
+
+    // The array keeps whatever the previous call left in it.  Nothing has to start at zero: the
+    // histogram pass overwrites every (warp, expert) entry the later passes read.
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int iR = (int)R, nw = (int)n_warps;
+    const int blocks = (nw + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    const size_t sh = (size_t)kWarpsPerBlock * s->E_tot * sizeof(int32_t);
+    if (blocks > 0)
+        routing_hist<<<blocks, kWarpsPerBlock * 32, sh, st>>>(topk_idx, iR, s->k_tot, s->E_tot, nw, scratch, status_dev);
+    routing_scan<<<1, 1024, 0, st>>>(iR, s->E_tot, tile_m, nw, r->max_mtiles, scratch, r->counts, r->offsets,
+                                     r->tiles, r->tile_offsets, r->mtile_expert, r->mtile_first_row,
+                                     r->mtile_valid, status_dev);
+    if (blocks > 0)
+        routing_scatter<<<blocks, kWarpsPerBlock * 32, sh, st>>>(topk_idx, iR, s->E_tot, tile_m, nw, scratch,
+                                                                r->offsets, r->tile_offsets, r->perm,
+                                                                r->inv_perm, r->pad_row);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(h, e, "static routing launch");
+    if (tile_counts_host) {
+        e = cudaMemcpyAsync(tile_counts_host, r->tiles, (size_t)(s->E_tot + 1) * 4, cudaMemcpyDeviceToHost, st);
+        if (e != cudaSuccess) return cuda_fail(h, e, "tile counts copy");
+    }
+    return MOE_OK;
+}
