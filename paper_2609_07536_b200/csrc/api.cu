@@ -152,7 +152,8 @@ int32_t moe_workspace_bytes(const moe_shape *s, int32_t tile_m, int32_t tile_n, 
         b += align16((size_t)n_routing_warps(s) * E * 4); // per-warp histograms
         *routing_bytes = b + 16;
     }
-    if (y_bytes) *y_bytes = align16((size_t)s->TP * mt * tile_m * s->H * 2) + 16;
+    if (y_bytes)   // token-major: [T][L][k_tot * TP][ceil(H/L)]
+        *y_bytes = align16((size_t)s->T * s->L * s->k_tot * s->TP * (size_t)ceil_div(s->H, s->L) * 2) + 16;
     if (flags_bytes) {
         const size_t nts = (size_t)ceil_div(ceil_div(s->H, s->L), tile_n);
         *flags_bytes = ((size_t)kSplitCounterWords + (size_t)s->L * s->TP * mt * nts) * 4 + 16;
@@ -218,6 +219,7 @@ int32_t moe_gemm2_combine(moe_handle *h, const void *x_routed, const void *W2, c
     if (!shape_ok(s)) return MOE_ERR_SHAPE;
     if (!tile_ok(occ->tile_m, occ->tile_n)) return MOE_ERR_UNSUPPORTED;
     if (occ->comm_tile_m != kCommTileM || occ->comm_tile_n != kCommTileN) return MOE_ERR_UNSUPPORTED;
+    if ((ceil_div(s->H, s->L) % 8) != 0) return MOE_ERR_SHAPE;   // 16-byte column chunks per split
     if (s->T == 0) return MOE_OK;
     if (!x_routed || !W2 || !topk_w || !y_ws || !flags_ws) return MOE_ERR_NULL;
     if (n_mtiles < 0 || n_mtiles > r->max_mtiles) return MOE_ERR_SHAPE;
@@ -272,6 +274,14 @@ int32_t moe_gemm2_combine(moe_handle *h, const void *x_routed, const void *W2, c
     p.mtile_first_row = r->mtile_first_row;
     p.mtile_valid = r->mtile_valid;
     p.pad_row = r->pad_row;
+    p.perm = r->perm;
+    p.Q = s->k_tot * s->TP;
+    {   // column slab of one unit: the largest power of two with Q * slab_cols * 2 <= 8 KB, at most 1024
+        int sh = 10;
+        while (sh > 3 && ((int64_t)p.Q << sh) * 2 > 8192) --sh;
+        p.slab_shift = sh;
+        p.slab_cols = 1 << sh;
+    }
     p.topk_w = topk_w;
     p.Y = y_ws;
     p.status = status_dev;

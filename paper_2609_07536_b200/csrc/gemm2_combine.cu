@@ -80,6 +80,14 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map
         ::"r"(dst), "l"((unsigned long long)map), "r"(bar), "r"(x), "r"(y), "r"(z)
         : "memory");
 }
+// untiled bulk copy global -> shared; both addresses 16-byte aligned, size a multiple of 16
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+        : "memory");
+}
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t cols)
 {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(cols) : "memory");
@@ -120,6 +128,18 @@ __device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32])
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+__device__ __forceinline__ uint4 lds_v4(uint32_t addr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ float lds_f32(uint32_t addr)
+{
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+    return v;
+}
 __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p)
 {
     uint32_t v;
@@ -188,25 +208,33 @@ struct Control {
     unsigned long long tmem_empty[2];
     uint32_t tmem_base;
     volatile uint32_t abort;
+    unsigned long long comm_full[24];   // communication CTA: one barrier per warp and stage
+    float comm_w[12][256];              // ... and the per-row weights of the unit a warp reduces (Q <= 256)
 };
 
-// Bounded mbarrier wait.  Returns false on timeout or when another warp of the CTA gave up.
+// Bounded mbarrier wait, warp-collective: lane 0 polls (32 lanes polling the same barrier would
+// each occupy the shared-memory pipe), the result is broadcast.  Returns false on timeout or when
+// another warp of the CTA gave up.
 __device__ __forceinline__ bool wait_barrier(uint32_t bar, uint32_t parity, Control *ctl,
                                              unsigned long long deadline, uint32_t *status,
                                              uint32_t detail, uint32_t where)
 {
-    uint32_t spins = 0;
-    while (!mbar_try_wait(bar, parity)) {
-        if ((++spins & 63u) == 0u) {
-            if (ctl->abort) return false;
-            if (globaltimer_ns() > deadline) {
-                ctl->abort = 1u;
-                report(status, MOE_DEV_TIMEOUT, detail, where);
-                return false;
+    uint32_t ok = 1u;
+    if ((threadIdx.x & 31u) == 0u) {
+        uint32_t spins = 0;
+        while (!mbar_try_wait(bar, parity)) {
+            if ((++spins & 63u) == 0u) {
+                if (ctl->abort) { ok = 0u; break; }
+                if (globaltimer_ns() > deadline) {
+                    ctl->abort = 1u;
+                    report(status, MOE_DEV_TIMEOUT, detail, where);
+                    ok = 0u;
+                    break;
+                }
             }
         }
     }
-    return true;
+    return __shfl_sync(0xffffffffu, ok, 0) != 0u;
 }
 
 struct Tile {
@@ -333,9 +361,9 @@ __device__ void compute_cta(const FusedParams &P, uint8_t *ring, Control *ctl, i
         }
     } else if (warp >= 4 && warp < 4 + C::kEpiWarps) {
         // ---------------- epilogue: TMEM -> bf16 -> Y, then publish the tile
-        const int q = warp & 3;                    // TMEM lane quarter this warp may read
+        const int q4 = warp & 3;                   // TMEM lane quarter this warp may read
         const int half = (warp - 4) >> 2;          // column half of the tile
-        const int row_in_tile = q * 32 + lane;
+        const int row_in_tile = q4 * 32 + lane;
         const bool is_leader = (warp == 4 && lane == 0);
         __nv_bfloat16 *Y = reinterpret_cast<__nv_bfloat16 *>(P.Y);
         int it = 0;
@@ -351,18 +379,32 @@ __device__ void compute_cta(const FusedParams &P, uint8_t *ring, Control *ctl, i
                 const int n0 = t.s * P.split_w + t.i_n * TN;
                 const int col_end = min(P.H, (t.s + 1) * P.split_w);
                 const bool row_ok = row_in_tile < valid;
-                __nv_bfloat16 *yrow = Y + ((size_t)t.p * (size_t)P.R_pad + (size_t)t.mu * P.tile_m + row_in_tile) * (size_t)P.H;
+                // destination of this thread's row: the routed row belongs to flat assignment
+                // f = (token, slot); Y is token-major so that the combine reads one contiguous block
+                __nv_bfloat16 *ybase = Y;
+                int q = 0;
+                if (row_ok) {
+                    const int f = __ldg(&P.perm[__ldg(&P.mtile_first_row[t.mu]) + row_in_tile]);
+                    const int tok = f / P.k_tot;
+                    q = (f - tok * P.k_tot) * P.TP + t.p;
+                    ybase = Y + ((size_t)tok * P.L + t.s) * (size_t)P.Q * (size_t)P.split_w;
+                }
+                const int cis0 = n0 - t.s * P.split_w;   // column inside the split
 #pragma unroll
                 for (int cc = 0; cc < C::kColsPerHalf; cc += 32) {
                     const int col = half * C::kColsPerHalf + cc;
                     uint32_t r[32];
-                    tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * TN + col), r);
+                    tmem_ld_32x32(tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(a * TN + col), r);
                     tmem_ld_wait();
                     if (row_ok) {
 #pragma unroll
                         for (int v = 0; v < 4; ++v) {
                             const int c0 = n0 + col + v * 8;
                             if (c0 < col_end) {
+                                const int cis = cis0 + col + v * 8;
+                                const int slab = cis >> P.slab_shift;
+                                const int cin = cis & (P.slab_cols - 1);
+                                const int wslab = min(P.slab_cols, P.split_w - (slab << P.slab_shift));
                                 uint4 pk;
                                 __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(r[v * 8 + 0]), __uint_as_float(r[v * 8 + 1]));
                                 __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(r[v * 8 + 2]), __uint_as_float(r[v * 8 + 3]));
@@ -372,7 +414,7 @@ __device__ void compute_cta(const FusedParams &P, uint8_t *ring, Control *ctl, i
                                 pk.y = *reinterpret_cast<uint32_t *>(&h1);
                                 pk.z = *reinterpret_cast<uint32_t *>(&h2);
                                 pk.w = *reinterpret_cast<uint32_t *>(&h3);
-                                *reinterpret_cast<uint4 *>(yrow + c0) = pk;
+                                *reinterpret_cast<uint4 *>(ybase + ((size_t)slab * P.Q << P.slab_shift) + (size_t)q * wslab + cin) = pk;
                             }
                         }
                     }
@@ -413,16 +455,102 @@ __device__ __forceinline__ void fma_bf16x8(float (&acc)[8], const uint4 &v, floa
     }
 }
 
+// Communication CTA.  Y is token-major: the k_tot * TP partial rows of one (token, split, column
+// slab) are one contiguous block (a "unit", at most 8 KB).  Twelve warps work independently; warp w
+// serves units w, w+12, ... of its CTA.  Each warp owns two 8 KB stages of shared memory and one
+// mbarrier per stage: it fetches a unit with ONE bulk asynchronous copy (global -> shared), and
+// while that copy is in flight it reduces the previous unit in fp32 in (j, p) order with the token's
+// weights and stores the bf16 result into the owning rank's buffer.  No warp waits on another one:
+// the issue latency of the copies and the memory latency overlap across the twelve warps.
+constexpr int kCommWarps = 12;
+constexpr int kCommUnitBytes = 8192;
+constexpr int kCommWarpBytes = 2 * kCommUnitBytes;
+static_assert(kCommWarps * kCommWarpBytes <= kStageBytesTotal, "communication stages exceed the ring");
+
+struct CommUnit {
+    int t, d, s, slab, wslab, ucols;
+    float w;          // lane j: weight of slot j (0 when the slot has no source row)
+    bool live;
+};
+
 template <int TN>
-__device__ void comm_cta(const FusedParams &P, int c)
+__device__ void comm_cta(const FusedParams &P, uint8_t *ring, Control *ctl, int c)
 {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    constexpr int n_warps = kThreads / 32;
-    constexpr int kGroupCols = 256;               // 32 lanes x 8 bf16
-    const int Q = P.k_tot * P.TP;
-    const unsigned long long deadline = globaltimer_ns() + P.wait_ns;
-    const __nv_bfloat16 *Y = reinterpret_cast<const __nv_bfloat16 *>(P.Y);
     const bool wait_needed = (P.mode != MOE_MODE_COMBINE_ONLY);
+    const unsigned long long deadline = globaltimer_ns() + P.wait_ns;
+    // the wait for a copy only follows a readiness wait: it gets a later deadline so that the first
+    // report names the wait that really ran out
+    const unsigned long long deadline2 = deadline + P.wait_ns / 4 + 1000000ull;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < 2 * kCommWarps; ++i) mbar_init(smem_u32(&ctl->comm_full[i]), 1);
+        ctl->abort = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+    if (warp >= kCommWarps) return;
+    uint8_t *my_ring = ring + warp * kCommWarpBytes;
+    float *wq = ctl->comm_w[warp];
+    const __nv_bfloat16 *Y = reinterpret_cast<const __nv_bfloat16 *>(P.Y);
+
+    // reduce the unit sitting in stage `st` (its copy was issued one unit ago)
+    auto consume = [&](const CommUnit &u, int st, uint32_t parity) -> bool {
+        bool ok = wait_barrier(smem_u32(&ctl->comm_full[2 * warp + st]), parity, ctl, deadline2, P.status,
+                               (uint32_t)u.t, 43u);
+        if (!ok) return false;
+        const int n16 = u.ucols >> 3;
+        const uint32_t row_bytes = (uint32_t)u.wslab * 2u;
+        // per-row weights, read back as shared-memory broadcasts inside the unrolled loop
+        if (lane < P.k_tot)
+            for (int p = 0; p < P.TP; ++p) wq[lane * P.TP + p] = u.w;
+        __syncwarp();
+        const uint32_t wq_s = smem_u32(wq);
+        const uint32_t stage_s = smem_u32(my_ring + st * kCommUnitBytes);
+        __nv_bfloat16 *orow = reinterpret_cast<__nv_bfloat16 *>(P.out[u.d]) +
+                              (size_t)(u.t - u.d * P.tok_blk) * (size_t)P.H + u.s * P.split_w + (u.slab << P.slab_shift);
+        for (int c16 = lane; c16 < ((n16 + 31) & ~31); c16 += 32) {
+            float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            const uint32_t src = stage_s + (uint32_t)(c16 < n16 ? c16 : 0) * 16u;
+            for (int r0 = 0; r0 < P.Q; r0 += 8) {
+                uint4 v[8];
+                float w[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int r = min(r0 + i, P.Q - 1);
+                    v[i] = lds_v4(src + (uint32_t)r * row_bytes);
+                    w[i] = lds_f32(wq_s + (uint32_t)r * 4u);
+                    if (r0 + i >= P.Q) w[i] = 0.f;
+                }
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    // a slot without a source row holds bytes nobody wrote: drop them
+                    if (w[i] == 0.f) v[i] = make_uint4(0u, 0u, 0u, 0u);
+                    fma_bf16x8(acc, v[i], w[i]);
+                }
+            }
+            if (c16 < n16) {
+                uint4 pk;
+                __nv_bfloat162 h0 = __floats2bfloat162_rn(acc[0], acc[1]);
+                __nv_bfloat162 h1 = __floats2bfloat162_rn(acc[2], acc[3]);
+                __nv_bfloat162 h2 = __floats2bfloat162_rn(acc[4], acc[5]);
+                __nv_bfloat162 h3 = __floats2bfloat162_rn(acc[6], acc[7]);
+                pk.x = *reinterpret_cast<uint32_t *>(&h0);
+                pk.y = *reinterpret_cast<uint32_t *>(&h1);
+                pk.z = *reinterpret_cast<uint32_t *>(&h2);
+                pk.w = *reinterpret_cast<uint32_t *>(&h3);
+                __stcs(reinterpret_cast<uint4 *>(orow + c16 * 8), pk);
+            }
+        }
+        __syncwarp();   // all lanes are done with the stage (and with wq) before either is reused
+        return true;
+    };
+
+    int unit = 0;            // running unit number of this CTA
+    int n_mine = 0;          // units this warp has issued so far: stage n_mine & 1, parity (n_mine >> 1) & 1
+    CommUnit prev;
+    prev.live = false;
 
     for (int s = 0; s < P.L; ++s) {
         bool split_ready = !wait_needed;
@@ -438,26 +566,43 @@ __device__ void comm_cta(const FusedParams &P, int c)
             const int c0 = split_c0 + col_tile * kCommTileN;
             const int c1 = min(split_c1, c0 + kCommTileN);
             if (t0 >= t1 || c0 >= c1) continue;
-            const int groups = (c1 - c0 + kGroupCols - 1) / kGroupCols;
-            const int units = (t1 - t0) * groups;
-            __nv_bfloat16 *out_d = reinterpret_cast<__nv_bfloat16 *>(P.out[d]);
-            for (int u = warp; u < units; u += n_warps) {
-                const int tt = u / groups;
-                const int grp = u - tt * groups;
-                const int t = t0 + tt;
-                const int gcol0 = c0 + grp * kGroupCols;
-                const int col = gcol0 + lane * 8;
-                // routing of this token: lane j holds slot j
-                int my_row = -1;
-                float my_w = 0.f;
+            const int slab0 = (c0 - split_c0) >> P.slab_shift;
+            const int n_slabs = ((c1 - split_c0 + P.slab_cols - 1) >> P.slab_shift) - slab0;
+            const int n_units = (t1 - t0) * n_slabs;
+            // first unit of this tile that belongs to this warp
+            int k = (warp - unit % kCommWarps + kCommWarps) % kCommWarps;
+            // routing of a unit's token is fetched one unit ahead, off the per-unit critical path
+            int nxt_row = -1;
+            float nxt_w = 0.f;
+            if (k < n_units && lane < P.k_tot) {
+                const int tn = t0 + k / n_slabs;
+                nxt_row = __ldg(&P.pad_row[(size_t)tn * P.k_tot + lane]);
+                nxt_w = __ldg(&P.topk_w[(size_t)tn * P.k_tot + lane]);
+            }
+            for (; k < n_units; k += kCommWarps) {
+                CommUnit u;
+                u.t = t0 + k / n_slabs;
+                u.slab = slab0 + k % n_slabs;
+                u.d = d;
+                u.s = s;
+                u.wslab = min(P.slab_cols, P.split_w - (u.slab << P.slab_shift));            // layout pitch
+                u.ucols = min(u.wslab, split_c1 - split_c0 - (u.slab << P.slab_shift));       // real columns
+                u.live = true;
+                int my_row = nxt_row;
+                u.w = nxt_w;
+                if (k + kCommWarps < n_units && lane < P.k_tot) {
+                    const int tn = t0 + (k + kCommWarps) / n_slabs;
+                    nxt_row = __ldg(&P.pad_row[(size_t)tn * P.k_tot + lane]);
+                    nxt_w = __ldg(&P.topk_w[(size_t)tn * P.k_tot + lane]);
+                }
                 if (lane < P.k_tot) {
-                    my_row = __ldg(&P.pad_row[(size_t)t * P.k_tot + lane]);
-                    my_w = __ldg(&P.topk_w[(size_t)t * P.k_tot + lane]);
                     if (my_row >= P.R_pad) {
-                        report(P.status, MOE_DEV_OOB, (uint32_t)my_row, 41u);
+                        report(P.status, MOE_DEV_OOB, (uint32_t)my_row, 42u);
                         my_row = -1;
                     }
+                    if (my_row < 0) u.w = 0.f;
                 }
+                // ---- readiness of the producing tiles
                 if (!split_ready) {
                     uint32_t done = 0;
                     if (lane == 0) done = ld_acquire_u32(&P.split_done[s]);
@@ -465,70 +610,64 @@ __device__ void comm_cta(const FusedParams &P, int c)
                     if (done >= (uint32_t)P.W_comp) {
                         split_ready = true;
                     } else {
-                        // per-tile readiness: every (slot j, shard p, n-tile under this column group)
-                        const int nt = (min(c1, gcol0 + kGroupCols) - gcol0 + TN - 1) / TN;
-                        const int in0 = (gcol0 - split_c0) / TN;
+                        // per tile: every (slot j, shard p, n-tile under this slab)
+                        const int cs0 = u.slab << P.slab_shift;
+                        const int in0 = cs0 / TN;
+                        const int nt = (cs0 + u.ucols - 1) / TN - in0 + 1;
                         bool failed = false;
-                        for (int chk = lane; chk < Q * nt; chk += 32) {
+                        for (int chk = lane; chk < P.Q * nt && !failed; chk += 32) {
                             const int qq = chk / nt;
                             const int tn = chk - qq * nt;
                             const int j = qq / P.TP;
                             const int p = qq - j * P.TP;
-                            const int row = __ldg(&P.pad_row[(size_t)t * P.k_tot + j]);
+                            const int row = __ldg(&P.pad_row[(size_t)u.t * P.k_tot + j]);
                             if (row < 0 || row >= P.R_pad) continue;
-                            const int mu = row / P.tile_m;
-                            const int g = s * P.W_comp + (mu * P.TP + p) * P.NTs + in0 + tn;
+                            const int g = s * P.W_comp + ((row / P.tile_m) * P.TP + p) * P.NTs + in0 + tn;
                             uint32_t spins = 0;
                             while (ld_acquire_u32(&P.flags[g]) != P.epoch) {
-                                if ((++spins & 31u) == 0u && globaltimer_ns() > deadline) {
+                                if ((++spins & 31u) == 0u && (ctl->abort || globaltimer_ns() > deadline)) {
                                     report(P.status, MOE_DEV_TIMEOUT, (uint32_t)g, 40u);
                                     failed = true;
                                     break;
                                 }
                                 __nanosleep(64);
                             }
-                            if (failed) break;
                         }
-                        if (__any_sync(0xffffffffu, failed)) return;   // this warp gives up; others carry on
+                        if (__any_sync(0xffffffffu, failed)) {
+                            // this warp gives up; the copy it still has in flight must land first
+                            if (prev.live) consume(prev, (n_mine - 1) & 1, (uint32_t)((n_mine - 1) >> 1) & 1u);
+                            return;
+                        }
                     }
                     __syncwarp();
+                    // rows published through ordinary stores are read by the copy engine next
+                    asm volatile("fence.proxy.async;" ::: "memory");
                 }
-                // gather + weighted sum, fp32, fixed (j, p) order
-                float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-                const bool active = col < c1;
-                for (int q0 = 0; q0 < Q; q0 += 8) {
-                    uint4 v[8];
-                    float w[8];
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const int qq = q0 + i;
-                        const int j = (qq < Q) ? qq / P.TP : 0;
-                        const int p = qq - j * P.TP;
-                        const int row = __shfl_sync(0xffffffffu, my_row, j);
-                        w[i] = __shfl_sync(0xffffffffu, my_w, j);
-                        v[i] = make_uint4(0u, 0u, 0u, 0u);
-                        if (qq >= Q || row < 0) w[i] = 0.f;
-                        else if (active)
-                            v[i] = __ldcg(reinterpret_cast<const uint4 *>(Y + ((size_t)p * (size_t)P.R_pad + (size_t)row) * (size_t)P.H + col));
-                    }
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) fma_bf16x8(acc, v[i], w[i]);
+                // ---- issue this unit's copy, then reduce the previous unit while it is in flight
+                const int st = n_mine & 1;
+                if (lane == 0) {
+                    const uint32_t full = smem_u32(&ctl->comm_full[2 * warp + st]);
+                    const uint32_t bytes = (uint32_t)(P.Q * u.wslab) * 2u;
+                    const __nv_bfloat16 *src = Y + ((size_t)u.t * P.L + s) * (size_t)P.Q * (size_t)P.split_w +
+                                               ((size_t)u.slab * P.Q << P.slab_shift);
+                    mbar_arrive_expect_tx(full, bytes);
+                    bulk_load(smem_u32(my_ring + st * kCommUnitBytes), src, bytes, full);
                 }
-                if (active) {
-                    uint4 pk;
-                    __nv_bfloat162 h0 = __floats2bfloat162_rn(acc[0], acc[1]);
-                    __nv_bfloat162 h1 = __floats2bfloat162_rn(acc[2], acc[3]);
-                    __nv_bfloat162 h2 = __floats2bfloat162_rn(acc[4], acc[5]);
-                    __nv_bfloat162 h3 = __floats2bfloat162_rn(acc[6], acc[7]);
-                    pk.x = *reinterpret_cast<uint32_t *>(&h0);
-                    pk.y = *reinterpret_cast<uint32_t *>(&h1);
-                    pk.z = *reinterpret_cast<uint32_t *>(&h2);
-                    pk.w = *reinterpret_cast<uint32_t *>(&h3);
-                    __stcs(reinterpret_cast<uint4 *>(out_d + (size_t)(t - d * P.tok_blk) * (size_t)P.H + col), pk);
+                __syncwarp();
+                ++n_mine;
+                if (prev.live && !consume(prev, (n_mine - 2) & 1, (uint32_t)((n_mine - 2) >> 1) & 1u)) {
+                    // the previous copy never landed (reported); wait for the one just issued, then leave
+                    const unsigned long long drain = globaltimer_ns() + 2000000ull;
+                    while (!mbar_try_wait(smem_u32(&ctl->comm_full[2 * warp + st]), (uint32_t)((n_mine - 1) >> 1) & 1u) &&
+                           globaltimer_ns() < drain) {}
+                    return;
                 }
+                prev = u;
             }
+            unit += n_units;
         }
     }
+    if (prev.live) consume(prev, (n_mine - 1) & 1, (uint32_t)((n_mine - 1) >> 1) & 1u);
 }
 
 // --------------------------------------------------------------------------- kernel
@@ -545,7 +684,7 @@ moe_gemm2_combine_kernel(const __grid_constant__ FusedParams P)
     if (blockIdx.x == 0 && threadIdx.x < (unsigned)P.L) P.split_done_next[threadIdx.x] = 0u;
 
     if ((int)blockIdx.x < P.C)
-        comm_cta<TN>(P, (int)blockIdx.x);
+        comm_cta<TN>(P, ring, ctl, (int)blockIdx.x);
     else
         compute_cta<TN>(P, ring, ctl, (int)blockIdx.x - P.C);
 }

@@ -31,8 +31,9 @@ struct alignas(64) FusedParams {
     const int32_t *mtile_first_row;
     const int32_t *mtile_valid;
     const int32_t *pad_row;
+    const int32_t *perm;
     const float *topk_w;
-    void *Y;                       // bf16 [TP][R_pad][H]
+    void *Y;                       // bf16 [T][L][slabs][Q][slab cols], token-major
     uint32_t *flags;               // [L * W_comp] readiness per global tile (== epoch when ready)
     uint32_t *split_done;          // [L] tiles finished per split (this launch)
     uint32_t *split_done_next;     // [L] counters of the next launch, zeroed by this one
@@ -45,6 +46,7 @@ struct alignas(64) FusedParams {
     int32_t C, P, mode, withhold;
     int32_t tok_blk, tok_tiles_per_rank, comm_cols, comm_tiles;
     int32_t num_kb, last_ksteps;
+    int32_t Q, slab_cols, slab_shift;   // Q = k_tot * TP rows per unit; slab_cols = 1 << slab_shift
     uint32_t epoch;
 };
 
