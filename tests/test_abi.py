@@ -40,7 +40,7 @@ def test_workspace_sizes_and_argument_errors():
     s = B.make_shape(256, 256, 128, 8, 2, 1, 2, 1)
     rb, yb, fb, sb = B.moe_workspace_bytes(s, 64, 64)
     max_mtiles = 512 // 64 + 8
-    assert yb >= 1 * max_mtiles * 64 * 256 * 2 and sb == 16
+    assert yb >= 256 * 1 * 2 * 1 * 256 * 2 and sb == 16      # token-major partials: T x L x k_tot x TP x H/L
     assert fb >= (64 + 1 * 1 * max_mtiles * 4) * 4
     assert rb >= 3 * 512 * 4 + 3 * max_mtiles * 4
     with pytest.raises(B.MoeError) as e:
