@@ -231,6 +231,34 @@ def run_sweep(h, args, peaks):
     print(json.dumps({"sweep_summary": summary}))
 
 
+def calibrate(h, device, C_ref=32):
+    """Eq. 13 on this GPU: rho_ref = (time of one communication wave) / (time of one compute wave),
+    both measured with the role running alone on its share of the SMs at a fixed C_ref, on the
+    reference workload (DeepSeek-V2-Lite shape, T = 4096, uniform routing, 128x256, TP = EP = L = 2)."""
+    import torch
+    from dataclasses import replace
+    from paper_2609_07536_b200 import binding as B
+    from paper_2609_07536_b200 import workloads as wl
+    w = replace(wl.DSV2L, name="rho_ref", T=4096, routing="uniform", zipf_s=0.0, target_r_expert=0.0)
+    dw = DeviceWorkload(w, device, data="device")
+    step, (occ, lim, rho) = make_stepper(h, dw)
+    plan, counts = step(C_ref)
+    torch.cuda.synchronize()
+    P = lim.G - C_ref
+    t_comp = statistics.median(time_fused(step, torch, 0, 3, 15, mode=B.MOE_MODE_GEMM_ONLY, P_override=P, reuse=counts))
+    t_comm = statistics.median(time_fused(step, torch, 1, 3, 15, mode=B.MOE_MODE_COMBINE_ONLY, C_override=C_ref, reuse=counts))
+    V_comp = -(-plan.W_comp // P)
+    V_comm = -(-plan.W_comm // C_ref)
+    wave_comp = t_comp / (V_comp * w.L)
+    wave_comm = t_comm / (V_comm * w.L)
+    print(json.dumps({"calibration": {
+        "workload": "DeepSeek-V2-Lite shape, T=4096, uniform, 128x256, TP=2, EP=2, L=2", "C_ref": C_ref, "P": P,
+        "t_gemm_only_us": t_comp, "compute_waves": V_comp * w.L, "us_per_compute_wave": wave_comp,
+        "t_combine_only_us": t_comm, "comm_waves": V_comm * w.L, "us_per_comm_wave": wave_comm,
+        "rho_ref": wave_comm / wave_comp, "K_ref": w.K, "tile_ref": [w.tile_m, w.tile_n],
+        "rows_ref": w.k_tot * w.TP + 1, "comm_cols_ref": min(1024, -(-w.H // w.L)), "D_ref": w.EP}}))
+
+
 # ----------------------------------------------------------------------------- CPU baseline
 
 def cpu_baseline(w, idx, wt, x_cpu, W2_cpu, budget_s=15.0):
@@ -304,6 +332,10 @@ def main():
                     help="time just this launch mode (for profiling): warmup + steps launches, short JSON")
     ap.add_argument("--force-C", type=int, default=0, help="with --only: communication CTAs (0 = analytical)")
     ap.add_argument("--data", default="seeded", choices=["seeded", "device"])
+    ap.add_argument("--tile", default="", help="GEMM tile MxN overriding the workload's (e.g. 256x256)")
+    ap.add_argument("--L", type=int, default=0, help="pipeline splits overriding the workload's")
+    ap.add_argument("--calibrate", action="store_true",
+                    help="one-time service-rate characterisation of the kernel family (Eq. 13): prints rho_ref")
     ap.add_argument("--sweep", action="store_true", help="selector-regret sweep on the DeepSeek-V2-Lite shape")
     ap.add_argument("--sweep-out", default="gpurun_out/sweep.json")
     ap.add_argument("--sweep-filter", default="", help="substring a sweep workload name must contain")
@@ -331,8 +363,17 @@ def main():
 
     if args.sweep:
         return run_sweep(h, args, peaks)
+    if args.calibrate:
+        return calibrate(h, device)
 
     w = wl.CONFIGS[args.workload]
+    if args.tile:
+        from dataclasses import replace
+        tm, tn = (int(v) for v in args.tile.split("x"))
+        w = replace(w, tile_m=tm, tile_n=tn)
+    if args.L:
+        from dataclasses import replace
+        w = replace(w, L=args.L)
     dw = DeviceWorkload(w, device, data=args.data if args.only else "seeded")
     step, (occ, lim, rho) = make_stepper(h, dw)
     K, W = max(1, args.steps), max(3, args.warmup)
@@ -342,7 +383,7 @@ def main():
                 "combine_only": B.MOE_MODE_COMBINE_ONLY}[args.only]
         kw = {}
         if args.only == "gemm_only":
-            kw = dict(P_override=(lim.G - args.force_C) if args.force_C else lim.G)
+            kw = dict(P_override=((lim.G - args.force_C) if args.force_C else lim.G) // occ.comp_slot_sms)
         elif args.only == "combine_only":
             kw = dict(C_override=args.force_C or lim.G)
         if args.only == "combine_only":   # Y must exist
@@ -412,7 +453,8 @@ def main():
     if rank == 0:
         # ---- the two roles alone (all SMs compute / all SMs communicate)
         G_sm = lim.G
-        gemm_only = statistics.median(time_fused(step, torch, 0, 2, 7, mode=B.MOE_MODE_GEMM_ONLY, P_override=G_sm))
+        gemm_only = statistics.median(time_fused(step, torch, 0, 2, 7, mode=B.MOE_MODE_GEMM_ONLY,
+                                                 P_override=G_sm // occ.comp_slot_sms))
         lim_all = G_sm
         comb_only = statistics.median(time_fused(step, torch, 1, 2, 7, mode=B.MOE_MODE_COMBINE_ONLY, C_override=G_sm))
         extra["gemm_only"] = {"us": gemm_only, "tflops": dw.flops / gemm_only / 1e6,

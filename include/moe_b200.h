@@ -74,6 +74,8 @@ typedef struct {
     int32_t tile_m, tile_n;           /* T_M^comp, T_N^comp */
     int32_t comm_tile_m, comm_tile_n; /* T_M^comm, T_N^comm */
     int32_t o_comp, o_comm;           /* resident CTAs per SM of each role */
+    int32_t comp_slot_sms;            /* SMs one compute slot occupies: 1, or 2 when a compute tile is run
+                                         by a pair of CTAs on two SMs; P(C) = o_comp * floor((G - R(C)) / comp_slot_sms) */
 } moe_occupancy;
 
 /* GPU residency limits and the user's overrides (Section III-D legal set; Section III-E:
@@ -100,7 +102,7 @@ typedef struct {
 typedef struct {
     int32_t comm_ctas;   /* C*   */
     int32_t R;           /* R(C*) = ceil(C / o_comm), SM positions reserved (Eq. 1) */
-    int32_t P;           /* P(C*) = o_comp (G - R), compute slots (Eq. 3) */
+    int32_t P;           /* P(C*) = o_comp floor((G - R) / comp_slot_sms), compute slots (Eq. 3) */
     int32_t W_comp;      /* Eq. 5, compute tiles per split */
     int32_t W_comm;      /* communication tiles per split on this GPU (Eq. 7 summed over ranks) */
     int32_t delta;       /* Delta_comp(C*) (tie breaker) */
@@ -145,7 +147,8 @@ int32_t moe_set_wait_limit_ns(moe_handle *h, uint64_t ns);
 
 /* Tile shape and residency of the GEMM2 kernel for (tile_m, tile_n), the communication tile,
  * the GPU limits and the stored service-rate constants (Section III-B, III-D, III-E).
- * tile_m in {64, 128}, tile_n in {64, 128, 256}.  Any output pointer may be NULL.  [host] */
+ * (tile_m, tile_n): tile_m in {64, 128} with tile_n in {64, 128, 256} (one CTA per tile), or
+ * (256, 256) (a pair of CTAs on two SMs per tile).  Any output pointer may be NULL.  [host] */
 int32_t moe_query_occupancy(moe_handle *h, int32_t tile_m, int32_t tile_n,
                             moe_occupancy *occ, moe_sm_limits *limits, moe_rho *rho);
 
@@ -216,7 +219,8 @@ int32_t moe_time_plan_partition(const int32_t *routed_tile_counts, int32_t n_set
  * out [host] array of EP [device] pointers, buffer d is bf16 [ceil(T/EP), H], fully overwritten
  * for the tokens rank d owns; y_ws / flags_ws / status_dev as sized by moe_workspace_bytes.
  * n_mtiles = S (host value from moe_build_routing).  Requires H % 8 == 0, K % 16 == 0,
- * 16-byte aligned pointers, 1 <= C, 1 <= P, R * o_comm >= C, R + ceil(P / o_comp) <= G. */
+ * ceil(H/L) % 8 == 0, 16-byte aligned pointers, 1 <= C, 1 <= P, R * o_comm >= C,
+ * R + ceil(P / o_comp) * comp_slot_sms <= G. */
 int32_t moe_gemm2_combine(moe_handle *h, const void *x_routed, const void *W2,
                           const int32_t *topk_idx, const float *topk_w,
                           const moe_shape *shape, const moe_occupancy *occ,

@@ -5,7 +5,8 @@ CPU-baseline leg may import it.  It shares no code with the library's host solve
 
 It follows the paper's Section III step by step, in the paper's order and notation:
   Eq. 1   R(C) = ceil(C / o_comm)
-  Eq. 3   P(C) = o_comp * (G - R(C))
+  Eq. 3   P(C) = o_comp * (G - R(C)); for a kernel family whose compute slot spans `slot_sms` SMs
+          (a tile run by a pair of CTAs) only whole slots count: o_comp * floor((G - R(C)) / slot_sms)
   Eq. 5   W_comp = g * (sum_e ceil(M_e / T_M)) * ceil(ceil(N/L) / T_N)
   Eq. 6   V_comp(C) = ceil(W_comp / P(C))
   Eq. 7   W_comm = ceil(ceil(M/D) / T_M^comm) * ceil(ceil(N/L) / T_N^comm)   (per split and rank)
@@ -114,15 +115,16 @@ def reservation(C: int, o_comm: int) -> int:
     return ceil_div(C, o_comm)                       # Eq. 1
 
 
-def compute_capacity(C: int, G: int, o_comp: int, o_comm: int) -> int:
-    return o_comp * (G - reservation(C, o_comm))     # Eq. 3
+def compute_capacity(C: int, G: int, o_comp: int, o_comm: int, slot_sms: int = 1) -> int:
+    free = G - reservation(C, o_comm)
+    return o_comp * (free // slot_sms) if free > 0 else 0     # Eq. 3
 
 
-def makespan(C: int, Wc: int, Wm: int, L: int, G: int, o_comp: int, o_comm: int, rho):
+def makespan(C: int, Wc: int, Wm: int, L: int, G: int, o_comp: int, o_comm: int, rho, slot_sms: int = 1):
     """T(C) of Eq. 12 with rho any exact number type (int, Fraction).  Returns
     (T, Delta_comp, R, P, [A_s], V_comm) or None when P(C) <= 0."""
     R = reservation(C, o_comm)
-    P = o_comp * (G - R)
+    P = compute_capacity(C, G, o_comp, o_comm, slot_sms)
     if P <= 0:
         return None
     A = [ceil_div((s + 1) * Wc, P) for s in range(L)]    # Eq. 9
@@ -137,14 +139,15 @@ def makespan(C: int, Wc: int, Wm: int, L: int, G: int, o_comp: int, o_comm: int,
 
 
 def select(Wc: int, Wm: int, L: int, G: int, o_comp: int, o_comm: int, C_max: int, rho_q: int,
-           force_comm_ctas: int = 0, selector_off: bool = False, default_C: int = 3) -> dict:
+           force_comm_ctas: int = 0, selector_off: bool = False, default_C: int = 3,
+           slot_sms: int = 1) -> dict:
     """Algorithm 1 in fixed point.  T_q is T(C) * 2^20 with rho replaced by rho_q / 2^20.
 
     Precedence (Section III-E): an explicit user value of C wins over everything; with the
     selector switched off the fixed default is used.  Either must be a legal C."""
     def evaluate(C):
         R = reservation(C, o_comm)
-        P = o_comp * (G - R)
+        P = compute_capacity(C, G, o_comp, o_comm, slot_sms)
         if P <= 0:
             return None
         V_comm = ceil_div(Wm, C)
@@ -178,11 +181,11 @@ def select(Wc: int, Wm: int, L: int, G: int, o_comp: int, o_comm: int, C_max: in
     return best
 
 
-def curve(Wc: int, Wm: int, L: int, G: int, o_comp: int, o_comm: int, C_max: int, rho) -> dict:
+def curve(Wc: int, Wm: int, L: int, G: int, o_comp: int, o_comm: int, C_max: int, rho, slot_sms: int = 1) -> dict:
     """{C: (T, Delta_comp)} for every legal C, rho exact (Fraction or int)."""
     out = {}
     for C in range(1, C_max + 1):
-        m = makespan(C, Wc, Wm, L, G, o_comp, o_comm, rho)
+        m = makespan(C, Wc, Wm, L, G, o_comp, o_comm, rho, slot_sms)
         if m is not None:
             out[C] = (m[0], m[1])
     return out

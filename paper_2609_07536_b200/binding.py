@@ -44,7 +44,8 @@ class moe_shape(C.Structure):
 
 
 class moe_occupancy(C.Structure):
-    _fields_ = [(n, C.c_int32) for n in ("tile_m", "tile_n", "comm_tile_m", "comm_tile_n", "o_comp", "o_comm")]
+    _fields_ = [(n, C.c_int32) for n in ("tile_m", "tile_n", "comm_tile_m", "comm_tile_n", "o_comp", "o_comm",
+                                                "comp_slot_sms")]
 
 
 class moe_sm_limits(C.Structure):

@@ -28,7 +28,11 @@ bool shape_ok(const moe_shape *s)
            s->L <= MOE_MAX_L && s->H % 8 == 0 && s->I % s->TP == 0 && (s->I / s->TP) % 16 == 0 &&
            (int64_t)s->T * s->k_tot < (int64_t)1 << 30;
 }
-bool tile_ok(int tile_m, int tile_n) { return (tile_m == 64 || tile_m == 128) && tile_n_slot(tile_n) >= 0; }
+bool tile_ok(int tile_m, int tile_n)
+{
+    return ((tile_m == 64 || tile_m == 128) && tile_n_slot(tile_n) >= 0) || (tile_m == 256 && tile_n == 256);
+}
+bool tile_m_ok(int tile_m) { return tile_m == 64 || tile_m == 128 || tile_m == 256; }
 
 int32_t max_mtiles_of(const moe_shape *s, int tile_m)
 {
@@ -80,6 +84,11 @@ int32_t moe_create(int32_t device, moe_handle **out)
             return MOE_ERR_CUDA;
         }
     }
+    e = pair_occupancy(&h->o_pair, &h->max_pairs);
+    if (e != cudaSuccess) {
+        delete h;
+        return MOE_ERR_CUDA;
+    }
     *out = h;
     return MOE_OK;
 }
@@ -110,11 +119,14 @@ int32_t moe_query_occupancy(moe_handle *h, int32_t tile_m, int32_t tile_n, moe_o
         occ->comm_tile_m = kCommTileM;
         occ->comm_tile_n = kCommTileN;
         // both roles are CTAs of the same kernel: one resident CTA per SM by shared memory
-        occ->o_comp = h->o_comp[tile_n_slot(tile_n)];
-        occ->o_comm = h->o_comp[tile_n_slot(tile_n)];
+        const bool pair = (tile_m == 256);
+        occ->o_comp = pair ? h->o_pair : h->o_comp[tile_n_slot(tile_n)];
+        occ->o_comm = occ->o_comp;
+        occ->comp_slot_sms = pair ? 2 : 1;
     }
     if (limits) {
-        limits->G = h->G;
+        // a pair tile needs both CTAs of a cluster resident: count only SMs that can host one
+        limits->G = (tile_m == 256) ? (2 * h->max_pairs < h->G ? 2 * h->max_pairs : h->G) : h->G;
         limits->C_max = h->G / 2;   // one-time saturation characterisation of this kernel family
         limits->force_comm_ctas = 0;
         limits->selector_off = 0;
@@ -156,7 +168,8 @@ int32_t moe_workspace_bytes(const moe_shape *s, int32_t tile_m, int32_t tile_n, 
         *y_bytes = align16((size_t)s->T * s->L * s->k_tot * s->TP * (size_t)ceil_div(s->H, s->L) * 2) + 16;
     if (flags_bytes) {
         const size_t nts = (size_t)ceil_div(ceil_div(s->H, s->L), tile_n);
-        *flags_bytes = ((size_t)kSplitCounterWords + (size_t)s->L * s->TP * mt * nts) * 4 + 16;
+        const size_t parts = (tile_m == 256) ? 2 : 1;   // a pair tile is published in two parts
+        *flags_bytes = ((size_t)kSplitCounterWords + (size_t)s->L * s->TP * mt * nts * parts) * 4 + 16;
     }
     if (status_bytes) *status_bytes = 16;
     return MOE_OK;
@@ -166,7 +179,7 @@ int32_t moe_routing_view(void *ws, const moe_shape *s, int32_t tile_m, moe_routi
 {
     if (!ws || !s || !out) return MOE_ERR_NULL;
     if (!shape_ok(s)) return MOE_ERR_SHAPE;
-    if (tile_m != 64 && tile_m != 128) return MOE_ERR_UNSUPPORTED;
+    if (!tile_m_ok(tile_m)) return MOE_ERR_UNSUPPORTED;
     if (!aligned16(ws)) return MOE_ERR_ALIGN;
     const size_t R = (size_t)s->T * s->k_tot, E = (size_t)s->E_tot;
     const size_t mt = (size_t)max_mtiles_of(s, tile_m);
@@ -196,7 +209,7 @@ int32_t moe_build_routing(moe_handle *h, const int32_t *topk_idx, const moe_shap
 {
     if (!h || !s || !r || !status_dev) return MOE_ERR_NULL;
     if (!shape_ok(s)) return MOE_ERR_SHAPE;
-    if (tile_m != 64 && tile_m != 128) return MOE_ERR_UNSUPPORTED;
+    if (!tile_m_ok(tile_m)) return MOE_ERR_UNSUPPORTED;
     if (s->T > 0 && !topk_idx) return MOE_ERR_NULL;
     if (r->max_mtiles < max_mtiles_of(s, tile_m)) return MOE_ERR_SHAPE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -236,12 +249,16 @@ int32_t moe_gemm2_combine(moe_handle *h, const void *x_routed, const void *W2, c
     const int C = (mode == MOE_MODE_GEMM_ONLY) ? 0 : plan->comm_ctas;
     const int Pc = (mode == MOE_MODE_COMBINE_ONLY) ? 0 : plan->P;
     const int o_comp = occ->o_comp > 0 ? occ->o_comp : 1, o_comm = occ->o_comm > 0 ? occ->o_comm : 1;
+    const bool pair = (occ->tile_m == 256);
+    const int slot_sms = pair ? 2 : 1;
+    if (occ->comp_slot_sms != slot_sms) return MOE_ERR_UNSUPPORTED;
     if (mode != MOE_MODE_GEMM_ONLY && C < 1) return MOE_ERR_PLAN_INFEASIBLE;
     if (mode != MOE_MODE_COMBINE_ONLY && Pc < 1) return MOE_ERR_PLAN_INFEASIBLE;
     if (mode == MOE_MODE_FUSED && (int64_t)plan->R * o_comm < C) return MOE_ERR_PLAN_INFEASIBLE;
     // every CTA must be resident at once: spinning communication CTAs may never keep a compute
     // CTA off the GPU (Section II-C: the legal set keeps positive compute capacity)
-    if (ceil_div(C, o_comm) + ceil_div(Pc, o_comp) > h->G) return MOE_ERR_PLAN_INFEASIBLE;
+    if (ceil_div(C, o_comm) + ceil_div(Pc, o_comp) * slot_sms > h->G) return MOE_ERR_PLAN_INFEASIBLE;
+    if (pair && (((C + 1) & ~1) + 2 * Pc > 2 * h->max_pairs)) return MOE_ERR_PLAN_INFEASIBLE;
 
     FusedParams p;
     memset(&p, 0, sizeof p);
@@ -250,10 +267,11 @@ int32_t moe_gemm2_combine(moe_handle *h, const void *x_routed, const void *W2, c
     p.T = s->T; p.H = s->H; p.K = K; p.TP = s->TP; p.EP = s->EP; p.L = s->L; p.k_tot = s->k_tot;
     p.S = n_mtiles;
     p.tile_m = occ->tile_m;
+    p.flag_parts = pair ? 2 : 1;
     p.split_w = (int32_t)ceil_div(s->H, s->L);
     p.NTs = (int32_t)ceil_div(p.split_w, TN);
     const int64_t Wc = (int64_t)s->TP * n_mtiles * p.NTs;
-    if (Wc * s->L >= (int64_t)1 << 31) return MOE_ERR_SHAPE;
+    if (Wc * s->L * 2 >= (int64_t)1 << 31) return MOE_ERR_SHAPE;
     p.W_comp = (int32_t)Wc;
     p.C = C; p.P = Pc; p.mode = mode; p.withhold = plan->debug_withhold_tile;
     p.tok_blk = (int32_t)ceil_div(s->T, s->EP);
@@ -323,7 +341,7 @@ int32_t moe_gemm2_combine(moe_handle *h, const void *x_routed, const void *W2, c
     {
         cuuint64_t dims[3] = {(cuuint64_t)s->I, (cuuint64_t)s->H, (cuuint64_t)s->E_tot};
         cuuint64_t strides[2] = {(cuuint64_t)s->I * 2, (cuuint64_t)s->H * s->I * 2};
-        cuuint32_t box[3] = {(cuuint32_t)kBlockK, (cuuint32_t)TN, 1};
+        cuuint32_t box[3] = {(cuuint32_t)kBlockK, (cuuint32_t)(pair ? TN / 2 : TN), 1};   // a pair CTA loads half the rows
         cuuint32_t es[3] = {1, 1, 1};
         CUresult cr = encode(&p.tmB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(W2), dims, strides,
                              box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -333,7 +351,7 @@ int32_t moe_gemm2_combine(moe_handle *h, const void *x_routed, const void *W2, c
             return MOE_ERR_CUDA;
         }
     }
-    e = fused_launch(TN, p, C + Pc, st);
+    e = pair ? pair_launch(p, ((C + 1) & ~1) + 2 * Pc, st) : fused_launch(TN, p, C + Pc, st);
     if (e != cudaSuccess) return cuda_fail(h, e, "fused launch");
     return MOE_OK;
 }

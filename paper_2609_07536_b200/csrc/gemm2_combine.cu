@@ -112,6 +112,70 @@ __device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, ui
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// ---- CTA-pair (cta_group::2) variants: one MMA spans the tensor cores and TMEM of two SMs
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t mapa_u32(uint32_t addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// each CTA of the pair loads its own operand half; completion is signalled on the leader's barrier
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, uint32_t leader_bar, int x, int y)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"((unsigned long long)map), "r"(leader_bar), "r"(x), "r"(y)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap *map, uint32_t leader_bar, int x, int y, int z)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"((unsigned long long)map), "r"(leader_bar), "r"(x), "r"(y), "r"(z)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_dst, uint32_t cols)
+{
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t cols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+// arrives on the barrier at the same shared-memory offset in both CTAs of the pair
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar)
+{
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+        ::"r"(bar), "h"((uint16_t)3)
+        : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
 // 32 lanes x 32 consecutive fp32 columns: thread i reads TMEM lane (base lane + i)
 __device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32])
 {
@@ -133,6 +197,10 @@ __device__ __forceinline__ uint4 lds_v4(uint32_t addr)
     uint4 v;
     asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
     return v;
+}
+__device__ __forceinline__ void sts_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 __device__ __forceinline__ float lds_f32(uint32_t addr)
 {
@@ -209,8 +277,19 @@ struct Control {
     uint32_t tmem_base;
     volatile uint32_t abort;
     unsigned long long comm_full[24];   // communication CTA: one barrier per warp and stage
-    float comm_w[12][256];              // ... and the per-row weights of the unit a warp reduces (Q <= 256)
 };
+
+// 32 KB after the control block, used by one role per CTA:
+//   communication CTA: per-row weights of the unit each warp reduces (12 warps x 256 floats)
+//   compute CTA      : per-epilogue-warp staging (8 warps x 2.5 KB + row pointers) for coalesced Y stores
+constexpr int kAuxBytes = 8 * 2560 + 8 * 256;
+constexpr int kEpiStagePitch = 80;    // 64 data bytes + 16 pad: conflict-free 16-byte stores
+struct EpiStage {
+    uint8_t data[32 * kEpiStagePitch];        // 32 rows x 32 bf16
+    unsigned long long rowptr[32];            // destination of each row for the group in hand (0 = skip)
+};
+static_assert(sizeof(EpiStage) * 8 <= kAuxBytes, "epilogue staging exceeds the aux region");
+static_assert(12 * 256 * 4 <= kAuxBytes, "communication weights exceed the aux region");
 
 // Bounded mbarrier wait, warp-collective: lane 0 polls (32 lanes polling the same barrier would
 // each occupy the shared-memory pipe), the result is broadcast.  Returns false on timeout or when
@@ -252,10 +331,98 @@ __device__ __forceinline__ Tile decode_tile(int g, const FusedParams &P)
     return t;
 }
 
+// --------------------------------------------------------------------------- epilogue helper
+
+// One thread = one accumulator row (TMEM lane).  Reads COLS fp32 columns starting at `col_first` of
+// the accumulator at `taddr`, rounds to bf16 and writes them to the row's place in the token-major Y:
+// slab = column slab inside the split, q = row of the unit (slot j, shard p).
+template <int COLS>
+__device__ __forceinline__ void store_accumulator_rows(const FusedParams &P, uint32_t taddr, int col_first, bool row_ok,
+                                                       __nv_bfloat16 *ybase, int q, int n0, int col_end, int cis0)
+{
+#pragma unroll
+    for (int cc = 0; cc < COLS; cc += 32) {
+        const int col = col_first + cc;
+        uint32_t r[32];
+        tmem_ld_32x32(taddr + (uint32_t)col, r);
+        tmem_ld_wait();
+        if (row_ok) {
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+                const int c0 = n0 + col + v * 8;
+                if (c0 < col_end) {
+                    const int cis = cis0 + col + v * 8;
+                    const int slab = cis >> P.slab_shift;
+                    const int cin = cis & (P.slab_cols - 1);
+                    const int wslab = min(P.slab_cols, P.split_w - (slab << P.slab_shift));
+                    uint4 pk;
+                    __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(r[v * 8 + 0]), __uint_as_float(r[v * 8 + 1]));
+                    __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(r[v * 8 + 2]), __uint_as_float(r[v * 8 + 3]));
+                    __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(r[v * 8 + 4]), __uint_as_float(r[v * 8 + 5]));
+                    __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(r[v * 8 + 6]), __uint_as_float(r[v * 8 + 7]));
+                    pk.x = *reinterpret_cast<uint32_t *>(&h0);
+                    pk.y = *reinterpret_cast<uint32_t *>(&h1);
+                    pk.z = *reinterpret_cast<uint32_t *>(&h2);
+                    pk.w = *reinterpret_cast<uint32_t *>(&h3);
+                    *reinterpret_cast<uint4 *>(ybase + ((size_t)slab * P.Q << P.slab_shift) + (size_t)q * wslab + cin) = pk;
+                }
+            }
+        }
+    }
+}
+
+// Same job with the stores coalesced: the warp's 32 rows x 32 columns go through a padded staging
+// buffer, so that four lanes write one row's 64 contiguous bytes (two full sectors) instead of every
+// lane writing 16 bytes of a different row.  Needs the 32-column group inside one column slab.
+template <int COLS>
+__device__ __forceinline__ void store_accumulator_rows_staged(const FusedParams &P, uint32_t taddr, int col_first, bool row_ok,
+                                                              __nv_bfloat16 *ybase, int q, int n0, int col_end, int cis0,
+                                                              EpiStage *stg)
+{
+    const int lane = threadIdx.x & 31;
+    const uint32_t stg_s = smem_u32(stg->data);
+    const uint32_t my_row_s = stg_s + (uint32_t)lane * kEpiStagePitch;
+    const int chunk = lane & 3;
+#pragma unroll 2
+    for (int cc = 0; cc < COLS; cc += 32) {
+        const int col = col_first + cc;
+        uint32_t r[32];
+        tmem_ld_32x32(taddr + (uint32_t)col, r);
+        // where this thread's row goes for this 32-column group
+        const int cis = cis0 + col;
+        const int slab = cis >> P.slab_shift;
+        const int wslab = min(P.slab_cols, P.split_w - (slab << P.slab_shift));
+        stg->rowptr[lane] = row_ok ? (unsigned long long)(ybase + ((size_t)slab * P.Q << P.slab_shift) + (size_t)q * wslab +
+                                                          (cis & (P.slab_cols - 1)))
+                                   : 0ull;
+        tmem_ld_wait();
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+            __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(r[v * 8 + 0]), __uint_as_float(r[v * 8 + 1]));
+            __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(r[v * 8 + 2]), __uint_as_float(r[v * 8 + 3]));
+            __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(r[v * 8 + 4]), __uint_as_float(r[v * 8 + 5]));
+            __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(r[v * 8 + 6]), __uint_as_float(r[v * 8 + 7]));
+            sts_v4(my_row_s + v * 16, *reinterpret_cast<uint32_t *>(&h0), *reinterpret_cast<uint32_t *>(&h1),
+                   *reinterpret_cast<uint32_t *>(&h2), *reinterpret_cast<uint32_t *>(&h3));
+        }
+        __syncwarp();
+        // four lanes per row, eight rows per store instruction
+        const bool col_ok = (n0 + col + chunk * 8) < col_end;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int row = i * 8 + (lane >> 2);
+            const unsigned long long dst = stg->rowptr[row];
+            const uint4 v = lds_v4(stg_s + (uint32_t)row * kEpiStagePitch + (uint32_t)chunk * 16u);
+            if (dst != 0ull && col_ok) *reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(dst) + chunk * 8) = v;
+        }
+        __syncwarp();
+    }
+}
+
 // --------------------------------------------------------------------------- compute CTA
 
 template <int TN>
-__device__ void compute_cta(const FusedParams &P, uint8_t *ring, Control *ctl, int b)
+__device__ void compute_cta(const FusedParams &P, uint8_t *ring, Control *ctl, uint8_t *aux, int b)
 {
     using C = Cfg<TN>;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -389,36 +556,14 @@ __device__ void compute_cta(const FusedParams &P, uint8_t *ring, Control *ctl, i
                     q = (f - tok * P.k_tot) * P.TP + t.p;
                     ybase = Y + ((size_t)tok * P.L + t.s) * (size_t)P.Q * (size_t)P.split_w;
                 }
-                const int cis0 = n0 - t.s * P.split_w;   // column inside the split
-#pragma unroll
-                for (int cc = 0; cc < C::kColsPerHalf; cc += 32) {
-                    const int col = half * C::kColsPerHalf + cc;
-                    uint32_t r[32];
-                    tmem_ld_32x32(tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(a * TN + col), r);
-                    tmem_ld_wait();
-                    if (row_ok) {
-#pragma unroll
-                        for (int v = 0; v < 4; ++v) {
-                            const int c0 = n0 + col + v * 8;
-                            if (c0 < col_end) {
-                                const int cis = cis0 + col + v * 8;
-                                const int slab = cis >> P.slab_shift;
-                                const int cin = cis & (P.slab_cols - 1);
-                                const int wslab = min(P.slab_cols, P.split_w - (slab << P.slab_shift));
-                                uint4 pk;
-                                __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(r[v * 8 + 0]), __uint_as_float(r[v * 8 + 1]));
-                                __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(r[v * 8 + 2]), __uint_as_float(r[v * 8 + 3]));
-                                __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(r[v * 8 + 4]), __uint_as_float(r[v * 8 + 5]));
-                                __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(r[v * 8 + 6]), __uint_as_float(r[v * 8 + 7]));
-                                pk.x = *reinterpret_cast<uint32_t *>(&h0);
-                                pk.y = *reinterpret_cast<uint32_t *>(&h1);
-                                pk.z = *reinterpret_cast<uint32_t *>(&h2);
-                                pk.w = *reinterpret_cast<uint32_t *>(&h3);
-                                *reinterpret_cast<uint4 *>(ybase + ((size_t)slab * P.Q << P.slab_shift) + (size_t)q * wslab + cin) = pk;
-                            }
-                        }
-                    }
-                }
+                if (P.slab_cols >= 32)
+                    store_accumulator_rows_staged<C::kColsPerHalf>(
+                        P, tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(a * TN), half * C::kColsPerHalf, row_ok,
+                        ybase, q, n0, col_end, n0 - t.s * P.split_w, reinterpret_cast<EpiStage *>(aux) + (warp - 4));
+                else
+                    store_accumulator_rows<C::kColsPerHalf>(P, tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(a * TN),
+                                                            half * C::kColsPerHalf, row_ok, ybase, q, n0, col_end,
+                                                            n0 - t.s * P.split_w);
                 // the accumulator buffer may be overwritten by the MMA of the tile after next
                 tc_fence_before();
                 __syncwarp();
@@ -440,6 +585,189 @@ __device__ void compute_cta(const FusedParams &P, uint8_t *ring, Control *ctl, i
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, C::kTmemCols);
+    }
+}
+
+
+// --------------------------------------------------------------------------- compute CTA pair
+//
+// 256 x 256 pair tile: two CTAs of a cluster (two SMs) compute one tile with tcgen05.mma.cta_group::2.
+// CTA `rank` loads its own 128 rows of x_routed and its own 128 of the 256 W2 rows of every k-block
+// (no multicast: each CTA issues its own loads), so a k-block costs 32 KB per SM instead of 48 KB.
+// Rank 0 (the leader) issues the MMAs; tcgen05.commit arrives on the barriers of both CTAs.
+//   full[stage]       only the leader's is used: armed by the leader for the bytes of both CTAs
+//   empty[stage]      one per CTA (its producer waits on it), signalled by the leader's commit
+//   tmem_full[a]      one per CTA (its epilogue waits on it), signalled by the leader's commit
+//   tmem_empty[a]     only the leader's is used: 8 local + 8 remote epilogue warps arrive
+struct PairCfg {
+    static constexpr int kTileN = 256;
+    static constexpr int kABytes = kMmaM * kBlockK * 2;                 // 16 KB: this CTA's 128 rows
+    static constexpr int kBBytes = (kTileN / 2) * kBlockK * 2;          // 16 KB: this CTA's 128 W2 rows
+    static constexpr int kStageBytes = kABytes + kBBytes;               // 32 KB
+    static constexpr int kStages = kStageBytesTotal / kStageBytes;      // 6
+    static constexpr int kTmemCols = 2 * kTileN;                        // two accumulator buffers
+    static constexpr int kEpiWarps = 8;
+    static constexpr int kEpiThreads = kEpiWarps * 32;
+    static constexpr int kColsPerHalf = kTileN / 2;
+};
+
+__device__ void compute_cta_pair(const FusedParams &P, uint8_t *ring, Control *ctl, uint8_t *aux, int b)
+{
+    using C = PairCfg;
+    constexpr int TN = C::kTileN;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    const bool leader_cta = (rank == 0);
+    const int total_tiles = P.L * P.W_comp;
+    const unsigned long long deadline = globaltimer_ns() + P.wait_ns;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < C::kStages; ++i) {
+            mbar_init(smem_u32(&ctl->full[i]), 1);
+            mbar_init(smem_u32(&ctl->empty[i]), 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(smem_u32(&ctl->tmem_full[i]), 1);
+            mbar_init(smem_u32(&ctl->tmem_empty[i]), 2 * C::kEpiWarps);
+        }
+        ctl->abort = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc_pair(smem_u32(&ctl->tmem_base), C::kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();          // the peer's barriers exist before anything arrives on them
+    tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    if (warp == 0) {
+        // ---------------- TMA producer (both CTAs): own operand halves, leader's full barrier
+        int stage = 0;
+        uint32_t phase = 0;
+        uint32_t armed = 0;
+        bool ok = true;
+        for (int g = b; g < total_tiles && ok; g += P.P) {
+            const Tile t = decode_tile(g, P);
+            const int e = __ldg(&P.mtile_expert[t.mu]);
+            const int row0 = __ldg(&P.mtile_first_row[t.mu]) + (int)rank * kMmaM;
+            const int n0 = t.s * P.split_w + t.i_n * TN + (int)rank * (TN / 2);
+            const int k0 = t.p * P.K;
+            for (int kb = 0; kb < P.num_kb; ++kb) {
+                ok = wait_barrier(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, deadline, P.status, (uint32_t)g, 10u);
+                if (!ok) break;
+                if (lane == 0) {
+                    const uint32_t own_full = smem_u32(&ctl->full[stage]);
+                    const uint32_t leader_full = mapa_u32(own_full, 0u);
+                    const uint32_t a_dst = smem_u32(ring + stage * C::kStageBytes);
+                    if (leader_cta) mbar_arrive_expect_tx(own_full, 2u * (uint32_t)C::kStageBytes);
+                    tma_load_2d_pair(a_dst, &P.tmA, leader_full, k0 + kb * kBlockK, row0);
+                    tma_load_3d_pair(a_dst + C::kABytes, &P.tmB, leader_full, k0 + kb * kBlockK, n0, e);
+                }
+                __syncwarp();
+                armed |= 1u << stage;
+                if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+            }
+        }
+        if (!ok && leader_cta) {
+            // wind-down: let the copies already issued land before shared memory is released
+            const unsigned long long drain = globaltimer_ns() + 2000000ull;
+            for (int sidx = 0; sidx < C::kStages; ++sidx) {
+                if (!(armed & (1u << sidx))) continue;
+                const uint32_t par = (sidx < stage) ? phase : (phase ^ 1u);
+                while (!mbar_try_wait(smem_u32(&ctl->full[sidx]), par) && globaltimer_ns() < drain) {}
+            }
+        }
+    } else if (warp == 1 && leader_cta) {
+        // ---------------- MMA issuer (leader CTA only)
+        constexpr uint32_t idesc = make_idesc(2 * kMmaM, TN);
+        int stage = 0;
+        uint32_t phase = 0;
+        int it = 0;
+        bool ok = true;
+        for (int g = b; g < total_tiles && ok; g += P.P, ++it) {
+            const int a = it & 1;
+            const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+            ok = wait_barrier(smem_u32(&ctl->tmem_empty[a]), acc_phase ^ 1u, ctl, deadline, P.status, (uint32_t)g, 20u);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + (uint32_t)(a * TN);
+            for (int kb = 0; kb < P.num_kb; ++kb) {
+                ok = wait_barrier(smem_u32(&ctl->full[stage]), phase, ctl, deadline, P.status, (uint32_t)g, 21u);
+                if (!ok) break;
+                tc_fence_after();
+                if (lane == 0) {
+                    const uint32_t a_addr = smem_u32(ring + stage * C::kStageBytes);
+                    const uint64_t a_desc = make_smem_desc(a_addr);
+                    const uint64_t b_desc = make_smem_desc(a_addr + C::kABytes);
+                    const int ksteps = (kb == P.num_kb - 1) ? P.last_ksteps : (kBlockK / kUmmaK);
+                    for (int k = 0; k < ksteps; ++k)
+                        tc_mma_bf16_pair(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
+                                         (kb > 0 || k > 0) ? 1u : 0u);
+                    tc_commit_pair(smem_u32(&ctl->empty[stage]));      // both CTAs may refill the stage
+                }
+                __syncwarp();
+                if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+            }
+            if (ok && lane == 0) tc_commit_pair(smem_u32(&ctl->tmem_full[a]));   // both epilogues may start
+            __syncwarp();
+        }
+    } else if (warp >= 4 && warp < 4 + C::kEpiWarps) {
+        // ---------------- epilogue (both CTAs): own 128 rows of the pair tile
+        const int q4 = warp & 3;
+        const int half = (warp - 4) >> 2;
+        const int row_in_tile = (int)rank * kMmaM + q4 * 32 + lane;
+        const bool is_leader = (warp == 4 && lane == 0);
+        __nv_bfloat16 *Y = reinterpret_cast<__nv_bfloat16 *>(P.Y);
+        int it = 0;
+        for (int g = b; g < total_tiles; g += P.P, ++it) {
+            const Tile t = decode_tile(g, P);
+            const int a = it & 1;
+            const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+            const bool ok = wait_barrier(smem_u32(&ctl->tmem_full[a]), acc_phase, ctl, deadline, P.status, (uint32_t)g, 30u);
+            if (ok) {
+                tc_fence_after();
+                const int valid = __ldg(&P.mtile_valid[t.mu]);
+                const int n0 = t.s * P.split_w + t.i_n * TN;
+                const int col_end = min(P.H, (t.s + 1) * P.split_w);
+                const bool row_ok = row_in_tile < valid;
+                __nv_bfloat16 *ybase = Y;
+                int q = 0;
+                if (row_ok) {
+                    const int f = __ldg(&P.perm[__ldg(&P.mtile_first_row[t.mu]) + row_in_tile]);
+                    const int tok = f / P.k_tot;
+                    q = (f - tok * P.k_tot) * P.TP + t.p;
+                    ybase = Y + ((size_t)tok * P.L + t.s) * (size_t)P.Q * (size_t)P.split_w;
+                }
+                if (P.slab_cols >= 32)
+                    store_accumulator_rows_staged<C::kColsPerHalf>(
+                        P, tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(a * TN), half * C::kColsPerHalf, row_ok,
+                        ybase, q, n0, col_end, n0 - t.s * P.split_w, reinterpret_cast<EpiStage *>(aux) + (warp - 4));
+                else
+                    store_accumulator_rows<C::kColsPerHalf>(P, tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(a * TN),
+                                                            half * C::kColsPerHalf, row_ok, ybase, q, n0, col_end,
+                                                            n0 - t.s * P.split_w);
+                // this CTA's half of the accumulator buffer is drained: tell the leader's MMA warp
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(mapa_u32(smem_u32(&ctl->tmem_empty[a]), 0u));
+            }
+            named_barrier(1, C::kEpiThreads);
+            if (ctl->abort) break;
+            if (is_leader && g != P.withhold) {
+                __threadfence();
+                st_release_u32(&P.flags[2 * g + (int)rank], P.epoch);
+                red_release_add_u32(&P.split_done[t.s], 1u);
+            }
+        }
+    }
+    // ---------------- teardown: nobody leaves while its peer may still touch its memory
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc_pair(tmem_base, C::kTmemCols);
     }
 }
 
@@ -474,7 +802,7 @@ struct CommUnit {
 };
 
 template <int TN>
-__device__ void comm_cta(const FusedParams &P, uint8_t *ring, Control *ctl, int c)
+__device__ void comm_cta(const FusedParams &P, uint8_t *ring, Control *ctl, uint8_t *aux, int c)
 {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const bool wait_needed = (P.mode != MOE_MODE_COMBINE_ONLY);
@@ -492,7 +820,7 @@ __device__ void comm_cta(const FusedParams &P, uint8_t *ring, Control *ctl, int 
     __syncthreads();
     if (warp >= kCommWarps) return;
     uint8_t *my_ring = ring + warp * kCommWarpBytes;
-    float *wq = ctl->comm_w[warp];
+    float *wq = reinterpret_cast<float *>(aux) + warp * 256;
     const __nv_bfloat16 *Y = reinterpret_cast<const __nv_bfloat16 *>(P.Y);
 
     // reduce the unit sitting in stage `st` (its copy was issued one unit ago)
@@ -607,7 +935,7 @@ __device__ void comm_cta(const FusedParams &P, uint8_t *ring, Control *ctl, int 
                     uint32_t done = 0;
                     if (lane == 0) done = ld_acquire_u32(&P.split_done[s]);
                     done = __shfl_sync(0xffffffffu, done, 0);
-                    if (done >= (uint32_t)P.W_comp) {
+                    if (done >= (uint32_t)(P.W_comp * P.flag_parts)) {
                         split_ready = true;
                     } else {
                         // per tile: every (slot j, shard p, n-tile under this slab)
@@ -622,7 +950,10 @@ __device__ void comm_cta(const FusedParams &P, uint8_t *ring, Control *ctl, int 
                             const int p = qq - j * P.TP;
                             const int row = __ldg(&P.pad_row[(size_t)u.t * P.k_tot + j]);
                             if (row < 0 || row >= P.R_pad) continue;
-                            const int g = s * P.W_comp + ((row / P.tile_m) * P.TP + p) * P.NTs + in0 + tn;
+                            const int mu = row / P.tile_m;
+                            // a pair tile is published in two parts, one per CTA: the row's part is its 128-row half
+                            const int part = (P.flag_parts == 2) ? ((row - mu * P.tile_m) >> 7) : 0;
+                            const int g = (s * P.W_comp + (mu * P.TP + p) * P.NTs + in0 + tn) * P.flag_parts + part;
                             uint32_t spins = 0;
                             while (ld_acquire_u32(&P.flags[g]) != P.epoch) {
                                 if ((++spins & 31u) == 0u && (ctl->abort || globaltimer_ns() > deadline)) {
@@ -680,18 +1011,38 @@ moe_gemm2_combine_kernel(const __grid_constant__ FusedParams P)
     // 128B-swizzled tiles need 1024-byte aligned bases
     uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     Control *ctl = reinterpret_cast<Control *>(ring + kStageBytesTotal);
+    uint8_t *aux = reinterpret_cast<uint8_t *>(ring + kStageBytesTotal + ((sizeof(Control) + 127) & ~(size_t)127));
 
     if (blockIdx.x == 0 && threadIdx.x < (unsigned)P.L) P.split_done_next[threadIdx.x] = 0u;
 
     if ((int)blockIdx.x < P.C)
-        comm_cta<TN>(P, ring, ctl, (int)blockIdx.x);
+        comm_cta<TN>(P, ring, ctl, aux, (int)blockIdx.x);
     else
-        compute_cta<TN>(P, ring, ctl, (int)blockIdx.x - P.C);
+        compute_cta<TN>(P, ring, ctl, aux, (int)blockIdx.x - P.C);
+}
+
+// Pair kernel: launched with clusters of two CTAs.  Communication CTAs are single CTAs (blockIdx < C);
+// with an odd C the cluster-mate of the last one has no role; compute pairs start at the next even index.
+__global__ void __launch_bounds__(kThreads, 1)
+moe_gemm2_combine_pair_kernel(const __grid_constant__ FusedParams P)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    Control *ctl = reinterpret_cast<Control *>(ring + kStageBytesTotal);
+    uint8_t *aux = reinterpret_cast<uint8_t *>(ring + kStageBytesTotal + ((sizeof(Control) + 127) & ~(size_t)127));
+
+    if (blockIdx.x == 0 && threadIdx.x < (unsigned)P.L) P.split_done_next[threadIdx.x] = 0u;
+
+    const int c_even = (P.C + 1) & ~1;
+    if ((int)blockIdx.x < P.C)
+        comm_cta<256>(P, ring, ctl, aux, (int)blockIdx.x);
+    else if ((int)blockIdx.x >= c_even)
+        compute_cta_pair(P, ring, ctl, aux, ((int)blockIdx.x - c_even) >> 1);
 }
 
 }  // namespace
 
-size_t fused_smem_bytes(int) { return (size_t)kStageBytesTotal + 1024 + sizeof(Control) + 64; }
+size_t fused_smem_bytes(int) { return (size_t)kStageBytesTotal + 1024 + ((sizeof(Control) + 127) & ~(size_t)127) + kAuxBytes; }
 
 template <int TN>
 static cudaError_t prepare()
@@ -716,6 +1067,47 @@ cudaError_t fused_occupancy(int tile_n, int *blocks_per_sm)
         return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, moe_gemm2_combine_kernel<256>, kThreads, sm);
     }
     return cudaErrorInvalidValue;
+}
+
+cudaError_t pair_occupancy(int *blocks_per_sm, int *max_clusters)
+{
+    const size_t sm = fused_smem_bytes(256);
+    cudaError_t e = cudaFuncSetAttribute(moe_gemm2_combine_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+    if (e != cudaSuccess) return e;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, moe_gemm2_combine_pair_kernel, kThreads, sm);
+    if (e != cudaSuccess) return e;
+    int dev = 0, n_sm = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(n_sm & ~1));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = sm;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaOccupancyMaxActiveClusters(max_clusters, moe_gemm2_combine_pair_kernel, &cfg);
+}
+
+cudaError_t pair_launch(const FusedParams &p, int grid, cudaStream_t stream)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = fused_smem_bytes(256);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, moe_gemm2_combine_pair_kernel, p);
 }
 
 cudaError_t fused_launch(int tile_n, const FusedParams &p, int grid, cudaStream_t stream)

@@ -46,6 +46,7 @@ struct alignas(64) FusedParams {
     int32_t C, P, mode, withhold;
     int32_t tok_blk, tok_tiles_per_rank, comm_cols, comm_tiles;
     int32_t num_kb, last_ksteps;
+    int32_t flag_parts;                 // readiness flags per tile: 1, or 2 for a CTA-pair tile
     int32_t Q, slab_cols, slab_shift;   // Q = k_tot * TP rows per unit; slab_cols = 1 << slab_shift
     uint32_t epoch;
 };
@@ -60,6 +61,8 @@ struct moe_handle {
     std::unordered_map<const void *, uint32_t> epochs;  // per flags workspace
     void *encode_tiled = nullptr;                       // cuTensorMapEncodeTiled
     int o_comp[3] = {0, 0, 0};                          // tile_n = 64, 128, 256
+    int o_pair = 0;                                     // CTA-pair kernel: resident CTAs per SM
+    int max_pairs = 0;                                  // ... and co-resident clusters of two
 };
 
 namespace moe {
@@ -71,6 +74,9 @@ int32_t cuda_fail(moe_handle *h, cudaError_t e, const char *what);
 size_t fused_smem_bytes(int tile_n);
 cudaError_t fused_occupancy(int tile_n, int *blocks_per_sm);
 cudaError_t fused_launch(int tile_n, const FusedParams &p, int grid, cudaStream_t stream);
+// CTA-pair kernel (256 x 256 tiles, clusters of two)
+cudaError_t pair_occupancy(int *blocks_per_sm, int *max_clusters);
+cudaError_t pair_launch(const FusedParams &p, int grid, cudaStream_t stream);
 // routing kernels (routing.cu)
 cudaError_t routing_launch(const int32_t *topk_idx, const moe_shape &s, int tile_m,
                            const moe_routing &r, uint32_t *status, cudaStream_t stream);

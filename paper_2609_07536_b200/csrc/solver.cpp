@@ -2,7 +2,7 @@
 //
 // Section III-D, Algorithm 1: for every legal C evaluate the wave-quantized makespan
 //   R(C) = ceil(C / o_comm)                      (Eq. 1)
-//   P(C) = o_comp (G - R(C))                     (Eq. 3)
+//   P(C) = o_comp floor((G - R(C)) / slot_sms)   (Eq. 3; slot_sms = SMs per compute slot)
 //   A_s  = ceil((s+1) W_comp / P)                (Eq. 9)
 //   q    = rho ceil(W_comm / C)                  (Eq. 8, Eq. 10)
 //   F_s  = max(A_s, F_{s-1}) + q,  T = F_{L-1}   (Eq. 11, Eq. 12)
@@ -30,10 +30,11 @@ struct Candidate {
 
 // One candidate.  32-bit divisions when every dividend fits (the common case), else 64-bit.
 inline bool evaluate(int32_t C, int64_t Wc, int64_t Wm, int32_t L, int32_t G, int32_t o_comp,
-                     int32_t o_comm, int64_t rho_q, bool small, Candidate *out)
+                     int32_t o_comm, int32_t slot_sms, int64_t rho_q, bool small, Candidate *out)
 {
     const int32_t R = (C + o_comm - 1) / o_comm;
-    const int64_t P = (int64_t)o_comp * (G - R);
+    // Eq. 3, with a compute slot that may span several SMs (a CTA pair): only whole slots count
+    const int64_t P = G > R ? (int64_t)o_comp * ((G - R) / slot_sms) : 0;
     if (P <= 0) return false;
     int64_t F = 0;
     int64_t V_comp;
@@ -78,7 +79,7 @@ extern "C" int32_t plan_partition(const int32_t *routed_tile_counts, int32_t n_e
     if (n_experts < 0 || shape->T < 0 || shape->H < 1 || shape->L < 1 || shape->L > MOE_MAX_L ||
         shape->EP < 1 || shape->TP < 1 || shape->I < 1 || shape->k_tot < 1 ||
         occ->tile_m < 1 || occ->tile_n < 1 || occ->comm_tile_m < 1 || occ->comm_tile_n < 1 ||
-        occ->o_comp < 1 || occ->o_comm < 1 || limits->G < 1)
+        occ->o_comp < 1 || occ->o_comm < 1 || occ->comp_slot_sms < 1 || limits->G < 1)
         return MOE_ERR_SHAPE;
 
     // Eq. 16: sum of the routed tile counts; Eq. 5: compute tiles per split (g = TP groups).
@@ -123,7 +124,7 @@ extern "C" int32_t plan_partition(const int32_t *routed_tile_counts, int32_t n_e
     const double scaled = rho_v * (double)(1 << kRhoShift) + 0.5;
     const int64_t rho_q = (int64_t)scaled;  // scaled >= 0.5: truncation is floor
 
-    const int32_t L = shape->L, G = limits->G, o_comp = occ->o_comp, o_comm = occ->o_comm;
+    const int32_t L = shape->L, G = limits->G, o_comp = occ->o_comp, o_comm = occ->o_comm, slot = occ->comp_slot_sms;
     const bool small = (int64_t)L * Wc < (int64_t)0x7FFFFF00 && Wm < (int64_t)0x7FFFFF00 &&
                        (int64_t)o_comp * G < (int64_t)0x7FFFFF00;
 
@@ -132,11 +133,11 @@ extern "C" int32_t plan_partition(const int32_t *routed_tile_counts, int32_t n_e
     if (limits->force_comm_ctas > 0 || limits->selector_off) {
         const int32_t C = limits->force_comm_ctas > 0 ? limits->force_comm_ctas : limits->default_C;
         if (C < 1) return MOE_ERR_PLAN_INFEASIBLE;
-        have = evaluate(C, Wc, Wm, L, G, o_comp, o_comm, rho_q, small, &best);
+        have = evaluate(C, Wc, Wm, L, G, o_comp, o_comm, slot, rho_q, small, &best);
     } else {
         for (int32_t C = 1; C <= limits->C_max; ++C) {
             Candidate c;
-            if (!evaluate(C, Wc, Wm, L, G, o_comp, o_comm, rho_q, small, &c)) break;  // P only falls
+            if (!evaluate(C, Wc, Wm, L, G, o_comp, o_comm, slot, rho_q, small, &c)) break;  // P only falls
             // ascending C: a strict improvement of (T, Delta) is needed to replace the incumbent
             if (!have || c.T_q < best.T_q || (c.T_q == best.T_q && c.delta < best.delta)) {
                 best = c;

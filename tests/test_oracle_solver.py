@@ -41,6 +41,9 @@ def test_a100_reduction():
         assert sr.reservation(C, 1) == C
         assert sr.compute_capacity(C, 108, 2, 1) == 2 * (108 - C)
     assert sr.reservation(5, 2) == 3 and sr.reservation(6, 2) == 3 and sr.reservation(7, 4) == 2
+    # a compute slot spanning two SMs: only whole pairs count, and none when nothing is left
+    assert sr.compute_capacity(20, 148, 1, 1, 2) == 64 and sr.compute_capacity(21, 148, 1, 1, 2) == 63
+    assert sr.compute_capacity(147, 148, 1, 1, 2) == 0 and sr.compute_capacity(200, 148, 1, 1, 2) == 0
 
 
 def test_work_terms_of_the_examples():

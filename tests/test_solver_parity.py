@@ -27,7 +27,7 @@ def _oracle_plan(tiles, shape, occ, lim, rho):
     rho_q = sr.quantise_rho(r)
     sel = sr.select(Wc, Wm, shape.L, lim.G, occ.o_comp, occ.o_comm, lim.C_max, rho_q,
                     force_comm_ctas=lim.force_comm_ctas, selector_off=bool(lim.selector_off),
-                    default_C=lim.default_C)
+                    default_C=lim.default_C, slot_sms=occ.comp_slot_sms)
     sel["rho_q"] = rho_q
     return sel
 
@@ -48,7 +48,7 @@ def _rand_inputs(rng):
                          rng.choice([128, 512, 1408]) * TP, E, rng.choice([1, 2, 8]), TP,
                          rng.choice([1, 2, 4, 8]), rng.choice([1, 2, 4, 8]))
     occ = B.moe_occupancy(tile_m, tile_n, rng.choice([64, 128]), rng.choice([512, 1024]),
-                          rng.choice([1, 2]), rng.choice([1, 2, 4]))
+                          rng.choice([1, 2]), rng.choice([1, 2, 4]), rng.choice([1, 1, 2]))
     lim = B.moe_sm_limits(rng.choice([4, 108, 148]), rng.randint(1, 160), 0, 0, 3)
     rho = B.moe_rho(rng.uniform(0.05, 30.0), rng.choice([352, 704]), 128, rng.choice([128, 256]),
                     rng.choice([2, 4]), 17, 1024, rng.choice([B.MOE_RHO_PAPER, B.MOE_RHO_LOCAL]))
@@ -109,7 +109,7 @@ def test_baseline_shapes(w):
     idx, _, _ = wl.make_routing(w)
     r = rr.build_routing(idx, w.E_tot, w.tile_m)
     shape = B.make_shape(w.T, w.H, w.I, w.E_tot, w.k_tot, w.TP, w.EP, w.L)
-    occ = B.moe_occupancy(w.tile_m, w.tile_n, 128, 1024, 1, 1)
+    occ = B.moe_occupancy(w.tile_m, w.tile_n, 128, 1024, 1, 1, 1)
     lim = B.moe_sm_limits(148, 74, 0, 0, 3)
     for mode in (B.MOE_RHO_PAPER, B.MOE_RHO_LOCAL):
         rho = B.moe_rho(2.5, 704, 128, 256, 2, 17, 1024, mode)
@@ -123,7 +123,7 @@ def test_golden_examples_through_the_library(golden_dir):
     # Ex.C and Ex.D of the hand-worked examples, expressed as library inputs
     # Ex.C: W_comp = 8192 = TP 2 x S 1024 x 4 n-tiles ; W_comm = 64 (one rank of 8192 tokens)
     shape = B.make_shape(8192, 2048, 1408, 64, 8, 2, 1, 2)
-    occ = B.moe_occupancy(128, 256, 128, 1024, 1, 1)
+    occ = B.moe_occupancy(128, 256, 128, 1024, 1, 1, 1)
     lim = B.moe_sm_limits(148, 74, 0, 0, 3)
     rho = B.moe_rho(3.0, 704, 128, 256, 1, 17, 1024, B.MOE_RHO_PAPER)
     plan = B.plan_partition([16] * 64, occ, lim, shape, rho)
@@ -132,7 +132,7 @@ def test_golden_examples_through_the_library(golden_dir):
     assert plan.pred_T_q == 137 << 20 and plan.rho_q == 3145728
     # Ex.D: o_comm = 2, W_comp = 1000 = 1 x 1000 x 1, W_comm = 37, L = 4, rho = 2.5
     shape = B.make_shape(37 * 128, 1024, 704, 10, 8, 1, 1, 4)
-    occ = B.moe_occupancy(128, 256, 128, 1024, 1, 2)
+    occ = B.moe_occupancy(128, 256, 128, 1024, 1, 2, 1)
     lim = B.moe_sm_limits(148, 32, 0, 0, 3)
     rho = B.moe_rho(2.5, 704, 128, 256, 1, 17, 1024, B.MOE_RHO_PAPER)
     plan = B.plan_partition([100] * 10, occ, lim, shape, rho)
@@ -141,11 +141,30 @@ def test_golden_examples_through_the_library(golden_dir):
     assert plan.pred_T_q == 34 << 20
 
 
+def test_pair_slots():
+    # a compute slot that spans two SMs (CTA pair): P(C) = floor((G - C) / 2); an odd C strands one SM
+    shape = B.make_shape(16384, 2048, 1408, 66, 8, 2, 2, 2)
+    occ = B.moe_occupancy(256, 256, 128, 1024, 1, 1, 2)
+    rho = B.moe_rho(9.0, 704, 128, 256, 2, 17, 1024, B.MOE_RHO_LOCAL)
+    for C in (1, 2, 7, 20, 146, 147):
+        lim = B.moe_sm_limits(148, 74, C, 0, 3)
+        if (148 - C) // 2 < 1:
+            with pytest.raises(B.MoeError):
+                B.plan_partition([8] * 66, occ, lim, shape, rho)
+            continue
+        plan = B.plan_partition([8] * 66, occ, lim, shape, rho)
+        assert plan.P == (148 - C) // 2 and plan.R == C
+        _same(plan, _oracle_plan([8] * 66, shape, occ, lim, rho))
+    lim = B.moe_sm_limits(148, 74, 0, 0, 3)
+    plan = B.plan_partition([8] * 66, occ, lim, shape, rho)
+    assert plan.comm_ctas % 2 == 0           # an odd C never beats the even one below it by the model
+
+
 def test_solver_cost_is_small():
     # not a benchmark: only guards against an accidental blow-up (ctypes overhead dominates here)
     w = wl.DSV2L
     shape = B.make_shape(w.T, w.H, w.I, w.E_tot, w.k_tot, w.TP, w.EP, w.L)
-    occ = B.moe_occupancy(128, 256, 128, 1024, 1, 1)
+    occ = B.moe_occupancy(128, 256, 128, 1024, 1, 1, 1)
     lim = B.moe_sm_limits(148, 74, 0, 0, 3)
     rho = B.moe_rho(2.5, 704, 128, 256, 2, 17, 1024, B.MOE_RHO_LOCAL)
     tiles = [17] * 66
