@@ -387,7 +387,7 @@ def main():
         elif args.only == "combine_only":
             kw = dict(C_override=args.force_C or lim.G)
         if args.only == "combine_only":   # Y must exist
-            step(0, mode=B.MOE_MODE_GEMM_ONLY, P_override=lim.G)
+            step(0, mode=B.MOE_MODE_GEMM_ONLY, P_override=lim.G // occ.comp_slot_sms)
         ts = time_fused(step, torch, (args.force_C if args.only == "fused" else (1 if args.only == "combine_only" else 0)),
                         args.warmup, K, mode=mode, **kw)
         med = statistics.median(ts)

@@ -773,6 +773,33 @@ __device__ void compute_cta_pair(const FusedParams &P, uint8_t *ring, Control *c
 
 // --------------------------------------------------------------------------- communication CTA
 
+// two fp32 FMAs in one instruction (sm_100): acc = x * w + acc on packed pairs
+__device__ __forceinline__ unsigned long long ffma2(unsigned long long x, unsigned long long w, unsigned long long acc)
+{
+    unsigned long long d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(x), "l"(w), "l"(acc));
+    return d;
+}
+__device__ __forceinline__ unsigned long long pack_f32x2(uint32_t lo, uint32_t hi)
+{
+    unsigned long long d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
+    return d;
+}
+__device__ __forceinline__ void unpack_f32x2(unsigned long long v, float &lo, float &hi)
+{
+    uint32_t a, b;
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(a), "=r"(b) : "l"(v));
+    lo = __uint_as_float(a);
+    hi = __uint_as_float(b);
+}
+// acc[i] (a pair of fp32) += w * (the two bf16 of word i), for the four words of v
+__device__ __forceinline__ void fma2_bf16x8(unsigned long long (&acc)[4], const uint4 &v, unsigned long long ww)
+{
+    const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) acc[i] = ffma2(pack_f32x2(u[i] << 16, u[i] & 0xFFFF0000u), ww, acc[i]);
+}
 __device__ __forceinline__ void fma_bf16x8(float (&acc)[8], const uint4 &v, float w)
 {
     const uint32_t u[4] = {v.x, v.y, v.z, v.w};
@@ -799,6 +826,7 @@ struct CommUnit {
     int t, d, s, slab, wslab, ucols;
     float w;          // lane j: weight of slot j (0 when the slot has no source row)
     bool live;
+    bool all_valid;   // every slot of the token has a source row
 };
 
 template <int TN>
@@ -838,6 +866,43 @@ __device__ void comm_cta(const FusedParams &P, uint8_t *ring, Control *ctl, uint
         const uint32_t stage_s = smem_u32(my_ring + st * kCommUnitBytes);
         __nv_bfloat16 *orow = reinterpret_cast<__nv_bfloat16 *>(P.out[u.d]) +
                               (size_t)(u.t - u.d * P.tok_blk) * (size_t)P.H + u.s * P.split_w + (u.slab << P.slab_shift);
+        if (u.all_valid && P.Q <= 16) {
+            // common case: every slot has a source row and the unit has at most 16 rows: weights stay in
+            // registers as packed pairs, rows are fetched eight at a time, two FMAs per instruction
+            unsigned long long ww[16];
+#pragma unroll
+            for (int r = 0; r < 16; ++r) {
+                const uint32_t wb = __float_as_uint(r < P.Q ? lds_f32(wq_s + (uint32_t)r * 4u) : 0.f);
+                ww[r] = pack_f32x2(wb, wb);
+            }
+            for (int c16 = lane; c16 < n16; c16 += 32) {
+                unsigned long long acc[4] = {0ull, 0ull, 0ull, 0ull};
+                const uint32_t src = stage_s + (uint32_t)c16 * 16u;
+#pragma unroll
+                for (int r0 = 0; r0 < 16; r0 += 8) {
+                    if (r0 < P.Q) {
+                        uint4 v[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) v[i] = lds_v4(src + (uint32_t)min(r0 + i, P.Q - 1) * row_bytes);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) fma2_bf16x8(acc, v[i], ww[r0 + i]);   // rows past Q carry weight 0
+                    }
+                }
+                float f[8];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) unpack_f32x2(acc[i], f[2 * i], f[2 * i + 1]);
+                uint4 pk;
+                __nv_bfloat162 h0 = __floats2bfloat162_rn(f[0], f[1]);
+                __nv_bfloat162 h1 = __floats2bfloat162_rn(f[2], f[3]);
+                __nv_bfloat162 h2 = __floats2bfloat162_rn(f[4], f[5]);
+                __nv_bfloat162 h3 = __floats2bfloat162_rn(f[6], f[7]);
+                pk.x = *reinterpret_cast<uint32_t *>(&h0);
+                pk.y = *reinterpret_cast<uint32_t *>(&h1);
+                pk.z = *reinterpret_cast<uint32_t *>(&h2);
+                pk.w = *reinterpret_cast<uint32_t *>(&h3);
+                __stcs(reinterpret_cast<uint4 *>(orow + c16 * 8), pk);
+            }
+        } else
         for (int c16 = lane; c16 < ((n16 + 31) & ~31); c16 += 32) {
             float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
             const uint32_t src = stage_s + (uint32_t)(c16 < n16 ? c16 : 0) * 16u;
@@ -930,6 +995,7 @@ __device__ void comm_cta(const FusedParams &P, uint8_t *ring, Control *ctl, uint
                     }
                     if (my_row < 0) u.w = 0.f;
                 }
+                u.all_valid = __all_sync(0xffffffffu, lane >= P.k_tot || my_row >= 0);
                 // ---- readiness of the producing tiles
                 if (!split_ready) {
                     uint32_t done = 0;
