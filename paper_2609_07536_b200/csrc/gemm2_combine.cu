@@ -8,17 +8,21 @@
 //                   b, b+P, b+2P, ... of the split-major sequence in which the expert
 //                   problems of one split are contiguous).
 //
-// Compute CTA (warp-specialised):
-//   warp 0      TMA producer: x_routed tile (128 rows x 64 k) and W2 tile (tile_n rows x 64 k)
-//               into a ring of 128B-swizzled shared-memory stages;
-//   warp 1      MMA issuer: tcgen05.mma (M = 128, N = tile_n, K = 16, bf16 -> fp32) into one of
-//               two TMEM accumulator buffers; tcgen05.commit frees stages / publishes the tile;
-//   warps 4-11  epilogue: tcgen05.ld -> bf16 -> Y (tile-padded), then the tile's readiness flag
-//               (st.release.gpu) and the split counter (red.release.gpu).
-// Communication CTA (16 warps): a warp owns (token, 256-column group) units of its
-//   communication tile; it waits for the producing tiles (ld.acquire.gpu; bounded), gathers the
-//   k_tot * TP rows with 16-byte loads, accumulates in fp32 in (j, p) order and stores bf16 into
-//   the owning rank's buffer.
+// Compute CTA (warp-specialised; tile_m x tile_n with tile_m in {64, 128}):
+//   warps 0, 2  TMA producers (one thread each): warp 0 the x_routed tile (128 rows x 64 k), warp 2 the
+//               W2 tile (tile_n rows x 64 k) of every k-block, into a ring of 128B-swizzled stages;
+//   warp 1      MMA issuer (one thread): tcgen05.mma (M = 128, N = tile_n, K = 16, bf16 -> fp32) into one
+//               of two TMEM accumulator buffers; tcgen05.commit frees stages / publishes the tile;
+//   warps 4-11  epilogue: tcgen05.ld -> bf16 -> Y, then the tile's readiness flag (st.release.gpu) and
+//               the split counter (red.release.gpu).
+// Compute CTA pair (256 x 256 tiles): the same roles in both CTAs of a cluster of two; one
+//   tcgen05.mma.cta_group::2 spans both SMs, each CTA loads only its own operand halves.
+// Y is token-major: the epilogue scatters each accumulator row to its (token, slot, shard) place, so
+//   that the k_tot * TP partial rows of one (token, split, column slab) form one contiguous block.
+// Communication CTA (12 independent warps): a warp fetches such a block with one bulk asynchronous
+//   copy into its own double-buffered shared-memory stage (the readiness of the producing tiles is
+//   checked first: split counter, else per-tile flags with ld.acquire.gpu; bounded), sums the rows in
+//   fp32 in (j, p) order with the token's weights and stores bf16 into the owning rank's buffer.
 //
 // Every wait is bounded: after `wait_ns` the waiter records MOE_DEV_TIMEOUT and the CTA winds
 // down (pending bulk copies are drained, TMEM is released).
@@ -316,6 +320,25 @@ __device__ __forceinline__ bool wait_barrier(uint32_t bar, uint32_t parity, Cont
     return __shfl_sync(0xffffffffu, ok, 0) != 0u;
 }
 
+// The same wait for a loop that a single thread runs on its own (no broadcast).
+__device__ __forceinline__ bool wait_barrier_1t(uint32_t bar, uint32_t parity, Control *ctl,
+                                                unsigned long long deadline, uint32_t *status,
+                                                uint32_t detail, uint32_t where)
+{
+    uint32_t spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 63u) == 0u) {
+            if (ctl->abort) return false;
+            if (globaltimer_ns() > deadline) {
+                ctl->abort = 1u;
+                report(status, MOE_DEV_TIMEOUT, detail, where);
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
 struct Tile {
     int s, mu, p, i_n;
 };
@@ -449,66 +472,68 @@ __device__ void compute_cta(const FusedParams &P, uint8_t *ring, Control *ctl, u
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
 
-    if (warp == 0) {
-        // ---------------- TMA producer: the whole warp walks the loop, lane 0 issues
-        int stage = 0;
-        uint32_t phase = 0;
-        uint32_t armed = 0;  // bit s: stage s was handed to the TMA unit at least once
-        bool ok = true;
-        for (int g = b; g < total_tiles && ok; g += P.P) {
-            const Tile t = decode_tile(g, P);
-            const int e = __ldg(&P.mtile_expert[t.mu]);
-            const int row0 = __ldg(&P.mtile_first_row[t.mu]);
-            const int n0 = t.s * P.split_w + t.i_n * TN;
-            const int k0 = t.p * P.K;
-            for (int kb = 0; kb < P.num_kb; ++kb) {
-                ok = wait_barrier(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, deadline, P.status, (uint32_t)g, 10u);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                if (lane == 0) {
+    if (warp == 0 || warp == 2) {
+        // ---------------- TMA producers: warp 0 loads the x_routed tile, warp 2 the W2 tile of every
+        // k-block; both complete on the same full barrier.  One thread per warp runs the whole loop (no
+        // per-iteration warp broadcast); the others park below.
+        const bool load_a = (warp == 0);
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            uint32_t armed = 0;  // bit s: stage s was handed to the TMA unit at least once
+            bool ok = true;
+            for (int g = b; g < total_tiles && ok; g += P.P) {
+                const Tile t = decode_tile(g, P);
+                const int e = __ldg(&P.mtile_expert[t.mu]);
+                const int row0 = __ldg(&P.mtile_first_row[t.mu]);
+                const int n0 = t.s * P.split_w + t.i_n * TN;
+                int kx = t.p * P.K;
+                for (int kb = 0; kb < P.num_kb; ++kb, kx += kBlockK) {
+                    ok = wait_barrier_1t(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, deadline, P.status, (uint32_t)g, 10u);
+                    if (!ok) break;
                     const uint32_t full = smem_u32(&ctl->full[stage]);
                     const uint32_t a_dst = smem_u32(ring + stage * C::kStageBytes);
-                    mbar_arrive_expect_tx(full, (uint32_t)C::kStageBytes);
-                    tma_load_2d(a_dst, &P.tmA, full, k0 + kb * kBlockK, row0);
-                    tma_load_3d(a_dst + C::kABytes, &P.tmB, full, k0 + kb * kBlockK, n0, e);
+                    if (load_a) {
+                        mbar_arrive_expect_tx(full, (uint32_t)C::kStageBytes);
+                        tma_load_2d(a_dst, &P.tmA, full, kx, row0);
+                    } else {
+                        tma_load_3d(a_dst + C::kABytes, &P.tmB, full, kx, n0, e);
+                    }
+                    armed |= 1u << stage;
+                    if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
                 }
-                __syncwarp();
-                armed |= 1u << stage;
-                if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+            }
+            if (!ok) {
+                // wind-down: let the copies already issued land before shared memory is released
+                // (bounded; a stage consumed meanwhile has completed its phase and passes at once)
+                const unsigned long long drain = globaltimer_ns() + 2000000ull;
+                for (int sidx = 0; sidx < C::kStages; ++sidx) {
+                    if (!(armed & (1u << sidx))) continue;
+                    const uint32_t par = (sidx < stage) ? phase : (phase ^ 1u);
+                    while (!mbar_try_wait(smem_u32(&ctl->full[sidx]), par) && globaltimer_ns() < drain) {}
+                }
             }
         }
-        if (!ok) {
-            // wind-down: let the copies already issued land before shared memory is released
-            // (bounded; a stage consumed meanwhile has completed its phase and passes at once)
-            const unsigned long long drain = globaltimer_ns() + 2000000ull;
-            for (int sidx = 0; sidx < C::kStages; ++sidx) {
-                if (!(armed & (1u << sidx))) continue;
-                // parity of the phase this stage was last armed in
-                const uint32_t par = (sidx < stage) ? phase : (phase ^ 1u);
-                while (!mbar_try_wait(smem_u32(&ctl->full[sidx]), par) && globaltimer_ns() < drain) {}
-            }
-        }
+        __syncwarp();
     } else if (warp == 1) {
-        // ---------------- MMA issuer: the whole warp walks the loop, lane 0 issues
-        constexpr uint32_t idesc = make_idesc(kMmaM, TN);
-        int stage = 0;
-        uint32_t phase = 0;
-        int it = 0;
-        bool ok = true;
-        for (int g = b; g < total_tiles && ok; g += P.P, ++it) {
-            const int a = it & 1;
-            const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
-            ok = wait_barrier(smem_u32(&ctl->tmem_empty[a]), acc_phase ^ 1u, ctl, deadline, P.status, (uint32_t)g, 20u);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t d_tmem = tmem_base + (uint32_t)(a * TN);
-            for (int kb = 0; kb < P.num_kb; ++kb) {
-                ok = wait_barrier(smem_u32(&ctl->full[stage]), phase, ctl, deadline, P.status, (uint32_t)g, 21u);
-                ok = __all_sync(0xffffffffu, ok);
+        // ---------------- MMA issuer: one thread runs the whole loop
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc(kMmaM, TN);
+            int stage = 0;
+            uint32_t phase = 0;
+            int it = 0;
+            bool ok = true;
+            for (int g = b; g < total_tiles && ok; g += P.P, ++it) {
+                const int a = it & 1;
+                const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+                ok = wait_barrier_1t(smem_u32(&ctl->tmem_empty[a]), acc_phase ^ 1u, ctl, deadline, P.status, (uint32_t)g, 20u);
                 if (!ok) break;
                 tc_fence_after();
-                if (lane == 0) {
+                const uint32_t d_tmem = tmem_base + (uint32_t)(a * TN);
+                for (int kb = 0; kb < P.num_kb; ++kb) {
+                    ok = wait_barrier_1t(smem_u32(&ctl->full[stage]), phase, ctl, deadline, P.status, (uint32_t)g, 21u);
+                    if (!ok) break;
+                    tc_fence_after();
                     const uint32_t a_addr = smem_u32(ring + stage * C::kStageBytes);
                     const uint64_t a_desc = make_smem_desc(a_addr);
                     const uint64_t b_desc = make_smem_desc(a_addr + C::kABytes);
@@ -519,13 +544,12 @@ __device__ void compute_cta(const FusedParams &P, uint8_t *ring, Control *ctl, u
                                     (kb > 0 || k > 0) ? 1u : 0u);
                     }
                     tc_commit(smem_u32(&ctl->empty[stage]));   // stage reusable once these MMAs have read it
+                    if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
                 }
-                __syncwarp();
-                if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+                if (ok) tc_commit(smem_u32(&ctl->tmem_full[a]));  // accumulator complete
             }
-            if (ok && lane == 0) tc_commit(smem_u32(&ctl->tmem_full[a]));  // accumulator complete
-            __syncwarp();
         }
+        __syncwarp();
     } else if (warp >= 4 && warp < 4 + C::kEpiWarps) {
         // ---------------- epilogue: TMEM -> bf16 -> Y, then publish the tile
         const int q4 = warp & 3;                   // TMEM lane quarter this warp may read
@@ -641,62 +665,68 @@ __device__ void compute_cta_pair(const FusedParams &P, uint8_t *ring, Control *c
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
 
-    if (warp == 0) {
-        // ---------------- TMA producer (both CTAs): own operand halves, leader's full barrier
-        int stage = 0;
-        uint32_t phase = 0;
-        uint32_t armed = 0;
-        bool ok = true;
-        for (int g = b; g < total_tiles && ok; g += P.P) {
-            const Tile t = decode_tile(g, P);
-            const int e = __ldg(&P.mtile_expert[t.mu]);
-            const int row0 = __ldg(&P.mtile_first_row[t.mu]) + (int)rank * kMmaM;
-            const int n0 = t.s * P.split_w + t.i_n * TN + (int)rank * (TN / 2);
-            const int k0 = t.p * P.K;
-            for (int kb = 0; kb < P.num_kb; ++kb) {
-                ok = wait_barrier(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, deadline, P.status, (uint32_t)g, 10u);
-                if (!ok) break;
-                if (lane == 0) {
+    if (warp == 0 || warp == 2) {
+        // ---------------- TMA producers (both CTAs): warp 0 loads this CTA's x_routed rows, warp 2 its W2
+        // rows; both complete on the leader's full barrier.  Two issuing threads halve the serial issue
+        // latency per k-block.  One thread per warp runs the whole loop; the others park below.
+        const bool load_a = (warp == 0);
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            uint32_t armed = 0;
+            bool ok = true;
+            for (int g = b; g < total_tiles && ok; g += P.P) {
+                const Tile t = decode_tile(g, P);
+                const int e = __ldg(&P.mtile_expert[t.mu]);
+                const int row0 = __ldg(&P.mtile_first_row[t.mu]) + (int)rank * kMmaM;
+                const int n0 = t.s * P.split_w + t.i_n * TN + (int)rank * (TN / 2);
+                int kx = t.p * P.K;
+                for (int kb = 0; kb < P.num_kb; ++kb, kx += kBlockK) {
                     const uint32_t own_full = smem_u32(&ctl->full[stage]);
-                    const uint32_t leader_full = mapa_u32(own_full, 0u);
+                    ok = wait_barrier_1t(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, deadline, P.status, (uint32_t)g, 10u);
+                    if (!ok) break;
+                    const uint32_t leader_full = own_full & 0xFEFFFFFFu;   // same offset in the leader CTA (rank 0)
                     const uint32_t a_dst = smem_u32(ring + stage * C::kStageBytes);
-                    if (leader_cta) mbar_arrive_expect_tx(own_full, 2u * (uint32_t)C::kStageBytes);
-                    tma_load_2d_pair(a_dst, &P.tmA, leader_full, k0 + kb * kBlockK, row0);
-                    tma_load_3d_pair(a_dst + C::kABytes, &P.tmB, leader_full, k0 + kb * kBlockK, n0, e);
+                    if (load_a) {
+                        if (leader_cta) mbar_arrive_expect_tx(own_full, 2u * (uint32_t)C::kStageBytes);
+                        tma_load_2d_pair(a_dst, &P.tmA, leader_full, kx, row0);
+                    } else {
+                        tma_load_3d_pair(a_dst + C::kABytes, &P.tmB, leader_full, kx, n0, e);
+                    }
+                    armed |= 1u << stage;
+                    if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
                 }
-                __syncwarp();
-                armed |= 1u << stage;
-                if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+            }
+            if (!ok && leader_cta) {
+                // wind-down: let the copies already issued land before shared memory is released
+                const unsigned long long drain = globaltimer_ns() + 2000000ull;
+                for (int sidx = 0; sidx < C::kStages; ++sidx) {
+                    if (!(armed & (1u << sidx))) continue;
+                    const uint32_t par = (sidx < stage) ? phase : (phase ^ 1u);
+                    while (!mbar_try_wait(smem_u32(&ctl->full[sidx]), par) && globaltimer_ns() < drain) {}
+                }
             }
         }
-        if (!ok && leader_cta) {
-            // wind-down: let the copies already issued land before shared memory is released
-            const unsigned long long drain = globaltimer_ns() + 2000000ull;
-            for (int sidx = 0; sidx < C::kStages; ++sidx) {
-                if (!(armed & (1u << sidx))) continue;
-                const uint32_t par = (sidx < stage) ? phase : (phase ^ 1u);
-                while (!mbar_try_wait(smem_u32(&ctl->full[sidx]), par) && globaltimer_ns() < drain) {}
-            }
-        }
+        __syncwarp();
     } else if (warp == 1 && leader_cta) {
-        // ---------------- MMA issuer (leader CTA only)
-        constexpr uint32_t idesc = make_idesc(2 * kMmaM, TN);
-        int stage = 0;
-        uint32_t phase = 0;
-        int it = 0;
-        bool ok = true;
-        for (int g = b; g < total_tiles && ok; g += P.P, ++it) {
-            const int a = it & 1;
-            const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
-            ok = wait_barrier(smem_u32(&ctl->tmem_empty[a]), acc_phase ^ 1u, ctl, deadline, P.status, (uint32_t)g, 20u);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t d_tmem = tmem_base + (uint32_t)(a * TN);
-            for (int kb = 0; kb < P.num_kb; ++kb) {
-                ok = wait_barrier(smem_u32(&ctl->full[stage]), phase, ctl, deadline, P.status, (uint32_t)g, 21u);
+        // ---------------- MMA issuer (leader CTA only): one thread runs the whole loop
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc(2 * kMmaM, TN);
+            int stage = 0;
+            uint32_t phase = 0;
+            int it = 0;
+            bool ok = true;
+            for (int g = b; g < total_tiles && ok; g += P.P, ++it) {
+                const int a = it & 1;
+                const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+                ok = wait_barrier_1t(smem_u32(&ctl->tmem_empty[a]), acc_phase ^ 1u, ctl, deadline, P.status, (uint32_t)g, 20u);
                 if (!ok) break;
                 tc_fence_after();
-                if (lane == 0) {
+                const uint32_t d_tmem = tmem_base + (uint32_t)(a * TN);
+                for (int kb = 0; kb < P.num_kb; ++kb) {
+                    ok = wait_barrier_1t(smem_u32(&ctl->full[stage]), phase, ctl, deadline, P.status, (uint32_t)g, 21u);
+                    if (!ok) break;
+                    tc_fence_after();
                     const uint32_t a_addr = smem_u32(ring + stage * C::kStageBytes);
                     const uint64_t a_desc = make_smem_desc(a_addr);
                     const uint64_t b_desc = make_smem_desc(a_addr + C::kABytes);
@@ -705,13 +735,12 @@ __device__ void compute_cta_pair(const FusedParams &P, uint8_t *ring, Control *c
                         tc_mma_bf16_pair(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
                                          (kb > 0 || k > 0) ? 1u : 0u);
                     tc_commit_pair(smem_u32(&ctl->empty[stage]));      // both CTAs may refill the stage
+                    if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
                 }
-                __syncwarp();
-                if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+                if (ok) tc_commit_pair(smem_u32(&ctl->tmem_full[a]));   // both epilogues may start
             }
-            if (ok && lane == 0) tc_commit_pair(smem_u32(&ctl->tmem_full[a]));   // both epilogues may start
-            __syncwarp();
         }
+        __syncwarp();
     } else if (warp >= 4 && warp < 4 + C::kEpiWarps) {
         // ---------------- epilogue (both CTAs): own 128 rows of the pair tile
         const int q4 = warp & 3;
