@@ -86,6 +86,10 @@ typedef struct {
     int32_t force_comm_ctas; /* > 0: use exactly this C */
     int32_t selector_off;    /* != 0: use default_C */
     int32_t default_C;       /* the fixed count used when the selector is off */
+    int32_t drain_help;      /* != 0: compute CTAs that run out of GEMM tiles serve the communication tiles
+                                that are left (an extension of this library, not in the paper: with it the
+                                selector models the tail after the last compute wave as served by every SM);
+                                0: the paper's static partition and its recurrence exactly */
 } moe_sm_limits;
 
 /* Relative wave service rate (Eq. 13-15). */
@@ -110,6 +114,8 @@ typedef struct {
     int64_t rho_q;       /* rho scaled by 2^20 and rounded to nearest */
     int32_t mode;        /* MOE_MODE_* (plan_partition writes MOE_MODE_FUSED) */
     int32_t debug_withhold_tile; /* test hook: global tile whose readiness is never raised; -1 = none */
+    int32_t drain_help;  /* copied from moe_sm_limits: compute CTAs help with the communication tail */
+    int32_t reserved;
 } moe_plan;
 
 /* Views into the routing workspace, all [device] int32. */
@@ -153,8 +159,9 @@ int32_t moe_query_occupancy(moe_handle *h, int32_t tile_m, int32_t tile_n,
                             moe_occupancy *occ, moe_sm_limits *limits, moe_rho *rho);
 
 /* Sizes of the caller-allocated workspaces [bytes]: routing arrays, the tile-padded GEMM2
- * output Y (bf16 [TP][T_M * max_mtiles][H]), readiness flags + split counters (must be
- * zero-filled once before first use and not shared between handles), status (16 bytes). */
+ * output Y (bf16, token-major: [T][L][k_tot * TP][ceil(H/L)]), readiness flags + split counters +
+ * tile claims (must be zero-filled once before first use and not shared between handles), status
+ * (16 bytes). */
 int32_t moe_workspace_bytes(const moe_shape *shape, int32_t tile_m, int32_t tile_n,
                             size_t *routing_bytes, size_t *y_bytes, size_t *flags_bytes,
                             size_t *status_bytes);

@@ -140,12 +140,17 @@ def makespan(C: int, Wc: int, Wm: int, L: int, G: int, o_comp: int, o_comm: int,
 
 def select(Wc: int, Wm: int, L: int, G: int, o_comp: int, o_comm: int, C_max: int, rho_q: int,
            force_comm_ctas: int = 0, selector_off: bool = False, default_C: int = 3,
-           slot_sms: int = 1) -> dict:
+           slot_sms: int = 1, drain_help: bool = False) -> dict:
     """Algorithm 1 in fixed point.  T_q is T(C) * 2^20 with rho replaced by rho_q / 2^20.
 
     Precedence (Section III-E): an explicit user value of C wins over everything; with the
     selector switched off the fixed default is used.  Either must be a legal C."""
     def evaluate(C):
+        if drain_help:
+            m = makespan_drain_help(C, Wc, Wm, L, G, o_comp, o_comm, rho_q, slot_sms)
+            if m is None:
+                return None
+            return dict(comm_ctas=C, R=m[2], P=m[3], T_q=m[0], delta=m[1], W_comp=Wc, W_comm=Wm)
         R = reservation(C, o_comm)
         P = compute_capacity(C, G, o_comp, o_comm, slot_sms)
         if P <= 0:
@@ -179,6 +184,32 @@ def select(Wc: int, Wm: int, L: int, G: int, o_comp: int, o_comm: int, C_max: in
     if best is None:
         raise ValueError("no legal C")
     return best
+
+
+def makespan_drain_help(C: int, Wc: int, Wm: int, L: int, G: int, o_comp: int, o_comm: int, rho_q: int,
+                        slot_sms: int = 1):
+    """Extension of the recurrence (not in the paper) for a kernel family whose compute CTAs serve
+    communication tiles once their GEMM tiles are done.  Fixed point, rho_q = rho * 2^20.
+      * splits 0..L-2: Eq. 11 unchanged, C workers;
+      * at A_{L-1} (last compute wave over) the tiles still queued -- whole waves of C, at most
+        (L-1) W_comm -- plus the last split's W_comm tiles are served by C + H workers, where
+        H = P * slot_sms / o_comp is the number of CTAs that were computing.
+    Returns (T_q, Delta_comp, R, P) or None when P(C) <= 0."""
+    R = reservation(C, o_comm)
+    P = compute_capacity(C, G, o_comp, o_comm, slot_sms)
+    if P <= 0:
+        return None
+    q = rho_q * ceil_div(Wm, C)
+    F = 0
+    for s in range(L - 1):
+        F = max(ceil_div((s + 1) * Wc, P) * RHO_ONE, F) + q
+    A_last = ceil_div(L * Wc, P) * RHO_ONE
+    backlog = 0
+    if F > A_last and rho_q > 0:
+        backlog = min(ceil_div(F - A_last, rho_q) * C, (L - 1) * Wm)
+    workers = C + P * slot_sms // o_comp
+    T_q = A_last + rho_q * ceil_div(backlog + Wm, workers)
+    return T_q, ceil_div(Wc, P) * P - Wc, R, P
 
 
 def curve(Wc: int, Wm: int, L: int, G: int, o_comp: int, o_comm: int, C_max: int, rho, slot_sms: int = 1) -> dict:

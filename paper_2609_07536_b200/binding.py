@@ -49,7 +49,8 @@ class moe_occupancy(C.Structure):
 
 
 class moe_sm_limits(C.Structure):
-    _fields_ = [(n, C.c_int32) for n in ("G", "C_max", "force_comm_ctas", "selector_off", "default_C")]
+    _fields_ = [(n, C.c_int32) for n in ("G", "C_max", "force_comm_ctas", "selector_off", "default_C",
+                                                "drain_help")]
 
 
 class moe_rho(C.Structure):
@@ -59,7 +60,8 @@ class moe_rho(C.Structure):
 
 class moe_plan(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("comm_ctas", "R", "P", "W_comp", "W_comm", "delta")] + [
-        ("pred_T_q", C.c_int64), ("rho_q", C.c_int64), ("mode", C.c_int32), ("debug_withhold_tile", C.c_int32)]
+        ("pred_T_q", C.c_int64), ("rho_q", C.c_int64), ("mode", C.c_int32), ("debug_withhold_tile", C.c_int32),
+        ("drain_help", C.c_int32), ("reserved", C.c_int32)]
 
 
 class moe_routing(C.Structure):

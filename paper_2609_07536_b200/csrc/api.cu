@@ -19,7 +19,19 @@ inline size_t align16(size_t x) { return (x + 15) & ~(size_t)15; }
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 
-constexpr int kSplitCounterWords = 64;  // 2 parities x MOE_MAX_L counters, padded
+constexpr int kSplitCounterWords = 64;  // 2 parities x MOE_MAX_L split counters, then 2 x MOE_MAX_L steal counters, padded
+
+int64_t comm_tiles_of(const moe_shape *s)
+{
+    const int64_t blk = ceil_div(s->T, s->EP);
+    int64_t tok_tiles = 0;
+    for (int d = 0; d < s->EP; ++d) {
+        int64_t own = (int64_t)s->T - (int64_t)d * blk;
+        if (own > blk) own = blk;
+        if (own > 0) tok_tiles += ceil_div(own, kCommTileM);
+    }
+    return tok_tiles * ceil_div(ceil_div(s->H, s->L), kCommTileN);
+}
 
 bool shape_ok(const moe_shape *s)
 {
@@ -131,6 +143,7 @@ int32_t moe_query_occupancy(moe_handle *h, int32_t tile_m, int32_t tile_n, moe_o
         limits->force_comm_ctas = 0;
         limits->selector_off = 0;
         limits->default_C = 3;      // the fixed count of the upstream path (Section II-C)
+        limits->drain_help = 1;
     }
     if (rho) {
         // one-time service-rate characterisation of this kernel family on B200 (Eq. 13):
@@ -169,7 +182,8 @@ int32_t moe_workspace_bytes(const moe_shape *s, int32_t tile_m, int32_t tile_n, 
     if (flags_bytes) {
         const size_t nts = (size_t)ceil_div(ceil_div(s->H, s->L), tile_n);
         const size_t parts = (tile_m == 256) ? 2 : 1;   // a pair tile is published in two parts
-        *flags_bytes = ((size_t)kSplitCounterWords + (size_t)s->L * s->TP * mt * nts * parts) * 4 + 16;
+        *flags_bytes = ((size_t)kSplitCounterWords + (size_t)s->L * s->TP * mt * nts * parts +
+                        (size_t)s->L * (size_t)comm_tiles_of(s)) * 4 + 16;
     }
     if (status_bytes) *status_bytes = 16;
     return MOE_OK;
@@ -274,6 +288,7 @@ int32_t moe_gemm2_combine(moe_handle *h, const void *x_routed, const void *W2, c
     if (Wc * s->L * 2 >= (int64_t)1 << 31) return MOE_ERR_SHAPE;
     p.W_comp = (int32_t)Wc;
     p.C = C; p.P = Pc; p.mode = mode; p.withhold = plan->debug_withhold_tile;
+    p.drain_help = (mode == MOE_MODE_FUSED && plan->drain_help) ? 1 : 0;
     p.tok_blk = (int32_t)ceil_div(s->T, s->EP);
     p.tok_tiles_per_rank = (int32_t)ceil_div(p.tok_blk, kCommTileM);
     p.comm_cols = (int32_t)ceil_div(p.split_w, kCommTileN);
@@ -320,7 +335,10 @@ int32_t moe_gemm2_combine(moe_handle *h, const void *x_routed, const void *W2, c
     p.epoch = ep;
     p.split_done = flags_ws + (ep & 1u) * MOE_MAX_L;
     p.split_done_next = flags_ws + ((ep + 1u) & 1u) * MOE_MAX_L;
+    p.steal = flags_ws + 2 * MOE_MAX_L + (ep & 1u) * MOE_MAX_L;
+    p.steal_next = flags_ws + 2 * MOE_MAX_L + ((ep + 1u) & 1u) * MOE_MAX_L;
     p.flags = flags_ws + kSplitCounterWords;
+    p.claims = p.flags + (size_t)s->L * (size_t)p.W_comp * p.flag_parts;
 
     // tensor maps (Section II-A operands): x_routed [R, I] and W2 [E_tot, H, I], k contiguous
     EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(h->encode_tiled);

@@ -281,6 +281,7 @@ struct Control {
     uint32_t tmem_base;
     volatile uint32_t abort;
     unsigned long long comm_full[24];   // communication CTA: one barrier per warp and stage
+    volatile int claim_slot[2];         // ... and the CTA-wide result of a tile claim
 };
 
 // 32 KB after the control block, used by one role per CTA:
@@ -859,10 +860,11 @@ struct CommUnit {
 };
 
 template <int TN>
-__device__ void comm_cta(const FusedParams &P, uint8_t *ring, Control *ctl, uint8_t *aux, int c)
+__device__ void comm_cta(const FusedParams &P, uint8_t *ring, Control *ctl, uint8_t *aux, int c, bool helper)
 {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const bool wait_needed = (P.mode != MOE_MODE_COMBINE_ONLY);
+    const bool claiming = (P.drain_help != 0);   // tiles are claimed, so that a helper and the tile's own CTA never both serve it
     const unsigned long long deadline = globaltimer_ns() + P.wait_ns;
     // the wait for a copy only follows a readiness wait: it gets a later deadline so that the first
     // report names the wait that really ran out
@@ -871,6 +873,7 @@ __device__ void comm_cta(const FusedParams &P, uint8_t *ring, Control *ctl, uint
     if (threadIdx.x == 0) {
         for (int i = 0; i < 2 * kCommWarps; ++i) mbar_init(smem_u32(&ctl->comm_full[i]), 1);
         ctl->abort = 0u;
+        ctl->claim_slot[0] = ctl->claim_slot[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -973,124 +976,181 @@ __device__ void comm_cta(const FusedParams &P, uint8_t *ring, Control *ctl, uint
     int n_mine = 0;          // units this warp has issued so far: stage n_mine & 1, parity (n_mine >> 1) & 1
     CommUnit prev;
     prev.live = false;
+    uint32_t ready_mask = wait_needed ? 0u : 0xffffffffu;   // bit s: split s is known to be complete
 
-    for (int s = 0; s < P.L; ++s) {
-        bool split_ready = !wait_needed;
+    // serve communication tile ct of split s; false when this warp had to give up (reported)
+    auto serve_tile = [&](int s, int ct) -> bool {
         const int split_c0 = s * P.split_w;
         const int split_c1 = min(P.H, split_c0 + P.split_w);
-        for (int ct = c; ct < P.comm_tiles; ct += P.C) {
-            const int tok_tile = ct / P.comm_cols;
-            const int col_tile = ct - tok_tile * P.comm_cols;
-            const int d = tok_tile / P.tok_tiles_per_rank;
-            const int ti = tok_tile - d * P.tok_tiles_per_rank;
-            const int t0 = d * P.tok_blk + ti * kCommTileM;
-            const int t1 = min(min(P.T, (d + 1) * P.tok_blk), t0 + kCommTileM);
-            const int c0 = split_c0 + col_tile * kCommTileN;
-            const int c1 = min(split_c1, c0 + kCommTileN);
-            if (t0 >= t1 || c0 >= c1) continue;
-            const int slab0 = (c0 - split_c0) >> P.slab_shift;
-            const int n_slabs = ((c1 - split_c0 + P.slab_cols - 1) >> P.slab_shift) - slab0;
-            const int n_units = (t1 - t0) * n_slabs;
-            // first unit of this tile that belongs to this warp
-            int k = (warp - unit % kCommWarps + kCommWarps) % kCommWarps;
-            // routing of a unit's token is fetched one unit ahead, off the per-unit critical path
-            int nxt_row = -1;
-            float nxt_w = 0.f;
-            if (k < n_units && lane < P.k_tot) {
-                const int tn = t0 + k / n_slabs;
+        const int tok_tile = ct / P.comm_cols;
+        const int col_tile = ct - tok_tile * P.comm_cols;
+        const int d = tok_tile / P.tok_tiles_per_rank;
+        const int ti = tok_tile - d * P.tok_tiles_per_rank;
+        const int t0 = d * P.tok_blk + ti * kCommTileM;
+        const int t1 = min(min(P.T, (d + 1) * P.tok_blk), t0 + kCommTileM);
+        const int c0 = split_c0 + col_tile * kCommTileN;
+        const int c1 = min(split_c1, c0 + kCommTileN);
+        if (t0 >= t1 || c0 >= c1) return true;
+        const int slab0 = (c0 - split_c0) >> P.slab_shift;
+        const int n_slabs = ((c1 - split_c0 + P.slab_cols - 1) >> P.slab_shift) - slab0;
+        const int n_units = (t1 - t0) * n_slabs;
+        // first unit of this tile that belongs to this warp
+        int k = (warp - unit % kCommWarps + kCommWarps) % kCommWarps;
+        // routing of a unit's token is fetched one unit ahead, off the per-unit critical path
+        int nxt_row = -1;
+        float nxt_w = 0.f;
+        if (k < n_units && lane < P.k_tot) {
+            const int tn = t0 + k / n_slabs;
+            nxt_row = __ldg(&P.pad_row[(size_t)tn * P.k_tot + lane]);
+            nxt_w = __ldg(&P.topk_w[(size_t)tn * P.k_tot + lane]);
+        }
+        for (; k < n_units; k += kCommWarps) {
+            CommUnit u;
+            u.t = t0 + k / n_slabs;
+            u.slab = slab0 + k % n_slabs;
+            u.d = d;
+            u.s = s;
+            u.wslab = min(P.slab_cols, P.split_w - (u.slab << P.slab_shift));            // layout pitch
+            u.ucols = min(u.wslab, split_c1 - split_c0 - (u.slab << P.slab_shift));       // real columns
+            u.live = true;
+            int my_row = nxt_row;
+            u.w = nxt_w;
+            if (k + kCommWarps < n_units && lane < P.k_tot) {
+                const int tn = t0 + (k + kCommWarps) / n_slabs;
                 nxt_row = __ldg(&P.pad_row[(size_t)tn * P.k_tot + lane]);
                 nxt_w = __ldg(&P.topk_w[(size_t)tn * P.k_tot + lane]);
             }
-            for (; k < n_units; k += kCommWarps) {
-                CommUnit u;
-                u.t = t0 + k / n_slabs;
-                u.slab = slab0 + k % n_slabs;
-                u.d = d;
-                u.s = s;
-                u.wslab = min(P.slab_cols, P.split_w - (u.slab << P.slab_shift));            // layout pitch
-                u.ucols = min(u.wslab, split_c1 - split_c0 - (u.slab << P.slab_shift));       // real columns
-                u.live = true;
-                int my_row = nxt_row;
-                u.w = nxt_w;
-                if (k + kCommWarps < n_units && lane < P.k_tot) {
-                    const int tn = t0 + (k + kCommWarps) / n_slabs;
-                    nxt_row = __ldg(&P.pad_row[(size_t)tn * P.k_tot + lane]);
-                    nxt_w = __ldg(&P.topk_w[(size_t)tn * P.k_tot + lane]);
+            if (lane < P.k_tot) {
+                if (my_row >= P.R_pad) {
+                    report(P.status, MOE_DEV_OOB, (uint32_t)my_row, 42u);
+                    my_row = -1;
                 }
-                if (lane < P.k_tot) {
-                    if (my_row >= P.R_pad) {
-                        report(P.status, MOE_DEV_OOB, (uint32_t)my_row, 42u);
-                        my_row = -1;
-                    }
-                    if (my_row < 0) u.w = 0.f;
-                }
-                u.all_valid = __all_sync(0xffffffffu, lane >= P.k_tot || my_row >= 0);
-                // ---- readiness of the producing tiles
-                if (!split_ready) {
-                    uint32_t done = 0;
-                    if (lane == 0) done = ld_acquire_u32(&P.split_done[s]);
-                    done = __shfl_sync(0xffffffffu, done, 0);
-                    if (done >= (uint32_t)(P.W_comp * P.flag_parts)) {
-                        split_ready = true;
-                    } else {
-                        // per tile: every (slot j, shard p, n-tile under this slab)
-                        const int cs0 = u.slab << P.slab_shift;
-                        const int in0 = cs0 / TN;
-                        const int nt = (cs0 + u.ucols - 1) / TN - in0 + 1;
-                        bool failed = false;
-                        for (int chk = lane; chk < P.Q * nt && !failed; chk += 32) {
-                            const int qq = chk / nt;
-                            const int tn = chk - qq * nt;
-                            const int j = qq / P.TP;
-                            const int p = qq - j * P.TP;
-                            const int row = __ldg(&P.pad_row[(size_t)u.t * P.k_tot + j]);
-                            if (row < 0 || row >= P.R_pad) continue;
-                            const int mu = row / P.tile_m;
-                            // a pair tile is published in two parts, one per CTA: the row's part is its 128-row half
-                            const int part = (P.flag_parts == 2) ? ((row - mu * P.tile_m) >> 7) : 0;
-                            const int g = (s * P.W_comp + (mu * P.TP + p) * P.NTs + in0 + tn) * P.flag_parts + part;
-                            uint32_t spins = 0;
-                            while (ld_acquire_u32(&P.flags[g]) != P.epoch) {
-                                if ((++spins & 31u) == 0u && (ctl->abort || globaltimer_ns() > deadline)) {
-                                    report(P.status, MOE_DEV_TIMEOUT, (uint32_t)g, 40u);
-                                    failed = true;
-                                    break;
-                                }
-                                __nanosleep(64);
+                if (my_row < 0) u.w = 0.f;
+            }
+            u.all_valid = __all_sync(0xffffffffu, lane >= P.k_tot || my_row >= 0);
+            // ---- readiness of the producing tiles
+            if (!((ready_mask >> s) & 1u)) {
+                uint32_t done = 0;
+                if (lane == 0) done = ld_acquire_u32(&P.split_done[s]);
+                done = __shfl_sync(0xffffffffu, done, 0);
+                if (done >= (uint32_t)(P.W_comp * P.flag_parts)) {
+                    ready_mask |= 1u << s;
+                } else {
+                    // per tile: every (slot j, shard p, n-tile under this slab)
+                    const int cs0 = u.slab << P.slab_shift;
+                    const int in0 = cs0 / TN;
+                    const int nt = (cs0 + u.ucols - 1) / TN - in0 + 1;
+                    bool failed = false;
+                    for (int chk = lane; chk < P.Q * nt && !failed; chk += 32) {
+                        const int qq = chk / nt;
+                        const int tn = chk - qq * nt;
+                        const int j = qq / P.TP;
+                        const int p = qq - j * P.TP;
+                        const int row = __ldg(&P.pad_row[(size_t)u.t * P.k_tot + j]);
+                        if (row < 0 || row >= P.R_pad) continue;
+                        const int mu = row / P.tile_m;
+                        // a pair tile is published in two parts, one per CTA: the row's part is its 128-row half
+                        const int part = (P.flag_parts == 2) ? ((row - mu * P.tile_m) >> 7) : 0;
+                        const int g = (s * P.W_comp + (mu * P.TP + p) * P.NTs + in0 + tn) * P.flag_parts + part;
+                        uint32_t spins = 0;
+                        while (ld_acquire_u32(&P.flags[g]) != P.epoch) {
+                            if ((++spins & 31u) == 0u && (ctl->abort || globaltimer_ns() > deadline)) {
+                                report(P.status, MOE_DEV_TIMEOUT, (uint32_t)g, 40u);
+                                failed = true;
+                                break;
                             }
-                        }
-                        if (__any_sync(0xffffffffu, failed)) {
-                            // this warp gives up; the copy it still has in flight must land first
-                            if (prev.live) consume(prev, (n_mine - 1) & 1, (uint32_t)((n_mine - 1) >> 1) & 1u);
-                            return;
+                            __nanosleep(64);
                         }
                     }
-                    __syncwarp();
-                    // rows published through ordinary stores are read by the copy engine next
-                    asm volatile("fence.proxy.async;" ::: "memory");
-                }
-                // ---- issue this unit's copy, then reduce the previous unit while it is in flight
-                const int st = n_mine & 1;
-                if (lane == 0) {
-                    const uint32_t full = smem_u32(&ctl->comm_full[2 * warp + st]);
-                    const uint32_t bytes = (uint32_t)(P.Q * u.wslab) * 2u;
-                    const __nv_bfloat16 *src = Y + ((size_t)u.t * P.L + s) * (size_t)P.Q * (size_t)P.split_w +
-                                               ((size_t)u.slab * P.Q << P.slab_shift);
-                    mbar_arrive_expect_tx(full, bytes);
-                    bulk_load(smem_u32(my_ring + st * kCommUnitBytes), src, bytes, full);
+                    if (__any_sync(0xffffffffu, failed)) {
+                        // this warp gives up; the copy it still has in flight must land first
+                        if (prev.live) consume(prev, (n_mine - 1) & 1, (uint32_t)((n_mine - 1) >> 1) & 1u);
+                        prev.live = false;
+                        unit += n_units;
+                        return false;
+                    }
                 }
                 __syncwarp();
-                ++n_mine;
-                if (prev.live && !consume(prev, (n_mine - 2) & 1, (uint32_t)((n_mine - 2) >> 1) & 1u)) {
-                    // the previous copy never landed (reported); wait for the one just issued, then leave
-                    const unsigned long long drain = globaltimer_ns() + 2000000ull;
-                    while (!mbar_try_wait(smem_u32(&ctl->comm_full[2 * warp + st]), (uint32_t)((n_mine - 1) >> 1) & 1u) &&
-                           globaltimer_ns() < drain) {}
-                    return;
-                }
-                prev = u;
+                // rows published through ordinary stores are read by the copy engine next
+                asm volatile("fence.proxy.async;" ::: "memory");
             }
-            unit += n_units;
+            // ---- issue this unit's copy, then reduce the previous unit while it is in flight
+            const int st = n_mine & 1;
+            if (lane == 0) {
+                const uint32_t full = smem_u32(&ctl->comm_full[2 * warp + st]);
+                const uint32_t bytes = (uint32_t)(P.Q * u.wslab) * 2u;
+                const __nv_bfloat16 *src = Y + ((size_t)u.t * P.L + s) * (size_t)P.Q * (size_t)P.split_w +
+                                           ((size_t)u.slab * P.Q << P.slab_shift);
+                mbar_arrive_expect_tx(full, bytes);
+                bulk_load(smem_u32(my_ring + st * kCommUnitBytes), src, bytes, full);
+            }
+            __syncwarp();
+            ++n_mine;
+            if (prev.live && !consume(prev, (n_mine - 2) & 1, (uint32_t)((n_mine - 2) >> 1) & 1u)) {
+                // the previous copy never landed (reported); wait for the one just issued, then leave
+                const unsigned long long drain = globaltimer_ns() + 2000000ull;
+                while (!mbar_try_wait(smem_u32(&ctl->comm_full[2 * warp + st]), (uint32_t)((n_mine - 1) >> 1) & 1u) &&
+                       globaltimer_ns() < drain) {}
+                prev.live = false;
+                unit += n_units;
+                return false;
+            }
+            prev = u;
+        }
+        unit += n_units;
+        return true;
+    };
+
+    // CTA-wide decision taken by one thread and read by all twelve working warps.  Two result slots
+    // alternate, so one barrier per decision is enough.
+    int n_decisions = 0;
+    auto broadcast = [&](int value_from_warp0_lane0) -> int {
+        volatile int *slot = &ctl->claim_slot[n_decisions & 1];
+        if (warp == 0 && lane == 0) *slot = value_from_warp0_lane0;
+        named_barrier(3, kCommWarps * 32);
+        ++n_decisions;
+        return *slot;
+    };
+    bool dead = false;   // this warp gave up; it keeps meeting the others at the decision barriers
+
+    if (!helper) {
+        for (int s = 0; s < P.L; ++s) {
+            for (int ct = c; ct < P.comm_tiles; ct += P.C) {
+                if (claiming) {
+                    int mine = 0;
+                    if (warp == 0 && lane == 0) mine = (atomicExch(&P.claims[s * P.comm_tiles + ct], P.epoch) != P.epoch) ? 1 : 0;
+                    mine = broadcast(mine);
+                    if (ctl->abort) { s = P.L; break; }
+                    if (!mine) continue;      // a helper took it
+                }
+                if (!dead && !serve_tile(s, ct)) {
+                    dead = true;
+                    ctl->abort = 1u;
+                    if (!claiming) return;    // no CTA-wide barriers in this mode: the warp may leave
+                }
+            }
+        }
+    } else {
+        // a compute CTA that ran out of GEMM tiles: take unclaimed tiles from the back, last split first
+        for (int s = P.L - 1; s >= 0; --s) {
+            for (;;) {
+                int ct = -1;
+                if (warp == 0 && lane == 0) {
+                    for (;;) {
+                        const uint32_t idx = atomicAdd(&P.steal[s], 1u);
+                        if (idx >= (uint32_t)P.comm_tiles) break;
+                        const int cand = P.comm_tiles - 1 - (int)idx;
+                        if (atomicExch(&P.claims[s * P.comm_tiles + cand], P.epoch) != P.epoch) { ct = cand; break; }
+                    }
+                }
+                ct = broadcast(ct);
+                if (ctl->abort) { s = -1; break; }
+                if (ct < 0) break;
+                if (!dead && !serve_tile(s, ct)) {
+                    dead = true;
+                    ctl->abort = 1u;
+                }
+            }
         }
     }
     if (prev.live) consume(prev, (n_mine - 1) & 1, (uint32_t)((n_mine - 1) >> 1) & 1u);
@@ -1108,12 +1168,18 @@ moe_gemm2_combine_kernel(const __grid_constant__ FusedParams P)
     Control *ctl = reinterpret_cast<Control *>(ring + kStageBytesTotal);
     uint8_t *aux = reinterpret_cast<uint8_t *>(ring + kStageBytesTotal + ((sizeof(Control) + 127) & ~(size_t)127));
 
-    if (blockIdx.x == 0 && threadIdx.x < (unsigned)P.L) P.split_done_next[threadIdx.x] = 0u;
+    if (blockIdx.x == 0 && threadIdx.x < (unsigned)P.L) {
+        P.split_done_next[threadIdx.x] = 0u;
+        P.steal_next[threadIdx.x] = 0u;
+    }
 
     if ((int)blockIdx.x < P.C)
-        comm_cta<TN>(P, ring, ctl, aux, (int)blockIdx.x);
-    else
+        comm_cta<TN>(P, ring, ctl, aux, (int)blockIdx.x, false);
+    else {
         compute_cta<TN>(P, ring, ctl, aux, (int)blockIdx.x - P.C);
+        // out of GEMM tiles: help with the communication that is left (all TMA and TMEM traffic is over)
+        if (P.drain_help && P.mode == MOE_MODE_FUSED && !ctl->abort) comm_cta<TN>(P, ring, ctl, aux, 0, true);
+    }
 }
 
 // Pair kernel: launched with clusters of two CTAs.  Communication CTAs are single CTAs (blockIdx < C);
@@ -1126,13 +1192,18 @@ moe_gemm2_combine_pair_kernel(const __grid_constant__ FusedParams P)
     Control *ctl = reinterpret_cast<Control *>(ring + kStageBytesTotal);
     uint8_t *aux = reinterpret_cast<uint8_t *>(ring + kStageBytesTotal + ((sizeof(Control) + 127) & ~(size_t)127));
 
-    if (blockIdx.x == 0 && threadIdx.x < (unsigned)P.L) P.split_done_next[threadIdx.x] = 0u;
+    if (blockIdx.x == 0 && threadIdx.x < (unsigned)P.L) {
+        P.split_done_next[threadIdx.x] = 0u;
+        P.steal_next[threadIdx.x] = 0u;
+    }
 
     const int c_even = (P.C + 1) & ~1;
     if ((int)blockIdx.x < P.C)
-        comm_cta<256>(P, ring, ctl, aux, (int)blockIdx.x);
-    else if ((int)blockIdx.x >= c_even)
+        comm_cta<256>(P, ring, ctl, aux, (int)blockIdx.x, false);
+    else if ((int)blockIdx.x >= c_even) {
         compute_cta_pair(P, ring, ctl, aux, ((int)blockIdx.x - c_even) >> 1);
+        if (P.drain_help && P.mode == MOE_MODE_FUSED && !ctl->abort) comm_cta<256>(P, ring, ctl, aux, 0, true);
+    }
 }
 
 }  // namespace

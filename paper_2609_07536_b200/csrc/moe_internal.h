@@ -37,6 +37,9 @@ struct alignas(64) FusedParams {
     uint32_t *flags;               // [L * W_comp] readiness per global tile (== epoch when ready)
     uint32_t *split_done;          // [L] tiles finished per split (this launch)
     uint32_t *split_done_next;     // [L] counters of the next launch, zeroed by this one
+    uint32_t *steal;               // [L] communication tiles handed to helper CTAs so far (this launch)
+    uint32_t *steal_next;          // [L] ... of the next launch, zeroed by this one
+    uint32_t *claims;              // [L * comm_tiles] == epoch once a CTA has taken the tile
     uint32_t *status;              // 4 words
     void *out[MOE_MAX_EP];
     unsigned long long wait_ns;
@@ -46,6 +49,7 @@ struct alignas(64) FusedParams {
     int32_t C, P, mode, withhold;
     int32_t tok_blk, tok_tiles_per_rank, comm_cols, comm_tiles;
     int32_t num_kb, last_ksteps;
+    int32_t drain_help;                 // compute CTAs serve communication tiles once their GEMM tiles are done
     int32_t flag_parts;                 // readiness flags per tile: 1, or 2 for a CTA-pair tile
     int32_t Q, slab_cols, slab_shift;   // Q = k_tot * TP rows per unit; slab_cols = 1 << slab_shift
     uint32_t epoch;

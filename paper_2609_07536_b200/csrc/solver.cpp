@@ -30,7 +30,7 @@ struct Candidate {
 
 // One candidate.  32-bit divisions when every dividend fits (the common case), else 64-bit.
 inline bool evaluate(int32_t C, int64_t Wc, int64_t Wm, int32_t L, int32_t G, int32_t o_comp,
-                     int32_t o_comm, int32_t slot_sms, int64_t rho_q, bool small, Candidate *out)
+                     int32_t o_comm, int32_t slot_sms, int64_t rho_q, bool small, bool drain_help, Candidate *out)
 {
     const int32_t R = (C + o_comm - 1) / o_comm;
     // Eq. 3, with a compute slot that may span several SMs (a CTA pair): only whole slots count
@@ -38,7 +38,27 @@ inline bool evaluate(int32_t C, int64_t Wc, int64_t Wm, int32_t L, int32_t G, in
     if (P <= 0) return false;
     int64_t F = 0;
     int64_t V_comp;
-    if (small) {
+    if (drain_help) {
+        // Extension (not in the paper): once the last compute wave is over, the compute CTAs serve
+        // communication tiles too.  Splits 0..L-2 follow Eq. 11; the tiles still queued at A_{L-1}
+        // (whole waves of C) plus the last split's W_comm are served by C + H workers, H = the CTAs
+        // that were computing.
+        const int64_t v_comm = ceil_div64(Wm, C);
+        const int64_t q = rho_q * v_comm;
+        for (int32_t s = 0; s + 1 < L; ++s) {
+            const int64_t A = ceil_div64((int64_t)(s + 1) * Wc, P) << kRhoShift;
+            F = (A > F ? A : F) + q;
+        }
+        const int64_t A_last = ceil_div64((int64_t)L * Wc, P) << kRhoShift;
+        int64_t backlog = 0;
+        if (F > A_last && rho_q > 0) {
+            backlog = ceil_div64(F - A_last, rho_q) * C;
+            if (backlog > (int64_t)(L - 1) * Wm) backlog = (int64_t)(L - 1) * Wm;
+        }
+        const int64_t workers = (int64_t)C + P * slot_sms / o_comp;
+        F = A_last + rho_q * ceil_div64(backlog + Wm, workers);
+        V_comp = ceil_div64(Wc, P);
+    } else if (small) {
         const uint32_t p = (uint32_t)P, wc = (uint32_t)Wc;
         const uint32_t v_comm = ceil_div32((uint32_t)Wm, (uint32_t)C);
         const int64_t q = rho_q * (int64_t)v_comm;
@@ -133,11 +153,11 @@ extern "C" int32_t plan_partition(const int32_t *routed_tile_counts, int32_t n_e
     if (limits->force_comm_ctas > 0 || limits->selector_off) {
         const int32_t C = limits->force_comm_ctas > 0 ? limits->force_comm_ctas : limits->default_C;
         if (C < 1) return MOE_ERR_PLAN_INFEASIBLE;
-        have = evaluate(C, Wc, Wm, L, G, o_comp, o_comm, slot, rho_q, small, &best);
+        have = evaluate(C, Wc, Wm, L, G, o_comp, o_comm, slot, rho_q, small, limits->drain_help != 0, &best);
     } else {
         for (int32_t C = 1; C <= limits->C_max; ++C) {
             Candidate c;
-            if (!evaluate(C, Wc, Wm, L, G, o_comp, o_comm, slot, rho_q, small, &c)) break;  // P only falls
+            if (!evaluate(C, Wc, Wm, L, G, o_comp, o_comm, slot, rho_q, small, limits->drain_help != 0, &c)) break;  // P only falls
             // ascending C: a strict improvement of (T, Delta) is needed to replace the incumbent
             if (!have || c.T_q < best.T_q || (c.T_q == best.T_q && c.delta < best.delta)) {
                 best = c;
@@ -157,6 +177,8 @@ extern "C" int32_t plan_partition(const int32_t *routed_tile_counts, int32_t n_e
     out->rho_q = rho_q;
     out->mode = MOE_MODE_FUSED;
     out->debug_withhold_tile = -1;
+    out->drain_help = limits->drain_help != 0 ? 1 : 0;
+    out->reserved = 0;
     return MOE_OK;
 }
 

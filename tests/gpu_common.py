@@ -53,7 +53,7 @@ def build_routing(w: wl.Workload, topk_idx: np.ndarray, ws: B.Workspace = None):
 
 
 def run_layer(w: wl.Workload, topk_idx, topk_w, x, W2, force_C=0, mode=B.MOE_MODE_FUSED, ws=None,
-              withhold=-1, check_status=True, P_override=None):
+              withhold=-1, check_status=True, P_override=None, drain_help=None):
     """x, W2: bf16 torch tensors (CPU or CUDA).  Returns (list of EP outputs on CPU as float32,
     plan, workspace, S)."""
     h = handle()
@@ -61,6 +61,8 @@ def run_layer(w: wl.Workload, topk_idx, topk_w, x, W2, force_C=0, mode=B.MOE_MOD
     ws, idx_dev, S = build_routing(w, topk_idx, ws)
     occ, lim, rho = B.moe_query_occupancy(h, w.tile_m, w.tile_n)
     lim.force_comm_ctas = force_C
+    if drain_help is not None:
+        lim.drain_help = int(drain_help)
     tiles = ws.tile_counts[:shape.E_tot].tolist()
     plan = B.plan_partition(tiles, occ, lim, shape, rho)
     plan.mode = mode

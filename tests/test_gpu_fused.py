@@ -140,6 +140,39 @@ def test_bitwise_identical_across_C_P_and_runs():
                 assert np.array_equal(a, b), (C, P, rep)
 
 
+def test_drain_help_and_tile_families_change_nothing_but_time():
+    # compute CTAs helping with the communication tail, or another GEMM tile family, may only change
+    # who writes a value and when: the bits must be the same
+    w = replace(wl.GRANITE, name="dh", T=2000, L=2)
+    idx, wt, _ = wl.make_routing(w)
+    x, W2 = wl.make_data(w)
+    base = None
+    for tile in ((128, 256), (128, 128), (256, 256)):
+        for dh in (0, 1):
+            for C in (0, 1, 9, 60):
+                wt_ = replace(w, tile_m=tile[0], tile_n=tile[1])
+                outs, plan, ws, S, st = G.run_layer(wt_, idx, wt, x, W2, force_C=C, drain_help=dh)
+                assert st.code == 0 and plan.drain_help == dh
+                bits = [torch.from_numpy(o).bfloat16().view(torch.int16).numpy() for o in outs]
+                if base is None:
+                    base = bits
+                for a, b in zip(base, bits):
+                    assert np.array_equal(a, b), (tile, dh, C)
+    expect, _ = _oracle_tokens(w, idx, wt, x, W2)
+    got = np.concatenate([o[:len(G.tokens_of_rank(w.T, w.EP, d))] for d, o in enumerate(outs)])
+    assert np.max(np.abs(got - expect)) <= G.tolerance(expect)
+
+
+def test_pair_tiles_against_oracle():
+    for kw in (dict(T=777, E=5, k=2, H=1536, I=512, TP=2, EP=3, L=4),      # partial n-tile at the split end
+               dict(T=300, E=3, k=1, H=256, I=64, TP=1, EP=1, L=1),         # m-tiles with an empty second half
+               dict(T=1030, E=70, k=2, H=512, I=256, TP=2, EP=8, L=2)):     # empty experts
+        base = dict(name="pair", routing_seed=3, data_seed=4, tile_m=256, tile_n=256)
+        base.update(kw)
+        _check_against_oracle(replace(wl.TINY, **base))
+    _check_against_oracle(replace(wl.DSV2L, tile_m=256, tile_n=256), n_random=96)
+
+
 def test_ep_concat_invariance_and_tp_within_tolerance():
     w = replace(wl.QWEN, name="ep", T=1200, E=16)
     idx, wt, _ = wl.make_routing(w)

@@ -27,7 +27,7 @@ def _oracle_plan(tiles, shape, occ, lim, rho):
     rho_q = sr.quantise_rho(r)
     sel = sr.select(Wc, Wm, shape.L, lim.G, occ.o_comp, occ.o_comm, lim.C_max, rho_q,
                     force_comm_ctas=lim.force_comm_ctas, selector_off=bool(lim.selector_off),
-                    default_C=lim.default_C, slot_sms=occ.comp_slot_sms)
+                    default_C=lim.default_C, slot_sms=occ.comp_slot_sms, drain_help=bool(lim.drain_help))
     sel["rho_q"] = rho_q
     return sel
 
@@ -36,7 +36,7 @@ def _same(plan, sel):
     assert (plan.comm_ctas, plan.R, plan.P) == (sel["comm_ctas"], sel["R"], sel["P"])
     assert (plan.W_comp, plan.W_comm, plan.delta) == (sel["W_comp"], sel["W_comm"], sel["delta"])
     assert plan.pred_T_q == sel["T_q"] and plan.rho_q == sel["rho_q"]
-    assert plan.mode == B.MOE_MODE_FUSED and plan.debug_withhold_tile == -1
+    assert plan.mode == B.MOE_MODE_FUSED and plan.debug_withhold_tile == -1 and plan.reserved == 0
 
 
 def _rand_inputs(rng):
@@ -49,7 +49,7 @@ def _rand_inputs(rng):
                          rng.choice([1, 2, 4, 8]), rng.choice([1, 2, 4, 8]))
     occ = B.moe_occupancy(tile_m, tile_n, rng.choice([64, 128]), rng.choice([512, 1024]),
                           rng.choice([1, 2]), rng.choice([1, 2, 4]), rng.choice([1, 1, 2]))
-    lim = B.moe_sm_limits(rng.choice([4, 108, 148]), rng.randint(1, 160), 0, 0, 3)
+    lim = B.moe_sm_limits(rng.choice([4, 108, 148]), rng.randint(1, 160), 0, 0, 3, rng.choice([0, 0, 1]))
     rho = B.moe_rho(rng.uniform(0.05, 30.0), rng.choice([352, 704]), 128, rng.choice([128, 256]),
                     rng.choice([2, 4]), 17, 1024, rng.choice([B.MOE_RHO_PAPER, B.MOE_RHO_LOCAL]))
     tiles = [rng.randint(0, 40) for _ in range(E)]
@@ -158,6 +158,29 @@ def test_pair_slots():
     lim = B.moe_sm_limits(148, 74, 0, 0, 3)
     plan = B.plan_partition([8] * 66, occ, lim, shape, rho)
     assert plan.comm_ctas % 2 == 0           # an odd C never beats the even one below it by the model
+
+
+def test_drain_help_model():
+    # the extension: after the last compute wave every SM serves communication tiles
+    shape = B.make_shape(16384, 2048, 1408, 66, 8, 2, 2, 4)
+    occ = B.moe_occupancy(128, 256, 128, 1024, 1, 1, 1)
+    rho = B.moe_rho(9.0, 704, 128, 256, 2, 17, 1024, B.MOE_RHO_LOCAL)
+    tiles = [17] * 66
+    picks = {}
+    for dh in (0, 1):
+        lim = B.moe_sm_limits(148, 74, 0, 0, 3, dh)
+        plan = B.plan_partition(tiles, occ, lim, shape, rho)
+        _same(plan, _oracle_plan(tiles, shape, occ, lim, rho))
+        assert plan.drain_help == dh
+        picks[dh] = plan
+    # helpers shorten the tail, so the model never predicts a longer makespan and never asks for more C
+    assert picks[1].pred_T_q <= picks[0].pred_T_q and picks[1].comm_ctas <= picks[0].comm_ctas
+    # closed form for L = 1: T = A_0 + rho * ceil(W_comm / (C + P))
+    shape1 = B.make_shape(4096, 2048, 1408, 66, 8, 2, 1, 1)
+    lim = B.moe_sm_limits(148, 74, 10, 0, 3, 1)
+    plan = B.plan_partition(tiles, occ, lim, shape1, rho)
+    A0 = -(-plan.W_comp // plan.P)
+    assert plan.pred_T_q == (A0 << 20) + plan.rho_q * -(-plan.W_comm // (10 + plan.P))
 
 
 def test_solver_cost_is_small():
