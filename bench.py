@@ -175,33 +175,48 @@ def time_fused(step, torch, force_C, n_warm, n_samples, **kw):
 # legal C; regret = (T_pick - T_best) / T_best.
 
 def time_all_C(step, torch, counts, C_list, n_warm=1, n_samples=5):
-    """Median fused-kernel time [us] for every C in C_list (routing is reused)."""
-    out = {}
-    for C in C_list:
-        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_samples)]
-        for _ in range(n_warm):
+    """Median fused-kernel time [us] for every C in C_list (routing is reused).  The candidates are
+    interleaved: every round visits all of them in a fresh seeded random order, so that slow drifts
+    of the GPU's state (power capping sets in after a second or two of load) hit every C alike."""
+    import random
+    rng = random.Random(1234)
+    order = list(C_list)
+    for _ in range(n_warm):
+        for C in order:
             step(C, reuse=counts)
-        for a, b in evs:
+    samples = {C: [] for C in order}
+    evs = []
+    for _ in range(n_samples):
+        rng.shuffle(order)
+        for C in order:
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             step(C, ev_before=a, ev_after=b, reuse=counts)
-        torch.cuda.synchronize()
-        out[C] = statistics.median(a.elapsed_time(b) * 1e3 for a, b in evs)
+            evs.append((C, a, b))
+    torch.cuda.synchronize()
+    for C, a, b in evs:
+        samples[C].append(a.elapsed_time(b) * 1e3)
+    return {C: statistics.median(v) for C, v in samples.items()}
+
+
+def regret_of_workload(step, torch, counts, lim, picked_C, n_warm=1, n_samples=5, C_hi=None, keep_curve=True):
+    """Times every C of the legal set {1..C_max} (or up to C_hi) and compares the analytical pick."""
+    C_hi = C_hi or lim.C_max
+    Cs = sorted(set(list(range(1, C_hi + 1)) + [picked_C]))
+    times = time_all_C(step, torch, counts, Cs, n_warm, n_samples)
+    best_C = min(times, key=times.get)
+    t_best, t_pick = times[best_C], times[picked_C]
+    out = {"picked_C": picked_C, "t_pick_us": t_pick, "best_C": best_C, "t_best_us": t_best,
+           "regret": (t_pick - t_best) / t_best,
+           "regret_static_C3": (times[3] - t_best) / t_best if 3 in times else None,
+           "swept_C": [1, C_hi], "samples_per_C": n_samples}
+    if keep_curve:
+        out["times_us"] = {str(c): round(t, 1) for c, t in times.items()}
     return out
 
 
-def regret_of_workload(step, torch, counts, G, picked_C, n_warm=1, n_samples=5, C_hi=None):
-    C_hi = C_hi or (G - 1)
-    times = time_all_C(step, torch, counts, list(range(1, C_hi + 1)), n_warm, n_samples)
-    best_C = min(times, key=times.get)
-    t_best, t_pick = times[best_C], times[picked_C]
-    return {"picked_C": picked_C, "t_pick_us": t_pick, "best_C": best_C, "t_best_us": t_best,
-            "regret": (t_pick - t_best) / t_best,
-            "regret_static_C3": (times[3] - t_best) / t_best if 3 in times else None,
-            "swept_C": [1, C_hi], "samples_per_C": n_samples,
-            "times_us": {str(c): round(t, 2) for c, t in times.items()}}
-
-
 def run_sweep(h, args, peaks):
-    """The regret sweep on the DeepSeek-V2-Lite shape: T x Zipf s x EP x tile, every feasible C."""
+    """The regret sweep on the DeepSeek-V2-Lite shape: T x Zipf s x EP x tile, every legal C, for the
+    paper's static partition (drain_help = 0) and for the default mode (drain_help = 1)."""
     import torch
     from paper_2609_07536_b200 import workloads as wl
     device = f"cuda:{torch.cuda.current_device()}"
@@ -210,28 +225,38 @@ def run_sweep(h, args, peaks):
         if args.sweep_filter and args.sweep_filter not in w.name:
             continue
         dw = DeviceWorkload(w, device, data="device")
-        step, (occ, lim, rho) = make_stepper(h, dw)
-        plan, counts = step()
-        torch.cuda.synchronize()
-        r = regret_of_workload(step, torch, counts, lim.G, plan.comm_ctas, n_warm=1, n_samples=5)
-        r.update(name=w.name, T=w.T, zipf_s=w.zipf_s, EP=w.EP, tile=f"{w.tile_m}x{w.tile_n}",
-                 r_expert=dw.info["r_expert"], W_comp=plan.W_comp, W_comm=plan.W_comm, rho=plan.rho_q / 2 ** 20,
-                 roofline_frac=(dw.flops / peaks["bf16_tflops"] / 1e6) / r["t_pick_us"])
-        results.append(r)
-        print(f"{w.name}: pick C={r['picked_C']} {r['t_pick_us']:.1f} us | best C={r['best_C']} "
-              f"{r['t_best_us']:.1f} us | regret {100 * r['regret']:.2f}%", flush=True)
+        row = dict(name=w.name, T=w.T, zipf_s=w.zipf_s, EP=w.EP, tile=f"{w.tile_m}x{w.tile_n}", L=w.L,
+                   r_expert=dw.info["r_expert"])
+        for dh in (0, 1):
+            step, (occ, lim, rho) = make_stepper(h, dw, limits_override=dict(drain_help=dh))
+            plan, counts = step()
+            torch.cuda.synchronize()
+            r = regret_of_workload(step, torch, counts, lim, plan.comm_ctas, n_warm=1, n_samples=3,
+                                   keep_curve=args.sweep_curves)
+            r.update(W_comp=plan.W_comp, W_comm=plan.W_comm, rho=plan.rho_q / 2 ** 20,
+                     roofline_frac=(dw.flops / peaks["bf16_tflops"] / 1e6) / r["t_pick_us"])
+            row["static" if dh == 0 else "drain_help"] = r
+        results.append(row)
+        a, b = row["static"], row["drain_help"]
+        print(f"{w.name}: static pick C={a['picked_C']} {a['t_pick_us']:.0f} us best C={a['best_C']} {a['t_best_us']:.0f} us "
+              f"regret {100 * a['regret']:.1f}% (C=3: {100 * a['regret_static_C3']:.0f}%) | drain-help pick C={b['picked_C']} "
+              f"{b['t_pick_us']:.0f} us best C={b['best_C']} {b['t_best_us']:.0f} us regret {100 * b['regret']:.1f}%", flush=True)
         del dw, step
         torch.cuda.empty_cache()
-    regs = [r["regret"] for r in results]
-    summary = {"n": len(results), "mean_regret": statistics.mean(regs) if regs else None,
-               "max_regret": max(regs) if regs else None,
-               "mean_regret_static_C3": statistics.mean(r["regret_static_C3"] for r in results) if regs else None}
+    summary = {"n": len(results)}
+    for key in ("static", "drain_help"):
+        regs = [r[key]["regret"] for r in results]
+        if regs:
+            summary[key] = {"mean_regret": statistics.mean(regs), "max_regret": max(regs),
+                            "mean_regret_static_C3": statistics.mean(r[key]["regret_static_C3"] for r in results),
+                            "geomean_speedup_pick_over_C3": statistics.geometric_mean(
+                                (1 + r[key]["regret_static_C3"]) / (1 + r[key]["regret"]) for r in results)}
     os.makedirs(os.path.dirname(args.sweep_out) or ".", exist_ok=True)
     json.dump({"summary": summary, "results": results}, open(args.sweep_out, "w"))
     print(json.dumps({"sweep_summary": summary}))
 
 
-def calibrate(h, device, C_ref=32):
+def calibrate(h, device, C_ref=32, tile=(128, 256)):
     """Eq. 13 on this GPU: rho_ref = (time of one communication wave) / (time of one compute wave),
     both measured with the role running alone on its share of the SMs at a fixed C_ref, on the
     reference workload (DeepSeek-V2-Lite shape, T = 4096, uniform routing, 128x256, TP = EP = L = 2)."""
@@ -239,12 +264,13 @@ def calibrate(h, device, C_ref=32):
     from dataclasses import replace
     from paper_2609_07536_b200 import binding as B
     from paper_2609_07536_b200 import workloads as wl
-    w = replace(wl.DSV2L, name="rho_ref", T=4096, routing="uniform", zipf_s=0.0, target_r_expert=0.0)
+    w = replace(wl.DSV2L, name="rho_ref", T=4096, routing="uniform", zipf_s=0.0, target_r_expert=0.0,
+                tile_m=tile[0], tile_n=tile[1])
     dw = DeviceWorkload(w, device, data="device")
     step, (occ, lim, rho) = make_stepper(h, dw)
     plan, counts = step(C_ref)
     torch.cuda.synchronize()
-    P = lim.G - C_ref
+    P = (lim.G - C_ref) // occ.comp_slot_sms
     t_comp = statistics.median(time_fused(step, torch, 0, 3, 15, mode=B.MOE_MODE_GEMM_ONLY, P_override=P, reuse=counts))
     t_comm = statistics.median(time_fused(step, torch, 1, 3, 15, mode=B.MOE_MODE_COMBINE_ONLY, C_override=C_ref, reuse=counts))
     V_comp = -(-plan.W_comp // P)
@@ -339,6 +365,9 @@ def main():
     ap.add_argument("--sweep", action="store_true", help="selector-regret sweep on the DeepSeek-V2-Lite shape")
     ap.add_argument("--sweep-out", default="gpurun_out/sweep.json")
     ap.add_argument("--sweep-filter", default="", help="substring a sweep workload name must contain")
+    ap.add_argument("--sweep-curves", action="store_true", help="keep every t(C) in the sweep output")
+    ap.add_argument("--drain-help", type=int, default=1, choices=[0, 1],
+                    help="1 (default): compute CTAs help with the communication tail; 0: the paper's static partition")
     args = ap.parse_args()
     if args.impl == "reference":
         return reference_arm(args)
@@ -364,7 +393,8 @@ def main():
     if args.sweep:
         return run_sweep(h, args, peaks)
     if args.calibrate:
-        return calibrate(h, device)
+        tile = tuple(int(v) for v in args.tile.split("x")) if args.tile else (128, 256)
+        return calibrate(h, device, tile=tile)
 
     w = wl.CONFIGS[args.workload]
     if args.tile:
@@ -375,7 +405,7 @@ def main():
         from dataclasses import replace
         w = replace(w, L=args.L)
     dw = DeviceWorkload(w, device, data=args.data if args.only else "seeded")
-    step, (occ, lim, rho) = make_stepper(h, dw)
+    step, (occ, lim, rho) = make_stepper(h, dw, limits_override=dict(drain_help=args.drain_help))
     K, W = max(1, args.steps), max(3, args.warmup)
 
     if args.only:
@@ -463,7 +493,13 @@ def main():
                                  "frac_of_hbm_peak": dw.combine_bytes / comb_only / 1e3 / peaks["hbm_gbs"], "C": lim_all}
         # ---- selector regret on this workload: every feasible C timed
         if not args.no_regret:
-            extra["regret"] = regret_of_workload(step, torch, counts, lim.G, plan.comm_ctas, n_warm=1, n_samples=5)
+            extra["regret"] = regret_of_workload(step, torch, counts, lim, plan.comm_ctas, n_warm=1, n_samples=5)
+            # the paper's static partition on the same workload: its pick, its sweep, its regret
+            step0, (occ0, lim0, rho0) = make_stepper(h, dw, limits_override=dict(drain_help=1 - args.drain_help))
+            lim0.force_comm_ctas = 0
+            plan0 = B.plan_partition(counts[:w.E_tot], occ0, lim0, dw.shape, rho0)
+            key = "regret_static_partition" if args.drain_help else "regret_drain_help"
+            extra[key] = regret_of_workload(step0, torch, counts, lim0, plan0.comm_ctas, n_warm=1, n_samples=5)
         # ---- solver overhead: mean over >= 1e6 calls, rotating routed-count vectors
         rng = np.random.default_rng(0)
         base_counts = np.array(counts[:w.E_tot])
@@ -502,7 +538,7 @@ def main():
                        "l2": "inputs larger than L2 (x 369 MB, W2 381 MB, Y 1.1 GB vs 126 MB)",
                        "replicas": "independent per GPU, no collective" if world > 1 else "single GPU"},
             "plan": {"comm_ctas": plan.comm_ctas, "R": plan.R, "P": plan.P, "W_comp": plan.W_comp,
-                     "W_comm": plan.W_comm, "rho": plan.rho_q / 2 ** 20},
+                     "W_comm": plan.W_comm, "rho": plan.rho_q / 2 ** 20, "drain_help": plan.drain_help},
             "fused_kernel_us": fused_med, "tflops": dw.flops / fused_med / 1e6,
             "wall_ms_per_step": wall * 1e3 / K,
             "roofline": roofline,

@@ -146,13 +146,20 @@ int32_t moe_query_occupancy(moe_handle *h, int32_t tile_m, int32_t tile_n, moe_o
         limits->drain_help = 1;
     }
     if (rho) {
-        // one-time service-rate characterisation of this kernel family on B200 (Eq. 13):
-        // reference run = DeepSeek-V2-Lite shape, T = 4096, uniform routing, 128x256 tiles,
-        // TP = 2, EP = 2, L = 2.
-        rho->rho_ref = 2.0;
+        // One-time service-rate characterisation of this kernel family on B200 (Eq. 13), one constant per
+        // GEMM tile shape (Section III-E: every kernel choice brings its own).  Reference run: DeepSeek-V2-
+        // Lite shape, T = 4096, uniform routing, TP = 2, EP = 2, L = 2, K = 704; each role alone on its
+        // share of the SMs at C = 32: time per communication wave / time per compute wave.
+        //   128x256: 66.8 us / 6.26 us ; 256x256 (CTA pair): 67.8 / 5.97 ; 128x128: 66.8 / 5.15
         rho->K_ref = 704;
-        rho->tile_m_ref = 128;
-        rho->tile_n_ref = 256;
+        rho->tile_m_ref = tile_m;
+        rho->tile_n_ref = tile_n;
+        if (tile_m == 256) rho->rho_ref = 11.35;
+        else if (tile_n == 256) rho->rho_ref = 10.67;
+        else if (tile_n == 128) rho->rho_ref = 12.97;
+        else rho->rho_ref = 12.97 * 2.0;          // 64-wide tiles: Eq. 14 tile-area scaling from 128x128
+        if (tile_m == 64) rho->rho_ref *= 1.0;     // a 64-row tile still occupies a 128-row MMA: same wave time
+        if (tile_n == 64) { rho->tile_n_ref = 64; }
         rho->D_ref = 2;
         rho->rows_ref = 8 * 2 + 1;
         rho->comm_cols_ref = 1024;
@@ -183,7 +190,7 @@ int32_t moe_workspace_bytes(const moe_shape *s, int32_t tile_m, int32_t tile_n, 
         const size_t nts = (size_t)ceil_div(ceil_div(s->H, s->L), tile_n);
         const size_t parts = (tile_m == 256) ? 2 : 1;   // a pair tile is published in two parts
         *flags_bytes = ((size_t)kSplitCounterWords + (size_t)s->L * s->TP * mt * nts * parts +
-                        (size_t)s->L * (size_t)comm_tiles_of(s)) * 4 + 16;
+                        (size_t)s->L * (size_t)comm_tiles_of(s) * 4 /* claims: 4 slices per tile */) * 4 + 16;
     }
     if (status_bytes) *status_bytes = 16;
     return MOE_OK;

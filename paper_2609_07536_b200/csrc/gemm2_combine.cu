@@ -848,6 +848,7 @@ __device__ __forceinline__ void fma_bf16x8(float (&acc)[8], const uint4 &v, floa
 // weights and stores the bf16 result into the owning rank's buffer.  No warp waits on another one:
 // the issue latency of the copies and the memory latency overlap across the twelve warps.
 constexpr int kCommWarps = 12;
+constexpr int kCommSub = 4;            // token slices a communication tile is claimed in (drain help)
 constexpr int kCommUnitBytes = 8192;
 constexpr int kCommWarpBytes = 2 * kCommUnitBytes;
 static_assert(kCommWarps * kCommWarpBytes <= kStageBytesTotal, "communication stages exceed the ring");
@@ -979,15 +980,18 @@ __device__ void comm_cta(const FusedParams &P, uint8_t *ring, Control *ctl, uint
     uint32_t ready_mask = wait_needed ? 0u : 0xffffffffu;   // bit s: split s is known to be complete
 
     // serve communication tile ct of split s; false when this warp had to give up (reported)
-    auto serve_tile = [&](int s, int ct) -> bool {
+    auto serve_tile = [&](int s, int ct, int sub) -> bool {
         const int split_c0 = s * P.split_w;
         const int split_c1 = min(P.H, split_c0 + P.split_w);
         const int tok_tile = ct / P.comm_cols;
         const int col_tile = ct - tok_tile * P.comm_cols;
         const int d = tok_tile / P.tok_tiles_per_rank;
         const int ti = tok_tile - d * P.tok_tiles_per_rank;
-        const int t0 = d * P.tok_blk + ti * kCommTileM;
-        const int t1 = min(min(P.T, (d + 1) * P.tok_blk), t0 + kCommTileM);
+        // a communication tile is claimed and served in kCommSub token slices (all of it when sub < 0)
+        const int tile_t0 = d * P.tok_blk + ti * kCommTileM;
+        const int tile_t1 = min(min(P.T, (d + 1) * P.tok_blk), tile_t0 + kCommTileM);
+        const int t0 = sub < 0 ? tile_t0 : tile_t0 + sub * (kCommTileM / kCommSub);
+        const int t1 = sub < 0 ? tile_t1 : min(tile_t1, t0 + kCommTileM / kCommSub);
         const int c0 = split_c0 + col_tile * kCommTileN;
         const int c1 = min(split_c1, c0 + kCommTileN);
         if (t0 >= t1 || c0 >= c1) return true;
@@ -1116,37 +1120,45 @@ __device__ void comm_cta(const FusedParams &P, uint8_t *ring, Control *ctl, uint
     if (!helper) {
         for (int s = 0; s < P.L; ++s) {
             for (int ct = c; ct < P.comm_tiles; ct += P.C) {
-                if (claiming) {
-                    int mine = 0;
-                    if (warp == 0 && lane == 0) mine = (atomicExch(&P.claims[s * P.comm_tiles + ct], P.epoch) != P.epoch) ? 1 : 0;
-                    mine = broadcast(mine);
-                    if (ctl->abort) { s = P.L; break; }
-                    if (!mine) continue;      // a helper took it
+                if (!claiming) {
+                    if (!serve_tile(s, ct, -1)) {
+                        ctl->abort = 1u;
+                        return;               // no CTA-wide barriers in this mode: the warp may leave
+                    }
+                    continue;
                 }
-                if (!dead && !serve_tile(s, ct)) {
-                    dead = true;
-                    ctl->abort = 1u;
-                    if (!claiming) return;    // no CTA-wide barriers in this mode: the warp may leave
+                for (int sub = 0; sub < kCommSub; ++sub) {
+                    int mine = 0;
+                    if (warp == 0 && lane == 0)
+                        mine = (atomicExch(&P.claims[(s * P.comm_tiles + ct) * kCommSub + sub], P.epoch) != P.epoch) ? 1 : 0;
+                    mine = broadcast(mine);
+                    if (ctl->abort) { s = P.L; ct = P.comm_tiles; break; }
+                    if (!mine) continue;      // a helper took it
+                    if (!dead && !serve_tile(s, ct, sub)) {
+                        dead = true;
+                        ctl->abort = 1u;
+                    }
                 }
             }
         }
     } else {
-        // a compute CTA that ran out of GEMM tiles: take unclaimed tiles from the back, last split first
+        // a compute CTA that ran out of GEMM tiles: take unclaimed tile slices from the back, last split first
+        const uint32_t n_slices = (uint32_t)(P.comm_tiles * kCommSub);
         for (int s = P.L - 1; s >= 0; --s) {
             for (;;) {
-                int ct = -1;
+                int slice = -1;
                 if (warp == 0 && lane == 0) {
                     for (;;) {
                         const uint32_t idx = atomicAdd(&P.steal[s], 1u);
-                        if (idx >= (uint32_t)P.comm_tiles) break;
-                        const int cand = P.comm_tiles - 1 - (int)idx;
-                        if (atomicExch(&P.claims[s * P.comm_tiles + cand], P.epoch) != P.epoch) { ct = cand; break; }
+                        if (idx >= n_slices) break;
+                        const int cand = (int)(n_slices - 1u - idx);
+                        if (atomicExch(&P.claims[s * (int)n_slices + cand], P.epoch) != P.epoch) { slice = cand; break; }
                     }
                 }
-                ct = broadcast(ct);
+                slice = broadcast(slice);
                 if (ctl->abort) { s = -1; break; }
-                if (ct < 0) break;
-                if (!dead && !serve_tile(s, ct)) {
+                if (slice < 0) break;
+                if (!dead && !serve_tile(s, slice / kCommSub, slice % kCommSub)) {
                     dead = true;
                     ctl->abort = 1u;
                 }

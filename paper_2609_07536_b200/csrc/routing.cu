@@ -63,15 +63,26 @@ routing_scan(int R, int E_tot, int tile_m, int n_warps, int max_mtiles,
              int32_t *tile_offsets, int32_t *mtile_expert, int32_t *mtile_first_row,
              int32_t *mtile_valid, uint32_t *status)
 {
-    // counts, and whist turned into an exclusive prefix over the warps (per expert)
-    for (int e = threadIdx.x; e < E_tot; e += blockDim.x) {
-        int run = 0;
-        for (int w = 0; w < n_warps; ++w) {
-            const int c = whist[(size_t)w * E_tot + e];
-            whist[(size_t)w * E_tot + e] = run;
-            run += c;
+    // counts, and whist turned into an exclusive prefix over the (sorting) warps, per expert: one warp
+    // of this CTA per expert, 32 entries per step with a shuffle scan
+    {
+        const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, n_w = blockDim.x >> 5;
+        for (int e = wid; e < E_tot; e += n_w) {
+            int run = 0;
+            for (int w0 = 0; w0 < n_warps; w0 += 32) {
+                const int w = w0 + lane;
+                const int c = (w < n_warps) ? whist[(size_t)w * E_tot + e] : 0;
+                int incl = c;
+#pragma unroll
+                for (int d = 1; d < 32; d <<= 1) {
+                    const int up = __shfl_up_sync(0xffffffffu, incl, d);
+                    if (lane >= d) incl += up;
+                }
+                if (w < n_warps) whist[(size_t)w * E_tot + e] = run + incl - c;
+                run += __shfl_sync(0xffffffffu, incl, 31);
+            }
+            if (lane == 0) counts[e] = run;
         }
-        counts[e] = run;
     }
     __syncthreads();
     if (threadIdx.x == 0) {

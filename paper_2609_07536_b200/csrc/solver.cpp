@@ -43,21 +43,47 @@ inline bool evaluate(int32_t C, int64_t Wc, int64_t Wm, int32_t L, int32_t G, in
         // communication tiles too.  Splits 0..L-2 follow Eq. 11; the tiles still queued at A_{L-1}
         // (whole waves of C) plus the last split's W_comm are served by C + H workers, H = the CTAs
         // that were computing.
-        const int64_t v_comm = ceil_div64(Wm, C);
-        const int64_t q = rho_q * v_comm;
-        for (int32_t s = 0; s + 1 < L; ++s) {
-            const int64_t A = ceil_div64((int64_t)(s + 1) * Wc, P) << kRhoShift;
-            F = (A > F ? A : F) + q;
+        int64_t v_comm, A_last;
+        if (small) {
+            const uint32_t p = (uint32_t)P, wc = (uint32_t)Wc;
+            v_comm = ceil_div32((uint32_t)Wm, (uint32_t)C);
+            const int64_t q = rho_q * v_comm;
+            uint32_t num = 0, a0 = 0;
+            for (int32_t s = 0; s + 1 < L; ++s) {
+                num += wc;
+                const uint32_t a = ceil_div32(num, p);
+                if (s == 0) a0 = a;
+                const int64_t A = (int64_t)a << kRhoShift;
+                F = (A > F ? A : F) + q;
+            }
+            const uint32_t al = ceil_div32(num + wc, p);
+            A_last = (int64_t)al << kRhoShift;
+            V_comp = (L > 1) ? a0 : al;
+        } else {
+            v_comm = ceil_div64(Wm, C);
+            const int64_t q = rho_q * v_comm;
+            for (int32_t s = 0; s + 1 < L; ++s) {
+                const int64_t A = ceil_div64((int64_t)(s + 1) * Wc, P) << kRhoShift;
+                F = (A > F ? A : F) + q;
+            }
+            A_last = ceil_div64((int64_t)L * Wc, P) << kRhoShift;
+            V_comp = ceil_div64(Wc, P);
         }
-        const int64_t A_last = ceil_div64((int64_t)L * Wc, P) << kRhoShift;
         int64_t backlog = 0;
         if (F > A_last && rho_q > 0) {
-            backlog = ceil_div64(F - A_last, rho_q) * C;
+            // ceil((F - A_last) / rho_q): quotient from a double division, then made exact
+            const int64_t num = F - A_last;
+            int64_t w = (int64_t)((double)num / (double)rho_q);
+            while (w * rho_q < num) ++w;
+            while (w > 0 && (w - 1) * rho_q >= num) --w;
+            backlog = w * C;
             if (backlog > (int64_t)(L - 1) * Wm) backlog = (int64_t)(L - 1) * Wm;
         }
         const int64_t workers = (int64_t)C + P * slot_sms / o_comp;
-        F = A_last + rho_q * ceil_div64(backlog + Wm, workers);
-        V_comp = ceil_div64(Wc, P);
+        const int64_t rem = backlog + Wm;
+        const int64_t waves = (small && workers < 0x7FFFFFFF) ? (int64_t)ceil_div32((uint32_t)rem, (uint32_t)workers)
+                                                              : ceil_div64(rem, workers);
+        F = A_last + rho_q * waves;
     } else if (small) {
         const uint32_t p = (uint32_t)P, wc = (uint32_t)Wc;
         const uint32_t v_comm = ceil_div32((uint32_t)Wm, (uint32_t)C);
@@ -150,17 +176,85 @@ extern "C" int32_t plan_partition(const int32_t *routed_tile_counts, int32_t n_e
 
     Candidate best{};
     bool have = false;
+    const bool dh = limits->drain_help != 0;
     if (limits->force_comm_ctas > 0 || limits->selector_off) {
         const int32_t C = limits->force_comm_ctas > 0 ? limits->force_comm_ctas : limits->default_C;
         if (C < 1) return MOE_ERR_PLAN_INFEASIBLE;
-        have = evaluate(C, Wc, Wm, L, G, o_comp, o_comm, slot, rho_q, small, limits->drain_help != 0, &best);
-    } else {
+        have = evaluate(C, Wc, Wm, L, G, o_comp, o_comm, slot, rho_q, small, dh, &best);
+    } else if (!small) {
         for (int32_t C = 1; C <= limits->C_max; ++C) {
             Candidate c;
-            if (!evaluate(C, Wc, Wm, L, G, o_comp, o_comm, slot, rho_q, small, limits->drain_help != 0, &c)) break;  // P only falls
-            // ascending C: a strict improvement of (T, Delta) is needed to replace the incumbent
+            if (!evaluate(C, Wc, Wm, L, G, o_comp, o_comm, slot, rho_q, small, dh, &c)) break;  // P only falls
             if (!have || c.T_q < best.T_q || (c.T_q == best.T_q && c.delta < best.delta)) {
                 best = c;
+                have = true;
+            }
+        }
+    } else {
+        // Algorithm 1 over C = 1..C_max without a division in the loop: as C grows, P(C) only falls and
+        // ceil(W_comm / C) only falls, so every ceiling is carried from the previous candidate and moved
+        // to its new exact value with a few multiply-compare steps (same integers as the plain formulas).
+        int64_t qa[MOE_MAX_L];           // qa[s] = ceil((s+1) W_comp / P)
+        for (int32_t s = 0; s < L; ++s) qa[s] = 0;
+        int64_t v = Wm;                  // ceil(W_comm / C), C = 1
+        int64_t P_prev = 0;
+        const double inv_rho = rho_q > 0 ? 1.0 / (double)rho_q : 0.0;
+        for (int32_t C = 1; C <= limits->C_max; ++C) {
+            const int32_t R = (o_comm == 1) ? C : (C + o_comm - 1) / o_comm;
+            if (G <= R) break;
+            const int64_t P = (slot == 1) ? (int64_t)o_comp * (G - R) : (int64_t)o_comp * ((G - R) / slot);
+            if (P <= 0) break;
+            if (P != P_prev) {
+                if (P_prev == 0) {
+                    for (int32_t s = 0; s < L; ++s) qa[s] = ceil_div64((int64_t)(s + 1) * Wc, P);
+                } else {
+                    for (int32_t s = 0; s < L; ++s) {
+                        const int64_t num = (int64_t)(s + 1) * Wc;
+                        int64_t q = qa[s];
+                        while (q * P < num) ++q;
+                        qa[s] = q;
+                    }
+                }
+                P_prev = P;
+            }
+            while (v > 1 && (v - 1) * C >= Wm) --v;
+            const int64_t qc = rho_q * v;
+            int64_t F = 0;
+            if (!dh) {
+                for (int32_t s = 0; s < L; ++s) {                       // Eq. 11
+                    const int64_t A = qa[s] << kRhoShift;
+                    F = (A > F ? A : F) + qc;
+                }
+            } else {
+                for (int32_t s = 0; s + 1 < L; ++s) {
+                    const int64_t A = qa[s] << kRhoShift;
+                    F = (A > F ? A : F) + qc;
+                }
+                const int64_t A_last = qa[L - 1] << kRhoShift;
+                int64_t backlog = 0;
+                if (F > A_last && rho_q > 0) {
+                    const int64_t num = F - A_last;
+                    int64_t w = (int64_t)((double)num * inv_rho);
+                    while (w * rho_q < num) ++w;
+                    while (w > 0 && (w - 1) * rho_q >= num) --w;
+                    backlog = w * C;
+                    if (backlog > (int64_t)(L - 1) * Wm) backlog = (int64_t)(L - 1) * Wm;
+                }
+                const int64_t workers = (int64_t)C + P * slot / o_comp;
+                const int64_t rem = backlog + Wm;
+                int64_t waves = rem > 0 ? 1 : 0;
+                if (rem > 8 * workers) waves = ceil_div64(rem, workers);
+                else while (waves * workers < rem) ++waves;
+                F = A_last + rho_q * waves;
+            }
+            const int64_t delta = qa[0] * P - Wc;                        // tie breaker, V_comp = qa[0]
+            // ascending C: a strict improvement of (T, Delta) is needed to replace the incumbent
+            if (!have || F < best.T_q || (F == best.T_q && delta < best.delta)) {
+                best.T_q = F;
+                best.delta = delta;
+                best.C = C;
+                best.R = R;
+                best.P = (int32_t)P;
                 have = true;
             }
         }
