@@ -190,7 +190,7 @@ int32_t moe_workspace_bytes(const moe_shape *s, int32_t tile_m, int32_t tile_n, 
         const size_t nts = (size_t)ceil_div(ceil_div(s->H, s->L), tile_n);
         const size_t parts = (tile_m == 256) ? 2 : 1;   // a pair tile is published in two parts
         *flags_bytes = ((size_t)kSplitCounterWords + (size_t)s->L * s->TP * mt * nts * parts +
-                        (size_t)s->L * (size_t)comm_tiles_of(s) * 4 /* claims: 4 slices per tile */) * 4 + 16;
+                        (size_t)s->L * (size_t)comm_tiles_of(s) * 4 /* claims, with room for 4 slices per tile */) * 4 + 16;
     }
     if (status_bytes) *status_bytes = 16;
     return MOE_OK;

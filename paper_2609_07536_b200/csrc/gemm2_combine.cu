@@ -848,7 +848,7 @@ __device__ __forceinline__ void fma_bf16x8(float (&acc)[8], const uint4 &v, floa
 // weights and stores the bf16 result into the owning rank's buffer.  No warp waits on another one:
 // the issue latency of the copies and the memory latency overlap across the twelve warps.
 constexpr int kCommWarps = 12;
-constexpr int kCommSub = 4;            // token slices a communication tile is claimed in (drain help)
+constexpr int kCommSub = 1;            // token slices a communication tile is claimed in (finer slices measured slower)
 constexpr int kCommUnitBytes = 8192;
 constexpr int kCommWarpBytes = 2 * kCommUnitBytes;
 static_assert(kCommWarps * kCommWarpBytes <= kStageBytesTotal, "communication stages exceed the ring");
