@@ -29,6 +29,8 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "fused GEMM2+combine us/layer (whole step: routing build + analytical plan + fused kernel)"
+# workload -> (dram__bytes_read.sum + dram__bytes_write.sum of one fused launch, (tile_m, tile_n, L) it was captured at)
+NCU_TRAFFIC_BYTES = {"dsv2lite": (2188667000 + 1138103000, (128, 256, 2))}
 
 
 def load_peaks():
@@ -522,11 +524,12 @@ def main():
             "kernel_us": fused_med, "roofline_us": max(t_flops_us, t_hbm_us),
             "frac_of_sustained": (ach / peaks["bf16_tflops_sustained"]) if tensor_bound and peaks.get("bf16_tflops_sustained") else None,
         }
-        traffic_path = os.path.join(ROOT, "profiles", "traffic.json")
-        if os.path.exists(traffic_path):
-            tr = json.load(open(traffic_path)).get(w.name)
-            if tr:
-                roofline["traffic"] = tr["bytes_per_launch"]
+        # DRAM read + write bytes of one fused launch from the ncu capture summarised in
+        # profiles/fused_gemm2_combine_dsv2lite_ncu.md (same workload, same launch configuration)
+        if w.name in NCU_TRAFFIC_BYTES and (w.tile_m, w.tile_n, w.L) == NCU_TRAFFIC_BYTES[w.name][1]:
+            roofline["traffic"] = NCU_TRAFFIC_BYTES[w.name][0]
+            roofline["traffic_algorithmic"] = (w.R * w.I * 2 * w.L + w.E_tot * w.H * w.I * 2 +
+                                               2 * w.T * w.L * w.k_tot * w.TP * (-(-w.H // w.L)) * 2 + w.T * w.H * 2)
         line = {
             "metric": METRIC, "value": step_us / world, "unit": "us/layer", "n_gpus": world, "steps": K, "warmup": W,
             "ms_per_step": step_us / 1e3, "higher_is_better": False, "scaling": "weak",

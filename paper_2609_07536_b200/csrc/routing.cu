@@ -102,15 +102,18 @@ routing_scan(int R, int E_tot, int tile_m, int n_warps, int max_mtiles,
         if (toff > max_mtiles) report(status, MOE_DEV_OOB, (uint32_t)toff, 2u);
     }
     __syncthreads();
-    for (int e = threadIdx.x; e < E_tot; e += blockDim.x) {
-        const int c = counts[e], off = offsets[e], toff = tile_offsets[e], nt = tiles[e];
-        for (int i = 0; i < nt; ++i) {
-            const int mu = toff + i;
-            if (mu >= max_mtiles) break;
-            mtile_expert[mu] = e;
-            mtile_first_row[mu] = off + i * tile_m;
-            mtile_valid[mu] = min(tile_m, c - i * tile_m);
+    // m-tile table, one thread per m-tile: the expert is found by bisection in the tile prefix
+    const int S = min(tile_offsets[E_tot], max_mtiles);
+    for (int mu = threadIdx.x; mu < S; mu += blockDim.x) {
+        int lo = 0, hi = E_tot - 1;          // largest e with tile_offsets[e] <= mu
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (tile_offsets[mid] <= mu) lo = mid; else hi = mid - 1;
         }
+        const int e = lo, i = mu - tile_offsets[e];
+        mtile_expert[mu] = e;
+        mtile_first_row[mu] = offsets[e] + i * tile_m;
+        mtile_valid[mu] = min(tile_m, counts[e] - i * tile_m);
     }
 }
 
