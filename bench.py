@@ -42,6 +42,25 @@ def load_peaks():
     return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
 
 
+# ----------------------------------------------------------------------------- replicas
+
+def max_over_ranks(values, world, device="cpu"):
+    """Replicas only: every rank runs the same independent workload, the job's time is the slowest rank's.
+    Works on any initialised process group (NCCL on the GPU machine, gloo in the CPU tests)."""
+    if world <= 1:
+        return [float(v) for v in values]
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(v) for v in values], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.tolist()]
+
+
+def job_value(us_per_layer_slowest_rank, world):
+    """N independent replicas finish N layers in the time of the slowest one: us per layer of the whole job."""
+    return us_per_layer_slowest_rank / max(1, world)
+
+
 # ----------------------------------------------------------------------------- clocks
 
 class ClockSampler:
@@ -476,10 +495,7 @@ def main():
     d2h = out_h.numel() * 2 + (w.E_tot + 1) * 4 + 16
 
     # ---- max over ranks
-    if world > 1:
-        t = torch.tensor([step_us, fused_med, e2e_us], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        step_us, fused_med, e2e_us = (float(v) for v in t.tolist())
+    step_us, fused_med, e2e_us = max_over_ranks([step_us, fused_med, e2e_us], world, device)
 
     extra = {}
     if rank == 0:
@@ -531,7 +547,7 @@ def main():
             roofline["traffic_algorithmic"] = (w.R * w.I * 2 * w.L + w.E_tot * w.H * w.I * 2 +
                                                2 * w.T * w.L * w.k_tot * w.TP * (-(-w.H // w.L)) * 2 + w.T * w.H * 2)
         line = {
-            "metric": METRIC, "value": step_us / world, "unit": "us/layer", "n_gpus": world, "steps": K, "warmup": W,
+            "metric": METRIC, "value": job_value(step_us, world), "unit": "us/layer", "n_gpus": world, "steps": K, "warmup": W,
             "ms_per_step": step_us / 1e3, "higher_is_better": False, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": w.name, "T": w.T, "H": w.H, "I": w.I, "E": w.E, "k": w.k,
@@ -545,7 +561,7 @@ def main():
             "fused_kernel_us": fused_med, "tflops": dw.flops / fused_med / 1e6,
             "wall_ms_per_step": wall * 1e3 / K,
             "roofline": roofline,
-            "e2e": {"value": e2e_us / world, "unit": "us/layer", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "e2e": {"value": job_value(e2e_us, world), "unit": "us/layer", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": Ke},
             "gpu_launches": 4 * K,
             "clocks": clocks,
