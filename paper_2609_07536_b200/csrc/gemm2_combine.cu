@@ -13,7 +13,7 @@
 //               W2 tile (tile_n rows x 64 k) of every k-block, into a ring of 128B-swizzled stages;
 //   warp 1      MMA issuer (one thread): tcgen05.mma (M = 128, N = tile_n, K = 16, bf16 -> fp32) into one
 //               of two TMEM accumulator buffers; tcgen05.commit frees stages / publishes the tile;
-//   warps 4-11  epilogue: tcgen05.ld -> bf16 -> Y, then the tile's readiness flag (st.release.gpu) and
+//   warps 4-15  epilogue: tcgen05.ld -> bf16 -> Y, then the tile's readiness flag (st.release.gpu) and
 //               the split counter (red.release.gpu).
 // Compute CTA pair (256 x 256 tiles): the same roles in both CTAs of a cluster of two; one
 //   tcgen05.mma.cta_group::2 spans both SMs, each CTA loads only its own operand halves.
@@ -268,9 +268,9 @@ struct Cfg {
     static constexpr int kStageBytes = kABytes + kBBytes;
     static constexpr int kStages = kStageBytesTotal / kStageBytes;  // 8 / 6 / 4
     static constexpr int kTmemCols = 2 * TN;                     // two accumulator buffers
-    static constexpr int kEpiWarps = 8;
+    static constexpr int kEpiWarps = 12;                          // warps 4..15: three column groups x four lane quarters
     static constexpr int kEpiThreads = kEpiWarps * 32;
-    static constexpr int kColsPerHalf = TN / 2;
+    static constexpr int kColsPerGroup = ((TN / 32 + 2) / 3) * 32;  // 32-column rounds dealt to the groups: 96 / 64 / 32
 };
 
 struct Control {
@@ -286,14 +286,14 @@ struct Control {
 
 // 32 KB after the control block, used by one role per CTA:
 //   communication CTA: per-row weights of the unit each warp reduces (12 warps x 256 floats)
-//   compute CTA      : per-epilogue-warp staging (8 warps x 2.5 KB + row pointers) for coalesced Y stores
-constexpr int kAuxBytes = 8 * 2560 + 8 * 256;
+//   compute CTA      : per-epilogue-warp staging (12 warps x 2.5 KB + row pointers) for coalesced Y stores
+constexpr int kAuxBytes = 12 * 2560 + 12 * 256;
 constexpr int kEpiStagePitch = 80;    // 64 data bytes + 16 pad: conflict-free 16-byte stores
 struct EpiStage {
     uint8_t data[32 * kEpiStagePitch];        // 32 rows x 32 bf16
     unsigned long long rowptr[32];            // destination of each row for the group in hand (0 = skip)
 };
-static_assert(sizeof(EpiStage) * 8 <= kAuxBytes, "epilogue staging exceeds the aux region");
+static_assert(sizeof(EpiStage) * 12 <= kAuxBytes, "epilogue staging exceeds the aux region");
 static_assert(12 * 256 * 4 <= kAuxBytes, "communication weights exceed the aux region");
 
 // Bounded mbarrier wait, warp-collective: lane 0 polls (32 lanes polling the same barrier would
@@ -360,12 +360,11 @@ __device__ __forceinline__ Tile decode_tile(int g, const FusedParams &P)
 // One thread = one accumulator row (TMEM lane).  Reads COLS fp32 columns starting at `col_first` of
 // the accumulator at `taddr`, rounds to bf16 and writes them to the row's place in the token-major Y:
 // slab = column slab inside the split, q = row of the unit (slot j, shard p).
-template <int COLS>
-__device__ __forceinline__ void store_accumulator_rows(const FusedParams &P, uint32_t taddr, int col_first, bool row_ok,
+__device__ __forceinline__ void store_accumulator_rows(const FusedParams &P, uint32_t taddr, int col_first, int n_cols, bool row_ok,
                                                        __nv_bfloat16 *ybase, int q, int n0, int col_end, int cis0)
 {
-#pragma unroll
-    for (int cc = 0; cc < COLS; cc += 32) {
+#pragma unroll 1
+    for (int cc = 0; cc < n_cols; cc += 32) {
         const int col = col_first + cc;
         uint32_t r[32];
         tmem_ld_32x32(taddr + (uint32_t)col, r);
@@ -398,8 +397,7 @@ __device__ __forceinline__ void store_accumulator_rows(const FusedParams &P, uin
 // Same job with the stores coalesced: the warp's 32 rows x 32 columns go through a padded staging
 // buffer, so that four lanes write one row's 64 contiguous bytes (two full sectors) instead of every
 // lane writing 16 bytes of a different row.  Needs the 32-column group inside one column slab.
-template <int COLS>
-__device__ __forceinline__ void store_accumulator_rows_staged(const FusedParams &P, uint32_t taddr, int col_first, bool row_ok,
+__device__ __forceinline__ void store_accumulator_rows_staged(const FusedParams &P, uint32_t taddr, int col_first, int n_cols, bool row_ok,
                                                               __nv_bfloat16 *ybase, int q, int n0, int col_end, int cis0,
                                                               EpiStage *stg)
 {
@@ -407,8 +405,8 @@ __device__ __forceinline__ void store_accumulator_rows_staged(const FusedParams 
     const uint32_t stg_s = smem_u32(stg->data);
     const uint32_t my_row_s = stg_s + (uint32_t)lane * kEpiStagePitch;
     const int chunk = lane & 3;
-#pragma unroll 2
-    for (int cc = 0; cc < COLS; cc += 32) {
+#pragma unroll 1
+    for (int cc = 0; cc < n_cols; cc += 32) {
         const int col = col_first + cc;
         uint32_t r[32];
         tmem_ld_32x32(taddr + (uint32_t)col, r);
@@ -554,7 +552,9 @@ __device__ void compute_cta(const FusedParams &P, uint8_t *ring, Control *ctl, u
     } else if (warp >= 4 && warp < 4 + C::kEpiWarps) {
         // ---------------- epilogue: TMEM -> bf16 -> Y, then publish the tile
         const int q4 = warp & 3;                   // TMEM lane quarter this warp may read
-        const int half = (warp - 4) >> 2;          // column half of the tile
+        const int grp = (warp - 4) >> 2;           // column group of the tile
+        const int col_first = grp * C::kColsPerGroup;
+        const int n_cols = max(0, min(C::kColsPerGroup, TN - col_first));
         const int row_in_tile = q4 * 32 + lane;
         const bool is_leader = (warp == 4 && lane == 0);
         __nv_bfloat16 *Y = reinterpret_cast<__nv_bfloat16 *>(P.Y);
@@ -582,12 +582,12 @@ __device__ void compute_cta(const FusedParams &P, uint8_t *ring, Control *ctl, u
                     ybase = Y + ((size_t)tok * P.L + t.s) * (size_t)P.Q * (size_t)P.split_w;
                 }
                 if (P.slab_cols >= 32)
-                    store_accumulator_rows_staged<C::kColsPerHalf>(
-                        P, tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(a * TN), half * C::kColsPerHalf, row_ok,
+                    store_accumulator_rows_staged(
+                        P, tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(a * TN), col_first, n_cols, row_ok,
                         ybase, q, n0, col_end, n0 - t.s * P.split_w, reinterpret_cast<EpiStage *>(aux) + (warp - 4));
                 else
-                    store_accumulator_rows<C::kColsPerHalf>(P, tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(a * TN),
-                                                            half * C::kColsPerHalf, row_ok, ybase, q, n0, col_end,
+                    store_accumulator_rows(P, tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(a * TN),
+                                                            col_first, n_cols, row_ok, ybase, q, n0, col_end,
                                                             n0 - t.s * P.split_w);
                 // the accumulator buffer may be overwritten by the MMA of the tile after next
                 tc_fence_before();
@@ -631,9 +631,9 @@ struct PairCfg {
     static constexpr int kStageBytes = kABytes + kBBytes;               // 32 KB
     static constexpr int kStages = kStageBytesTotal / kStageBytes;      // 6
     static constexpr int kTmemCols = 2 * kTileN;                        // two accumulator buffers
-    static constexpr int kEpiWarps = 8;
+    static constexpr int kEpiWarps = 12;
     static constexpr int kEpiThreads = kEpiWarps * 32;
-    static constexpr int kColsPerHalf = kTileN / 2;
+    static constexpr int kColsPerGroup = ((kTileN / 32 + 2) / 3) * 32;  // 96, 96, 64
 };
 
 __device__ void compute_cta_pair(const FusedParams &P, uint8_t *ring, Control *ctl, uint8_t *aux, int b)
@@ -745,7 +745,9 @@ __device__ void compute_cta_pair(const FusedParams &P, uint8_t *ring, Control *c
     } else if (warp >= 4 && warp < 4 + C::kEpiWarps) {
         // ---------------- epilogue (both CTAs): own 128 rows of the pair tile
         const int q4 = warp & 3;
-        const int half = (warp - 4) >> 2;
+        const int grp = (warp - 4) >> 2;
+        const int col_first = grp * C::kColsPerGroup;
+        const int n_cols = max(0, min(C::kColsPerGroup, TN - col_first));
         const int row_in_tile = (int)rank * kMmaM + q4 * 32 + lane;
         const bool is_leader = (warp == 4 && lane == 0);
         __nv_bfloat16 *Y = reinterpret_cast<__nv_bfloat16 *>(P.Y);
@@ -770,12 +772,12 @@ __device__ void compute_cta_pair(const FusedParams &P, uint8_t *ring, Control *c
                     ybase = Y + ((size_t)tok * P.L + t.s) * (size_t)P.Q * (size_t)P.split_w;
                 }
                 if (P.slab_cols >= 32)
-                    store_accumulator_rows_staged<C::kColsPerHalf>(
-                        P, tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(a * TN), half * C::kColsPerHalf, row_ok,
+                    store_accumulator_rows_staged(
+                        P, tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(a * TN), col_first, n_cols, row_ok,
                         ybase, q, n0, col_end, n0 - t.s * P.split_w, reinterpret_cast<EpiStage *>(aux) + (warp - 4));
                 else
-                    store_accumulator_rows<C::kColsPerHalf>(P, tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(a * TN),
-                                                            half * C::kColsPerHalf, row_ok, ybase, q, n0, col_end,
+                    store_accumulator_rows(P, tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(a * TN),
+                                                            col_first, n_cols, row_ok, ybase, q, n0, col_end,
                                                             n0 - t.s * P.split_w);
                 // this CTA's half of the accumulator buffer is drained: tell the leader's MMA warp
                 tc_fence_before();
