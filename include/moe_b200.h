@@ -241,6 +241,20 @@ int32_t moe_get_status(moe_handle *h, const uint32_t *status_dev, moe_status *ho
 /* Clears the device status (asynchronous memset). */
 int32_t moe_clear_status(moe_handle *h, uint32_t *status_dev, void *stream);
 
+/* ---- the whole step on device-resident inputs -----------------------------------------------
+ * One call for routing build -> wait for the tile counts -> plan_partition -> fused launch
+ * (Section III-E: the manager sits between dispatch and launch; the counts are read on the host).
+ * Inputs and workspaces as for moe_build_routing / moe_gemm2_combine; tile_counts_pinned [host, pinned]
+ * E_tot + 1 ints; limits_or_null = NULL uses moe_query_occupancy's limits; plan_out may be NULL.
+ * Returns after the fused kernel has been launched (asynchronous on `stream`); the only host wait
+ * inside is the one for the tile counts.  ev_before / ev_after: optional cudaEvent_t handles (NULL = none)
+ * recorded on `stream` right before and right after the fused launch, for timing it. */
+int32_t moe_layer(moe_handle *h, const void *x_routed, const void *W2, const int32_t *topk_idx,
+                  const float *topk_w, const moe_shape *shape, int32_t tile_m, int32_t tile_n,
+                  const moe_sm_limits *limits_or_null, const moe_routing *routing,
+                  int32_t *tile_counts_pinned, void *const *out, void *y_ws, uint32_t *flags_ws,
+                  uint32_t *status_dev, moe_plan *plan_out, void *ev_before, void *ev_after, void *stream);
+
 /* ---- the whole step from host buffers ---------------------------------------------------
  * The call a user without device-resident activations makes: copies x_routed, topk_idx and
  * topk_w from (pinned) host memory into `arena`, builds the routing, waits for the tile

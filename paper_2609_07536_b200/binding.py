@@ -29,7 +29,7 @@ EXPORTS = [
     "moe_query_occupancy", "moe_workspace_bytes", "moe_routing_view", "moe_build_routing",
     "moe_build_routing_static",
     "plan_partition", "moe_time_plan_partition", "moe_gemm2_combine", "moe_get_status", "moe_clear_status",
-    "moe_host_arena_bytes", "moe_layer_host",
+    "moe_layer", "moe_host_arena_bytes", "moe_layer_host",
 ]
 
 
@@ -107,6 +107,8 @@ def lib():
                                         i32, P(moe_plan), P(vp), vp, vp, vp, vp]
         L.moe_get_status.argtypes = [vp, vp, P(moe_status), vp]
         L.moe_clear_status.argtypes = [vp, vp, vp]
+        L.moe_layer.argtypes = [vp, vp, vp, vp, vp, P(moe_shape), i32, i32, P(moe_sm_limits), P(moe_routing), vp,
+                                P(vp), vp, vp, vp, P(moe_plan), vp, vp, vp]
         L.moe_host_arena_bytes.argtypes = [P(moe_shape), i32, i32, P(C.c_size_t)]
         L.moe_layer_host.argtypes = [vp, vp, vp, vp, vp, P(moe_shape), i32, i32, P(moe_sm_limits), vp,
                                      C.c_size_t, vp, vp, P(moe_plan), vp]
@@ -240,6 +242,35 @@ def moe_get_status(h, status_dev, stream=None, check: bool = True) -> moe_status
 
 def moe_clear_status(h, status_dev, stream=None):
     _check(lib().moe_clear_status(h, _ptr(status_dev), _stream(stream)), "moe_clear_status", h)
+
+
+class LayerCall:
+    """moe_layer with its arguments marshalled once (for a loop that repeats the same call)."""
+
+    def __init__(self, h, x_routed, W2, topk_idx, topk_w, ws: "Workspace", limits=None, stream=None):
+        self._stream = _stream(stream)
+        self.h, self.ws = h, ws
+        self.outs = (C.c_void_p * len(ws.out))(*[_ptr(o) for o in ws.out])
+        self.plan = moe_plan()
+        self.limits = limits
+        self.args = (h, _ptr(x_routed), _ptr(W2), _ptr(topk_idx), _ptr(topk_w), C.byref(ws.shape), ws.tile_m,
+                     ws.tile_n, C.byref(limits) if limits is not None else None, C.byref(ws.routing),
+                     _ptr(ws.tile_counts), self.outs, _ptr(ws.y_ws), _ptr(ws.flags_ws), _ptr(ws.status),
+                     C.byref(self.plan))
+        self.keep = (x_routed, W2, topk_idx, topk_w)
+
+    def __call__(self, ev_before=None, ev_after=None) -> moe_plan:
+        """ev_before / ev_after: torch.cuda.Event objects that have been recorded at least once (so that
+        their CUDA handles exist); they are re-recorded around the fused launch."""
+        eb = ev_before.cuda_event if ev_before is not None else None
+        ea = ev_after.cuda_event if ev_after is not None else None
+        _check(lib().moe_layer(*self.args, eb, ea, self._stream), "moe_layer", self.h)
+        return self.plan
+
+
+def moe_layer(h, x_routed, W2, topk_idx, topk_w, ws: "Workspace", limits=None, stream=None) -> moe_plan:
+    """Routing build -> tile counts to the host -> analytical plan -> fused launch, in one library call."""
+    return LayerCall(h, x_routed, W2, topk_idx, topk_w, ws, limits, stream)()
 
 
 def moe_host_arena_bytes(shape, tile_m, tile_n) -> int:

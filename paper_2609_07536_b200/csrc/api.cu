@@ -400,6 +400,37 @@ int32_t moe_clear_status(moe_handle *h, uint32_t *status_dev, void *stream)
     return e == cudaSuccess ? MOE_OK : cuda_fail(h, e, "status clear");
 }
 
+// ---- whole step on device-resident inputs -----------------------------------------------------
+
+int32_t moe_layer(moe_handle *h, const void *x_routed, const void *W2, const int32_t *topk_idx,
+                  const float *topk_w, const moe_shape *s, int32_t tile_m, int32_t tile_n,
+                  const moe_sm_limits *limits_or_null, const moe_routing *routing,
+                  int32_t *tile_counts_pinned, void *const *out, void *y_ws, uint32_t *flags_ws,
+                  uint32_t *status_dev, moe_plan *plan_out, void *ev_before, void *ev_after, void *stream)
+{
+    if (!h || !s || !routing || !tile_counts_pinned) return MOE_ERR_NULL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t rc = moe_build_routing(h, topk_idx, s, tile_m, routing, tile_counts_pinned, status_dev, st);
+    if (rc != MOE_OK) return rc;
+    cudaError_t e = cudaStreamSynchronize(st);       // the tile counts are on the host now
+    if (e != cudaSuccess) return cuda_fail(h, e, "tile counts sync");
+    moe_occupancy occ;
+    moe_sm_limits lim;
+    moe_rho rho;
+    rc = moe_query_occupancy(h, tile_m, tile_n, &occ, &lim, &rho);
+    if (rc != MOE_OK) return rc;
+    if (limits_or_null) lim = *limits_or_null;
+    moe_plan plan;
+    rc = plan_partition(tile_counts_pinned, s->E_tot, &occ, &lim, s, &rho, &plan);
+    if (rc != MOE_OK) return rc;
+    if (plan_out) *plan_out = plan;
+    if (ev_before) cudaEventRecord(static_cast<cudaEvent_t>(ev_before), st);
+    rc = moe_gemm2_combine(h, x_routed, W2, topk_idx, topk_w, s, &occ, routing, tile_counts_pinned[s->E_tot], &plan,
+                           out, y_ws, flags_ws, status_dev, st);
+    if (ev_after) cudaEventRecord(static_cast<cudaEvent_t>(ev_after), st);
+    return rc;
+}
+
 // ---- whole step from host buffers ----------------------------------------------------------
 
 namespace {

@@ -302,3 +302,26 @@ def test_host_buffer_entry_point_matches_device_path():
     got = out_h.float().numpy()
     cat = np.concatenate([o[:len(G.tokens_of_rank(w.T, w.EP, d))] for d, o in enumerate(dev)])
     assert np.array_equal(got, cat)
+
+
+def test_single_call_layer_matches_the_stepwise_path():
+    h = G.handle()
+    w = replace(wl.GRANITE, name="layer", T=1500)
+    idx, wt, _ = wl.make_routing(w)
+    x, W2 = wl.make_data(w)
+    ref_outs, plan, ws, S, st = G.run_layer(w, idx, wt, x, W2)
+    ref_outs = [o.copy() for o in ref_outs]
+    for o in ws.out:
+        o.fill_(float("nan"))
+    xd, Wd = x.cuda(), W2.cuda()
+    idx_d, wt_d = torch.from_numpy(idx).cuda(), torch.from_numpy(wt).cuda()
+    ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ea.record(); eb.record()
+    call = B.LayerCall(h, xd, Wd, idx_d, wt_d, ws)
+    p2 = call(ea, eb)
+    torch.cuda.synchronize()
+    assert B.moe_get_status(h, ws.status).code == 0
+    assert (p2.comm_ctas, p2.P, p2.W_comp) == (plan.comm_ctas, plan.P, plan.W_comp)
+    assert ea.elapsed_time(eb) > 0
+    for a, o in zip(ref_outs, ws.out):
+        assert np.array_equal(a, o.float().cpu().numpy(), equal_nan=True)
