@@ -218,13 +218,13 @@ __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p)
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
-__device__ __forceinline__ void st_release_u32(uint32_t *p, uint32_t v)
+__device__ __forceinline__ void st_relaxed_u32(uint32_t *p, uint32_t v)
 {
-    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+    asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
-__device__ __forceinline__ void red_release_add_u32(uint32_t *p, uint32_t v)
+__device__ __forceinline__ void red_relaxed_add_u32(uint32_t *p, uint32_t v)
 {
-    asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+    asm volatile("red.relaxed.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 __device__ __forceinline__ void named_barrier(int id, int threads)
 {
@@ -269,7 +269,6 @@ struct Cfg {
     static constexpr int kStages = kStageBytesTotal / kStageBytes;  // 8 / 6 / 4
     static constexpr int kTmemCols = 2 * TN;                     // two accumulator buffers
     static constexpr int kEpiWarps = 12;                          // warps 4..15: three column groups x four lane quarters
-    static constexpr int kEpiThreads = kEpiWarps * 32;
     static constexpr int kColsPerGroup = ((TN / 32 + 2) / 3) * 32;  // 32-column rounds dealt to the groups: 96 / 64 / 32
 };
 
@@ -278,6 +277,8 @@ struct Control {
     unsigned long long empty[8];
     unsigned long long tmem_full[2];
     unsigned long long tmem_empty[2];
+    unsigned long long epi_done[2];     // every epilogue warp has stored its rows of the tile (per accumulator buffer)
+    unsigned long long pub_done[2];     // the publisher warp has raised that tile's flag
     uint32_t tmem_base;
     volatile uint32_t abort;
     unsigned long long comm_full[24];   // communication CTA: one barrier per warp and stage
@@ -460,6 +461,8 @@ __device__ void compute_cta(const FusedParams &P, uint8_t *ring, Control *ctl, u
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&ctl->tmem_full[i]), 1);
             mbar_init(smem_u32(&ctl->tmem_empty[i]), C::kEpiWarps);
+            mbar_init(smem_u32(&ctl->epi_done[i]), C::kEpiWarps);
+            mbar_init(smem_u32(&ctl->pub_done[i]), 1);
         }
         ctl->abort = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -476,15 +479,20 @@ __device__ void compute_cta(const FusedParams &P, uint8_t *ring, Control *ctl, u
         // k-block; both complete on the same full barrier.  One thread per warp runs the whole loop (no
         // per-iteration warp broadcast); the others park below.
         const bool load_a = (warp == 0);
-        if (lane == 0) {
+        if (lane == 0 && b < total_tiles) {
             int stage = 0;
             uint32_t phase = 0;
             uint32_t armed = 0;  // bit s: stage s was handed to the TMA unit at least once
             bool ok = true;
+            // the m-tile table entries of the NEXT tile are fetched while this tile's k-blocks are issued, so
+            // that the two dependent global loads never stall the stream of copies at a tile boundary
+            Tile t = decode_tile(b, P);
+            int e = __ldg(&P.mtile_expert[t.mu]);
+            int row0 = __ldg(&P.mtile_first_row[t.mu]);
             for (int g = b; g < total_tiles && ok; g += P.P) {
-                const Tile t = decode_tile(g, P);
-                const int e = __ldg(&P.mtile_expert[t.mu]);
-                const int row0 = __ldg(&P.mtile_first_row[t.mu]);
+                const Tile t_next = decode_tile(min(g + P.P, total_tiles - 1), P);
+                const int e_next = __ldg(&P.mtile_expert[t_next.mu]);
+                const int row0_next = __ldg(&P.mtile_first_row[t_next.mu]);
                 const int n0 = t.s * P.split_w + t.i_n * TN;
                 int kx = t.p * P.K;
                 for (int kb = 0; kb < P.num_kb; ++kb, kx += kBlockK) {
@@ -501,6 +509,9 @@ __device__ void compute_cta(const FusedParams &P, uint8_t *ring, Control *ctl, u
                     armed |= 1u << stage;
                     if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
                 }
+                t = t_next;
+                e = e_next;
+                row0 = row0_next;
             }
             if (!ok) {
                 // wind-down: let the copies already issued land before shared memory is released
@@ -537,10 +548,19 @@ __device__ void compute_cta(const FusedParams &P, uint8_t *ring, Control *ctl, u
                     const uint64_t a_desc = make_smem_desc(a_addr);
                     const uint64_t b_desc = make_smem_desc(a_addr + C::kABytes);
                     const int ksteps = (kb == P.num_kb - 1) ? P.last_ksteps : (kBlockK / kUmmaK);
-                    for (int k = 0; k < ksteps; ++k) {
-                        // advancing K by 16 bf16 = 32 bytes inside the swizzle row: +2 in the address field
-                        tc_mma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
-                                    (kb > 0 || k > 0) ? 1u : 0u);
+                    // advancing K by 16 bf16 = 32 bytes inside the swizzle row: +2 in the address field.
+                    // The full k-block is written out: the issuing thread has to stay ahead of the tensor
+                    // pipe, and the rolled loop (variable trip count, 64-bit adds) costs it twice the cycles.
+                    const uint32_t acc0 = kb > 0 ? 1u : 0u;
+                    if (ksteps == kBlockK / kUmmaK) {
+                        tc_mma_bf16(d_tmem, a_desc, b_desc, idesc, acc0);
+                        tc_mma_bf16(d_tmem, a_desc + 2ull, b_desc + 2ull, idesc, 1u);
+                        tc_mma_bf16(d_tmem, a_desc + 4ull, b_desc + 4ull, idesc, 1u);
+                        tc_mma_bf16(d_tmem, a_desc + 6ull, b_desc + 6ull, idesc, 1u);
+                    } else {
+                        for (int k = 0; k < ksteps; ++k)
+                            tc_mma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
+                                        k > 0 ? 1u : acc0);
                     }
                     tc_commit(smem_u32(&ctl->empty[stage]));   // stage reusable once these MMAs have read it
                     if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
@@ -556,18 +576,33 @@ __device__ void compute_cta(const FusedParams &P, uint8_t *ring, Control *ctl, u
         const int col_first = grp * C::kColsPerGroup;
         const int n_cols = max(0, min(C::kColsPerGroup, TN - col_first));
         const int row_in_tile = q4 * 32 + lane;
-        const bool is_leader = (warp == 4 && lane == 0);
         __nv_bfloat16 *Y = reinterpret_cast<__nv_bfloat16 *>(P.Y);
+        // Row bookkeeping runs ahead of the accumulators: the m-tile table entries are fetched two tiles
+        // ahead and the row's flat assignment one tile ahead, so that these dependent global loads are
+        // not in the way between an accumulator becoming ready and its first store.
+        int valid = 0, f_row = 0, valid_n = 0, first_n = 0;
+        if (b < total_tiles) {
+            const int mu0 = decode_tile(b, P).mu;
+            const int mu1 = decode_tile(min(b + P.P, total_tiles - 1), P).mu;
+            valid = __ldg(&P.mtile_valid[mu0]);
+            const int first0 = __ldg(&P.mtile_first_row[mu0]);
+            valid_n = __ldg(&P.mtile_valid[mu1]);
+            first_n = __ldg(&P.mtile_first_row[mu1]);
+            if (row_in_tile < valid) f_row = __ldg(&P.perm[first0 + row_in_tile]);
+        }
         int it = 0;
         for (int g = b; g < total_tiles; g += P.P, ++it) {
             const Tile t = decode_tile(g, P);
             const int a = it & 1;
             const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+            const int mu_nn = decode_tile(min(g + 2 * P.P, total_tiles - 1), P).mu;
+            const int valid_nn = __ldg(&P.mtile_valid[mu_nn]);
+            const int first_nn = __ldg(&P.mtile_first_row[mu_nn]);
+            const int f_row_n = (row_in_tile < valid_n) ? __ldg(&P.perm[first_n + row_in_tile]) : 0;
             bool ok = wait_barrier(smem_u32(&ctl->tmem_full[a]), acc_phase, ctl, deadline, P.status, (uint32_t)g, 30u);
             ok = __all_sync(0xffffffffu, ok);
             if (ok) {
                 tc_fence_after();
-                const int valid = __ldg(&P.mtile_valid[t.mu]);
                 const int n0 = t.s * P.split_w + t.i_n * TN;
                 const int col_end = min(P.H, (t.s + 1) * P.split_w);
                 const bool row_ok = row_in_tile < valid;
@@ -576,7 +611,7 @@ __device__ void compute_cta(const FusedParams &P, uint8_t *ring, Control *ctl, u
                 __nv_bfloat16 *ybase = Y;
                 int q = 0;
                 if (row_ok) {
-                    const int f = __ldg(&P.perm[__ldg(&P.mtile_first_row[t.mu]) + row_in_tile]);
+                    const int f = f_row;
                     const int tok = f / P.k_tot;
                     q = (f - tok * P.k_tot) * P.TP + t.p;
                     ybase = Y + ((size_t)tok * P.L + t.s) * (size_t)P.Q * (size_t)P.split_w;
@@ -594,15 +629,39 @@ __device__ void compute_cta(const FusedParams &P, uint8_t *ring, Control *ctl, u
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&ctl->tmem_empty[a]));
             }
-            // every epilogue warp reaches this barrier, also after a failed wait
-            named_barrier(1, C::kEpiThreads);
-            if (ctl->abort) break;
-            if (is_leader && g != P.withhold) {
-                __threadfence();
-                st_release_u32(&P.flags[g], P.epoch);
-                red_release_add_u32(&P.split_done[t.s], 1u);
+            // hand the tile to the publisher warp.  Its barrier is reused every other tile, so the warp
+            // first makes sure that the tile two back has been published (it normally has, long ago).
+            if (ok && it >= 2)
+                ok = wait_barrier(smem_u32(&ctl->pub_done[a]), (uint32_t)((it - 2) >> 1) & 1u, ctl, deadline, P.status,
+                                  (uint32_t)g, 31u);
+            if (!ok) break;
+            __syncwarp();   // the lanes' stores are ordered before lane 0's arrival
+            if (lane == 0) mbar_arrive(smem_u32(&ctl->epi_done[a]));
+            valid = valid_n;
+            f_row = f_row_n;
+            valid_n = valid_nn;
+            first_n = first_nn;
+        }
+    } else if (warp == 3) {
+        // ---------------- publisher: one thread raises the readiness flag of every finished tile.  The
+        // release costs a microsecond or more (it waits for the CTA's stores to be performed); here it
+        // is off the path of the epilogue warps, which go straight on to the next accumulator.
+        if (lane == 0) {
+            int it = 0;
+            for (int g = b; g < total_tiles; g += P.P, ++it) {
+                const int a = it & 1;
+                if (!wait_barrier_1t(smem_u32(&ctl->epi_done[a]), (uint32_t)(it >> 1) & 1u, ctl, deadline, P.status,
+                                     (uint32_t)g, 32u))
+                    break;
+                if (g != P.withhold) {
+                    __threadfence();   // release: the epilogue warps' stores (observed through epi_done) come first
+                    st_relaxed_u32(&P.flags[g], P.epoch);
+                    red_relaxed_add_u32(&P.split_done[g / P.W_comp], 1u);
+                }
+                mbar_arrive(smem_u32(&ctl->pub_done[a]));
             }
         }
+        __syncwarp();
     }
     // ---------------- teardown
     tc_fence_before();
@@ -632,7 +691,6 @@ struct PairCfg {
     static constexpr int kStages = kStageBytesTotal / kStageBytes;      // 6
     static constexpr int kTmemCols = 2 * kTileN;                        // two accumulator buffers
     static constexpr int kEpiWarps = 12;
-    static constexpr int kEpiThreads = kEpiWarps * 32;
     static constexpr int kColsPerGroup = ((kTileN / 32 + 2) / 3) * 32;  // 96, 96, 64
 };
 
@@ -654,6 +712,8 @@ __device__ void compute_cta_pair(const FusedParams &P, uint8_t *ring, Control *c
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&ctl->tmem_full[i]), 1);
             mbar_init(smem_u32(&ctl->tmem_empty[i]), 2 * C::kEpiWarps);
+            mbar_init(smem_u32(&ctl->epi_done[i]), C::kEpiWarps);
+            mbar_init(smem_u32(&ctl->pub_done[i]), 1);
         }
         ctl->abort = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -671,15 +731,19 @@ __device__ void compute_cta_pair(const FusedParams &P, uint8_t *ring, Control *c
         // rows; both complete on the leader's full barrier.  Two issuing threads halve the serial issue
         // latency per k-block.  One thread per warp runs the whole loop; the others park below.
         const bool load_a = (warp == 0);
-        if (lane == 0) {
+        if (lane == 0 && b < total_tiles) {
             int stage = 0;
             uint32_t phase = 0;
             uint32_t armed = 0;
             bool ok = true;
+            // next tile's table entries are fetched one tile ahead (see compute_cta)
+            Tile t = decode_tile(b, P);
+            int e = __ldg(&P.mtile_expert[t.mu]);
+            int row0 = __ldg(&P.mtile_first_row[t.mu]) + (int)rank * kMmaM;
             for (int g = b; g < total_tiles && ok; g += P.P) {
-                const Tile t = decode_tile(g, P);
-                const int e = __ldg(&P.mtile_expert[t.mu]);
-                const int row0 = __ldg(&P.mtile_first_row[t.mu]) + (int)rank * kMmaM;
+                const Tile t_next = decode_tile(min(g + P.P, total_tiles - 1), P);
+                const int e_next = __ldg(&P.mtile_expert[t_next.mu]);
+                const int row0_next = __ldg(&P.mtile_first_row[t_next.mu]) + (int)rank * kMmaM;
                 const int n0 = t.s * P.split_w + t.i_n * TN + (int)rank * (TN / 2);
                 int kx = t.p * P.K;
                 for (int kb = 0; kb < P.num_kb; ++kb, kx += kBlockK) {
@@ -697,6 +761,9 @@ __device__ void compute_cta_pair(const FusedParams &P, uint8_t *ring, Control *c
                     armed |= 1u << stage;
                     if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
                 }
+                t = t_next;
+                e = e_next;
+                row0 = row0_next;
             }
             if (!ok && leader_cta) {
                 // wind-down: let the copies already issued land before shared memory is released
@@ -732,9 +799,17 @@ __device__ void compute_cta_pair(const FusedParams &P, uint8_t *ring, Control *c
                     const uint64_t a_desc = make_smem_desc(a_addr);
                     const uint64_t b_desc = make_smem_desc(a_addr + C::kABytes);
                     const int ksteps = (kb == P.num_kb - 1) ? P.last_ksteps : (kBlockK / kUmmaK);
-                    for (int k = 0; k < ksteps; ++k)
-                        tc_mma_bf16_pair(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
-                                         (kb > 0 || k > 0) ? 1u : 0u);
+                    const uint32_t acc0 = kb > 0 ? 1u : 0u;
+                    if (ksteps == kBlockK / kUmmaK) {   // written out: see compute_cta
+                        tc_mma_bf16_pair(d_tmem, a_desc, b_desc, idesc, acc0);
+                        tc_mma_bf16_pair(d_tmem, a_desc + 2ull, b_desc + 2ull, idesc, 1u);
+                        tc_mma_bf16_pair(d_tmem, a_desc + 4ull, b_desc + 4ull, idesc, 1u);
+                        tc_mma_bf16_pair(d_tmem, a_desc + 6ull, b_desc + 6ull, idesc, 1u);
+                    } else {
+                        for (int k = 0; k < ksteps; ++k)
+                            tc_mma_bf16_pair(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
+                                             k > 0 ? 1u : acc0);
+                    }
                     tc_commit_pair(smem_u32(&ctl->empty[stage]));      // both CTAs may refill the stage
                     if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
                 }
@@ -749,24 +824,39 @@ __device__ void compute_cta_pair(const FusedParams &P, uint8_t *ring, Control *c
         const int col_first = grp * C::kColsPerGroup;
         const int n_cols = max(0, min(C::kColsPerGroup, TN - col_first));
         const int row_in_tile = (int)rank * kMmaM + q4 * 32 + lane;
-        const bool is_leader = (warp == 4 && lane == 0);
         __nv_bfloat16 *Y = reinterpret_cast<__nv_bfloat16 *>(P.Y);
+        // Row bookkeeping runs ahead of the accumulators: the m-tile table entries are fetched two tiles
+        // ahead and the row's flat assignment one tile ahead, so that these dependent global loads are
+        // not in the way between an accumulator becoming ready and its first store.
+        int valid = 0, f_row = 0, valid_n = 0, first_n = 0;
+        if (b < total_tiles) {
+            const int mu0 = decode_tile(b, P).mu;
+            const int mu1 = decode_tile(min(b + P.P, total_tiles - 1), P).mu;
+            valid = __ldg(&P.mtile_valid[mu0]);
+            const int first0 = __ldg(&P.mtile_first_row[mu0]);
+            valid_n = __ldg(&P.mtile_valid[mu1]);
+            first_n = __ldg(&P.mtile_first_row[mu1]);
+            if (row_in_tile < valid) f_row = __ldg(&P.perm[first0 + row_in_tile]);
+        }
         int it = 0;
         for (int g = b; g < total_tiles; g += P.P, ++it) {
             const Tile t = decode_tile(g, P);
             const int a = it & 1;
             const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+            const int mu_nn = decode_tile(min(g + 2 * P.P, total_tiles - 1), P).mu;
+            const int valid_nn = __ldg(&P.mtile_valid[mu_nn]);
+            const int first_nn = __ldg(&P.mtile_first_row[mu_nn]);
+            const int f_row_n = (row_in_tile < valid_n) ? __ldg(&P.perm[first_n + row_in_tile]) : 0;
             const bool ok = wait_barrier(smem_u32(&ctl->tmem_full[a]), acc_phase, ctl, deadline, P.status, (uint32_t)g, 30u);
             if (ok) {
                 tc_fence_after();
-                const int valid = __ldg(&P.mtile_valid[t.mu]);
                 const int n0 = t.s * P.split_w + t.i_n * TN;
                 const int col_end = min(P.H, (t.s + 1) * P.split_w);
                 const bool row_ok = row_in_tile < valid;
                 __nv_bfloat16 *ybase = Y;
                 int q = 0;
                 if (row_ok) {
-                    const int f = __ldg(&P.perm[__ldg(&P.mtile_first_row[t.mu]) + row_in_tile]);
+                    const int f = f_row;
                     const int tok = f / P.k_tot;
                     q = (f - tok * P.k_tot) * P.TP + t.p;
                     ybase = Y + ((size_t)tok * P.L + t.s) * (size_t)P.Q * (size_t)P.split_w;
@@ -784,14 +874,37 @@ __device__ void compute_cta_pair(const FusedParams &P, uint8_t *ring, Control *c
                 __syncwarp();
                 if (lane == 0) mbar_arrive_cluster(mapa_u32(smem_u32(&ctl->tmem_empty[a]), 0u));
             }
-            named_barrier(1, C::kEpiThreads);
-            if (ctl->abort) break;
-            if (is_leader && g != P.withhold) {
-                __threadfence();
-                st_release_u32(&P.flags[2 * g + (int)rank], P.epoch);
-                red_release_add_u32(&P.split_done[t.s], 1u);
+            // hand the tile to the publisher warp (see compute_cta)
+            bool ok2 = ok;
+            if (ok2 && it >= 2)
+                ok2 = wait_barrier(smem_u32(&ctl->pub_done[a]), (uint32_t)((it - 2) >> 1) & 1u, ctl, deadline, P.status,
+                                   (uint32_t)g, 31u);
+            if (!ok2) break;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctl->epi_done[a]));
+            valid = valid_n;
+            f_row = f_row_n;
+            valid_n = valid_nn;
+            first_n = first_nn;
+        }
+    } else if (warp == 3) {
+        // ---------------- publisher (both CTAs): raises this CTA's flag of every finished pair tile
+        if (lane == 0) {
+            int it = 0;
+            for (int g = b; g < total_tiles; g += P.P, ++it) {
+                const int a = it & 1;
+                if (!wait_barrier_1t(smem_u32(&ctl->epi_done[a]), (uint32_t)(it >> 1) & 1u, ctl, deadline, P.status,
+                                     (uint32_t)g, 32u))
+                    break;
+                if (g != P.withhold) {
+                    __threadfence();
+                    st_relaxed_u32(&P.flags[2 * g + (int)rank], P.epoch);
+                    red_relaxed_add_u32(&P.split_done[g / P.W_comp], 1u);
+                }
+                mbar_arrive(smem_u32(&ctl->pub_done[a]));
             }
         }
+        __syncwarp();
     }
     // ---------------- teardown: nobody leaves while its peer may still touch its memory
     tc_fence_before();
