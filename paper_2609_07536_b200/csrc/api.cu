@@ -19,19 +19,7 @@ inline size_t align16(size_t x) { return (x + 15) & ~(size_t)15; }
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 
-constexpr int kSplitCounterWords = 64;  // 2 parities x MOE_MAX_L split counters, then 2 x MOE_MAX_L steal counters, padded
-
-int64_t comm_tiles_of(const moe_shape *s)
-{
-    const int64_t blk = ceil_div(s->T, s->EP);
-    int64_t tok_tiles = 0;
-    for (int d = 0; d < s->EP; ++d) {
-        int64_t own = (int64_t)s->T - (int64_t)d * blk;
-        if (own > blk) own = blk;
-        if (own > 0) tok_tiles += ceil_div(own, kCommTileM);
-    }
-    return tok_tiles * ceil_div(ceil_div(s->H, s->L), kCommTileN);
-}
+constexpr int kSplitCounterWords = 64;  // 2 parities x MOE_MAX_L split counters (32-bit), then 2 x MOE_MAX_L work queues (64-bit), padded
 
 bool shape_ok(const moe_shape *s)
 {
@@ -189,8 +177,7 @@ int32_t moe_workspace_bytes(const moe_shape *s, int32_t tile_m, int32_t tile_n, 
     if (flags_bytes) {
         const size_t nts = (size_t)ceil_div(ceil_div(s->H, s->L), tile_n);
         const size_t parts = (tile_m == 256) ? 2 : 1;   // a pair tile is published in two parts
-        *flags_bytes = ((size_t)kSplitCounterWords + (size_t)s->L * s->TP * mt * nts * parts +
-                        (size_t)s->L * (size_t)comm_tiles_of(s) * 4 /* claims, with room for 4 slices per tile */) * 4 + 16;
+        *flags_bytes = ((size_t)kSplitCounterWords + (size_t)s->L * s->TP * mt * nts * parts) * 4 + 16;
     }
     if (status_bytes) *status_bytes = 16;
     return MOE_OK;
@@ -342,10 +329,9 @@ int32_t moe_gemm2_combine(moe_handle *h, const void *x_routed, const void *W2, c
     p.epoch = ep;
     p.split_done = flags_ws + (ep & 1u) * MOE_MAX_L;
     p.split_done_next = flags_ws + ((ep + 1u) & 1u) * MOE_MAX_L;
-    p.steal = flags_ws + 2 * MOE_MAX_L + (ep & 1u) * MOE_MAX_L;
-    p.steal_next = flags_ws + 2 * MOE_MAX_L + ((ep + 1u) & 1u) * MOE_MAX_L;
+    p.queue = reinterpret_cast<unsigned long long *>(flags_ws + 2 * MOE_MAX_L) + (ep & 1u) * MOE_MAX_L;
+    p.queue_next = reinterpret_cast<unsigned long long *>(flags_ws + 2 * MOE_MAX_L) + ((ep + 1u) & 1u) * MOE_MAX_L;
     p.flags = flags_ws + kSplitCounterWords;
-    p.claims = p.flags + (size_t)s->L * (size_t)p.W_comp * p.flag_parts;
 
     // tensor maps (Section II-A operands): x_routed [R, I] and W2 [E_tot, H, I], k contiguous
     EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(h->encode_tiled);

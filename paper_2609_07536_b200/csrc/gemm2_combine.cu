@@ -135,9 +135,12 @@ __device__ __forceinline__ void cluster_sync_all()
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
+// Arrival that hands back an accumulator buffer.  Relaxed on purpose: what it orders are this warp's
+// TMEM reads, which tcgen05.wait::ld and tcgen05.fence::before_thread_sync have completed; a release
+// at cluster scope would also wait for the warp's outstanding global stores of Y (thousands of cycles).
+__device__ __forceinline__ void mbar_arrive_cluster_relaxed(uint32_t cluster_addr)
 {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+    asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 // each CTA of the pair loads its own operand half; completion is signalled on the leader's barrier
 __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, uint32_t leader_bar, int x, int y)
@@ -226,10 +229,6 @@ __device__ __forceinline__ void red_relaxed_add_u32(uint32_t *p, uint32_t v)
 {
     asm volatile("red.relaxed.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
-__device__ __forceinline__ void named_barrier(int id, int threads)
-{
-    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
-}
 
 // Shared-memory matrix descriptor of a K-major, 128B-swizzled operand tile whose rows are
 // 128 bytes (64 bf16): 8-row groups are 1024 bytes apart (stride byte offset), the leading
@@ -282,7 +281,6 @@ struct Control {
     uint32_t tmem_base;
     volatile uint32_t abort;
     unsigned long long comm_full[24];   // communication CTA: one barrier per warp and stage
-    volatile int claim_slot[2];         // ... and the CTA-wide result of a tile claim
 };
 
 // 32 KB after the control block, used by one role per CTA:
@@ -872,7 +870,7 @@ __device__ void compute_cta_pair(const FusedParams &P, uint8_t *ring, Control *c
                 // this CTA's half of the accumulator buffer is drained: tell the leader's MMA warp
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive_cluster(mapa_u32(smem_u32(&ctl->tmem_empty[a]), 0u));
+                if (lane == 0) mbar_arrive_cluster_relaxed(mapa_u32(smem_u32(&ctl->tmem_empty[a]), 0u));
             }
             // hand the tile to the publisher warp (see compute_cta)
             bool ok2 = ok;
@@ -963,7 +961,6 @@ __device__ __forceinline__ void fma_bf16x8(float (&acc)[8], const uint4 &v, floa
 // weights and stores the bf16 result into the owning rank's buffer.  No warp waits on another one:
 // the issue latency of the copies and the memory latency overlap across the twelve warps.
 constexpr int kCommWarps = 12;
-constexpr int kCommSub = 1;            // token slices a communication tile is claimed in (finer slices measured slower)
 constexpr int kCommUnitBytes = 8192;
 constexpr int kCommWarpBytes = 2 * kCommUnitBytes;
 static_assert(kCommWarps * kCommWarpBytes <= kStageBytesTotal, "communication stages exceed the ring");
@@ -989,7 +986,6 @@ __device__ void comm_cta(const FusedParams &P, uint8_t *ring, Control *ctl, uint
     if (threadIdx.x == 0) {
         for (int i = 0; i < 2 * kCommWarps; ++i) mbar_init(smem_u32(&ctl->comm_full[i]), 1);
         ctl->abort = 0u;
-        ctl->claim_slot[0] = ctl->claim_slot[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -1094,19 +1090,89 @@ __device__ void comm_cta(const FusedParams &P, uint8_t *ring, Control *ctl, uint
     prev.live = false;
     uint32_t ready_mask = wait_needed ? 0u : 0xffffffffu;   // bit s: split s is known to be complete
 
+    // One unit: wait until the GEMM tiles under it are published (unless its split is known to be
+    // complete), start its copy, then reduce the previous unit of this warp while the copy is in flight.
+    // False when the warp had to give up (reported); nothing of this warp is in flight then.
+    auto unit_step = [&](CommUnit &u) -> bool {
+        // ---- readiness of the producing tiles
+        if (!((ready_mask >> u.s) & 1u)) {
+            uint32_t done = 0;
+            if (lane == 0) done = ld_acquire_u32(&P.split_done[u.s]);
+            done = __shfl_sync(0xffffffffu, done, 0);
+            if (done >= (uint32_t)(P.W_comp * P.flag_parts)) {
+                ready_mask |= 1u << u.s;
+            } else {
+                // per tile: every (slot j, shard p, n-tile under this slab)
+                const int cs0 = u.slab << P.slab_shift;
+                const int in0 = cs0 / TN;
+                const int nt = (cs0 + u.ucols - 1) / TN - in0 + 1;
+                bool failed = false;
+                for (int chk = lane; chk < P.Q * nt && !failed; chk += 32) {
+                    const int qq = chk / nt;
+                    const int tn = chk - qq * nt;
+                    const int j = qq / P.TP;
+                    const int p = qq - j * P.TP;
+                    const int row = __ldg(&P.pad_row[(size_t)u.t * P.k_tot + j]);
+                    if (row < 0 || row >= P.R_pad) continue;
+                    const int mu = row / P.tile_m;
+                    // a pair tile is published in two parts, one per CTA: the row's part is its 128-row half
+                    const int part = (P.flag_parts == 2) ? ((row - mu * P.tile_m) >> 7) : 0;
+                    const int g = (u.s * P.W_comp + (mu * P.TP + p) * P.NTs + in0 + tn) * P.flag_parts + part;
+                    uint32_t spins = 0;
+                    while (ld_acquire_u32(&P.flags[g]) != P.epoch) {
+                        if ((++spins & 31u) == 0u && (ctl->abort || globaltimer_ns() > deadline)) {
+                            report(P.status, MOE_DEV_TIMEOUT, (uint32_t)g, 40u);
+                            failed = true;
+                            break;
+                        }
+                        __nanosleep(64);
+                    }
+                }
+                if (__any_sync(0xffffffffu, failed)) {
+                    // this warp gives up; the copy it still has in flight must land first
+                    if (prev.live) consume(prev, (n_mine - 1) & 1, (uint32_t)((n_mine - 1) >> 1) & 1u);
+                    prev.live = false;
+                    return false;
+                }
+            }
+            __syncwarp();
+            // rows published through ordinary stores are read by the copy engine next
+            asm volatile("fence.proxy.async;" ::: "memory");
+        }
+        // ---- issue this unit's copy, then reduce the previous unit while it is in flight
+        const int st = n_mine & 1;
+        if (lane == 0) {
+            const uint32_t full = smem_u32(&ctl->comm_full[2 * warp + st]);
+            const uint32_t bytes = (uint32_t)(P.Q * u.wslab) * 2u;
+            const __nv_bfloat16 *src = Y + ((size_t)u.t * P.L + u.s) * (size_t)P.Q * (size_t)P.split_w +
+                                       ((size_t)u.slab * P.Q << P.slab_shift);
+            mbar_arrive_expect_tx(full, bytes);
+            bulk_load(smem_u32(my_ring + st * kCommUnitBytes), src, bytes, full);
+        }
+        __syncwarp();
+        ++n_mine;
+        if (prev.live && !consume(prev, (n_mine - 2) & 1, (uint32_t)((n_mine - 2) >> 1) & 1u)) {
+            // the previous copy never landed (reported); wait for the one just issued, then leave
+            const unsigned long long drain = globaltimer_ns() + 2000000ull;
+            while (!mbar_try_wait(smem_u32(&ctl->comm_full[2 * warp + st]), (uint32_t)((n_mine - 1) >> 1) & 1u) &&
+                   globaltimer_ns() < drain) {}
+            prev.live = false;
+            return false;
+        }
+        prev = u;
+        return true;
+    };
+
     // serve communication tile ct of split s; false when this warp had to give up (reported)
-    auto serve_tile = [&](int s, int ct, int sub) -> bool {
+    auto serve_tile = [&](int s, int ct) -> bool {
         const int split_c0 = s * P.split_w;
         const int split_c1 = min(P.H, split_c0 + P.split_w);
         const int tok_tile = ct / P.comm_cols;
         const int col_tile = ct - tok_tile * P.comm_cols;
         const int d = tok_tile / P.tok_tiles_per_rank;
         const int ti = tok_tile - d * P.tok_tiles_per_rank;
-        // a communication tile is claimed and served in kCommSub token slices (all of it when sub < 0)
-        const int tile_t0 = d * P.tok_blk + ti * kCommTileM;
-        const int tile_t1 = min(min(P.T, (d + 1) * P.tok_blk), tile_t0 + kCommTileM);
-        const int t0 = sub < 0 ? tile_t0 : tile_t0 + sub * (kCommTileM / kCommSub);
-        const int t1 = sub < 0 ? tile_t1 : min(tile_t1, t0 + kCommTileM / kCommSub);
+        const int t0 = d * P.tok_blk + ti * kCommTileM;
+        const int t1 = min(min(P.T, (d + 1) * P.tok_blk), t0 + kCommTileM);
         const int c0 = split_c0 + col_tile * kCommTileN;
         const int c1 = min(split_c1, c0 + kCommTileN);
         if (t0 >= t1 || c0 >= c1) return true;
@@ -1147,136 +1213,120 @@ __device__ void comm_cta(const FusedParams &P, uint8_t *ring, Control *ctl, uint
                 if (my_row < 0) u.w = 0.f;
             }
             u.all_valid = __all_sync(0xffffffffu, lane >= P.k_tot || my_row >= 0);
-            // ---- readiness of the producing tiles
-            if (!((ready_mask >> s) & 1u)) {
-                uint32_t done = 0;
-                if (lane == 0) done = ld_acquire_u32(&P.split_done[s]);
-                done = __shfl_sync(0xffffffffu, done, 0);
-                if (done >= (uint32_t)(P.W_comp * P.flag_parts)) {
-                    ready_mask |= 1u << s;
-                } else {
-                    // per tile: every (slot j, shard p, n-tile under this slab)
-                    const int cs0 = u.slab << P.slab_shift;
-                    const int in0 = cs0 / TN;
-                    const int nt = (cs0 + u.ucols - 1) / TN - in0 + 1;
-                    bool failed = false;
-                    for (int chk = lane; chk < P.Q * nt && !failed; chk += 32) {
-                        const int qq = chk / nt;
-                        const int tn = chk - qq * nt;
-                        const int j = qq / P.TP;
-                        const int p = qq - j * P.TP;
-                        const int row = __ldg(&P.pad_row[(size_t)u.t * P.k_tot + j]);
-                        if (row < 0 || row >= P.R_pad) continue;
-                        const int mu = row / P.tile_m;
-                        // a pair tile is published in two parts, one per CTA: the row's part is its 128-row half
-                        const int part = (P.flag_parts == 2) ? ((row - mu * P.tile_m) >> 7) : 0;
-                        const int g = (s * P.W_comp + (mu * P.TP + p) * P.NTs + in0 + tn) * P.flag_parts + part;
-                        uint32_t spins = 0;
-                        while (ld_acquire_u32(&P.flags[g]) != P.epoch) {
-                            if ((++spins & 31u) == 0u && (ctl->abort || globaltimer_ns() > deadline)) {
-                                report(P.status, MOE_DEV_TIMEOUT, (uint32_t)g, 40u);
-                                failed = true;
-                                break;
-                            }
-                            __nanosleep(64);
-                        }
-                    }
-                    if (__any_sync(0xffffffffu, failed)) {
-                        // this warp gives up; the copy it still has in flight must land first
-                        if (prev.live) consume(prev, (n_mine - 1) & 1, (uint32_t)((n_mine - 1) >> 1) & 1u);
-                        prev.live = false;
-                        unit += n_units;
-                        return false;
-                    }
-                }
-                __syncwarp();
-                // rows published through ordinary stores are read by the copy engine next
-                asm volatile("fence.proxy.async;" ::: "memory");
-            }
-            // ---- issue this unit's copy, then reduce the previous unit while it is in flight
-            const int st = n_mine & 1;
-            if (lane == 0) {
-                const uint32_t full = smem_u32(&ctl->comm_full[2 * warp + st]);
-                const uint32_t bytes = (uint32_t)(P.Q * u.wslab) * 2u;
-                const __nv_bfloat16 *src = Y + ((size_t)u.t * P.L + s) * (size_t)P.Q * (size_t)P.split_w +
-                                           ((size_t)u.slab * P.Q << P.slab_shift);
-                mbar_arrive_expect_tx(full, bytes);
-                bulk_load(smem_u32(my_ring + st * kCommUnitBytes), src, bytes, full);
-            }
-            __syncwarp();
-            ++n_mine;
-            if (prev.live && !consume(prev, (n_mine - 2) & 1, (uint32_t)((n_mine - 2) >> 1) & 1u)) {
-                // the previous copy never landed (reported); wait for the one just issued, then leave
-                const unsigned long long drain = globaltimer_ns() + 2000000ull;
-                while (!mbar_try_wait(smem_u32(&ctl->comm_full[2 * warp + st]), (uint32_t)((n_mine - 1) >> 1) & 1u) &&
-                       globaltimer_ns() < drain) {}
-                prev.live = false;
+            if (!unit_step(u)) {
                 unit += n_units;
                 return false;
             }
-            prev = u;
         }
         unit += n_units;
         return true;
     };
 
-    // CTA-wide decision taken by one thread and read by all twelve working warps.  Two result slots
-    // alternate, so one barrier per decision is enough.
-    int n_decisions = 0;
-    auto broadcast = [&](int value_from_warp0_lane0) -> int {
-        volatile int *slot = &ctl->claim_slot[n_decisions & 1];
-        if (warp == 0 && lane == 0) *slot = value_from_warp0_lane0;
-        named_barrier(3, kCommWarps * 32);
-        ++n_decisions;
-        return *slot;
-    };
-    bool dead = false;   // this warp gave up; it keeps meeting the others at the decision barriers
-
-    if (!helper) {
-        for (int s = 0; s < P.L; ++s) {
-            for (int ct = c; ct < P.comm_tiles; ct += P.C) {
-                if (!claiming) {
-                    if (!serve_tile(s, ct, -1)) {
-                        ctl->abort = 1u;
-                        return;               // no CTA-wide barriers in this mode: the warp may leave
-                    }
-                    continue;
+    // serve items [i0, i1) of split s on this warp alone.  An item is one token x one communication
+    // column tile (token-major numbering); its units are the column slabs of that tile.
+    auto serve_items = [&](int s, uint32_t i0, uint32_t i1) -> bool {
+        const int split_c0 = s * P.split_w;
+        const int split_c1 = min(P.H, split_c0 + P.split_w);
+        int nxt_row = -1;
+        float nxt_w = 0.f;
+        if (lane < P.k_tot) {
+            const int tn = (int)(i0 / (uint32_t)P.comm_cols);
+            nxt_row = __ldg(&P.pad_row[(size_t)tn * P.k_tot + lane]);
+            nxt_w = __ldg(&P.topk_w[(size_t)tn * P.k_tot + lane]);
+        }
+        for (uint32_t item = i0; item < i1; ++item) {
+            const int tok = (int)(item / (uint32_t)P.comm_cols);
+            const int col_tile = (int)(item - (uint32_t)tok * (uint32_t)P.comm_cols);
+            int my_row = nxt_row;
+            float my_w = nxt_w;
+            if (item + 1 < i1 && lane < P.k_tot) {
+                const int tn = (int)((item + 1) / (uint32_t)P.comm_cols);
+                nxt_row = __ldg(&P.pad_row[(size_t)tn * P.k_tot + lane]);
+                nxt_w = __ldg(&P.topk_w[(size_t)tn * P.k_tot + lane]);
+            }
+            if (lane < P.k_tot) {
+                if (my_row >= P.R_pad) {
+                    report(P.status, MOE_DEV_OOB, (uint32_t)my_row, 42u);
+                    my_row = -1;
                 }
-                for (int sub = 0; sub < kCommSub; ++sub) {
-                    int mine = 0;
-                    if (warp == 0 && lane == 0)
-                        mine = (atomicExch(&P.claims[(s * P.comm_tiles + ct) * kCommSub + sub], P.epoch) != P.epoch) ? 1 : 0;
-                    mine = broadcast(mine);
-                    if (ctl->abort) { s = P.L; ct = P.comm_tiles; break; }
-                    if (!mine) continue;      // a helper took it
-                    if (!dead && !serve_tile(s, ct, sub)) {
-                        dead = true;
-                        ctl->abort = 1u;
-                    }
-                }
+                if (my_row < 0) my_w = 0.f;
+            }
+            const bool all_valid = __all_sync(0xffffffffu, lane >= P.k_tot || my_row >= 0);
+            const int c0 = split_c0 + col_tile * kCommTileN;
+            const int c1 = min(split_c1, c0 + kCommTileN);
+            if (c0 >= c1) continue;
+            const int slab0 = (c0 - split_c0) >> P.slab_shift;
+            const int slab1 = (c1 - split_c0 + P.slab_cols - 1) >> P.slab_shift;
+            for (int slab = slab0; slab < slab1; ++slab) {
+                CommUnit u;
+                u.t = tok;
+                u.d = tok / P.tok_blk;
+                u.s = s;
+                u.slab = slab;
+                u.wslab = min(P.slab_cols, P.split_w - (slab << P.slab_shift));
+                u.ucols = min(u.wslab, split_c1 - split_c0 - (slab << P.slab_shift));
+                u.w = my_w;
+                u.live = true;
+                u.all_valid = all_valid;
+                if (!unit_step(u)) return false;
             }
         }
-    } else {
-        // a compute CTA that ran out of GEMM tiles: take unclaimed tile slices from the back, last split first
-        const uint32_t n_slices = (uint32_t)(P.comm_tiles * kCommSub);
-        for (int s = P.L - 1; s >= 0; --s) {
-            for (;;) {
-                int slice = -1;
-                if (warp == 0 && lane == 0) {
-                    for (;;) {
-                        const uint32_t idx = atomicAdd(&P.steal[s], 1u);
-                        if (idx >= n_slices) break;
-                        const int cand = (int)(n_slices - 1u - idx);
-                        if (atomicExch(&P.claims[s * (int)n_slices + cand], P.epoch) != P.epoch) { slice = cand; break; }
-                    }
-                }
-                slice = broadcast(slice);
-                if (ctl->abort) { s = -1; break; }
-                if (slice < 0) break;
-                if (!dead && !serve_tile(s, slice / kCommSub, slice % kCommSub)) {
-                    dead = true;
+        return true;
+    };
+
+    if (!claiming) {
+        // the paper's static map: communication tile ct belongs to CTA ct mod C (Section III-A)
+        for (int s = 0; s < P.L; ++s)
+            for (int ct = c; ct < P.comm_tiles; ct += P.C)
+                if (!serve_tile(s, ct)) {
                     ctl->abort = 1u;
+                    return;
                 }
+    } else {
+        // Drain help: work is handed out dynamically, to warps.  Every split has a two-ended queue of
+        // its items in one 64-bit word (low half: items taken from the front, high half: from the back).
+        // Warps of the communication CTAs take from the front, split 0 first; warps of compute CTAs that
+        // have run out of GEMM tiles take from the back, last split first.  One atomic add claims a
+        // range; ranges shrink towards the end so that the last ones finish together.  The next claim is
+        // issued before the current range is served, which hides the latency of the atomic.
+        const uint32_t n_items = (uint32_t)P.T * (uint32_t)P.comm_cols;
+        int s = helper ? P.L - 1 : 0;
+        unsigned long long old = 0;
+        uint32_t chunk = 0;
+        auto claim = [&](int split) {   // lane 0 issues the atomic; the result is picked up later
+            if (lane == 0) {
+                const unsigned long long q = *reinterpret_cast<volatile unsigned long long *>(&P.queue[split]);
+                const uint32_t taken = (uint32_t)q + (uint32_t)(q >> 32);
+                const uint32_t rem = taken < n_items ? n_items - taken : 0u;
+                chunk = min(8u, max(1u, rem >> 12));
+                old = atomicAdd(&P.queue[split], helper ? ((unsigned long long)chunk << 32) : (unsigned long long)chunk);
+            }
+        };
+        claim(s);
+        while (s >= 0 && s < P.L) {
+            const unsigned long long o = __shfl_sync(0xffffffffu, old, 0);
+            const uint32_t ch = __shfl_sync(0xffffffffu, chunk, 0);
+            const uint32_t f = (uint32_t)o, bk = (uint32_t)(o >> 32);
+            const uint32_t hi = bk < n_items ? n_items - bk : 0u;    // items [hi, n) are taken from the back
+            uint32_t i0, i1;
+            if (!helper) {
+                i0 = f;
+                i1 = min(f + ch, hi);
+            } else {
+                i1 = hi;
+                i0 = max(f, hi > ch ? hi - ch : 0u);
+            }
+            const int cur = s;
+            if (i0 >= i1) {                      // this split is handed out: go on to the next one
+                s += helper ? -1 : 1;
+                if (s >= 0 && s < P.L) claim(s);
+                continue;
+            }
+            claim(s);
+            if (ctl->abort) break;
+            if (!serve_items(cur, i0, i1)) {
+                ctl->abort = 1u;
+                return;
             }
         }
     }
@@ -1297,7 +1347,7 @@ moe_gemm2_combine_kernel(const __grid_constant__ FusedParams P)
 
     if (blockIdx.x == 0 && threadIdx.x < (unsigned)P.L) {
         P.split_done_next[threadIdx.x] = 0u;
-        P.steal_next[threadIdx.x] = 0u;
+        P.queue_next[threadIdx.x] = 0ull;
     }
 
     if ((int)blockIdx.x < P.C)
@@ -1321,7 +1371,7 @@ moe_gemm2_combine_pair_kernel(const __grid_constant__ FusedParams P)
 
     if (blockIdx.x == 0 && threadIdx.x < (unsigned)P.L) {
         P.split_done_next[threadIdx.x] = 0u;
-        P.steal_next[threadIdx.x] = 0u;
+        P.queue_next[threadIdx.x] = 0ull;
     }
 
     const int c_even = (P.C + 1) & ~1;

@@ -37,9 +37,8 @@ struct alignas(64) FusedParams {
     uint32_t *flags;               // [L * W_comp] readiness per global tile (== epoch when ready)
     uint32_t *split_done;          // [L] tiles finished per split (this launch)
     uint32_t *split_done_next;     // [L] counters of the next launch, zeroed by this one
-    uint32_t *steal;               // [L] communication tiles handed to helper CTAs so far (this launch)
-    uint32_t *steal_next;          // [L] ... of the next launch, zeroed by this one
-    uint32_t *claims;              // [L * comm_tiles] == epoch once a CTA has taken the tile
+    unsigned long long *queue;     // [L] drain help: items of the split handed out so far, front | back << 32
+    unsigned long long *queue_next;  // [L] ... of the next launch, zeroed by this one
     uint32_t *status;              // 4 words
     void *out[MOE_MAX_EP];
     unsigned long long wait_ns;
