@@ -1377,7 +1377,11 @@ moe_gemm2_combine_pair_kernel(const __grid_constant__ FusedParams P)
     const int c_even = (P.C + 1) & ~1;
     if ((int)blockIdx.x < P.C)
         comm_cta<256>(P, ring, ctl, aux, (int)blockIdx.x, false);
-    else if ((int)blockIdx.x >= c_even) {
+    else if ((int)blockIdx.x < c_even) {
+        // odd C: the last communication CTA's cluster-mate cannot compute (no partner).  With dynamic work
+        // distribution it serves communication work as well; under the static map it has no tile list.
+        if (P.drain_help && P.mode == MOE_MODE_FUSED) comm_cta<256>(P, ring, ctl, aux, (int)blockIdx.x, false);
+    } else {
         compute_cta_pair(P, ring, ctl, aux, ((int)blockIdx.x - c_even) >> 1);
         if (P.drain_help && P.mode == MOE_MODE_FUSED && !ctl->abort) comm_cta<256>(P, ring, ctl, aux, 0, true);
     }

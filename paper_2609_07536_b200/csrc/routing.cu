@@ -212,7 +212,7 @@ extern "C" int32_t moe_build_routing_static(moe_handle *h, const int32_t *topk_i
     if (s->T < 0 || s->k_tot < 1 || s->k_tot > 32 || s->E_tot < 1 || s->E_tot > 1024 ||
         (int64_t)s->T * s->k_tot >= (int64_t)1 << 30)
         return MOE_ERR_SHAPE;
-    if (tile_m != 64 && tile_m != 128) return MOE_ERR_UNSUPPORTED;
+    if (tile_m != 64 && tile_m != 128 && tile_m != 256) return MOE_ERR_UNSUPPORTED;
     if (s->T > 0 && !topk_idx) return MOE_ERR_NULL;
     const int64_t R = (int64_t)s->T * s->k_tot;
     if (r->max_mtiles < (int32_t)(R / tile_m + s->E_tot)) return MOE_ERR_SHAPE;

@@ -72,17 +72,17 @@ GRANITE = Workload("granite3moe", T=4096, H=1536, I=512, E=40, k=8, TP=2, EP=2,
                    tile_m=128, tile_n=256, L=1, routing="zipf", zipf_s=1.0,
                    target_r_expert=2.5, routing_seed=0, data_seed=1)
 QWEN = Workload("qwen15moe", T=8192, H=2048, I=1408, E=60, k=4, TP=2, EP=2,
-                tile_m=128, tile_n=256, L=2, routing="zipf", zipf_s=1.0,
+                tile_m=256, tile_n=256, L=2, routing="zipf", zipf_s=1.0,
                 target_r_expert=2.5, routing_seed=0, data_seed=1)
 DSV2L = Workload("dsv2lite", T=16384, H=2048, I=1408, E=64, k=6, n_shared=2, TP=2, EP=2,
-                 tile_m=128, tile_n=256, L=2, routing="zipf", zipf_s=1.2,
+                 tile_m=256, tile_n=256, L=2, routing="zipf", zipf_s=1.2,
                  target_r_expert=3.0, routing_seed=0, data_seed=1)
 
 CONFIGS = {w.name: w for w in (TINY, GRANITE, QWEN, DSV2L)}
 
 
 def sweep_workloads(T_list=(1024, 2048, 4096, 8192, 16384, 32768), s_list=(0.0, 0.6, 1.2),
-                    EP_list=(1, 2, 4), tiles=((128, 128), (128, 256))):
+                    EP_list=(1, 2, 4), tiles=((128, 256), (256, 256))):
     """The selector-regret sweep on the DeepSeek-V2-Lite shape."""
     out = []
     for iT, T in enumerate(T_list):

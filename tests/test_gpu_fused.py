@@ -92,7 +92,7 @@ def test_qwen_config_sampled():
 
 
 def test_dsv2lite_config_sampled_in_bench_configuration():
-    # the launch configuration bench.py times: analytical plan, 128x256 tiles, L = 2
+    # the launch configuration bench.py times: analytical plan, 256x256 CTA-pair tiles, L = 2
     _check_against_oracle(wl.DSV2L, n_random=160)
 
 
@@ -104,11 +104,15 @@ def test_dsv2lite_config_sampled_in_bench_configuration():
     dict(T=1030, E=70, k=2, H=512, I=256, TP=2, EP=8, tile_m=128, tile_n=128, L=8),  # empty experts, L = 8
     dict(T=200, E=6, k=2, n_shared=2, H=256, I=128, TP=1, EP=1, tile_m=128, tile_n=64, L=2),  # shared experts
 ], ids=lambda kw: "-".join(f"{k}{v}" for k, v in kw.items()))
-def test_edge_shapes(kw):
+@pytest.mark.parametrize("drain_help", [0, 1], ids=["static", "drain_help"])
+def test_edge_shapes(kw, drain_help):
+    # both ways of handing out the communication work: the paper's static tile -> CTA map, and warps
+    # pulling token ranges from the two-ended queue (for a forced C that leaves most of it to helpers)
     base = dict(name="edge", routing_seed=3, data_seed=4, TP=1, EP=1, L=1)
     base.update(kw)
     w = replace(wl.TINY, **base)
-    _check_against_oracle(w)
+    _check_against_oracle(w, drain_help=drain_help)
+    _check_against_oracle(w, drain_help=drain_help, force_C=2)
 
 
 def test_one_hot_expert_and_forced_counts():
