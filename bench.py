@@ -569,7 +569,7 @@ def main():
             "roofline": roofline,
             "e2e": {"value": job_value(e2e_us, world), "unit": "us/layer", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": Ke},
-            "gpu_launches": 4 * K,
+            "gpu_launches": 5 * K,
             "clocks": clocks,
             "paper_context": {"hardware": "4xA100-SXM4-40GB", "mean_regret": 0.0322, "solver_us": 0.157,
                               "geomean_speedup_over_comet": 2.528},

@@ -57,63 +57,79 @@ routing_hist(const int32_t *__restrict__ topk_idx, int R, int k_tot, int E_tot, 
     }
 }
 
-__global__ void __launch_bounds__(1024)
-routing_scan(int R, int E_tot, int tile_m, int n_warps, int max_mtiles,
-             int32_t *__restrict__ whist, int32_t *counts, int32_t *offsets, int32_t *tiles,
-             int32_t *tile_offsets, int32_t *mtile_expert, int32_t *mtile_first_row,
-             int32_t *mtile_valid, uint32_t *status)
+// Per expert (one CTA each): counts[e], and whist[.][e] turned into an exclusive prefix over the
+// sorting warps.  Thread t owns a contiguous run of warps; the run sums are scanned across the CTA.
+constexpr int kScanThreads = 256;
+__global__ void __launch_bounds__(kScanThreads)
+routing_scan_columns(int E_tot, int n_warps, int32_t *__restrict__ whist, int32_t *__restrict__ counts)
 {
-    // counts, and whist turned into an exclusive prefix over the (sorting) warps, per expert: one warp
-    // of this CTA per expert, 32 entries per step with a shuffle scan
-    {
-        const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, n_w = blockDim.x >> 5;
-        for (int e = wid; e < E_tot; e += n_w) {
-            int run = 0;
-            for (int w0 = 0; w0 < n_warps; w0 += 32) {
-                const int w = w0 + lane;
-                const int c = (w < n_warps) ? whist[(size_t)w * E_tot + e] : 0;
-                int incl = c;
+    __shared__ int warp_sum[kScanThreads / 32];
+    const int e = blockIdx.x, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const int chunk = (n_warps + kScanThreads - 1) / kScanThreads;
+    const int w_lo = min(n_warps, tid * chunk), w_hi = min(n_warps, w_lo + chunk);
+    int sum = 0;
+    for (int w = w_lo; w < w_hi; ++w) sum += whist[(size_t)w * E_tot + e];
+    int incl = sum;
 #pragma unroll
-                for (int d = 1; d < 32; d <<= 1) {
-                    const int up = __shfl_up_sync(0xffffffffu, incl, d);
-                    if (lane >= d) incl += up;
-                }
-                if (w < n_warps) whist[(size_t)w * E_tot + e] = run + incl - c;
-                run += __shfl_sync(0xffffffffu, incl, 31);
-            }
-            if (lane == 0) counts[e] = run;
-        }
+    for (int d = 1; d < 32; d <<= 1) {
+        const int up = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += up;
     }
+    if (lane == 31) warp_sum[wid] = incl;
+    __syncthreads();
+    int base = incl - sum;
+    for (int i = 0; i < wid; ++i) base += warp_sum[i];
+    for (int w = w_lo; w < w_hi; ++w) {
+        const int c = whist[(size_t)w * E_tot + e];
+        whist[(size_t)w * E_tot + e] = base;
+        base += c;
+    }
+    if (tid == kScanThreads - 1) counts[e] = base;
+}
+
+// Offsets, tile counts and the m-tile table from the per-expert counts (one CTA; the prefix over the
+// experts is serial but runs in shared memory).  Dynamic shared memory: 3 * (E_tot + 1) ints.
+__global__ void __launch_bounds__(1024)
+routing_finalize(int E_tot, int tile_m, int max_mtiles, const int32_t *__restrict__ counts,
+                 int32_t *__restrict__ offsets, int32_t *__restrict__ tiles, int32_t *__restrict__ tile_offsets,
+                 int32_t *__restrict__ mtile_expert, int32_t *__restrict__ mtile_first_row,
+                 int32_t *__restrict__ mtile_valid, uint32_t *status)
+{
+    extern __shared__ int32_t fin[];
+    int32_t *s_cnt = fin, *s_off = fin + (E_tot + 1), *s_toff = fin + 2 * (E_tot + 1);
+    for (int e = threadIdx.x; e < E_tot; e += blockDim.x) s_cnt[e] = counts[e];
     __syncthreads();
     if (threadIdx.x == 0) {
         int off = 0, toff = 0;
         for (int e = 0; e < E_tot; ++e) {
-            const int c = counts[e];
-            const int nt = (c + tile_m - 1) / tile_m;
-            offsets[e] = off;
-            tile_offsets[e] = toff;
-            tiles[e] = nt;
-            off += c;
-            toff += nt;
+            s_off[e] = off;
+            s_toff[e] = toff;
+            off += s_cnt[e];
+            toff += (s_cnt[e] + tile_m - 1) / tile_m;
         }
-        offsets[E_tot] = off;
-        tile_offsets[E_tot] = toff;
-        tiles[E_tot] = toff;  // S rides behind the per-expert counts for the host copy
+        s_off[E_tot] = off;
+        s_toff[E_tot] = toff;
         if (toff > max_mtiles) report(status, MOE_DEV_OOB, (uint32_t)toff, 2u);
     }
     __syncthreads();
+    for (int e = threadIdx.x; e <= E_tot; e += blockDim.x) {
+        offsets[e] = s_off[e];
+        tile_offsets[e] = s_toff[e];
+        // S rides behind the per-expert tile counts for the host copy
+        tiles[e] = (e < E_tot) ? s_toff[e + 1] - s_toff[e] : s_toff[E_tot];
+    }
     // m-tile table, one thread per m-tile: the expert is found by bisection in the tile prefix
-    const int S = min(tile_offsets[E_tot], max_mtiles);
+    const int S = min(s_toff[E_tot], max_mtiles);
     for (int mu = threadIdx.x; mu < S; mu += blockDim.x) {
         int lo = 0, hi = E_tot - 1;          // largest e with tile_offsets[e] <= mu
         while (lo < hi) {
             const int mid = (lo + hi + 1) >> 1;
-            if (tile_offsets[mid] <= mu) lo = mid; else hi = mid - 1;
+            if (s_toff[mid] <= mu) lo = mid; else hi = mid - 1;
         }
-        const int e = lo, i = mu - tile_offsets[e];
+        const int e = lo, i = mu - s_toff[e];
         mtile_expert[mu] = e;
-        mtile_first_row[mu] = offsets[e] + i * tile_m;
-        mtile_valid[mu] = min(tile_m, counts[e] - i * tile_m);
+        mtile_first_row[mu] = s_off[e] + i * tile_m;
+        mtile_valid[mu] = min(tile_m, s_cnt[e] - i * tile_m);
     }
 }
 
@@ -165,9 +181,10 @@ cudaError_t routing_launch(const int32_t *topk_idx, const moe_shape &s, int tile
     if (blocks > 0)
         routing_hist<<<blocks, kWarpsPerBlock * 32, sh, stream>>>(topk_idx, R, s.k_tot, s.E_tot, n_warps,
                                                                   r.scratch, status);
-    routing_scan<<<1, 1024, 0, stream>>>(R, s.E_tot, tile_m, n_warps, r.max_mtiles, r.scratch, r.counts,
-                                         r.offsets, r.tiles, r.tile_offsets, r.mtile_expert,
-                                         r.mtile_first_row, r.mtile_valid, status);
+    routing_scan_columns<<<s.E_tot, kScanThreads, 0, stream>>>(s.E_tot, n_warps, r.scratch, r.counts);
+    routing_finalize<<<1, 1024, 3 * (size_t)(s.E_tot + 1) * sizeof(int32_t), stream>>>(
+        s.E_tot, tile_m, r.max_mtiles, r.counts, r.offsets, r.tiles, r.tile_offsets, r.mtile_expert,
+        r.mtile_first_row, r.mtile_valid, status);
     if (blocks > 0)
         routing_scatter<<<blocks, kWarpsPerBlock * 32, sh, stream>>>(
             topk_idx, R, s.E_tot, tile_m, n_warps, r.scratch, r.offsets, r.tile_offsets, r.perm,
@@ -249,9 +266,10 @@ extern "C" int32_t moe_build_routing_static(moe_handle *h, const int32_t *topk_i
     const size_t sh = (size_t)kWarpsPerBlock * s->E_tot * sizeof(int32_t);
     if (blocks > 0)
         routing_hist<<<blocks, kWarpsPerBlock * 32, sh, st>>>(topk_idx, iR, s->k_tot, s->E_tot, nw, scratch, status_dev);
-    routing_scan<<<1, 1024, 0, st>>>(iR, s->E_tot, tile_m, nw, r->max_mtiles, scratch, r->counts, r->offsets,
-                                     r->tiles, r->tile_offsets, r->mtile_expert, r->mtile_first_row,
-                                     r->mtile_valid, status_dev);
+    routing_scan_columns<<<s->E_tot, kScanThreads, 0, st>>>(s->E_tot, nw, scratch, r->counts);
+    routing_finalize<<<1, 1024, 3 * (size_t)(s->E_tot + 1) * sizeof(int32_t), st>>>(
+        s->E_tot, tile_m, r->max_mtiles, r->counts, r->offsets, r->tiles, r->tile_offsets, r->mtile_expert,
+        r->mtile_first_row, r->mtile_valid, status_dev);
     if (blocks > 0)
         routing_scatter<<<blocks, kWarpsPerBlock * 32, sh, st>>>(topk_idx, iR, s->E_tot, tile_m, nw, scratch,
                                                                 r->offsets, r->tile_offsets, r->perm,
