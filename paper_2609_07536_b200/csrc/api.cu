@@ -311,6 +311,8 @@ int32_t moe_gemm2_combine(moe_handle *h, const void *x_routed, const void *W2, c
     }
     p.topk_w = topk_w;
     p.Y = y_ws;
+    p.wide_store = (p.slab_cols >= 32 && p.split_w % 16 == 0 && s->H % 16 == 0 &&
+                    (reinterpret_cast<uintptr_t>(y_ws) & 31u) == 0) ? 1 : 0;
     p.status = status_dev;
     for (int d = 0; d < s->EP; ++d) p.out[d] = out[d];
 

@@ -393,6 +393,45 @@ __device__ __forceinline__ void store_accumulator_rows(const FusedParams &P, uin
     }
 }
 
+// Same job with 256-bit stores: every lane writes 32 bytes (one full sector) of its own row, twice
+// per 32-column group, straight from registers.  Needs every 16-column group whole and 32-byte aligned
+// (FusedParams::wide_store).  No shared memory and no intra-warp hand-over: this is the fastest of the
+// three when the epilogue is what limits a short-K tile.
+__device__ __forceinline__ void st_global_v8(void *p, const uint32_t (&w)[8])
+{
+    asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]),
+                 "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
+}
+__device__ __forceinline__ void store_accumulator_rows_wide(const FusedParams &P, uint32_t taddr, int col_first, int n_cols, bool row_ok,
+                                                            __nv_bfloat16 *ybase, int q, int n0, int col_end, int cis0)
+{
+#pragma unroll 1
+    for (int cc = 0; cc < n_cols; cc += 32) {
+        const int col = col_first + cc;
+        uint32_t r[32];
+        tmem_ld_32x32(taddr + (uint32_t)col, r);
+        const int cis = cis0 + col;
+        const int slab = cis >> P.slab_shift;
+        const int wslab = min(P.slab_cols, P.split_w - (slab << P.slab_shift));
+        __nv_bfloat16 *dst = ybase + ((size_t)slab * P.Q << P.slab_shift) + (size_t)q * wslab + (cis & (P.slab_cols - 1));
+        tmem_ld_wait();
+        if (row_ok) {
+#pragma unroll
+            for (int v = 0; v < 2; ++v) {
+                if (n0 + col + v * 16 < col_end) {
+                    uint32_t w[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[v * 16 + 2 * i]), __uint_as_float(r[v * 16 + 2 * i + 1]));
+                        w[i] = *reinterpret_cast<uint32_t *>(&h);
+                    }
+                    st_global_v8(dst + v * 16, w);
+                }
+            }
+        }
+    }
+}
+
 // Same job with the stores coalesced: the warp's 32 rows x 32 columns go through a padded staging
 // buffer, so that four lanes write one row's 64 contiguous bytes (two full sectors) instead of every
 // lane writing 16 bytes of a different row.  Needs the 32-column group inside one column slab.
@@ -614,7 +653,10 @@ __device__ void compute_cta(const FusedParams &P, uint8_t *ring, Control *ctl, u
                     q = (f - tok * P.k_tot) * P.TP + t.p;
                     ybase = Y + ((size_t)tok * P.L + t.s) * (size_t)P.Q * (size_t)P.split_w;
                 }
-                if (P.slab_cols >= 32)
+                if (P.wide_store)
+                    store_accumulator_rows_wide(P, tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(a * TN), col_first,
+                                                n_cols, row_ok, ybase, q, n0, col_end, n0 - t.s * P.split_w);
+                else if (P.slab_cols >= 32)
                     store_accumulator_rows_staged(
                         P, tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(a * TN), col_first, n_cols, row_ok,
                         ybase, q, n0, col_end, n0 - t.s * P.split_w, reinterpret_cast<EpiStage *>(aux) + (warp - 4));
@@ -859,7 +901,10 @@ __device__ void compute_cta_pair(const FusedParams &P, uint8_t *ring, Control *c
                     q = (f - tok * P.k_tot) * P.TP + t.p;
                     ybase = Y + ((size_t)tok * P.L + t.s) * (size_t)P.Q * (size_t)P.split_w;
                 }
-                if (P.slab_cols >= 32)
+                if (P.wide_store)
+                    store_accumulator_rows_wide(P, tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(a * TN), col_first,
+                                                n_cols, row_ok, ybase, q, n0, col_end, n0 - t.s * P.split_w);
+                else if (P.slab_cols >= 32)
                     store_accumulator_rows_staged(
                         P, tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(a * TN), col_first, n_cols, row_ok,
                         ybase, q, n0, col_end, n0 - t.s * P.split_w, reinterpret_cast<EpiStage *>(aux) + (warp - 4));
