@@ -86,9 +86,11 @@ typedef struct {
     int32_t force_comm_ctas; /* > 0: use exactly this C */
     int32_t selector_off;    /* != 0: use default_C */
     int32_t default_C;       /* the fixed count used when the selector is off */
-    int32_t drain_help;      /* != 0: compute CTAs that run out of GEMM tiles serve the communication tiles
-                                that are left (an extension of this library, not in the paper: with it the
-                                selector models the tail after the last compute wave as served by every SM);
+    int32_t drain_help;      /* != 0: compute CTAs that run out of GEMM tiles serve the communication work
+                                that is left, and the work is handed out dynamically (warps pull token ranges
+                                from a queue per split) instead of by the static tile -> CTA map (an extension
+                                of this library, not in the paper: with it the selector models the tail after
+                                the last compute wave as served by every SM);
                                 0: the paper's static partition and its recurrence exactly */
 } moe_sm_limits;
 
@@ -160,7 +162,7 @@ int32_t moe_query_occupancy(moe_handle *h, int32_t tile_m, int32_t tile_n,
 
 /* Sizes of the caller-allocated workspaces [bytes]: routing arrays, the tile-padded GEMM2
  * output Y (bf16, token-major: [T][L][k_tot * TP][ceil(H/L)]), readiness flags + split counters +
- * tile claims (must be zero-filled once before first use and not shared between handles), status
+ * work queues (must be zero-filled once before first use and not shared between handles), status
  * (16 bytes). */
 int32_t moe_workspace_bytes(const moe_shape *shape, int32_t tile_m, int32_t tile_n,
                             size_t *routing_bytes, size_t *y_bytes, size_t *flags_bytes,
