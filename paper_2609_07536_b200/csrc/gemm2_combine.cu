@@ -3,7 +3,8 @@
 //
 //   blockIdx <  C : communication CTA c (Section II-B: consumes published results; the same
 //                   C CTAs serve all splits in sequence; CTA c takes communication tiles
-//                   c, c+C, ... of a split).
+//                   c, c+C, ... of a split -- or, with drain help, its warps pull token ranges
+//                   from a queue per split that former compute CTAs also serve).
 //   blockIdx >= C : compute CTA b = blockIdx - C (Section III-C: takes global tiles
 //                   b, b+P, b+2P, ... of the split-major sequence in which the expert
 //                   problems of one split are contiguous).
@@ -13,8 +14,9 @@
 //               W2 tile (tile_n rows x 64 k) of every k-block, into a ring of 128B-swizzled stages;
 //   warp 1      MMA issuer (one thread): tcgen05.mma (M = 128, N = tile_n, K = 16, bf16 -> fp32) into one
 //               of two TMEM accumulator buffers; tcgen05.commit frees stages / publishes the tile;
-//   warps 4-15  epilogue: tcgen05.ld -> bf16 -> Y, then the tile's readiness flag (st.release.gpu) and
-//               the split counter (red.release.gpu).
+//   warps 4-15  epilogue: tcgen05.ld -> bf16 -> Y (three column groups x four TMEM lane quarters);
+//   warp 3      publisher (one thread): once the twelve epilogue warps have stored a tile, release fence,
+//               then the tile's readiness flag and the split counter.
 // Compute CTA pair (256 x 256 tiles): the same roles in both CTAs of a cluster of two; one
 //   tcgen05.mma.cta_group::2 spans both SMs, each CTA loads only its own operand halves.
 // Y is token-major: the epilogue scatters each accumulator row to its (token, slot, shard) place, so
@@ -197,7 +199,18 @@ __device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32])
         : "r"(taddr)
         : "memory");
 }
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// The same wait, naming the registers a preceding tcgen05.ld fills: the compiler then cannot move a use
+// of them above the wait (it sees only opaque asm statements, not the asynchronous write).
+__device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32])
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                   "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+                   "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+                   "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+                 :
+                 : "memory");
+}
 
 __device__ __forceinline__ uint4 lds_v4(uint32_t addr)
 {
@@ -367,7 +380,7 @@ __device__ __forceinline__ void store_accumulator_rows(const FusedParams &P, uin
         const int col = col_first + cc;
         uint32_t r[32];
         tmem_ld_32x32(taddr + (uint32_t)col, r);
-        tmem_ld_wait();
+        tmem_ld_wait(r);
         if (row_ok) {
 #pragma unroll
             for (int v = 0; v < 4; ++v) {
@@ -402,33 +415,38 @@ __device__ __forceinline__ void st_global_v8(void *p, const uint32_t (&w)[8])
     asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]),
                  "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
 }
+// one 32-column group of this thread's row: bf16, two 32-byte stores
+__device__ __forceinline__ void emit_wide(const FusedParams &P, const uint32_t (&r)[32], int col, bool row_ok,
+                                          __nv_bfloat16 *ybase, int q, int n0, int col_end, int cis0)
+{
+    if (!row_ok) return;
+    const int cis = cis0 + col;
+    const int slab = cis >> P.slab_shift;
+    const int wslab = min(P.slab_cols, P.split_w - (slab << P.slab_shift));
+    __nv_bfloat16 *dst = ybase + ((size_t)slab * P.Q << P.slab_shift) + (size_t)q * wslab + (cis & (P.slab_cols - 1));
+#pragma unroll
+    for (int v = 0; v < 2; ++v) {
+        if (n0 + col + v * 16 < col_end) {
+            uint32_t w[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[v * 16 + 2 * i]), __uint_as_float(r[v * 16 + 2 * i + 1]));
+                w[i] = *reinterpret_cast<uint32_t *>(&h);
+            }
+            st_global_v8(dst + v * 16, w);
+        }
+    }
+}
 __device__ __forceinline__ void store_accumulator_rows_wide(const FusedParams &P, uint32_t taddr, int col_first, int n_cols, bool row_ok,
                                                             __nv_bfloat16 *ybase, int q, int n0, int col_end, int cis0)
 {
+    // (reading the next group from TMEM while this one is stored was measured: no gain, 13 more registers)
 #pragma unroll 1
     for (int cc = 0; cc < n_cols; cc += 32) {
-        const int col = col_first + cc;
         uint32_t r[32];
-        tmem_ld_32x32(taddr + (uint32_t)col, r);
-        const int cis = cis0 + col;
-        const int slab = cis >> P.slab_shift;
-        const int wslab = min(P.slab_cols, P.split_w - (slab << P.slab_shift));
-        __nv_bfloat16 *dst = ybase + ((size_t)slab * P.Q << P.slab_shift) + (size_t)q * wslab + (cis & (P.slab_cols - 1));
-        tmem_ld_wait();
-        if (row_ok) {
-#pragma unroll
-            for (int v = 0; v < 2; ++v) {
-                if (n0 + col + v * 16 < col_end) {
-                    uint32_t w[8];
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[v * 16 + 2 * i]), __uint_as_float(r[v * 16 + 2 * i + 1]));
-                        w[i] = *reinterpret_cast<uint32_t *>(&h);
-                    }
-                    st_global_v8(dst + v * 16, w);
-                }
-            }
-        }
+        tmem_ld_32x32(taddr + (uint32_t)(col_first + cc), r);
+        tmem_ld_wait(r);
+        emit_wide(P, r, col_first + cc, row_ok, ybase, q, n0, col_end, cis0);
     }
 }
 
@@ -455,7 +473,7 @@ __device__ __forceinline__ void store_accumulator_rows_staged(const FusedParams 
         stg->rowptr[lane] = row_ok ? (unsigned long long)(ybase + ((size_t)slab * P.Q << P.slab_shift) + (size_t)q * wslab +
                                                           (cis & (P.slab_cols - 1)))
                                    : 0ull;
-        tmem_ld_wait();
+        tmem_ld_wait(r);
 #pragma unroll
         for (int v = 0; v < 4; ++v) {
             __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(r[v * 8 + 0]), __uint_as_float(r[v * 8 + 1]));
@@ -722,7 +740,7 @@ __device__ void compute_cta(const FusedParams &P, uint8_t *ring, Control *ctl, u
 //   full[stage]       only the leader's is used: armed by the leader for the bytes of both CTAs
 //   empty[stage]      one per CTA (its producer waits on it), signalled by the leader's commit
 //   tmem_full[a]      one per CTA (its epilogue waits on it), signalled by the leader's commit
-//   tmem_empty[a]     only the leader's is used: 8 local + 8 remote epilogue warps arrive
+//   tmem_empty[a]     only the leader's is used: 12 local + 12 remote epilogue warps arrive
 struct PairCfg {
     static constexpr int kTileN = 256;
     static constexpr int kABytes = kMmaM * kBlockK * 2;                 // 16 KB: this CTA's 128 rows
@@ -1022,7 +1040,7 @@ __device__ void comm_cta(const FusedParams &P, uint8_t *ring, Control *ctl, uint
 {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const bool wait_needed = (P.mode != MOE_MODE_COMBINE_ONLY);
-    const bool claiming = (P.drain_help != 0);   // tiles are claimed, so that a helper and the tile's own CTA never both serve it
+    const bool claiming = (P.drain_help != 0);   // work is handed out dynamically (queue per split) instead of by the static map
     const unsigned long long deadline = globaltimer_ns() + P.wait_ns;
     // the wait for a copy only follows a readiness wait: it gets a later deadline so that the first
     // report names the wait that really ran out

@@ -82,7 +82,7 @@ CONFIGS = {w.name: w for w in (TINY, GRANITE, QWEN, DSV2L)}
 
 
 def sweep_workloads(T_list=(1024, 2048, 4096, 8192, 16384, 32768), s_list=(0.0, 0.6, 1.2),
-                    EP_list=(1, 2, 4), tiles=((128, 256), (256, 256))):
+                    EP_list=(1, 2, 4), tiles=((128, 128), (128, 256), (256, 256))):
     """The selector-regret sweep on the DeepSeek-V2-Lite shape."""
     out = []
     for iT, T in enumerate(T_list):
