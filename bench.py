@@ -387,6 +387,9 @@ def main():
     ap.add_argument("--sweep-out", default="gpurun_out/sweep.json")
     ap.add_argument("--sweep-filter", default="", help="substring a sweep workload name must contain")
     ap.add_argument("--sweep-curves", action="store_true", help="keep every t(C) in the sweep output")
+    ap.add_argument("--counts", default="host", choices=["host", "device"],
+                    help="host: tile counts copied to the host, exact plan (default); device: no copy and no wait, "
+                         "plan from the normalised-load estimate (Section III-E)")
     ap.add_argument("--drain-help", type=int, default=1, choices=[0, 1],
                     help="1 (default): compute CTAs help with the communication tail; 0: the paper's static partition")
     args = ap.parse_args()
@@ -455,7 +458,7 @@ def main():
     # ---- device-resident timing: EXACTLY K steps between two barriers.  One step = one moe_layer call:
     # routing build -> tile counts on the host -> plan_partition -> fused launch.
     lim.force_comm_ctas = 0
-    layer = B.LayerCall(h, dw.x, dw.W2, dw.idx_d, dw.wt_d, dw.ws, limits=lim)
+    layer = B.LayerCall(h, dw.x, dw.W2, dw.idx_d, dw.wt_d, dw.ws, limits=lim, counts_on_device=(args.counts == "device"))
     for _ in range(W):
         plan = layer()
     fused_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]

@@ -61,6 +61,7 @@ enum { MOE_MODE_FUSED = 0, MOE_MODE_GEMM_ONLY = 1, MOE_MODE_COMBINE_ONLY = 2 };
 enum { MOE_RHO_PAPER = 0, MOE_RHO_LOCAL = 1 };
 #define MOE_MAX_EP 8
 #define MOE_MAX_L 8
+#define MOE_MTILES_ON_DEVICE (-1)   /* moe_gemm2_combine: read the m-tile count from routing->tiles[E_tot] on the device */
 
 typedef struct moe_handle moe_handle;
 
@@ -209,6 +210,13 @@ int32_t moe_build_routing_static(moe_handle *h, const int32_t *topk_idx, const m
 int32_t plan_partition(const int32_t *routed_tile_counts, int32_t n_experts,
                        const moe_occupancy *occ, const moe_sm_limits *limits,
                        const moe_shape *shape, const moe_rho *rho, moe_plan *out);
+/* The same selection when the routed counts exist only on the device (Section III-E): instead of
+ * a device-to-host copy and a synchronisation made for scheduling alone, the counts are replaced
+ * by a normalised-load estimate, R = T * k_tot assignments spread evenly over the E_tot experts:
+ * ceil(ceil(R / E_tot) / tile_m) tiles each (the paper gives no formula; this is the reading taken).
+ * out->W_comp then is the estimate, not the launch's tile count.  [host] */
+int32_t plan_partition_estimate(const moe_occupancy *occ, const moe_sm_limits *limits,
+                                const moe_shape *shape, const moe_rho *rho, moe_plan *out);
 
 /* Mean cost [ns] of one plan_partition() call over `iters` calls rotating through n_sets
  * routed-count vectors (n_sets x n_experts ints, back to back).  The paper reports the
@@ -229,7 +237,9 @@ int32_t moe_time_plan_partition(const int32_t *routed_tile_counts, int32_t n_set
  * for the tokens rank d owns; y_ws / flags_ws / status_dev as sized by moe_workspace_bytes.
  * n_mtiles = S (host value from moe_build_routing).  Requires H % 8 == 0, K % 16 == 0,
  * ceil(H/L) % 8 == 0, 16-byte aligned pointers, 1 <= C, 1 <= P, R * o_comm >= C,
- * R + ceil(P / o_comp) * comp_slot_sms <= G. */
+ * R + ceil(P / o_comp) * comp_slot_sms <= G. 
+ * n_mtiles = MOE_MTILES_ON_DEVICE: the kernel reads S from the routing workspace itself (no host copy of
+ * the counts is needed; the plan then comes from plan_partition_estimate). */
 int32_t moe_gemm2_combine(moe_handle *h, const void *x_routed, const void *W2,
                           const int32_t *topk_idx, const float *topk_w,
                           const moe_shape *shape, const moe_occupancy *occ,
@@ -249,7 +259,9 @@ int32_t moe_clear_status(moe_handle *h, uint32_t *status_dev, void *stream);
  * Inputs and workspaces as for moe_build_routing / moe_gemm2_combine; tile_counts_pinned [host, pinned]
  * E_tot + 1 ints; limits_or_null = NULL uses moe_query_occupancy's limits; plan_out may be NULL.
  * Returns after the fused kernel has been launched (asynchronous on `stream`); the only host wait
- * inside is the one for the tile counts.  ev_before / ev_after: optional cudaEvent_t handles (NULL = none)
+ * inside is the one for the tile counts.  tile_counts_pinned = NULL selects the device-only-counts
+ * path of Section III-E: no copy, no wait; the plan comes from plan_partition_estimate and the kernel
+ * reads the tile count on the device (the whole call is then asynchronous and can be stream-captured).  ev_before / ev_after: optional cudaEvent_t handles (NULL = none)
  * recorded on `stream` right before and right after the fused launch, for timing it. */
 int32_t moe_layer(moe_handle *h, const void *x_routed, const void *W2, const int32_t *topk_idx,
                   const float *topk_w, const moe_shape *shape, int32_t tile_m, int32_t tile_n,

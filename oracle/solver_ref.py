@@ -54,6 +54,15 @@ def w_comp(tiles, g: int, N: int, L: int, T_N: int) -> int:
     return g * sum(int(t) for t in tiles) * ceil_div(ceil_div(N, L), T_N)
 
 
+def normalised_load_tiles(T: int, k_tot: int, E_tot: int, T_M: int) -> list:
+    """Section III-E, routed counts left on the device: the selector runs on a normalised-load estimate
+    instead of the counts.  The paper gives no formula; the reading taken: the R = T * k_tot
+    assignments are spread evenly, every expert holds ceil(R / E_tot) rows, so Eq. 16 sees
+    ceil(ceil(R / E_tot) / T_M) tiles per expert."""
+    per_expert = ceil_div(T * k_tot, E_tot)
+    return [ceil_div(per_expert, T_M)] * E_tot
+
+
 def w_comm_rank(M: int, D: int, N: int, L: int, T_Mc: int, T_Nc: int) -> int:
     """Eq. 7: communication tiles per split and rank (a rank owns about ceil(M/D) tokens)."""
     return ceil_div(ceil_div(M, D), T_Mc) * ceil_div(ceil_div(N, L), T_Nc)

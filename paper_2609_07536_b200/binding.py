@@ -28,7 +28,8 @@ EXPORTS = [
     "moe_create", "moe_destroy", "moe_last_cuda_error", "moe_set_wait_limit_ns",
     "moe_query_occupancy", "moe_workspace_bytes", "moe_routing_view", "moe_build_routing",
     "moe_build_routing_static",
-    "plan_partition", "moe_time_plan_partition", "moe_gemm2_combine", "moe_get_status", "moe_clear_status",
+    "plan_partition", "plan_partition_estimate", "moe_time_plan_partition", "moe_gemm2_combine", "moe_get_status",
+    "moe_clear_status",
     "moe_layer", "moe_host_arena_bytes", "moe_layer_host",
 ]
 
@@ -100,6 +101,8 @@ def lib():
         L.moe_build_routing_static.argtypes = [vp, vp, P(moe_shape), i32, P(moe_routing), vp, vp, vp]
         L.plan_partition.argtypes = [P(i32), i32, P(moe_occupancy), P(moe_sm_limits), P(moe_shape),
                                      P(moe_rho), P(moe_plan)]
+        L.plan_partition_estimate.argtypes = [P(moe_occupancy), P(moe_sm_limits), P(moe_shape), P(moe_rho),
+                                              P(moe_plan)]
         L.moe_time_plan_partition.argtypes = [P(i32), i32, i32, P(moe_occupancy), P(moe_sm_limits),
                                               P(moe_shape), P(moe_rho), C.c_int64, P(C.c_double),
                                               P(C.c_int64)]
@@ -209,6 +212,14 @@ def plan_partition(routed_tile_counts, occ, limits, shape, rho) -> moe_plan:
     return plan
 
 
+def plan_partition_estimate(occ, limits, shape, rho) -> moe_plan:
+    """The selection on the normalised-load estimate (routed counts left on the device)."""
+    plan = moe_plan()
+    _check(lib().plan_partition_estimate(C.byref(occ), C.byref(limits), C.byref(shape), C.byref(rho), C.byref(plan)),
+           "plan_partition_estimate")
+    return plan
+
+
 def moe_time_plan_partition(count_sets, occ, limits, shape, rho, iters: int) -> float:
     """count_sets: list of equally long routed-count vectors.  Returns mean ns per call."""
     n_sets, n = len(count_sets), len(count_sets[0])
@@ -247,7 +258,8 @@ def moe_clear_status(h, status_dev, stream=None):
 class LayerCall:
     """moe_layer with its arguments marshalled once (for a loop that repeats the same call)."""
 
-    def __init__(self, h, x_routed, W2, topk_idx, topk_w, ws: "Workspace", limits=None, stream=None):
+    def __init__(self, h, x_routed, W2, topk_idx, topk_w, ws: "Workspace", limits=None, stream=None,
+                 counts_on_device=False):
         self._stream = _stream(stream)
         self.h, self.ws = h, ws
         self.outs = (C.c_void_p * len(ws.out))(*[_ptr(o) for o in ws.out])
@@ -255,7 +267,8 @@ class LayerCall:
         self.limits = limits
         self.args = (h, _ptr(x_routed), _ptr(W2), _ptr(topk_idx), _ptr(topk_w), C.byref(ws.shape), ws.tile_m,
                      ws.tile_n, C.byref(limits) if limits is not None else None, C.byref(ws.routing),
-                     _ptr(ws.tile_counts), self.outs, _ptr(ws.y_ws), _ptr(ws.flags_ws), _ptr(ws.status),
+                     None if counts_on_device else _ptr(ws.tile_counts), self.outs, _ptr(ws.y_ws),
+                     _ptr(ws.flags_ws), _ptr(ws.status),
                      C.byref(self.plan))
         self.keep = (x_routed, W2, topk_idx, topk_w)
 
@@ -268,9 +281,11 @@ class LayerCall:
         return self.plan
 
 
-def moe_layer(h, x_routed, W2, topk_idx, topk_w, ws: "Workspace", limits=None, stream=None) -> moe_plan:
-    """Routing build -> tile counts to the host -> analytical plan -> fused launch, in one library call."""
-    return LayerCall(h, x_routed, W2, topk_idx, topk_w, ws, limits, stream)()
+def moe_layer(h, x_routed, W2, topk_idx, topk_w, ws: "Workspace", limits=None, stream=None,
+              counts_on_device=False) -> moe_plan:
+    """Routing build -> tile counts to the host -> analytical plan -> fused launch, in one library call.
+    counts_on_device: no copy and no wait; the plan comes from the normalised-load estimate."""
+    return LayerCall(h, x_routed, W2, topk_idx, topk_w, ws, limits, stream, counts_on_device)()
 
 
 def moe_host_arena_bytes(shape, tile_m, tile_n) -> int:

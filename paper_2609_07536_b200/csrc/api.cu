@@ -243,6 +243,8 @@ int32_t moe_gemm2_combine(moe_handle *h, const void *x_routed, const void *W2, c
     if ((ceil_div(s->H, s->L) % 8) != 0) return MOE_ERR_SHAPE;   // 16-byte column chunks per split
     if (s->T == 0) return MOE_OK;
     if (!x_routed || !W2 || !topk_w || !y_ws || !flags_ws) return MOE_ERR_NULL;
+    const bool counts_on_device = (n_mtiles == MOE_MTILES_ON_DEVICE);
+    if (counts_on_device) n_mtiles = r->max_mtiles;   // bound for the sizes checked on the host
     if (n_mtiles < 0 || n_mtiles > r->max_mtiles) return MOE_ERR_SHAPE;
     if (!aligned16(x_routed) || !aligned16(W2) || !aligned16(y_ws) || !aligned16(flags_ws) ||
         !aligned16(status_dev))
@@ -281,6 +283,7 @@ int32_t moe_gemm2_combine(moe_handle *h, const void *x_routed, const void *W2, c
     const int64_t Wc = (int64_t)s->TP * n_mtiles * p.NTs;
     if (Wc * s->L * 2 >= (int64_t)1 << 31) return MOE_ERR_SHAPE;
     p.W_comp = (int32_t)Wc;
+    p.S_dev = counts_on_device ? r->tiles + s->E_tot : nullptr;
     p.C = C; p.P = Pc; p.mode = mode; p.withhold = plan->debug_withhold_tile;
     p.drain_help = (mode == MOE_MODE_FUSED && plan->drain_help) ? 1 : 0;
     p.tok_blk = (int32_t)ceil_div(s->T, s->EP);
@@ -396,12 +399,14 @@ int32_t moe_layer(moe_handle *h, const void *x_routed, const void *W2, const int
                   int32_t *tile_counts_pinned, void *const *out, void *y_ws, uint32_t *flags_ws,
                   uint32_t *status_dev, moe_plan *plan_out, void *ev_before, void *ev_after, void *stream)
 {
-    if (!h || !s || !routing || !tile_counts_pinned) return MOE_ERR_NULL;
+    if (!h || !s || !routing) return MOE_ERR_NULL;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int32_t rc = moe_build_routing(h, topk_idx, s, tile_m, routing, tile_counts_pinned, status_dev, st);
     if (rc != MOE_OK) return rc;
-    cudaError_t e = cudaStreamSynchronize(st);       // the tile counts are on the host now
-    if (e != cudaSuccess) return cuda_fail(h, e, "tile counts sync");
+    if (tile_counts_pinned) {
+        cudaError_t e = cudaStreamSynchronize(st);       // the tile counts are on the host now
+        if (e != cudaSuccess) return cuda_fail(h, e, "tile counts sync");
+    }
     moe_occupancy occ;
     moe_sm_limits lim;
     moe_rho rho;
@@ -409,11 +414,13 @@ int32_t moe_layer(moe_handle *h, const void *x_routed, const void *W2, const int
     if (rc != MOE_OK) return rc;
     if (limits_or_null) lim = *limits_or_null;
     moe_plan plan;
-    rc = plan_partition(tile_counts_pinned, s->E_tot, &occ, &lim, s, &rho, &plan);
+    rc = tile_counts_pinned ? plan_partition(tile_counts_pinned, s->E_tot, &occ, &lim, s, &rho, &plan)
+                            : plan_partition_estimate(&occ, &lim, s, &rho, &plan);   // counts stay on the device
     if (rc != MOE_OK) return rc;
     if (plan_out) *plan_out = plan;
     if (ev_before) cudaEventRecord(static_cast<cudaEvent_t>(ev_before), st);
-    rc = moe_gemm2_combine(h, x_routed, W2, topk_idx, topk_w, s, &occ, routing, tile_counts_pinned[s->E_tot], &plan,
+    rc = moe_gemm2_combine(h, x_routed, W2, topk_idx, topk_w, s, &occ, routing,
+                           tile_counts_pinned ? tile_counts_pinned[s->E_tot] : MOE_MTILES_ON_DEVICE, &plan,
                            out, y_ws, flags_ws, status_dev, st);
     if (ev_after) cudaEventRecord(static_cast<cudaEvent_t>(ev_after), st);
     return rc;

@@ -355,11 +355,11 @@ __device__ __forceinline__ bool wait_barrier_1t(uint32_t bar, uint32_t parity, C
 struct Tile {
     int s, mu, p, i_n;
 };
-__device__ __forceinline__ Tile decode_tile(int g, const FusedParams &P)
+__device__ __forceinline__ Tile decode_tile(int g, const FusedParams &P, int W_comp)
 {
     Tile t;
-    t.s = g / P.W_comp;
-    const int idx = g - t.s * P.W_comp;
+    t.s = g / W_comp;
+    const int idx = g - t.s * W_comp;
     const int r = idx / P.NTs;
     t.i_n = idx - r * P.NTs;
     t.mu = r / P.TP;
@@ -500,11 +500,11 @@ __device__ __forceinline__ void store_accumulator_rows_staged(const FusedParams 
 // --------------------------------------------------------------------------- compute CTA
 
 template <int TN>
-__device__ void compute_cta(const FusedParams &P, uint8_t *ring, Control *ctl, uint8_t *aux, int b)
+__device__ void compute_cta(const FusedParams &P, int W_comp, uint8_t *ring, Control *ctl, uint8_t *aux, int b)
 {
     using C = Cfg<TN>;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int total_tiles = P.L * P.W_comp;
+    const int total_tiles = P.L * W_comp;
     const unsigned long long deadline = globaltimer_ns() + P.wait_ns;
 
     // setup: barriers (thread 0), TMEM allocation (warp 1)
@@ -541,11 +541,11 @@ __device__ void compute_cta(const FusedParams &P, uint8_t *ring, Control *ctl, u
             bool ok = true;
             // the m-tile table entries of the NEXT tile are fetched while this tile's k-blocks are issued, so
             // that the two dependent global loads never stall the stream of copies at a tile boundary
-            Tile t = decode_tile(b, P);
+            Tile t = decode_tile(b, P, W_comp);
             int e = __ldg(&P.mtile_expert[t.mu]);
             int row0 = __ldg(&P.mtile_first_row[t.mu]);
             for (int g = b; g < total_tiles && ok; g += P.P) {
-                const Tile t_next = decode_tile(min(g + P.P, total_tiles - 1), P);
+                const Tile t_next = decode_tile(min(g + P.P, total_tiles - 1), P, W_comp);
                 const int e_next = __ldg(&P.mtile_expert[t_next.mu]);
                 const int row0_next = __ldg(&P.mtile_first_row[t_next.mu]);
                 const int n0 = t.s * P.split_w + t.i_n * TN;
@@ -637,8 +637,8 @@ __device__ void compute_cta(const FusedParams &P, uint8_t *ring, Control *ctl, u
         // not in the way between an accumulator becoming ready and its first store.
         int valid = 0, f_row = 0, valid_n = 0, first_n = 0;
         if (b < total_tiles) {
-            const int mu0 = decode_tile(b, P).mu;
-            const int mu1 = decode_tile(min(b + P.P, total_tiles - 1), P).mu;
+            const int mu0 = decode_tile(b, P, W_comp).mu;
+            const int mu1 = decode_tile(min(b + P.P, total_tiles - 1), P, W_comp).mu;
             valid = __ldg(&P.mtile_valid[mu0]);
             const int first0 = __ldg(&P.mtile_first_row[mu0]);
             valid_n = __ldg(&P.mtile_valid[mu1]);
@@ -647,10 +647,10 @@ __device__ void compute_cta(const FusedParams &P, uint8_t *ring, Control *ctl, u
         }
         int it = 0;
         for (int g = b; g < total_tiles; g += P.P, ++it) {
-            const Tile t = decode_tile(g, P);
+            const Tile t = decode_tile(g, P, W_comp);
             const int a = it & 1;
             const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
-            const int mu_nn = decode_tile(min(g + 2 * P.P, total_tiles - 1), P).mu;
+            const int mu_nn = decode_tile(min(g + 2 * P.P, total_tiles - 1), P, W_comp).mu;
             const int valid_nn = __ldg(&P.mtile_valid[mu_nn]);
             const int first_nn = __ldg(&P.mtile_first_row[mu_nn]);
             const int f_row_n = (row_in_tile < valid_n) ? __ldg(&P.perm[first_n + row_in_tile]) : 0;
@@ -714,7 +714,7 @@ __device__ void compute_cta(const FusedParams &P, uint8_t *ring, Control *ctl, u
                 if (g != P.withhold) {
                     __threadfence();   // release: the epilogue warps' stores (observed through epi_done) come first
                     st_relaxed_u32(&P.flags[g], P.epoch);
-                    red_relaxed_add_u32(&P.split_done[g / P.W_comp], 1u);
+                    red_relaxed_add_u32(&P.split_done[g / W_comp], 1u);
                 }
                 mbar_arrive(smem_u32(&ctl->pub_done[a]));
             }
@@ -752,14 +752,14 @@ struct PairCfg {
     static constexpr int kColsPerGroup = ((kTileN / 32 + 2) / 3) * 32;  // 96, 96, 64
 };
 
-__device__ void compute_cta_pair(const FusedParams &P, uint8_t *ring, Control *ctl, uint8_t *aux, int b)
+__device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring, Control *ctl, uint8_t *aux, int b)
 {
     using C = PairCfg;
     constexpr int TN = C::kTileN;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
     const bool leader_cta = (rank == 0);
-    const int total_tiles = P.L * P.W_comp;
+    const int total_tiles = P.L * W_comp;
     const unsigned long long deadline = globaltimer_ns() + P.wait_ns;
 
     if (threadIdx.x == 0) {
@@ -795,11 +795,11 @@ __device__ void compute_cta_pair(const FusedParams &P, uint8_t *ring, Control *c
             uint32_t armed = 0;
             bool ok = true;
             // next tile's table entries are fetched one tile ahead (see compute_cta)
-            Tile t = decode_tile(b, P);
+            Tile t = decode_tile(b, P, W_comp);
             int e = __ldg(&P.mtile_expert[t.mu]);
             int row0 = __ldg(&P.mtile_first_row[t.mu]) + (int)rank * kMmaM;
             for (int g = b; g < total_tiles && ok; g += P.P) {
-                const Tile t_next = decode_tile(min(g + P.P, total_tiles - 1), P);
+                const Tile t_next = decode_tile(min(g + P.P, total_tiles - 1), P, W_comp);
                 const int e_next = __ldg(&P.mtile_expert[t_next.mu]);
                 const int row0_next = __ldg(&P.mtile_first_row[t_next.mu]) + (int)rank * kMmaM;
                 const int n0 = t.s * P.split_w + t.i_n * TN + (int)rank * (TN / 2);
@@ -888,8 +888,8 @@ __device__ void compute_cta_pair(const FusedParams &P, uint8_t *ring, Control *c
         // not in the way between an accumulator becoming ready and its first store.
         int valid = 0, f_row = 0, valid_n = 0, first_n = 0;
         if (b < total_tiles) {
-            const int mu0 = decode_tile(b, P).mu;
-            const int mu1 = decode_tile(min(b + P.P, total_tiles - 1), P).mu;
+            const int mu0 = decode_tile(b, P, W_comp).mu;
+            const int mu1 = decode_tile(min(b + P.P, total_tiles - 1), P, W_comp).mu;
             valid = __ldg(&P.mtile_valid[mu0]);
             const int first0 = __ldg(&P.mtile_first_row[mu0]);
             valid_n = __ldg(&P.mtile_valid[mu1]);
@@ -898,10 +898,10 @@ __device__ void compute_cta_pair(const FusedParams &P, uint8_t *ring, Control *c
         }
         int it = 0;
         for (int g = b; g < total_tiles; g += P.P, ++it) {
-            const Tile t = decode_tile(g, P);
+            const Tile t = decode_tile(g, P, W_comp);
             const int a = it & 1;
             const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
-            const int mu_nn = decode_tile(min(g + 2 * P.P, total_tiles - 1), P).mu;
+            const int mu_nn = decode_tile(min(g + 2 * P.P, total_tiles - 1), P, W_comp).mu;
             const int valid_nn = __ldg(&P.mtile_valid[mu_nn]);
             const int first_nn = __ldg(&P.mtile_first_row[mu_nn]);
             const int f_row_n = (row_in_tile < valid_n) ? __ldg(&P.perm[first_n + row_in_tile]) : 0;
@@ -960,7 +960,7 @@ __device__ void compute_cta_pair(const FusedParams &P, uint8_t *ring, Control *c
                 if (g != P.withhold) {
                     __threadfence();
                     st_relaxed_u32(&P.flags[2 * g + (int)rank], P.epoch);
-                    red_relaxed_add_u32(&P.split_done[g / P.W_comp], 1u);
+                    red_relaxed_add_u32(&P.split_done[g / W_comp], 1u);
                 }
                 mbar_arrive(smem_u32(&ctl->pub_done[a]));
             }
@@ -1036,7 +1036,7 @@ struct CommUnit {
 };
 
 template <int TN>
-__device__ void comm_cta(const FusedParams &P, uint8_t *ring, Control *ctl, uint8_t *aux, int c, bool helper)
+__device__ void comm_cta(const FusedParams &P, int W_comp, uint8_t *ring, Control *ctl, uint8_t *aux, int c, bool helper)
 {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const bool wait_needed = (P.mode != MOE_MODE_COMBINE_ONLY);
@@ -1162,7 +1162,7 @@ __device__ void comm_cta(const FusedParams &P, uint8_t *ring, Control *ctl, uint
             uint32_t done = 0;
             if (lane == 0) done = ld_acquire_u32(&P.split_done[u.s]);
             done = __shfl_sync(0xffffffffu, done, 0);
-            if (done >= (uint32_t)(P.W_comp * P.flag_parts)) {
+            if (done >= (uint32_t)(W_comp * P.flag_parts)) {
                 ready_mask |= 1u << u.s;
             } else {
                 // per tile: every (slot j, shard p, n-tile under this slab)
@@ -1180,7 +1180,7 @@ __device__ void comm_cta(const FusedParams &P, uint8_t *ring, Control *ctl, uint
                     const int mu = row / P.tile_m;
                     // a pair tile is published in two parts, one per CTA: the row's part is its 128-row half
                     const int part = (P.flag_parts == 2) ? ((row - mu * P.tile_m) >> 7) : 0;
-                    const int g = (u.s * P.W_comp + (mu * P.TP + p) * P.NTs + in0 + tn) * P.flag_parts + part;
+                    const int g = (u.s * W_comp + (mu * P.TP + p) * P.NTs + in0 + tn) * P.flag_parts + part;
                     uint32_t spins = 0;
                     while (ld_acquire_u32(&P.flags[g]) != P.epoch) {
                         if ((++spins & 31u) == 0u && (ctl->abort || globaltimer_ns() > deadline)) {
@@ -1398,6 +1398,13 @@ __device__ void comm_cta(const FusedParams &P, uint8_t *ring, Control *ctl, uint
 
 // --------------------------------------------------------------------------- kernel
 
+// Compute tiles per split of this launch (Eq. 5).  With the routed counts left on the device the m-tile
+// count is read from the routing workspace (the routing kernels ran earlier on the same stream).
+__device__ __forceinline__ int launch_w_comp(const FusedParams &P)
+{
+    return P.S_dev ? min(__ldg(P.S_dev), P.S) * P.TP * P.NTs : P.W_comp;
+}
+
 template <int TN>
 __global__ void __launch_bounds__(kThreads, 1)
 moe_gemm2_combine_kernel(const __grid_constant__ FusedParams P)
@@ -1413,12 +1420,13 @@ moe_gemm2_combine_kernel(const __grid_constant__ FusedParams P)
         P.queue_next[threadIdx.x] = 0ull;
     }
 
+    const int W_comp = launch_w_comp(P);
     if ((int)blockIdx.x < P.C)
-        comm_cta<TN>(P, ring, ctl, aux, (int)blockIdx.x, false);
+        comm_cta<TN>(P, W_comp, ring, ctl, aux, (int)blockIdx.x, false);
     else {
-        compute_cta<TN>(P, ring, ctl, aux, (int)blockIdx.x - P.C);
+        compute_cta<TN>(P, W_comp, ring, ctl, aux, (int)blockIdx.x - P.C);
         // out of GEMM tiles: help with the communication that is left (all TMA and TMEM traffic is over)
-        if (P.drain_help && P.mode == MOE_MODE_FUSED && !ctl->abort) comm_cta<TN>(P, ring, ctl, aux, 0, true);
+        if (P.drain_help && P.mode == MOE_MODE_FUSED && !ctl->abort) comm_cta<TN>(P, W_comp, ring, ctl, aux, 0, true);
     }
 }
 
@@ -1438,15 +1446,16 @@ moe_gemm2_combine_pair_kernel(const __grid_constant__ FusedParams P)
     }
 
     const int c_even = (P.C + 1) & ~1;
+    const int W_comp = launch_w_comp(P);
     if ((int)blockIdx.x < P.C)
-        comm_cta<256>(P, ring, ctl, aux, (int)blockIdx.x, false);
+        comm_cta<256>(P, W_comp, ring, ctl, aux, (int)blockIdx.x, false);
     else if ((int)blockIdx.x < c_even) {
         // odd C: the last communication CTA's cluster-mate cannot compute (no partner).  With dynamic work
         // distribution it serves communication work as well; under the static map it has no tile list.
-        if (P.drain_help && P.mode == MOE_MODE_FUSED) comm_cta<256>(P, ring, ctl, aux, (int)blockIdx.x, false);
+        if (P.drain_help && P.mode == MOE_MODE_FUSED) comm_cta<256>(P, W_comp, ring, ctl, aux, (int)blockIdx.x, false);
     } else {
-        compute_cta_pair(P, ring, ctl, aux, ((int)blockIdx.x - c_even) >> 1);
-        if (P.drain_help && P.mode == MOE_MODE_FUSED && !ctl->abort) comm_cta<256>(P, ring, ctl, aux, 0, true);
+        compute_cta_pair(P, W_comp, ring, ctl, aux, ((int)blockIdx.x - c_even) >> 1);
+        if (P.drain_help && P.mode == MOE_MODE_FUSED && !ctl->abort) comm_cta<256>(P, W_comp, ring, ctl, aux, 0, true);
     }
 }
 

@@ -30,6 +30,7 @@ struct alignas(64) FusedParams {
     const int32_t *mtile_expert;
     const int32_t *mtile_first_row;
     const int32_t *mtile_valid;
+    const int32_t *S_dev;          // != nullptr: the m-tile count is read here by the kernel (S and W_comp below are unset)
     const int32_t *pad_row;
     const int32_t *perm;
     const float *topk_w;

@@ -303,3 +303,23 @@ extern "C" int32_t moe_time_plan_partition(const int32_t *routed_tile_counts, in
     if (checksum) *checksum = sum;
     return rc;
 }
+
+// Section III-E: when the routed counts exist only on the device, the selector runs on a
+// normalised-load estimate instead of paying a device-to-host copy and a synchronisation for scheduling
+// alone.  The estimate spreads the R = T * k_tot assignments evenly over the E_tot experts:
+// every expert gets ceil(R / E_tot) rows, i.e. ceil(ceil(R / E_tot) / T_M) tiles (Eq. 16 on those counts).
+extern "C" int32_t plan_partition_estimate(const moe_occupancy *occ, const moe_sm_limits *limits,
+                                           const moe_shape *shape, const moe_rho *rho, moe_plan *out)
+{
+    if (!occ || !limits || !shape || !rho || !out) return MOE_ERR_NULL;
+    if (shape->E_tot < 1 || shape->E_tot > 1024 || shape->T < 0 || shape->k_tot < 1 || occ->tile_m < 1)
+        return MOE_ERR_SHAPE;
+    int32_t counts[1024];
+    const int64_t R = (int64_t)shape->T * shape->k_tot;
+    const int64_t per_expert = (R + shape->E_tot - 1) / shape->E_tot;
+    const int64_t tiles = (per_expert + occ->tile_m - 1) / occ->tile_m;
+    if (tiles > INT32_MAX) return MOE_ERR_SHAPE;
+    for (int32_t e = 0; e < shape->E_tot; ++e) counts[e] = (int32_t)tiles;
+    return plan_partition(counts, shape->E_tot, occ, limits, shape, rho, out);
+}
+

@@ -329,3 +329,32 @@ def test_single_call_layer_matches_the_stepwise_path():
     assert ea.elapsed_time(eb) > 0
     for a, o in zip(ref_outs, ws.out):
         assert np.array_equal(a, o.float().cpu().numpy(), equal_nan=True)
+
+
+@pytest.mark.parametrize("tile", [(128, 256), (256, 256)], ids=["128x256", "pair"])
+def test_counts_left_on_the_device_give_the_same_bits(tile):
+    # Section III-E: no copy of the routed counts and no wait; the plan comes from the normalised-load
+    # estimate and the kernel reads the m-tile count from the routing workspace.  A skewed routing
+    # makes the estimate differ from the true tile count; the output may not change by a bit.
+    h = G.handle()
+    w = replace(wl.DSV2L, name="devcounts", T=3000, tile_m=tile[0], tile_n=tile[1])
+    idx, wt, _ = wl.make_routing(w)
+    x, W2 = wl.make_data(w)
+    ref_outs, plan, ws, S, st = G.run_layer(w, idx, wt, x, W2)
+    ref_outs = [o.copy() for o in ref_outs]
+    xd, Wd = x.cuda(), W2.cuda()
+    idx_d, wt_d = torch.from_numpy(idx).cuda(), torch.from_numpy(wt).cuda()
+    for rep in range(2):
+        for o in ws.out:
+            o.fill_(float("nan"))
+        ws.tile_counts.fill_(-7)                       # must stay untouched
+        p2 = B.moe_layer(h, xd, Wd, idx_d, wt_d, ws, counts_on_device=True)
+        torch.cuda.synchronize()
+        assert B.moe_get_status(h, ws.status).code == 0
+        assert (ws.tile_counts == -7).all()
+        occ, lim, rho = B.moe_query_occupancy(h, w.tile_m, w.tile_n)
+        est = B.plan_partition_estimate(occ, lim, ws.shape, rho)
+        assert (p2.comm_ctas, p2.P, p2.W_comp) == (est.comm_ctas, est.P, est.W_comp)
+        assert p2.W_comp != plan.W_comp                # the estimate is not the true count here
+        for a, o in zip(ref_outs, ws.out):
+            assert np.array_equal(a, o.float().cpu().numpy(), equal_nan=True), rep

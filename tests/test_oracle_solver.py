@@ -172,3 +172,28 @@ def test_select_is_the_lexicographic_minimum_and_overrides():
         assert d["comm_ctas"] == min(cur)
     with pytest.raises(ValueError):
         sr.select(10, 10, 1, 4, 1, 1, 16, sr.RHO_ONE, force_comm_ctas=4)   # P = 0
+
+
+def test_normalised_load_estimate_brackets_the_true_tile_count():
+    # The estimate is exact for a perfectly even routing whose per-expert rows fill whole tiles, it never
+    # falls below the bound every routing obeys (sum_e ceil(M_e/T_M) >= ceil(R/T_M)), and no routing
+    # exceeds it by more than one tile per expert plus the rounding of R/E.
+    rng = random.Random(5)
+    for _ in range(300):
+        E, T_M = rng.randint(1, 80), rng.choice([64, 128, 256])
+        k = rng.randint(1, 8)
+        T = rng.randint(0, 5000)
+        R = T * k
+        est = sum(sr.normalised_load_tiles(T, k, E, T_M))
+        assert est >= sr.ceil_div(R, T_M)
+        assert est <= R // T_M + 2 * E
+        # any routing: random split of R rows over E experts
+        cuts = sorted(rng.randint(0, R) for _ in range(E - 1))
+        loads = [b - a for a, b in zip([0] + cuts, cuts + [R])]
+        true = sum(sr.ceil_div(m, T_M) for m in loads)
+        assert sr.ceil_div(R, T_M) <= true <= R // T_M + E
+    # even routing, whole tiles: exact
+    assert sr.normalised_load_tiles(4096, 6, 64, 128) == [3] * 64          # 384 rows per expert
+    assert sum(sr.normalised_load_tiles(4096, 6, 64, 128)) == sum(sr.ceil_div(384, 128) for _ in range(64))
+    assert sr.normalised_load_tiles(0, 6, 64, 128) == [0] * 64
+

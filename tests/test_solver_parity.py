@@ -195,3 +195,23 @@ def test_solver_cost_is_small():
     for _ in range(2000):
         B.plan_partition(tiles, occ, lim, shape, rho)
     assert (time.perf_counter() - t) / 2000 < 1e-3
+
+
+def test_estimate_plan_equals_the_oracle_on_the_normalised_counts():
+    # Section III-E, counts left on the device: the library's estimate is the oracle's, and the plan on
+    # it is bit-exact like any other
+    rng = random.Random(21)
+    n = 0
+    for _ in range(3000):
+        _, shape, occ, lim, rho = _rand_inputs(rng)
+        tiles = sr.normalised_load_tiles(shape.T, shape.k_tot, shape.E_tot, occ.tile_m)
+        try:
+            sel = _oracle_plan(tiles, shape, occ, lim, rho)
+        except ValueError:
+            with pytest.raises(B.MoeError) as e:
+                B.plan_partition_estimate(occ, lim, shape, rho)
+            assert e.value.code == B.MOE_ERR_PLAN_INFEASIBLE
+            continue
+        _same(B.plan_partition_estimate(occ, lim, shape, rho), sel)
+        n += 1
+    assert n > 2000
