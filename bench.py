@@ -329,9 +329,20 @@ def cpu_baseline(w, idx, wt, x_cpu, W2_cpu, budget_s=15.0):
     ref.gemm2_combine(xb, Wb, idx, wt, r["inv_perm"], tokens=toks)
     dt = time.perf_counter() - t0
     us_layer = dt / n * w.T * 1e6
+    # the same loops on one thread, on a small sample (about 2 s)
+    n1 = int(max(4, min(n, 2.0 / max(per_tok * cores, 1e-9))))
+    before = ref.set_threads(1)
+    try:
+        t0 = time.perf_counter()
+        ref.gemm2_combine(xb, Wb, idx, wt, r["inv_perm"], tokens=toks[:n1])
+        dt1 = time.perf_counter() - t0
+    finally:
+        ref.set_threads(before)
     return {"value": us_layer, "unit": "us/layer", "cores": cores, "kind": "oracle",
             "sample": f"{n} of {w.T} tokens (seeded random sample) timed in {dt:.2f} s, scaled by T/n; "
-                      f"routing reference not included"}, dt
+                      f"routing reference not included",
+            "single_thread": {"value": dt1 / n1 * w.T * 1e6, "unit": "us/layer",
+                              "sample": f"{n1} tokens in {dt1:.2f} s, scaled by T/n"}}, dt
 
 
 def reference_arm(args):
@@ -479,6 +490,14 @@ def main():
     step_us = t_beg.elapsed_time(t_end) * 1e3 / K
     fused_us = [a.elapsed_time(b) * 1e3 for a, b in fused_ev]
     fused_med = statistics.median(fused_us)
+    # 95% interval of that median: block-stratified bootstrap (blocks of consecutive steps keep the slow
+    # drift of the power-capped clock inside a block), 1000 resamples, seeded
+    import random as _random
+    _rng = _random.Random(0)
+    _blk = max(1, len(fused_us) // 10)
+    _blocks = [fused_us[i:i + _blk] for i in range(0, len(fused_us), _blk)]
+    _meds = sorted(statistics.median([v for b in _blocks for v in (_rng.choice(b) for _ in b)]) for _ in range(1000))
+    fused_ci = [_meds[25], _meds[974]]
     st = B.moe_get_status(h, dw.ws.status)
     assert st.code == 0
     counts = dw.ws.tile_counts[:w.E_tot + 1].tolist()
@@ -550,7 +569,7 @@ def main():
             "unit": "TFLOP/s" if tensor_bound else "GB/s", "frac": ach / peak, "traffic": None,
             "peak_source": peaks["source"] + (" (sustained: the kernel is timed inside the step loop)" if tensor_bound else ""),
             "kernel": "moe_gemm2_combine_pair_kernel" if w.tile_m == 256 else "moe_gemm2_combine_kernel",
-            "kernel_us": fused_med, "roofline_us": max(t_flops_us, t_hbm_us),
+            "kernel_us": fused_med, "kernel_us_ci95": fused_ci, "roofline_us": max(t_flops_us, t_hbm_us),
             "frac_of_burst_peak": (ach / peaks["bf16_tflops"]) if tensor_bound else None,
             "burst_peak": peaks["bf16_tflops"] if tensor_bound else None,
         }

@@ -53,6 +53,20 @@ int moe_ref_threads(void)
 #endif
 }
 
+/* Sets the number of threads the loops below may use (for the single-thread timing beside the
+ * all-cores one); returns the previous maximum.  No effect without OpenMP. */
+int moe_ref_set_threads(int n)
+{
+#ifdef _OPENMP
+    const int before = omp_get_max_threads();
+    if (n >= 1) omp_set_num_threads(n);
+    return before;
+#else
+    (void)n;
+    return 1;
+#endif
+}
+
 /*
  * tokens: list of n_tokens token ids to evaluate (NULL = tokens 0..n_tokens-1).
  * out   : [n_tokens][H] fp32, row r belongs to tokens[r].

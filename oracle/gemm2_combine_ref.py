@@ -41,6 +41,8 @@ def _load():
         lib.moe_ref_round_bf16.restype = None
         lib.moe_ref_threads.argtypes = []
         lib.moe_ref_threads.restype = ctypes.c_int
+        lib.moe_ref_set_threads.argtypes = [ctypes.c_int]
+        lib.moe_ref_set_threads.restype = ctypes.c_int
         _lib = lib
     return _lib
 
@@ -48,6 +50,11 @@ def _load():
 def threads() -> int:
     """Threads the C loops will use (OpenMP's maximum)."""
     return int(_load().moe_ref_threads())
+
+
+def set_threads(n: int) -> int:
+    """Limits the C loops to n threads; returns the previous maximum (to restore it)."""
+    return int(_load().moe_ref_set_threads(int(n)))
 
 
 def _ptr(a, ty):

@@ -268,3 +268,50 @@ def simulate(C: int, Wc: int, Wm: int, L: int, P: int, rho: Fraction) -> dict:
         prev = max(worker) if Wm > 0 else start
         finish.append(prev)
     return dict(publish=publish, finish=finish, T=finish[-1] if finish else Fraction(0))
+
+
+def simulate_drain_help(C: int, Wc: int, Wm: int, L: int, P: int, helpers: int, rho: Fraction) -> dict:
+    """Event-by-event simulation of the schedule the drain-help model stands for (no closed form):
+      * compute side as in simulate();
+      * the C communication CTAs serve splits 0..L-2 in order, each split in waves of at most C tiles,
+        a wave takes rho;
+      * at A = the publication time of the last split every wave of those splits that has not
+        completed goes back to the pool with the tiles it really holds, together with the last
+        split's Wm tiles; the pool is served by C + helpers workers, rho per tile, from time A.
+    The model (makespan_drain_help) counts C tiles for every wave that is still open at A and counts
+    idle gaps between splits as waves, so it can only over-estimate this simulation; the two agree
+    when nothing is open at A, and when the service up to A is gap-free and Wm is a multiple of C."""
+    rho = Fraction(rho)
+    clock = [Fraction(0)] * P
+    tile_end = []
+    for i in range(L * Wc):
+        b = i % P
+        clock[b] = clock[b] + 1
+        tile_end.append(clock[b])
+    publish = []
+    for s in range(L):
+        seg = tile_end[s * Wc:(s + 1) * Wc]
+        publish.append(max(seg) if seg else Fraction(0))
+    A = publish[L - 1]
+    pool = Wm
+    prev = Fraction(0)
+    gap_free = True
+    for s in range(L - 1):
+        start = max(publish[s], prev)
+        if s > 0 and publish[s] > prev:
+            gap_free = False
+        left, t = Wm, start
+        while left > 0:
+            n = min(C, left)
+            if t + rho > A:          # this wave is not complete at A: its tiles are pooled
+                pool += n
+            t += rho
+            left -= n
+        prev = t
+    workers = C + helpers
+    worker = [A] * workers
+    for j in range(pool):
+        worker[j % workers] += rho
+    T = max(worker) if pool > 0 else A
+    return dict(publish=publish, T=T, pool=pool, gap_free=gap_free, open_at_A=pool > Wm)
+

@@ -173,7 +173,7 @@ def test_drain_help_model():
         _same(plan, _oracle_plan(tiles, shape, occ, lim, rho))
         assert plan.drain_help == dh
         picks[dh] = plan
-    # helpers shorten the tail, so the model never predicts a longer makespan and never asks for more C
+    # on this workload the helpers shorten the predicted tail and the selector asks for fewer communication CTAs
     assert picks[1].pred_T_q <= picks[0].pred_T_q and picks[1].comm_ctas <= picks[0].comm_ctas
     # closed form for L = 1: T = A_0 + rho * ceil(W_comm / (C + P))
     shape1 = B.make_shape(4096, 2048, 1408, 66, 8, 2, 1, 1)
