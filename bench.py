@@ -288,22 +288,12 @@ def calibrate(h, device, C_ref=32, tile=(128, 256)):
     w = replace(wl.DSV2L, name="rho_ref", T=4096, routing="uniform", zipf_s=0.0, target_r_expert=0.0,
                 tile_m=tile[0], tile_n=tile[1])
     dw = DeviceWorkload(w, device, data="device")
-    step, (occ, lim, rho) = make_stepper(h, dw)
-    plan, counts = step(C_ref)
-    torch.cuda.synchronize()
-    P = (lim.G - C_ref) // occ.comp_slot_sms
-    t_comp = statistics.median(time_fused(step, torch, 0, 3, 15, mode=B.MOE_MODE_GEMM_ONLY, P_override=P, reuse=counts))
-    t_comm = statistics.median(time_fused(step, torch, 1, 3, 15, mode=B.MOE_MODE_COMBINE_ONLY, C_override=C_ref, reuse=counts))
-    V_comp = -(-plan.W_comp // P)
-    V_comm = -(-plan.W_comm // C_ref)
-    wave_comp = t_comp / (V_comp * w.L)
-    wave_comm = t_comm / (V_comm * w.L)
+    rho, wave_comp, wave_comm = B.moe_calibrate_rho(h, dw.x, dw.W2, dw.idx_d, dw.wt_d, dw.ws, C_ref=C_ref, n_samples=15)
     print(json.dumps({"calibration": {
-        "workload": "DeepSeek-V2-Lite shape, T=4096, uniform, 128x256, TP=2, EP=2, L=2", "C_ref": C_ref, "P": P,
-        "t_gemm_only_us": t_comp, "compute_waves": V_comp * w.L, "us_per_compute_wave": wave_comp,
-        "t_combine_only_us": t_comm, "comm_waves": V_comm * w.L, "us_per_comm_wave": wave_comm,
-        "rho_ref": wave_comm / wave_comp, "K_ref": w.K, "tile_ref": [w.tile_m, w.tile_n],
-        "rows_ref": w.k_tot * w.TP + 1, "comm_cols_ref": min(1024, -(-w.H // w.L)), "D_ref": w.EP}}))
+        "workload": f"DeepSeek-V2-Lite shape, T=4096, uniform, {w.tile_m}x{w.tile_n}, TP=2, EP=2, L=2", "C_ref": C_ref,
+        "us_per_compute_wave": wave_comp, "us_per_comm_wave": wave_comm,
+        "rho_ref": rho.rho_ref, "K_ref": rho.K_ref, "tile_ref": [rho.tile_m_ref, rho.tile_n_ref],
+        "rows_ref": rho.rows_ref, "comm_cols_ref": rho.comm_cols_ref, "D_ref": rho.D_ref}}))
 
 
 # ----------------------------------------------------------------------------- CPU baseline

@@ -269,6 +269,22 @@ int32_t moe_layer(moe_handle *h, const void *x_routed, const void *W2, const int
                   int32_t *tile_counts_pinned, void *const *out, void *y_ws, uint32_t *flags_ws,
                   uint32_t *status_dev, moe_plan *plan_out, void *ev_before, void *ev_after, void *stream);
 
+/* ---- one-time service-rate characterisation of a kernel family (Eq. 13, Section III-C) -------
+ * Measures rho_ref on the caller's reference workload (inputs and workspaces as for moe_layer): the
+ * GEMM alone on P(C_ref) compute slots and the combine alone on C_ref communication CTAs (static
+ * map), each n_samples (<= 64) launches after two warm-ups, median; rho_ref = time per communication
+ * wave / time per compute wave.  Fills *rho_out with the constant and its reference factors (K, tile,
+ * EP, rows per token, communication tile width; mode as moe_query_occupancy reports it), and
+ * wave_us_out[0..1] (optional) with the two wave times in microseconds.  Meant to run once per kernel
+ * family, never per workload; the stored constants of moe_query_occupancy were measured with it on
+ * the DeepSeek-V2-Lite shape, T = 4096, uniform routing, TP = EP = L = 2, C_ref = 32.
+ * Synchronises the stream; creates and destroys two CUDA events.  [host; device work on stream] */
+int32_t moe_calibrate_rho(moe_handle *h, const void *x_routed, const void *W2, const int32_t *topk_idx,
+                          const float *topk_w, const moe_shape *shape, int32_t tile_m, int32_t tile_n,
+                          int32_t C_ref, int32_t n_samples, const moe_routing *routing,
+                          int32_t *tile_counts_pinned, void *const *out, void *y_ws, uint32_t *flags_ws,
+                          uint32_t *status_dev, moe_rho *rho_out, double *wave_us_out, void *stream);
+
 /* ---- the whole step from host buffers ---------------------------------------------------
  * The call a user without device-resident activations makes: copies x_routed, topk_idx and
  * topk_w from (pinned) host memory into `arena`, builds the routing, waits for the tile

@@ -30,7 +30,7 @@ EXPORTS = [
     "moe_build_routing_static",
     "plan_partition", "plan_partition_estimate", "moe_time_plan_partition", "moe_gemm2_combine", "moe_get_status",
     "moe_clear_status",
-    "moe_layer", "moe_host_arena_bytes", "moe_layer_host",
+    "moe_layer", "moe_calibrate_rho", "moe_host_arena_bytes", "moe_layer_host",
 ]
 
 
@@ -112,6 +112,8 @@ def lib():
         L.moe_clear_status.argtypes = [vp, vp, vp]
         L.moe_layer.argtypes = [vp, vp, vp, vp, vp, P(moe_shape), i32, i32, P(moe_sm_limits), P(moe_routing), vp,
                                 P(vp), vp, vp, vp, P(moe_plan), vp, vp, vp]
+        L.moe_calibrate_rho.argtypes = [vp, vp, vp, vp, vp, P(moe_shape), i32, i32, i32, i32, P(moe_routing), vp,
+                                        P(vp), vp, vp, vp, P(moe_rho), P(C.c_double), vp]
         L.moe_host_arena_bytes.argtypes = [P(moe_shape), i32, i32, P(C.c_size_t)]
         L.moe_layer_host.argtypes = [vp, vp, vp, vp, vp, P(moe_shape), i32, i32, P(moe_sm_limits), vp,
                                      C.c_size_t, vp, vp, P(moe_plan), vp]
@@ -286,6 +288,20 @@ def moe_layer(h, x_routed, W2, topk_idx, topk_w, ws: "Workspace", limits=None, s
     """Routing build -> tile counts to the host -> analytical plan -> fused launch, in one library call.
     counts_on_device: no copy and no wait; the plan comes from the normalised-load estimate."""
     return LayerCall(h, x_routed, W2, topk_idx, topk_w, ws, limits, stream, counts_on_device)()
+
+
+def moe_calibrate_rho(h, x_routed, W2, topk_idx, topk_w, ws: "Workspace", C_ref: int = 32, n_samples: int = 15,
+                      stream=None):
+    """One-time service-rate characterisation (Eq. 13) on the workload in `ws`.  Returns (moe_rho,
+    us per compute wave, us per communication wave)."""
+    outs = (C.c_void_p * len(ws.out))(*[_ptr(o) for o in ws.out])
+    rho = moe_rho()
+    waves = (C.c_double * 2)()
+    _check(lib().moe_calibrate_rho(h, _ptr(x_routed), _ptr(W2), _ptr(topk_idx), _ptr(topk_w), C.byref(ws.shape),
+                                   ws.tile_m, ws.tile_n, C_ref, n_samples, C.byref(ws.routing),
+                                   _ptr(ws.tile_counts), outs, _ptr(ws.y_ws), _ptr(ws.flags_ws), _ptr(ws.status),
+                                   C.byref(rho), waves, _stream(stream)), "moe_calibrate_rho", h)
+    return rho, waves[0], waves[1]
 
 
 def moe_host_arena_bytes(shape, tile_m, tile_n) -> int:

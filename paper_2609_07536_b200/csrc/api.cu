@@ -3,6 +3,8 @@
 #include <cstring>
 #include <new>
 
+#include <algorithm>
+
 #include "moe_internal.h"
 
 namespace moe {
@@ -424,6 +426,76 @@ int32_t moe_layer(moe_handle *h, const void *x_routed, const void *W2, const int
                            out, y_ws, flags_ws, status_dev, st);
     if (ev_after) cudaEventRecord(static_cast<cudaEvent_t>(ev_after), st);
     return rc;
+}
+
+// ---- one-time service-rate characterisation (Eq. 13) ---------------------------------------
+
+int32_t moe_calibrate_rho(moe_handle *h, const void *x_routed, const void *W2, const int32_t *topk_idx,
+                          const float *topk_w, const moe_shape *s, int32_t tile_m, int32_t tile_n,
+                          int32_t C_ref, int32_t n_samples, const moe_routing *routing,
+                          int32_t *tile_counts_pinned, void *const *out, void *y_ws, uint32_t *flags_ws,
+                          uint32_t *status_dev, moe_rho *rho_out, double *wave_us_out, void *stream)
+{
+    if (!h || !s || !routing || !tile_counts_pinned || !rho_out) return MOE_ERR_NULL;
+    if (C_ref < 1 || n_samples < 1 || n_samples > 64) return MOE_ERR_SHAPE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t rc = moe_build_routing(h, topk_idx, s, tile_m, routing, tile_counts_pinned, status_dev, st);
+    if (rc != MOE_OK) return rc;
+    cudaError_t e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(h, e, "tile counts sync");
+    moe_occupancy occ;
+    moe_sm_limits lim;
+    moe_rho rho;
+    rc = moe_query_occupancy(h, tile_m, tile_n, &occ, &lim, &rho);
+    if (rc != MOE_OK) return rc;
+    lim.force_comm_ctas = C_ref;
+    lim.drain_help = 0;                       // each role alone on its share of the SMs
+    moe_plan plan;
+    rc = plan_partition(tile_counts_pinned, s->E_tot, &occ, &lim, s, &rho, &plan);
+    if (rc != MOE_OK) return rc;
+    if (plan.W_comp < 1 || plan.W_comm < 1) return MOE_ERR_SHAPE;
+    const int32_t S = tile_counts_pinned[s->E_tot];
+
+    cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+    if ((e = cudaEventCreate(&ev0)) != cudaSuccess) return cuda_fail(h, e, "event");
+    if ((e = cudaEventCreate(&ev1)) != cudaSuccess) { cudaEventDestroy(ev0); return cuda_fail(h, e, "event"); }
+    double med[2] = {0.0, 0.0};
+    for (int role = 0; role < 2 && rc == MOE_OK; ++role) {
+        moe_plan p = plan;
+        p.mode = role == 0 ? MOE_MODE_GEMM_ONLY : MOE_MODE_COMBINE_ONLY;   // GEMM first: it also fills Y
+        float t[64];
+        for (int i = -2; i < n_samples && rc == MOE_OK; ++i) {              // two warm-up launches
+            cudaEventRecord(ev0, st);
+            rc = moe_gemm2_combine(h, x_routed, W2, topk_idx, topk_w, s, &occ, routing, S, &p, out, y_ws,
+                                   flags_ws, status_dev, st);
+            cudaEventRecord(ev1, st);
+            if ((e = cudaEventSynchronize(ev1)) != cudaSuccess) rc = cuda_fail(h, e, "calibration launch");
+            if (rc == MOE_OK && i >= 0) cudaEventElapsedTime(&t[i], ev0, ev1);
+        }
+        if (rc == MOE_OK) {
+            std::sort(t, t + n_samples);
+            med[role] = 1e3 * (double)t[n_samples / 2];
+        }
+    }
+    cudaEventDestroy(ev0);
+    cudaEventDestroy(ev1);
+    if (rc != MOE_OK) return rc;
+    // Eq. 13: time per wave of each role; a launch runs L splits of V waves each
+    const double comp_waves = (double)ceil_div(plan.W_comp, plan.P) * s->L;
+    const double comm_waves = (double)ceil_div(plan.W_comm, C_ref) * s->L;
+    const double wave_comp = med[0] / comp_waves, wave_comm = med[1] / comm_waves;
+    if (!(wave_comp > 0.0)) return MOE_ERR_SHAPE;
+    if (wave_us_out) { wave_us_out[0] = wave_comp; wave_us_out[1] = wave_comm; }
+    *rho_out = rho;
+    rho_out->rho_ref = wave_comm / wave_comp;
+    rho_out->K_ref = s->I / s->TP;
+    rho_out->tile_m_ref = tile_m;
+    rho_out->tile_n_ref = tile_n;
+    rho_out->D_ref = s->EP;
+    rho_out->rows_ref = s->k_tot * s->TP + 1;
+    const int64_t split_w = ceil_div(s->H, s->L);
+    rho_out->comm_cols_ref = (int32_t)(split_w < kCommTileN ? split_w : kCommTileN);
+    return MOE_OK;
 }
 
 // ---- whole step from host buffers ----------------------------------------------------------

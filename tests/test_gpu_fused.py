@@ -358,3 +358,27 @@ def test_counts_left_on_the_device_give_the_same_bits(tile):
         assert p2.W_comp != plan.W_comp                # the estimate is not the true count here
         for a, o in zip(ref_outs, ws.out):
             assert np.array_equal(a, o.float().cpu().numpy(), equal_nan=True), rep
+
+
+def test_service_rate_characterisation_entry_point():
+    # Eq. 13 through the library: a positive, finite rho_ref with the reference factors of the workload
+    # it ran on, the device status clean, and two calls that agree within the run-to-run spread
+    h = G.handle()
+    w = replace(wl.DSV2L, name="rho_ref", T=2048, routing="uniform", zipf_s=0.0, target_r_expert=0.0,
+                tile_m=128, tile_n=256)
+    idx, wt, _ = wl.make_routing(w)
+    x, W2 = wl.make_data(w)
+    ws, idx_d, S = G.build_routing(w, idx, None)
+    xd, Wd, wt_d = x.cuda(), W2.cuda(), torch.from_numpy(wt).cuda()
+    vals = []
+    for _ in range(2):
+        rho, wave_comp, wave_comm = B.moe_calibrate_rho(h, xd, Wd, idx_d, wt_d, ws, C_ref=32, n_samples=7)
+        assert B.moe_get_status(h, ws.status).code == 0
+        assert wave_comp > 0 and wave_comm > 0 and abs(rho.rho_ref - wave_comm / wave_comp) < 1e-9
+        assert (rho.K_ref, rho.tile_m_ref, rho.tile_n_ref, rho.D_ref) == (w.K, 128, 256, w.EP)
+        assert rho.rows_ref == w.k_tot * w.TP + 1 and rho.comm_cols_ref == 1024
+        assert 1.0 < rho.rho_ref < 200.0
+        vals.append(rho.rho_ref)
+    assert abs(vals[0] - vals[1]) / vals[0] < 0.3
+    with pytest.raises(B.MoeError):
+        B.moe_calibrate_rho(h, xd, Wd, idx_d, wt_d, ws, C_ref=0)
