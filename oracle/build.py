@@ -6,23 +6,23 @@ import os
 import subprocess
 
 HERE = os.path.dirname(os.path.abspath(__file__))
-SRC = os.path.join(HERE, "gemm2_combine_ref.c")
+SRCS = [os.path.join(HERE, "gemm2_combine_ref.c"), os.path.join(HERE, "gemm1_act_ref.c")]
 OUT_DIR = os.path.join(HERE, "_build")
 LIB = os.path.join(OUT_DIR, "libmoe_oracle.so")
 
 
 def build(force: bool = False) -> str:
-    """Compile gemm2_combine_ref.c into a shared object and return its path.
+    """Compile the C sources of the oracle into one shared object and return its path.
 
     -O2, no fast-math, no FMA contraction: the loops keep the written order of fp32
     operations."""
     os.makedirs(OUT_DIR, exist_ok=True)
     if (not force and os.path.exists(LIB)
-            and os.path.getmtime(LIB) >= os.path.getmtime(SRC)):
+            and all(os.path.getmtime(LIB) >= os.path.getmtime(src) for src in SRCS)):
         return LIB
     tmp = LIB + f".tmp{os.getpid()}"
     cmd = ["gcc", "-O2", "-std=c11", "-fopenmp", "-ffp-contract=off", "-fno-fast-math",
-           "-shared", "-fPIC", "-o", tmp, SRC]
+           "-shared", "-fPIC", "-o", tmp] + SRCS + ["-lm"]
     subprocess.run(cmd, check=True)
     os.replace(tmp, LIB)
     return LIB

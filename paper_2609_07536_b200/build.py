@@ -14,8 +14,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmoe_b200.so")
-SOURCES = ["api.cu", "routing.cu", "gemm2_combine.cu", "solver.cpp"]
-HEADERS = [os.path.join(CSRC, "moe_internal.h"),
+SOURCES = ["api.cu", "routing.cu", "gemm2_combine.cu", "gemm1_act.cu", "solver.cpp"]
+HEADERS = [os.path.join(CSRC, "moe_internal.h"), os.path.join(CSRC, "sm100_device.cuh"),
            os.path.join(os.path.dirname(HERE), "include", "moe_b200.h")]
 
 
