@@ -269,6 +269,24 @@ int32_t moe_layer(moe_handle *h, const void *x_routed, const void *W2, const int
                   int32_t *tile_counts_pinned, void *const *out, void *y_ws, uint32_t *flags_ws,
                   uint32_t *status_dev, moe_plan *plan_out, void *ev_before, void *ev_after, void *stream);
 
+/* ---- the up-stream stage on the same GPU (Section II-A, steps 1-2; not changed by the paper) ------
+ * x_routed[r][i] = silu(g) * u with g = hidden[t] . W1[e][0][i], u = hidden[t] . W1[e][1][i] for the routed
+ * row r of assignment perm[r] = t * k_tot + j, e = topk_idx[t][j]; fp32 accumulation, bf16 result.  The
+ * paper says "a gated activation" without naming it: SiLU gating is the reading taken.  Produces the
+ * x_routed operand of moe_gemm2_combine in routed order.
+ *   hidden      [device] bf16 [T, H], 16-byte aligned; H % 16 == 0, H >= 64
+ *   W1          [device] bf16 [E_tot, 2, I, H] (plane 0 gate, plane 1 up; H contiguous); I % 16 == 0
+ *   routing     a routing workspace built by moe_build_routing with this tile_m; n_mtiles as for
+ *               moe_gemm2_combine (MOE_MTILES_ON_DEVICE allowed)
+ *   h_routed_ws [device] moe_gemm1_workspace_bytes() bytes: the gathered rows [R, H]
+ *   x_routed    [device] bf16 [R, I], 32-byte aligned, fully overwritten
+ * Asynchronous on `stream` (one gather launch, one persistent tcgen05 launch); device-side problems go
+ * to the status word like in moe_gemm2_combine. */
+int32_t moe_gemm1_workspace_bytes(const moe_shape *shape, size_t *h_routed_bytes);
+int32_t moe_gemm1_act(moe_handle *h, const void *hidden, const void *W1, const moe_shape *shape,
+                      int32_t tile_m, const moe_routing *routing, int32_t n_mtiles, void *h_routed_ws,
+                      void *x_routed, uint32_t *status_dev, void *stream);
+
 /* ---- one-time service-rate characterisation of a kernel family (Eq. 13, Section III-C) -------
  * Measures rho_ref on the caller's reference workload (inputs and workspaces as for moe_layer): the
  * GEMM alone on P(C_ref) compute slots and the combine alone on C_ref communication CTAs (static

@@ -23,6 +23,7 @@ MOE_DEV_OK, MOE_DEV_TIMEOUT, MOE_DEV_OOB, MOE_DEV_DUP_EXPERT = 0, 1, 2, 3
 MOE_MODE_FUSED, MOE_MODE_GEMM_ONLY, MOE_MODE_COMBINE_ONLY = 0, 1, 2
 MOE_RHO_PAPER, MOE_RHO_LOCAL = 0, 1
 MOE_MAX_EP, MOE_MAX_L = 8, 8
+MOE_MTILES_ON_DEVICE = -1
 
 EXPORTS = [
     "moe_create", "moe_destroy", "moe_last_cuda_error", "moe_set_wait_limit_ns",
@@ -31,6 +32,7 @@ EXPORTS = [
     "plan_partition", "plan_partition_estimate", "moe_time_plan_partition", "moe_gemm2_combine", "moe_get_status",
     "moe_clear_status",
     "moe_layer", "moe_calibrate_rho", "moe_host_arena_bytes", "moe_layer_host",
+    "moe_gemm1_workspace_bytes", "moe_gemm1_act",
 ]
 
 
@@ -114,6 +116,8 @@ def lib():
                                 P(vp), vp, vp, vp, P(moe_plan), vp, vp, vp]
         L.moe_calibrate_rho.argtypes = [vp, vp, vp, vp, vp, P(moe_shape), i32, i32, i32, i32, P(moe_routing), vp,
                                         P(vp), vp, vp, vp, P(moe_rho), P(C.c_double), vp]
+        L.moe_gemm1_workspace_bytes.argtypes = [P(moe_shape), P(C.c_size_t)]
+        L.moe_gemm1_act.argtypes = [vp, vp, vp, P(moe_shape), i32, P(moe_routing), i32, vp, vp, vp, vp]
         L.moe_host_arena_bytes.argtypes = [P(moe_shape), i32, i32, P(C.c_size_t)]
         L.moe_layer_host.argtypes = [vp, vp, vp, vp, vp, P(moe_shape), i32, i32, P(moe_sm_limits), vp,
                                      C.c_size_t, vp, vp, P(moe_plan), vp]
@@ -302,6 +306,19 @@ def moe_calibrate_rho(h, x_routed, W2, topk_idx, topk_w, ws: "Workspace", C_ref:
                                    _ptr(ws.tile_counts), outs, _ptr(ws.y_ws), _ptr(ws.flags_ws), _ptr(ws.status),
                                    C.byref(rho), waves, _stream(stream)), "moe_calibrate_rho", h)
     return rho, waves[0], waves[1]
+
+
+def moe_gemm1_workspace_bytes(shape) -> int:
+    b = C.c_size_t()
+    _check(lib().moe_gemm1_workspace_bytes(C.byref(shape), C.byref(b)), "moe_gemm1_workspace_bytes")
+    return b.value
+
+
+def moe_gemm1_act(h, hidden, W1, shape, tile_m, routing, n_mtiles, h_routed_ws, x_routed, status_dev, stream=None):
+    """Gather + grouped GEMM1 (gate, up) + silu(gate) * up -> x_routed [R, I] in routed order."""
+    _check(lib().moe_gemm1_act(h, _ptr(hidden), _ptr(W1), C.byref(shape), tile_m, C.byref(routing), n_mtiles,
+                               _ptr(h_routed_ws), _ptr(x_routed), _ptr(status_dev), _stream(stream)),
+           "moe_gemm1_act", h)
 
 
 def moe_host_arena_bytes(shape, tile_m, tile_n) -> int:

@@ -176,11 +176,6 @@ __device__ __forceinline__ void store_accumulator_rows(const FusedParams &P, uin
 // per 32-column group, straight from registers.  Needs every 16-column group whole and 32-byte aligned
 // (FusedParams::wide_store).  No shared memory and no intra-warp hand-over: this is the fastest of the
 // three when the epilogue is what limits a short-K tile.
-__device__ __forceinline__ void st_global_v8(void *p, const uint32_t (&w)[8])
-{
-    asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]),
-                 "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
-}
 // one 32-column group of this thread's row: bf16, two 32-byte stores
 __device__ __forceinline__ void emit_wide(const FusedParams &P, const uint32_t (&r)[32], int col, bool row_ok,
                                           __nv_bfloat16 *ybase, int q, int n0, int col_end, int cis0)

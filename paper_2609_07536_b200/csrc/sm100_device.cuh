@@ -186,6 +186,12 @@ __device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32])
                  : "memory");
 }
 
+// 256-bit global store (sm_100): 32 bytes, one full sector, from eight registers; p 32-byte aligned
+__device__ __forceinline__ void st_global_v8(void *p, const uint32_t (&w)[8])
+{
+    asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]),
+                 "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
+}
 __device__ __forceinline__ uint4 lds_v4(uint32_t addr)
 {
     uint4 v;

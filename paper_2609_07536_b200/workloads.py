@@ -191,6 +191,14 @@ def make_data(w: Workload):
     return x, W2
 
 
+def make_gemm1_data(w: Workload):
+    """Inputs of the up-stream stage: hidden states [T, H] ~ N(0, 1) (a normalised residual stream) and the
+    gate/up weights W1 [E_tot, 2, I, H] ~ N(0, 0.02), bf16, from the data seed."""
+    hidden = normal_bf16((w.T, w.H), w.data_seed + 101, std=1.0)
+    W1 = normal_bf16((w.E_tot, 2, w.I, w.H), w.data_seed + 102, std=0.02)
+    return hidden, W1
+
+
 def bf16_bits(t: torch.Tensor) -> np.ndarray:
     """bf16 tensor (CPU) -> numpy uint16 view of its bit patterns."""
     return t.contiguous().view(torch.int16).numpy().view(np.uint16)
