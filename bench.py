@@ -296,6 +296,57 @@ def calibrate(h, device, C_ref=32, tile=(128, 256)):
         "rows_ref": rho.rows_ref, "comm_cols_ref": rho.comm_cols_ref, "D_ref": rho.D_ref}}))
 
 
+# ----------------------------------------------------------------------------- up-stream stage (next row)
+
+def time_gemm1(h, dw, torch, n_warm=3, n_samples=9, cpu_rows=0):
+    """Gather + grouped GEMM1 + gated activation producing x_routed (Section II-A, steps 1-2), timed alone with
+    CUDA events on the workload's routing.  Not part of `value`: the paper leaves this stage unchanged."""
+    from paper_2609_07536_b200 import binding as B
+    from paper_2609_07536_b200 import workloads as wl
+    w = dw.w
+    g = torch.Generator(device=dw.x.device).manual_seed(w.data_seed + 101)
+    hidden = torch.randn((w.T, w.H), generator=g, device=dw.x.device).bfloat16()
+    W1 = (torch.randn((w.E_tot, 2, w.I, w.H), generator=g, device=dw.x.device) * 0.02).bfloat16()
+    hr = torch.empty(B.moe_gemm1_workspace_bytes(dw.shape), dtype=torch.uint8, device=dw.x.device)
+    xr = torch.empty((w.R, w.I), dtype=torch.bfloat16, device=dw.x.device)
+    B.moe_build_routing(h, dw.idx_d, dw.shape, w.tile_m, dw.ws.routing, dw.ws.tile_counts, dw.ws.status)
+    torch.cuda.synchronize()
+    S = int(dw.ws.tile_counts[w.E_tot])
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_samples)]
+    for i in range(n_warm + n_samples):
+        if i >= n_warm:
+            evs[i - n_warm][0].record()
+        B.moe_gemm1_act(h, hidden, W1, dw.shape, w.tile_m, dw.ws.routing, S, hr, xr, dw.ws.status)
+        if i >= n_warm:
+            evs[i - n_warm][1].record()
+    torch.cuda.synchronize()
+    assert B.moe_get_status(h, dw.ws.status).code == 0
+    us = statistics.median(a.elapsed_time(b) * 1e3 for a, b in evs)
+    flops = 4.0 * w.R * w.H * w.I
+    res = {"us": us, "tflops": flops / us / 1e6, "flops": flops,
+           "bytes_gather": 2.0 * w.R * w.H * 2, "launches": 2,
+           "what": "gather + grouped GEMM1 (gate, up) + silu(gate) * up -> x_routed; timed alone (burst peak applies)"}
+    if cpu_rows > 0:   # the oracle of this stage on a seeded sample of routed rows: parity check and CPU time
+        import numpy as np
+        from oracle import gemm1_act_ref as g1
+        from oracle import gemm2_combine_ref as g2
+        from oracle import routing_ref as rr
+        rows = np.sort(np.random.default_rng(0).choice(w.R, size=min(w.R, cpu_rows), replace=False)).astype(np.int32)
+        perm = rr.build_routing(dw.idx, w.E_tot, w.tile_m)["perm"]
+        hb, Wb = wl.bf16_bits(hidden.cpu()), wl.bf16_bits(W1.cpu())
+        t0 = time.perf_counter()
+        ref = g1.gemm1_act(hb, Wb, dw.idx, perm, rows=rows)
+        dt = time.perf_counter() - t0
+        got = xr.float().cpu().numpy()[rows]
+        rms = float(np.sqrt(np.mean(ref.astype(np.float64) ** 2)))
+        tol = 1e-2 * rms + 1e-3 + 2.0 ** -8 * np.abs(ref)
+        res["cpu_oracle"] = {"value": dt / len(rows) * w.R * 1e6, "unit": "us/layer", "cores": g2.threads(), "kind": "oracle",
+                             "sample": f"{len(rows)} of {w.R} routed rows in {dt:.2f} s, scaled by R/n"}
+        res["parity_on_sample"] = {"rows": int(len(rows)), "max_abs_err": float(np.max(np.abs(got - ref))),
+                                   "within_tolerance": bool(np.all(np.abs(got - ref) <= tol))}
+    return res
+
+
 # ----------------------------------------------------------------------------- CPU baseline
 
 def cpu_baseline(w, idx, wt, x_cpu, W2_cpu, budget_s=15.0):
@@ -376,7 +427,7 @@ def main():
     ap.add_argument("--workload", default="dsv2lite")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-regret", action="store_true")
-    ap.add_argument("--only", default="", choices=["", "fused", "gemm_only", "combine_only"],
+    ap.add_argument("--only", default="", choices=["", "fused", "gemm_only", "combine_only", "gemm1"],
                     help="time just this launch mode (for profiling): warmup + steps launches, short JSON")
     ap.add_argument("--force-C", type=int, default=0, help="with --only: communication CTAs (0 = analytical)")
     ap.add_argument("--data", default="seeded", choices=["seeded", "device"])
@@ -433,6 +484,11 @@ def main():
     step, (occ, lim, rho) = make_stepper(h, dw, limits_override=dict(drain_help=args.drain_help))
     K, W = max(1, args.steps), max(3, args.warmup)
 
+    if args.only == "gemm1":
+        res = time_gemm1(h, dw, torch, n_warm=max(1, args.warmup), n_samples=K)
+        print(json.dumps({"only": "gemm1", "workload": w.name, **res}))
+        B.moe_destroy(h)
+        return
     if args.only:
         mode = {"fused": B.MOE_MODE_FUSED, "gemm_only": B.MOE_MODE_GEMM_ONLY,
                 "combine_only": B.MOE_MODE_COMBINE_ONLY}[args.only]
@@ -544,6 +600,10 @@ def main():
         extra["solver_ns"] = B.moe_time_plan_partition(sets, occ, lim, dw.shape, rho, 1_000_000)
         if not args.no_cpu_baseline:
             extra["cpu_baseline"], _ = cpu_baseline(w, dw.idx, dw.wt, dw.x_cpu, dw.W2_cpu)
+        # ---- the up-stream stage (next row of the scope table), reported beside the headline, not in it
+        g1res = time_gemm1(h, dw, torch, cpu_rows=0 if args.no_cpu_baseline else 4096)
+        g1res["frac_of_bf16_peak"] = g1res["tflops"] / peaks["bf16_tflops"]
+        extra["gemm1_act"] = g1res
 
     if rank == 0:
         # the fused kernel is timed inside the K-step loop (power-capped steady state), so its tensor
