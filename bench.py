@@ -322,9 +322,22 @@ def time_gemm1(h, dw, torch, n_warm=3, n_samples=9, cpu_rows=0):
     torch.cuda.synchronize()
     assert B.moe_get_status(h, dw.ws.status).code == 0
     us = statistics.median(a.elapsed_time(b) * 1e3 for a, b in evs)
+    # the whole post-router layer (routing build -> GEMM1 + activation -> plan -> GEMM2 + combine), one call per step
+    W2 = dw.W2
+    lay = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_samples)]
+    for i in range(n_warm + n_samples):
+        if i >= n_warm:
+            lay[i - n_warm][0].record()
+        B.moe_post_router_layer(h, hidden, W1, W2, dw.idx_d, dw.wt_d, dw.ws, hr, xr)
+        if i >= n_warm:
+            lay[i - n_warm][1].record()
+    torch.cuda.synchronize()
+    assert B.moe_get_status(h, dw.ws.status).code == 0
+    layer_us = statistics.median(a.elapsed_time(b) * 1e3 for a, b in lay)
     flops = 4.0 * w.R * w.H * w.I
     res = {"us": us, "tflops": flops / us / 1e6, "flops": flops,
            "bytes_gather": 2.0 * w.R * w.H * 2, "launches": 2,
+           "post_router_layer_us": layer_us, "post_router_layer_launches": 7,
            "what": "gather + grouped GEMM1 (gate, up) + silu(gate) * up -> x_routed; timed alone (burst peak applies)"}
     if cpu_rows > 0:   # the oracle of this stage on a seeded sample of routed rows: parity check and CPU time
         import numpy as np

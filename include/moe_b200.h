@@ -287,6 +287,19 @@ int32_t moe_gemm1_act(moe_handle *h, const void *hidden, const void *W1, const m
                       int32_t tile_m, const moe_routing *routing, int32_t n_mtiles, void *h_routed_ws,
                       void *x_routed, uint32_t *status_dev, void *stream);
 
+/* ---- the post-router MoE layer on device-resident inputs (Section II-A: the three operations) ----
+ * Routing build -> moe_gemm1_act (launched at once: it reads the m-tile count on the device) -> wait for
+ * the tile counts (hidden behind GEMM1) -> plan_partition -> moe_gemm2_combine.  Arguments as for
+ * moe_gemm1_act and moe_layer; x_routed_ws [device] bf16 [R, I], 32-byte aligned, is the intermediate.
+ * tile_counts_pinned = NULL: no copy and no wait, plan from plan_partition_estimate.  A handle serves one
+ * such call at a time (it owns the event the wait uses).  Asynchronous on `stream` after the wait. */
+int32_t moe_post_router_layer(moe_handle *h, const void *hidden, const void *W1, const void *W2,
+                              const int32_t *topk_idx, const float *topk_w, const moe_shape *shape,
+                              int32_t tile_m, int32_t tile_n, const moe_sm_limits *limits_or_null,
+                              const moe_routing *routing, int32_t *tile_counts_pinned, void *h_routed_ws,
+                              void *x_routed_ws, void *const *out, void *y_ws, uint32_t *flags_ws,
+                              uint32_t *status_dev, moe_plan *plan_out, void *stream);
+
 /* ---- one-time service-rate characterisation of a kernel family (Eq. 13, Section III-C) -------
  * Measures rho_ref on the caller's reference workload (inputs and workspaces as for moe_layer): the
  * GEMM alone on P(C_ref) compute slots and the combine alone on C_ref communication CTAs (static

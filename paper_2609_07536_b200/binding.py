@@ -32,7 +32,7 @@ EXPORTS = [
     "plan_partition", "plan_partition_estimate", "moe_time_plan_partition", "moe_gemm2_combine", "moe_get_status",
     "moe_clear_status",
     "moe_layer", "moe_calibrate_rho", "moe_host_arena_bytes", "moe_layer_host",
-    "moe_gemm1_workspace_bytes", "moe_gemm1_act",
+    "moe_gemm1_workspace_bytes", "moe_gemm1_act", "moe_post_router_layer",
 ]
 
 
@@ -118,6 +118,8 @@ def lib():
                                         P(vp), vp, vp, vp, P(moe_rho), P(C.c_double), vp]
         L.moe_gemm1_workspace_bytes.argtypes = [P(moe_shape), P(C.c_size_t)]
         L.moe_gemm1_act.argtypes = [vp, vp, vp, P(moe_shape), i32, P(moe_routing), i32, vp, vp, vp, vp]
+        L.moe_post_router_layer.argtypes = [vp, vp, vp, vp, vp, vp, P(moe_shape), i32, i32, P(moe_sm_limits),
+                                            P(moe_routing), vp, vp, vp, P(vp), vp, vp, vp, P(moe_plan), vp]
         L.moe_host_arena_bytes.argtypes = [P(moe_shape), i32, i32, P(C.c_size_t)]
         L.moe_layer_host.argtypes = [vp, vp, vp, vp, vp, P(moe_shape), i32, i32, P(moe_sm_limits), vp,
                                      C.c_size_t, vp, vp, P(moe_plan), vp]
@@ -319,6 +321,20 @@ def moe_gemm1_act(h, hidden, W1, shape, tile_m, routing, n_mtiles, h_routed_ws, 
     _check(lib().moe_gemm1_act(h, _ptr(hidden), _ptr(W1), C.byref(shape), tile_m, C.byref(routing), n_mtiles,
                                _ptr(h_routed_ws), _ptr(x_routed), _ptr(status_dev), _stream(stream)),
            "moe_gemm1_act", h)
+
+
+def moe_post_router_layer(h, hidden, W1, W2, topk_idx, topk_w, ws: "Workspace", h_routed_ws, x_routed_ws,
+                          limits=None, stream=None, counts_on_device=False) -> moe_plan:
+    """Routing build -> GEMM1 + activation -> plan -> GEMM2 + combine, one library call."""
+    outs = (C.c_void_p * len(ws.out))(*[_ptr(o) for o in ws.out])
+    plan = moe_plan()
+    _check(lib().moe_post_router_layer(h, _ptr(hidden), _ptr(W1), _ptr(W2), _ptr(topk_idx), _ptr(topk_w),
+                                       C.byref(ws.shape), ws.tile_m, ws.tile_n,
+                                       C.byref(limits) if limits is not None else None, C.byref(ws.routing),
+                                       None if counts_on_device else _ptr(ws.tile_counts), _ptr(h_routed_ws),
+                                       _ptr(x_routed_ws), outs, _ptr(ws.y_ws), _ptr(ws.flags_ws), _ptr(ws.status),
+                                       C.byref(plan), _stream(stream)), "moe_post_router_layer", h)
+    return plan
 
 
 def moe_host_arena_bytes(shape, tile_m, tile_n) -> int:

@@ -91,12 +91,20 @@ int32_t moe_create(int32_t device, moe_handle **out)
         delete h;
         return MOE_ERR_CUDA;
     }
+    cudaEvent_t ev = nullptr;
+    e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
+    if (e != cudaSuccess) {
+        delete h;
+        return MOE_ERR_CUDA;
+    }
+    h->counts_event = ev;
     *out = h;
     return MOE_OK;
 }
 
 int32_t moe_destroy(moe_handle *h)
 {
+    if (h && h->counts_event) cudaEventDestroy(static_cast<cudaEvent_t>(h->counts_event));
     delete h;
     return MOE_OK;
 }
@@ -426,6 +434,48 @@ int32_t moe_layer(moe_handle *h, const void *x_routed, const void *W2, const int
                            out, y_ws, flags_ws, status_dev, st);
     if (ev_after) cudaEventRecord(static_cast<cudaEvent_t>(ev_after), st);
     return rc;
+}
+
+// ---- the post-router MoE layer on device-resident inputs (Section II-A: steps 1-3) -------------
+
+int32_t moe_post_router_layer(moe_handle *h, const void *hidden, const void *W1, const void *W2,
+                              const int32_t *topk_idx, const float *topk_w, const moe_shape *s, int32_t tile_m,
+                              int32_t tile_n, const moe_sm_limits *limits_or_null, const moe_routing *routing,
+                              int32_t *tile_counts_pinned, void *h_routed_ws, void *x_routed_ws, void *const *out,
+                              void *y_ws, uint32_t *flags_ws, uint32_t *status_dev, moe_plan *plan_out, void *stream)
+{
+    if (!h || !s || !routing) return MOE_ERR_NULL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t rc = moe_build_routing(h, topk_idx, s, tile_m, routing, tile_counts_pinned, status_dev, st);
+    if (rc != MOE_OK) return rc;
+    // GEMM1 reads the m-tile count on the device, so it is launched before the host waits for the counts:
+    // the wait and the planning are hidden behind it
+    if (tile_counts_pinned && h->counts_event) cudaEventRecord(static_cast<cudaEvent_t>(h->counts_event), st);
+    rc = moe_gemm1_act(h, hidden, W1, s, tile_m, routing, MOE_MTILES_ON_DEVICE, h_routed_ws, x_routed_ws, status_dev, st);
+    if (rc != MOE_OK) return rc;
+    moe_occupancy occ;
+    moe_sm_limits lim;
+    moe_rho rho;
+    rc = moe_query_occupancy(h, tile_m, tile_n, &occ, &lim, &rho);
+    if (rc != MOE_OK) return rc;
+    if (limits_or_null) lim = *limits_or_null;
+    moe_plan plan;
+    int32_t n_mtiles = MOE_MTILES_ON_DEVICE;
+    if (tile_counts_pinned) {
+        // the copy of the counts was queued right after the routing kernels, before GEMM1: wait for it alone
+        cudaEvent_t counts_ready = static_cast<cudaEvent_t>(h->counts_event);
+        if (!counts_ready) return MOE_ERR_CUDA;
+        cudaError_t e = cudaEventSynchronize(counts_ready);
+        if (e != cudaSuccess) return cuda_fail(h, e, "tile counts wait");
+        rc = plan_partition(tile_counts_pinned, s->E_tot, &occ, &lim, s, &rho, &plan);
+        n_mtiles = tile_counts_pinned[s->E_tot];
+    } else {
+        rc = plan_partition_estimate(&occ, &lim, s, &rho, &plan);
+    }
+    if (rc != MOE_OK) return rc;
+    if (plan_out) *plan_out = plan;
+    return moe_gemm2_combine(h, x_routed_ws, W2, topk_idx, topk_w, s, &occ, routing, n_mtiles, &plan, out, y_ws,
+                             flags_ws, status_dev, st);
 }
 
 // ---- one-time service-rate characterisation (Eq. 13) ---------------------------------------

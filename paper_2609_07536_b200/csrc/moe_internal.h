@@ -68,6 +68,7 @@ struct moe_handle {
     int o_comp[3] = {0, 0, 0};                          // tile_n = 64, 128, 256
     int o_pair = 0;                                     // CTA-pair kernel: resident CTAs per SM
     int max_pairs = 0;                                  // ... and co-resident clusters of two
+    void *counts_event = nullptr;                       // cudaEvent_t: "the tile counts have reached the host"
 };
 
 namespace moe {

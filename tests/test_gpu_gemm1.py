@@ -128,3 +128,34 @@ def test_argument_validation():
     with pytest.raises(B.MoeError) as e:
         B.moe_gemm1_act(h, hd, Wd, bad, w.tile_m, ws.routing, S, hr, x, ws.status)
     assert e.value.code == B.MOE_ERR_SHAPE
+
+
+@pytest.mark.parametrize("counts_on_device", [False, True], ids=["host_counts", "device_counts"])
+def test_post_router_layer_against_the_oracle_chain(counts_on_device):
+    # the three operations of Section II-A in one call, against the oracle's GEMM1 + activation (rounded to
+    # bf16 as the stored intermediate is) followed by the oracle's GEMM2 + combine
+    h = G.handle()
+    w = replace(wl.TINY, name="layer3", T=500, E=10, k=3, n_shared=1, H=256, I=256, TP=2, EP=2, L=2,
+                tile_m=128, tile_n=128, routing="zipf", zipf_s=1.0, target_r_expert=2.0)
+    idx, wt, _ = wl.make_routing(w)
+    hidden, W1 = wl.make_gemm1_data(w)
+    _, W2 = wl.make_data(w)
+    ws = B.alloc_workspace(G.shape_of(w), w.tile_m, w.tile_n)
+    hr = torch.empty(B.moe_gemm1_workspace_bytes(ws.shape), dtype=torch.uint8, device="cuda")
+    xr = torch.empty((w.R, w.I), dtype=torch.bfloat16, device="cuda")
+    idx_d, wt_d = torch.from_numpy(idx).cuda(), torch.from_numpy(wt).cuda()
+    for o in ws.out:
+        o.fill_(float("nan"))
+    plan = B.moe_post_router_layer(h, hidden.cuda(), W1.cuda(), W2.cuda(), idx_d, wt_d, ws, hr, xr,
+                                   counts_on_device=counts_on_device)
+    torch.cuda.synchronize()
+    assert B.moe_get_status(h, ws.status).code == 0 and plan.comm_ctas >= 1
+    r = rr.build_routing(idx, w.E_tot, w.tile_m)
+    x_ref = g1.gemm1_act(wl.bf16_bits(hidden), wl.bf16_bits(W1), idx, r["perm"])
+    x_bits = wl.bf16_bits(torch.from_numpy(x_ref).bfloat16())
+    expect = g2.gemm2_combine(x_bits, wl.bf16_bits(W2), idx, wt, r["inv_perm"])
+    outs = [o.float().cpu().numpy() for o in ws.out]
+    got = np.concatenate([o[:len(G.tokens_of_rank(w.T, w.EP, d))] for d, o in enumerate(outs)])
+    assert not np.isnan(got).any()
+    # the intermediate may differ from the oracle's by one bf16 step in a few places: same tolerance form
+    assert np.max(np.abs(got - expect)) <= G.tolerance(expect)
