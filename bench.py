@@ -446,6 +446,7 @@ def main():
     ap.add_argument("--data", default="seeded", choices=["seeded", "device"])
     ap.add_argument("--tile", default="", help="GEMM tile MxN overriding the workload's (e.g. 256x256)")
     ap.add_argument("--L", type=int, default=0, help="pipeline splits overriding the workload's")
+    ap.add_argument("--T", type=int, default=0, help="token count overriding the workload's (small-T studies)")
     ap.add_argument("--calibrate", action="store_true",
                     help="one-time service-rate characterisation of the kernel family (Eq. 13): prints rho_ref")
     ap.add_argument("--sweep", action="store_true", help="selector-regret sweep on the DeepSeek-V2-Lite shape")
@@ -493,6 +494,9 @@ def main():
     if args.L:
         from dataclasses import replace
         w = replace(w, L=args.L)
+    if args.T:
+        from dataclasses import replace
+        w = replace(w, T=args.T, name=f"{w.name}_T{args.T}")
     dw = DeviceWorkload(w, device, data=args.data if args.only else "seeded")
     step, (occ, lim, rho) = make_stepper(h, dw, limits_override=dict(drain_help=args.drain_help))
     K, W = max(1, args.steps), max(3, args.warmup)

@@ -261,7 +261,8 @@ int32_t moe_clear_status(moe_handle *h, uint32_t *status_dev, void *stream);
  * Returns after the fused kernel has been launched (asynchronous on `stream`); the only host wait
  * inside is the one for the tile counts.  tile_counts_pinned = NULL selects the device-only-counts
  * path of Section III-E: no copy, no wait; the plan comes from plan_partition_estimate and the kernel
- * reads the tile count on the device (the whole call is then asynchronous and can be stream-captured).  ev_before / ev_after: optional cudaEvent_t handles (NULL = none)
+ * reads the tile count on the device (the whole call is then asynchronous; it is not meant for graph replay: the launch epoch that marks
+ * this launch's flags is a kernel argument set by the host on every call).  ev_before / ev_after: optional cudaEvent_t handles (NULL = none)
  * recorded on `stream` right before and right after the fused launch, for timing it. */
 int32_t moe_layer(moe_handle *h, const void *x_routed, const void *W2, const int32_t *topk_idx,
                   const float *topk_w, const moe_shape *shape, int32_t tile_m, int32_t tile_n,
