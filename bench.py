@@ -252,7 +252,7 @@ def run_sweep(h, args, peaks):
             step, (occ, lim, rho) = make_stepper(h, dw, limits_override=dict(drain_help=dh))
             plan, counts = step()
             torch.cuda.synchronize()
-            r = regret_of_workload(step, torch, counts, lim, plan.comm_ctas, n_warm=1, n_samples=3,
+            r = regret_of_workload(step, torch, counts, lim, plan.comm_ctas, n_warm=1, n_samples=args.sweep_samples,
                                    keep_curve=args.sweep_curves)
             r.update(W_comp=plan.W_comp, W_comm=plan.W_comm, rho=plan.rho_q / 2 ** 20,
                      roofline_frac=(dw.flops / peaks["bf16_tflops"] / 1e6) / r["t_pick_us"])
@@ -453,6 +453,7 @@ def main():
     ap.add_argument("--sweep-out", default="gpurun_out/sweep.json")
     ap.add_argument("--sweep-filter", default="", help="substring a sweep workload name must contain")
     ap.add_argument("--sweep-curves", action="store_true", help="keep every t(C) in the sweep output")
+    ap.add_argument("--sweep-samples", type=int, default=5, help="timed samples per C in the sweep")
     ap.add_argument("--counts", default="host", choices=["host", "device"],
                     help="host: tile counts copied to the host, exact plan (default); device: no copy and no wait, "
                          "plan from the normalised-load estimate (Section III-E)")
