@@ -1,7 +1,7 @@
 """Benchmark of the MoE GEMM2 + GatherRS hot path on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload dsv2lite] [--impl reference]
-    python bench.py --sweep [--sweep-out gpurun_out/sweep.json]      (selector-regret sweep)
+    python bench.py --sweep [--sweep-out sweep.json]                 (selector-regret sweep)
 
 One step = one pass of the whole hot path over one batch: routing/tile-count build (GPU) ->
 tile counts to the host -> analytical plan (host) -> fused grouped GEMM2 + combine (GPU).
@@ -450,7 +450,7 @@ def main():
     ap.add_argument("--calibrate", action="store_true",
                     help="one-time service-rate characterisation of the kernel family (Eq. 13): prints rho_ref")
     ap.add_argument("--sweep", action="store_true", help="selector-regret sweep on the DeepSeek-V2-Lite shape")
-    ap.add_argument("--sweep-out", default="gpurun_out/sweep.json")
+    ap.add_argument("--sweep-out", default="sweep.json")
     ap.add_argument("--sweep-filter", default="", help="substring a sweep workload name must contain")
     ap.add_argument("--sweep-curves", action="store_true", help="keep every t(C) in the sweep output")
     ap.add_argument("--sweep-samples", type=int, default=5, help="timed samples per C in the sweep")
