@@ -296,6 +296,7 @@ int32_t moe_gemm2_combine(moe_handle *h, const void *x_routed, const void *W2, c
     p.S_dev = counts_on_device ? r->tiles + s->E_tot : nullptr;
     p.C = C; p.P = Pc; p.mode = mode; p.withhold = plan->debug_withhold_tile;
     p.drain_help = (mode == MOE_MODE_FUSED && plan->drain_help) ? 1 : 0;
+    p.tile_order = plan->drain_help ? 1 : 0;   // nothing waits for an early split then: x is read once
     p.tok_blk = (int32_t)ceil_div(s->T, s->EP);
     p.tok_tiles_per_rank = (int32_t)ceil_div(p.tok_blk, kCommTileM);
     p.comm_cols = (int32_t)ceil_div(p.split_w, kCommTileN);

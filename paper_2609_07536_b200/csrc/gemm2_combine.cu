@@ -7,7 +7,8 @@
 //                   from a queue per split that former compute CTAs also serve).
 //   blockIdx >= C : compute CTA b = blockIdx - C (Section III-C: takes global tiles
 //                   b, b+P, b+2P, ... of the split-major sequence in which the expert
-//                   problems of one split are contiguous).
+//                   problems of one split are contiguous; m-tile-major across the splits when
+//                   the communication work is handed out dynamically).
 //
 // Compute CTA (warp-specialised; tile_m x tile_n with tile_m in {64, 128}):
 //   warps 0, 2  TMA producers (one thread each): warp 0 the x_routed tile (128 rows x 64 k), warp 2 the
@@ -120,16 +121,33 @@ __device__ __forceinline__ bool wait_barrier_1t(uint32_t bar, uint32_t parity, C
 
 struct Tile {
     int s, mu, p, i_n;
+    int id;   // canonical tile number s * W_comp + (mu * TP + p) * NTs + i_n: indexes the readiness flags
 };
+// Tile g of the processing sequence.  Split-major (Section III-C: all tiles of split s precede those of
+// s + 1; inside a split the expert problems are contiguous), or, when the work is handed out dynamically
+// and nothing waits for an early split (drain help), m-tile-major: the n-tiles of ALL splits of one
+// (m-tile, K-shard) are adjacent, so that the x rows are read from DRAM once instead of once per split.
 __device__ __forceinline__ Tile decode_tile(int g, const FusedParams &P, int W_comp)
 {
     Tile t;
-    t.s = g / W_comp;
-    const int idx = g - t.s * W_comp;
-    const int r = idx / P.NTs;
-    t.i_n = idx - r * P.NTs;
-    t.mu = r / P.TP;
-    t.p = r - t.mu * P.TP;
+    if (P.tile_order == 0) {
+        t.s = g / W_comp;
+        const int idx = g - t.s * W_comp;
+        const int r = idx / P.NTs;
+        t.i_n = idx - r * P.NTs;
+        t.mu = r / P.TP;
+        t.p = r - t.mu * P.TP;
+        t.id = g;
+    } else {
+        const int per_m = P.L * P.NTs;
+        const int r = g / per_m;
+        const int j = g - r * per_m;
+        t.s = j / P.NTs;
+        t.i_n = j - t.s * P.NTs;
+        t.mu = r / P.TP;
+        t.p = r - t.mu * P.TP;
+        t.id = t.s * W_comp + r * P.NTs + t.i_n;
+    }
     return t;
 }
 
@@ -472,10 +490,11 @@ __device__ void compute_cta(const FusedParams &P, int W_comp, uint8_t *ring, Con
                 if (!wait_barrier_1t(smem_u32(&ctl->epi_done[a]), (uint32_t)(it >> 1) & 1u, ctl, deadline, P.status,
                                      (uint32_t)g, 32u))
                     break;
-                if (g != P.withhold) {
+                const Tile t = decode_tile(g, P, W_comp);
+                if (t.id != P.withhold) {
                     __threadfence();   // release: the epilogue warps' stores (observed through epi_done) come first
-                    st_relaxed_u32(&P.flags[g], P.epoch);
-                    red_relaxed_add_u32(&P.split_done[g / W_comp], 1u);
+                    st_relaxed_u32(&P.flags[t.id], P.epoch);
+                    red_relaxed_add_u32(&P.split_done[t.s], 1u);
                 }
                 mbar_arrive(smem_u32(&ctl->pub_done[a]));
             }
@@ -718,10 +737,11 @@ __device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring
                 if (!wait_barrier_1t(smem_u32(&ctl->epi_done[a]), (uint32_t)(it >> 1) & 1u, ctl, deadline, P.status,
                                      (uint32_t)g, 32u))
                     break;
-                if (g != P.withhold) {
+                const Tile t = decode_tile(g, P, W_comp);
+                if (t.id != P.withhold) {
                     __threadfence();
-                    st_relaxed_u32(&P.flags[2 * g + (int)rank], P.epoch);
-                    red_relaxed_add_u32(&P.split_done[g / W_comp], 1u);
+                    st_relaxed_u32(&P.flags[2 * t.id + (int)rank], P.epoch);
+                    red_relaxed_add_u32(&P.split_done[t.s], 1u);
                 }
                 mbar_arrive(smem_u32(&ctl->pub_done[a]));
             }

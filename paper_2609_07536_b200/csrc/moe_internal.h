@@ -50,6 +50,7 @@ struct alignas(64) FusedParams {
     int32_t tok_blk, tok_tiles_per_rank, comm_cols, comm_tiles;
     int32_t num_kb, last_ksteps;
     int32_t drain_help;                 // compute CTAs serve communication tiles once their GEMM tiles are done
+    int32_t tile_order;                 // 0: split-major tile sequence (the paper's); 1: m-tile-major across splits
     int32_t flag_parts;                 // readiness flags per tile: 1, or 2 for a CTA-pair tile
     int32_t Q, slab_cols, slab_shift;   // Q = k_tot * TP rows per unit; slab_cols = 1 << slab_shift
     int32_t wide_store;                 // every 16-column group of a Y row is whole and 32-byte aligned: 256-bit epilogue stores
