@@ -228,7 +228,8 @@ int32_t moe_time_plan_partition(const int32_t *routed_tile_counts, int32_t n_set
 
 /* ---- a3-a5: fused grouped GEMM2 + GatherRS combine --------------------------------------
  * Section II-A step 3, Section II-B (compute CTAs publish, communication CTAs consume),
- * Section III-C (CTA b takes global tiles b, b+P, ... of the split-major sequence),
+ * Section III-C (CTA b takes global tiles b, b+P, ... of the split-major sequence; with
+ * plan->drain_help the sequence is m-tile-major across the splits, so that x_routed is read once),
  * Section III-E (C* communication CTAs, R(C*) reserved SMs, P(C*) compute CTAs).
  *   out_d[t - d*ceil(T/EP)][:] = sum_j topk_w[t][j] * sum_p (x_routed[inv_perm[t,j]][Kp] . W2[e][:, Kp])
  * x_routed [device] bf16 [R, I]; W2 [device] bf16 [E_tot, H, I]; topk_w [device] fp32 [T, k_tot];
@@ -237,7 +238,7 @@ int32_t moe_time_plan_partition(const int32_t *routed_tile_counts, int32_t n_set
  * for the tokens rank d owns; y_ws / flags_ws / status_dev as sized by moe_workspace_bytes.
  * n_mtiles = S (host value from moe_build_routing).  Requires H % 8 == 0, K % 16 == 0,
  * ceil(H/L) % 8 == 0, 16-byte aligned pointers, 1 <= C, 1 <= P, R * o_comm >= C,
- * R + ceil(P / o_comp) * comp_slot_sms <= G. 
+ * R + ceil(P / o_comp) * comp_slot_sms <= G.
  * n_mtiles = MOE_MTILES_ON_DEVICE: the kernel reads S from the routing workspace itself (no host copy of
  * the counts is needed; the plan then comes from plan_partition_estimate). */
 int32_t moe_gemm2_combine(moe_handle *h, const void *x_routed, const void *W2,
