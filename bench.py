@@ -643,11 +643,15 @@ def main():
         }
         # DRAM read + write bytes of one fused launch from the ncu capture summarised in
         # profiles/fused_gemm2_combine_dsv2lite_ncu.md (same workload, same launch configuration)
+        x_passes = 1 if args.drain_help else w.L      # m-tile-major order reads x once, split-major once per split
+        all_bytes = (w.R * w.I * 2 * x_passes + w.E_tot * w.H * w.I * 2 +
+                     2 * w.T * w.L * w.k_tot * w.TP * (-(-w.H // w.L)) * 2 + w.T * w.H * 2)
+        # every byte the launch has to move through HBM (x, W2, Y written and read back, out): not part of the
+        # headline roofline, but the real bound at small T, where every expert's weights are read for a few rows
+        roofline["hbm_all_traffic_us"] = all_bytes / peaks["hbm_gbs"] / 1e3
         if w.name in NCU_TRAFFIC_BYTES and (w.tile_m, w.tile_n, w.L) == NCU_TRAFFIC_BYTES[w.name][1]:
             roofline["traffic"] = NCU_TRAFFIC_BYTES[w.name][0]
-            x_passes = 1 if args.drain_help else w.L      # m-tile-major order reads x once, split-major once per split
-            roofline["traffic_algorithmic"] = (w.R * w.I * 2 * x_passes + w.E_tot * w.H * w.I * 2 +
-                                               2 * w.T * w.L * w.k_tot * w.TP * (-(-w.H // w.L)) * 2 + w.T * w.H * 2)
+            roofline["traffic_algorithmic"] = all_bytes
         line = {
             "metric": METRIC, "value": job_value(step_us, world), "unit": "us/layer", "n_gpus": world, "steps": K, "warmup": W,
             "ms_per_step": step_us / 1e3, "higher_is_better": False, "scaling": "weak",
