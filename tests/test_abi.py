@@ -55,3 +55,16 @@ def test_workspace_sizes_and_argument_errors():
     assert B.lib().moe_workspace_bytes(None, 64, 64, None, None, None, None) == B.MOE_ERR_NULL
     assert B.lib().moe_destroy(None) == B.MOE_OK
     assert B.moe_host_arena_bytes(s, 64, 64) > rb + yb + fb
+
+
+def test_header_is_plain_c():
+    # the boundary is a C ABI: the header has to compile as C99 on its own (no C++-isms, no torch types)
+    import shutil
+    import subprocess
+    gcc = shutil.which("gcc")
+    if gcc is None:
+        pytest.skip("no C compiler here")
+    header = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "include", "moe_b200.h")
+    res = subprocess.run([gcc, "-std=c99", "-Wall", "-Werror", "-fsyntax-only", "-x", "c", header],
+                         capture_output=True, text=True)
+    assert res.returncode == 0, res.stderr
