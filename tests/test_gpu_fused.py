@@ -382,3 +382,32 @@ def test_service_rate_characterisation_entry_point():
     assert abs(vals[0] - vals[1]) / vals[0] < 0.3
     with pytest.raises(B.MoeError):
         B.moe_calibrate_rho(h, xd, Wd, idx_d, wt_d, ws, C_ref=0)
+
+
+def test_random_small_shapes_against_the_oracle():
+    # seeded fuzz over the argument space the kernels accept: tile families, splits, shards, ranks, ragged
+    # sizes, forced and analytical C, static map and dynamic hand-out; every token checked
+    rng = np.random.default_rng(2024)
+    n_done = 0
+    for case in range(36):
+        tile_m, tile_n = [(64, 64), (64, 128), (128, 64), (128, 128), (128, 256), (256, 256)][int(rng.integers(6))]
+        TP = int(rng.choice([1, 2, 4]))
+        K = int(rng.choice([16, 48, 64, 80, 128, 208]))
+        L = int(rng.choice([1, 2, 3, 4]))
+        H = int(rng.choice([64, 136, 256, 320, 768])) * L if rng.random() < 0.5 else int(rng.choice([64, 128, 264, 512, 1024]))
+        if (-(-H // L)) % 8 != 0 or H % 8 != 0:
+            continue
+        E = int(rng.integers(1, 20))
+        k = int(rng.integers(1, min(E, 4) + 1))
+        n_shared = int(rng.choice([0, 0, 1, 2]))
+        T = int(rng.choice([1, 7, 65, 200, 513, 900]))
+        EP = int(rng.choice([1, 2, 3, 4, 8]))
+        w = replace(wl.TINY, name=f"fuzz{case}", T=T, H=H, I=K * TP, E=E, k=k, n_shared=n_shared, TP=TP, EP=EP, L=L,
+                    tile_m=tile_m, tile_n=tile_n, routing="zipf" if rng.random() < 0.5 else "uniform",
+                    zipf_s=1.0, target_r_expert=0.0, routing_seed=100 + case, data_seed=200 + case)
+        kw = dict(drain_help=int(rng.integers(2)))
+        if rng.random() < 0.5:
+            kw["force_C"] = int(rng.choice([1, 2, 5, 33]))
+        _check_against_oracle(w, **kw)
+        n_done += 1
+    assert n_done >= 25

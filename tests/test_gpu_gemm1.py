@@ -159,3 +159,16 @@ def test_post_router_layer_against_the_oracle_chain(counts_on_device):
     assert not np.isnan(got).any()
     # the intermediate may differ from the oracle's by one bf16 step in a few places: same tolerance form
     assert np.max(np.abs(got - expect)) <= G.tolerance(expect)
+
+
+def test_random_small_shapes_against_the_oracle():
+    # seeded fuzz: ragged token counts, partial k-blocks and n-tiles, every m-tile size, empty experts
+    rng = np.random.default_rng(77)
+    for case in range(14):
+        tile_m = int(rng.choice([64, 128, 256]))
+        w = replace(wl.TINY, name=f"g1fuzz{case}", T=int(rng.choice([1, 9, 130, 257, 600])),
+                    H=int(rng.choice([64, 80, 144, 256, 528])), I=int(rng.choice([16, 48, 128, 144, 272])),
+                    E=int(rng.integers(1, 24)), k=1, n_shared=int(rng.choice([0, 1])), TP=1, EP=1, L=1,
+                    tile_m=tile_m, tile_n=256 if tile_m == 256 else 64, routing_seed=300 + case, data_seed=400 + case)
+        w = replace(w, k=int(rng.integers(1, min(w.E, 3) + 1)))
+        _check(w, counts_on_device=bool(rng.integers(2)))
