@@ -11,7 +11,10 @@
  *    nothing throws across this boundary;
  *  - pointers are tagged [host] or [device]; the library never allocates device memory:
  *    the caller owns every buffer and the stream (passed as void*, a cudaStream_t);
- *  - all launches are asynchronous on the given stream;
+ *  - all launches are asynchronous on the given stream; the handle's device must be the calling
+ *    thread's current CUDA device (checked by every launching call: MOE_ERR_UNSUPPORTED otherwise);
+ *  - a handle is not thread-safe: one host thread uses it at a time (it keeps the text of the last
+ *    error and the launch epoch of every flags workspace it has launched on);
  *  - device-side problems (a bounded wait that ran out, an index out of range) are reported
  *    through a 4-word status buffer in device memory, read back with moe_get_status();
  *  - bf16 tensors are passed as void*; layouts are row-major with the last index contiguous.
@@ -196,7 +199,9 @@ int32_t moe_build_routing(moe_handle *h, const int32_t *topk_idx, const moe_shap
  *  - All calls on one GPU share the array and it keeps the previous call's contents; the
  *    builder overwrites every entry it later reads, so nothing needs clearing, but two calls
  *    whose kernels overlap on the GPU (different streams) race: order them.
- *  - Every GPU that loads the library holds the 512 KiB until the process exits. */
+ *  - Every GPU that loads the library holds the 512 KiB until the process exits.
+ *  - The handle's device must be the calling thread's current CUDA device, on every call (the array's
+ *    address belongs to that device): otherwise MOE_ERR_UNSUPPORTED and nothing is launched. */
 int32_t moe_build_routing_static(moe_handle *h, const int32_t *topk_idx, const moe_shape *shape,
                                  int32_t tile_m, const moe_routing *routing,
                                  int32_t *tile_counts_host, uint32_t *status_dev, void *stream);

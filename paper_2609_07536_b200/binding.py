@@ -133,7 +133,7 @@ def lib():
 def _check(rc, what, handle=None):
     if rc != MOE_OK:
         detail = ""
-        if handle is not None and rc in (MOE_ERR_CUDA, MOE_ERR_STATIC_LIMIT):
+        if handle is not None and rc in (MOE_ERR_CUDA, MOE_ERR_STATIC_LIMIT, MOE_ERR_UNSUPPORTED):
             detail = (lib().moe_last_cuda_error(handle) or b"").decode()
         raise MoeError(rc, what, detail)
 

@@ -15,6 +15,19 @@ int32_t cuda_fail(moe_handle *h, cudaError_t e, const char *what)
     return MOE_ERR_CUDA;
 }
 
+int32_t require_handle_device(moe_handle *h, const char *who)
+{
+    int cur = -1;
+    const cudaError_t e = cudaGetDevice(&cur);
+    if (e != cudaSuccess) return cuda_fail(h, e, "cudaGetDevice");
+    if (cur != h->device) {
+        snprintf(h->err, sizeof h->err, "%s: the current CUDA device is %d, the handle was created on device %d",
+                 who, cur, h->device);
+        return MOE_ERR_UNSUPPORTED;
+    }
+    return MOE_OK;
+}
+
 namespace {
 
 inline size_t align16(size_t x) { return (x + 15) & ~(size_t)15; }
@@ -230,6 +243,7 @@ int32_t moe_build_routing(moe_handle *h, const int32_t *topk_idx, const moe_shap
     if (!tile_m_ok(tile_m)) return MOE_ERR_UNSUPPORTED;
     if (s->T > 0 && !topk_idx) return MOE_ERR_NULL;
     if (r->max_mtiles < max_mtiles_of(s, tile_m)) return MOE_ERR_SHAPE;
+    if (const int32_t rc = require_handle_device(h, "moe_build_routing")) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = routing_launch(topk_idx, *s, tile_m, *r, status_dev, st);
     if (e != cudaSuccess) return cuda_fail(h, e, "routing launch");
@@ -279,6 +293,7 @@ int32_t moe_gemm2_combine(moe_handle *h, const void *x_routed, const void *W2, c
     // CTA off the GPU (Section II-C: the legal set keeps positive compute capacity)
     if (ceil_div(C, o_comm) + ceil_div(Pc, o_comp) * slot_sms > h->G) return MOE_ERR_PLAN_INFEASIBLE;
     if (pair && (((C + 1) & ~1) + 2 * Pc > 2 * h->max_pairs)) return MOE_ERR_PLAN_INFEASIBLE;
+    if (const int32_t rc = require_handle_device(h, "moe_gemm2_combine")) return rc;
 
     FusedParams p;
     memset(&p, 0, sizeof p);

@@ -335,6 +335,7 @@ extern "C" int32_t moe_gemm1_act(moe_handle *h, const void *hidden, const void *
     const bool counts_on_device = (n_mtiles == MOE_MTILES_ON_DEVICE);
     if (counts_on_device) n_mtiles = r->max_mtiles;
     if (n_mtiles < 0 || n_mtiles > r->max_mtiles) return MOE_ERR_SHAPE;
+    if (const int32_t rc = moe::require_handle_device(h, "moe_gemm1_act")) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int R = s->T * s->k_tot;
 

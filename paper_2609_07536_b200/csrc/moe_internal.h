@@ -77,6 +77,10 @@ namespace moe {
 inline int tile_n_slot(int tile_n) { return tile_n == 64 ? 0 : tile_n == 128 ? 1 : tile_n == 256 ? 2 : -1; }
 
 int32_t cuda_fail(moe_handle *h, cudaError_t e, const char *what);
+// MOE_OK when the calling thread's current CUDA device is the handle's; MOE_ERR_UNSUPPORTED (with a
+// message in the handle) otherwise.  Every launching entry point checks it: kernels run on the
+// current device, the buffers and the cached residency belong to the handle's.
+int32_t require_handle_device(moe_handle *h, const char *who);
 // fused kernel (gemm2_combine.cu)
 size_t fused_smem_bytes(int tile_n);
 cudaError_t fused_occupancy(int tile_n, int *blocks_per_sm);

@@ -4,12 +4,13 @@
 // ceil(M_e / T_M) tiles along the token dimension; Eq. 16: their sum S.
 // The routed rows are the flat assignments f = t * k_tot + j in a *stable* order by expert.
 //
-// Three small launches (the data is a few hundred KB):
-//   1. hist     every warp histograms its own contiguous chunk of assignments;
-//   2. scan     one CTA: counts, exclusive offsets, tiles per expert and their prefix, the
-//               m-tile table, and per-(warp, expert) exclusive bases;
-//   3. scatter  every warp walks its chunk in order, 32 assignments at a time;
-//               match_any gives each lane its rank among equal experts -> stable.
+// Four small launches (the data is a few hundred KB):
+//   1. hist          every warp histograms its own contiguous chunk of assignments;
+//   2. scan_columns  one CTA per expert: exclusive prefix of that expert's histogram column over
+//                    the warps (the per-(warp, expert) bases) and the expert's count;
+//   3. finalize      one CTA: exclusive offsets, tiles per expert and their prefix, the m-tile table;
+//   4. scatter       every warp walks its chunk in order, 32 assignments at a time;
+//                    match_any gives each lane its rank among equal experts -> stable.
 
 #include "moe_internal.h"
 
@@ -242,20 +243,22 @@ extern "C" int32_t moe_build_routing_static(moe_handle *h, const int32_t *topk_i
         return MOE_ERR_STATIC_LIMIT;
     }
     if (h->device < 0 || h->device >= kMaxStaticDevices) return MOE_ERR_UNSUPPORTED;
+    // Every call, not only the first: the kernels below run on the CURRENT device, and the array's
+    // address is only meaningful on the device it was resolved for.  A caller whose current device
+    // is not the handle's gets an error instead of kernels that dereference another GPU's address.
+    {
+        const int32_t rc = require_handle_device(h, "moe_build_routing_static");
+        if (rc != MOE_OK) return rc;
+    }
 
-    // set-up, once per device: resolve the array's device address with that device current
+    // set-up, once per device: resolve the array's device address (the handle's device is current)
     int32_t *scratch = g_static_scratch_addr[h->device];
     if (!scratch) {
-        int cur = -1;
-        cudaError_t e = cudaGetDevice(&cur);
-        if (e != cudaSuccess) return cuda_fail(h, e, "cudaGetDevice");
-        if (cur != h->device && (e = cudaSetDevice(h->device)) != cudaSuccess) return cuda_fail(h, e, "cudaSetDevice");
         void *p = nullptr;
-        e = cudaGetSymbolAddress(&p, g_static_scratch);
-        if (cur != h->device) cudaSetDevice(cur);
+        const cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);
         if (e != cudaSuccess || !p) return cuda_fail(h, e, "cudaGetSymbolAddress(static scratch)");
         scratch = static_cast<int32_t *>(p);
-        g_static_scratch_addr[h->device] = scratch;
+        g_static_scratch_addr[h->device] = scratch;   // every writer stores the same value
     }
 
     // The array keeps whatever the previous call left in it.  Nothing has to start at zero: the

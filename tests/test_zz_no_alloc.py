@@ -2,8 +2,10 @@
 (serving loops with a frozen memory pool, frameworks that own the allocator, latency-critical
 sections).  Its scratch is a fixed array inside the library, so this test checks, through the
 C ABI, that it produces exactly what moe_build_routing produces with a caller-allocated
-workspace -- twice in a row on different inputs, because the shared array keeps the previous
-call's contents -- and that a problem too large for the array is refused with a clear error.
+workspace and what the CPU routing reference computes -- twice in a row on different inputs,
+because the shared array keeps the previous call's contents --, that the amount of free device
+memory does not move across the calls, and that a problem too large for the array is refused
+with a clear error.
 
 Collected last on purpose (file name), and independent of the other tests: it builds its own
 handle and workspaces, so it passes alone in a fresh process as well as after the others.
@@ -15,6 +17,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import routing_ref as rr
 from paper_2609_07536_b200 import binding as B
 from paper_2609_07536_b200 import workloads as wl
 
@@ -60,14 +63,45 @@ def test_static_scratch_variant_matches_the_workspace_variant_twice_in_a_row():
             ref, ref_counts, S_ref = _run(h, B.moe_build_routing, w, idx)
             got, got_counts, S = _run(h, B.moe_build_routing_static, w, idx, null_scratch=True)
             assert S == S_ref and torch.equal(ref_counts, got_counts)
+            want = rr.build_routing(idx, w.E_tot, w.tile_m)          # the CPU reference, directly
+            assert S == want["S"]
             for k in KEYS:                           # integer work: bit-exact
                 assert np.array_equal(ref[k], got[k]), (w.name, k)
+                n = len(want[k])
+                assert np.array_equal(got[k][:n], np.asarray(want[k], dtype=np.int32)), (w.name, k, "vs reference")
         # and the very same input twice
         idx, _, _ = wl.make_routing(wl.DSV2L)
         a, _, _ = _run(h, B.moe_build_routing_static, wl.DSV2L, idx, null_scratch=True)
         b, _, _ = _run(h, B.moe_build_routing_static, wl.DSV2L, idx, null_scratch=True)
         for k in KEYS:
             assert np.array_equal(a[k], b[k]), k
+    finally:
+        B.moe_destroy(h)
+
+
+def test_later_calls_leave_the_amount_of_free_device_memory_alone():
+    """The point of the entry point: nothing is allocated.  The first call may make the driver load
+    the module that holds the array; from the second call on, free device memory as the driver
+    reports it must not move (the test's own buffers are all allocated beforehand)."""
+    h = B.moe_create(0)
+    try:
+        w = replace(wl.GRANITE, T=2048, routing_seed=9)
+        idx, _, _ = wl.make_routing(w)
+        shape = B.make_shape(w.T, w.H, w.I, w.E_tot, w.k_tot, w.TP, w.EP, w.L)
+        ws = B.alloc_workspace(shape, w.tile_m, w.tile_n)
+        ws.routing.scratch = None
+        idx_d = torch.from_numpy(idx).cuda()
+        B.moe_build_routing_static(h, idx_d, shape, w.tile_m, ws.routing, ws.tile_counts, ws.status)
+        torch.cuda.synchronize()
+        free_before, _ = torch.cuda.mem_get_info()
+        reserved_before = torch.cuda.memory_reserved()
+        for _ in range(3):
+            B.moe_build_routing_static(h, idx_d, shape, w.tile_m, ws.routing, ws.tile_counts, ws.status)
+        torch.cuda.synchronize()
+        free_after, _ = torch.cuda.mem_get_info()
+        assert torch.cuda.memory_reserved() == reserved_before      # nothing went through torch's allocator
+        assert free_after == free_before, (free_before, free_after)  # nor through cudaMalloc
+        assert B.moe_get_status(h, ws.status).code == 0
     finally:
         B.moe_destroy(h)
 
