@@ -315,3 +315,235 @@ def simulate_drain_help(C: int, Wc: int, Wm: int, L: int, P: int, helpers: int, 
     T = max(worker) if pool > 0 else A
     return dict(publish=publish, T=T, pool=pool, gap_free=gap_free, open_at_A=pool > Wm)
 
+
+
+# ----------------------------------------------------------------------------- co-resident family
+# Re-derivation for a kernel family in which communication work shares SMs with compute (Section III-B
+# lets o_comm exceed 1; Section III-E asks a new kernel family to re-derive o_comp, o_comm, tile work, the
+# dependency recurrence, the legal range and the service rate).  Not in the paper: this library's own
+# extension, pinned by its reductions to the recurrences above, closed forms, hand-worked values and an
+# event simulation (tests/test_oracle_solver.py).
+#
+#   * the unit of communication capacity is a WARP.  A dedicated communication CTA is `warps_cta` warps;
+#     a compute CTA carries w co-resident communication warps (the second decision variable) and turns
+#     into `warps_cta` communication warps once its GEMM tiles are done (drain help);
+#   * a communication tile is `warps_cta` quanta, one per warp of a dedicated CTA, so that a dedicated CTA
+#     still serves a tile in rho compute waves (Eq. 10 with quanta and warps in place of tiles and CTAs);
+#   * bandwidth-coupled service rate: N warps streaming together are limited by HBM once N exceeds `n_sat`
+#     (the warp count whose aggregate demand equals the measured copy bandwidth); the time of one quantum is
+#     rho(N) = rho * max(N, n_sat) / n_sat (rounded up in fixed point);
+#   * a co-resident warp shares its SM's issue slots and memory path with a running GEMM: it serves
+#     `gamma` times slower than a dedicated warp (N_eff counts it as 1/gamma warps), and every co-resident
+#     warp stretches the compute wave by `beta`; with more than one split they also force the split-major
+#     tile order (x is read once per split), which stretches the compute wave by `order`.
+#   All four constants are fixed point (2^-20) except n_sat and warps_cta (integers).
+
+def coupled_rho(rho_q: int, n_workers: int, n_sat: int) -> int:
+    """rho(N) = rho * max(N, n_sat) / n_sat, rounded up to the next multiple of 2^-20."""
+    return ceil_div(rho_q * max(n_workers, n_sat), n_sat)
+
+
+def coupled_service(rho_q: int, quanta: int, n_workers: int, n_sat: int) -> int:
+    """Time to serve `quanta` with n_workers warps, in waves of n_workers: a wave in which n warps stream
+    together takes rho(n), so the full waves take rho(n_workers) each and a last partial wave of r quanta
+    takes rho(r).  Below saturation this is Eq. 8 and Eq. 10, rho * ceil(quanta / n_workers); far above it
+    it tends to rho * quanta / n_sat: the bytes at the bandwidth, however many warps share them."""
+    full, rest = divmod(quanta, n_workers)
+    return full * coupled_rho(rho_q, n_workers, n_sat) + (coupled_rho(rho_q, rest, n_sat) if rest else 0)
+
+
+def makespan_co_resident(C: int, w: int, Wc: int, Wm: int, L: int, G: int, o_comp: int, o_comm: int, rho_q: int,
+                         slot_sms: int, warps_cta: int, n_sat: int, beta_q: int, gamma_q: int, order_q: int):
+    """T(C, w) for the co-resident family with drain help, fixed point.  Returns
+    (T_q, Delta_comp, R, P) or None when P(C) <= 0."""
+    R = reservation(C, o_comm)
+    P = compute_capacity(C, G, o_comp, o_comm, slot_sms)
+    if P <= 0:
+        return None
+    n_sm = P * slot_sms // o_comp                              # SMs that compute
+    tau_q = RHO_ONE + w * beta_q + (order_q if (w > 0 and L > 1) else 0)     # one compute wave
+    Wq = Wm * warps_cta                                        # quanta per split
+    n_early = C * warps_cta + w * n_sm                         # warps that serve while the GEMM runs
+    n_eff = C * warps_cta + (w * n_sm * RHO_ONE) // gamma_q    # ... in dedicated-warp equivalents
+    A_last = ceil_div(L * Wc, P) * tau_q
+    if n_eff <= 0:
+        backlog = (L - 1) * Wq                                 # nobody serves before the GEMM is over
+    else:
+        q_wave = coupled_rho(rho_q, n_early, n_sat)
+        q = q_wave * ceil_div(Wq, n_eff)
+        F = 0
+        for s in range(L - 1):                                 # Eq. 11 on splits 0..L-2
+            F = max(ceil_div((s + 1) * Wc, P) * tau_q, F) + q
+        backlog = 0
+        if F > A_last and q_wave > 0:
+            backlog = min(ceil_div(F - A_last, q_wave) * n_eff, (L - 1) * Wq)
+    n_tail = (C + n_sm) * warps_cta + w * n_sm                 # every warp serves once the GEMM is over
+    T_q = A_last + coupled_service(rho_q, backlog + Wq, n_tail, n_sat)
+    return T_q, ceil_div(Wc, P) * P - Wc, R, P
+
+
+def select_co_resident(Wc: int, Wm: int, L: int, G: int, o_comp: int, o_comm: int, C_max: int, rho_q: int,
+                       slot_sms: int, w_max: int, C_co_max: int, warps_cta: int, n_sat: int, beta_q: int,
+                       gamma_q: int, order_q: int, force_comm_ctas: int = 0, selector_off: bool = False,
+                       default_C: int = 3, force_co_warps: int = -1) -> dict:
+    """Algorithm 1 over the product set: C in 1..C_max with w = 0, and C in 1..min(C_max, C_co_max) with
+    w in 1..w_max (a one-time characterisation bounds the dedicated CTAs worth trying beside co-resident
+    warps, as the paper's C <= 16 does for its family).  Lexicographic minimum of (T, Delta_comp, w, C).
+    Overrides as in select(): a forced C / a forced w restrict the set to that value."""
+    if force_comm_ctas > 0 or selector_off:
+        Cs0 = Cs1 = [force_comm_ctas if force_comm_ctas > 0 else default_C]
+        if Cs0[0] < 1:
+            raise ValueError("C must be at least 1")
+    else:
+        Cs0 = list(range(1, C_max + 1))
+        Cs1 = list(range(1, min(C_max, C_co_max) + 1))
+    ws = list(range(0, w_max + 1)) if force_co_warps < 0 else [min(force_co_warps, w_max)]
+    best = None
+    for w in ws:
+        for C in (Cs0 if w == 0 else Cs1):
+            m = makespan_co_resident(C, w, Wc, Wm, L, G, o_comp, o_comm, rho_q, slot_sms, warps_cta, n_sat,
+                                     beta_q, gamma_q, order_q)
+            if m is None:
+                continue
+            key = (m[0], m[1], w, C)
+            if best is None or key < best[0]:
+                best = (key, dict(comm_ctas=C, co_warps=w, R=m[2], P=m[3], T_q=m[0], delta=m[1], W_comp=Wc, W_comm=Wm))
+    if best is None:
+        raise ValueError("no legal (C, w)")
+    return best[1]
+
+
+def simulate_co_resident(C: int, w: int, Wc: int, Wm: int, L: int, P: int, n_sm: int, rho: Fraction,
+                         warps_cta: int, n_sat: int, beta: Fraction, gamma: Fraction, order: Fraction) -> dict:
+    """Event-by-event simulation of the schedule makespan_co_resident stands for (no closed form):
+      * P compute slots take tiles round-robin, a tile takes tau = 1 + w*beta (+ order when w > 0 and L > 1);
+      * while the GEMM runs, split s (once published, and after split s-1) is served in waves of at most
+        n_eff = C*warps_cta + floor(w*n_sm/gamma) quanta, a wave takes rho * max(N_early, n_sat) / n_sat;
+      * at A = the publication of the last split every wave that has not completed returns its quanta to
+        the pool, which with the last split's quanta is served by all N_tail warps, wave by wave; a wave in
+        which n warps stream together takes rho * max(n, n_sat) / n_sat.
+    As with simulate_drain_help the closed form can only over-estimate (it counts an open wave in full)."""
+    rho, beta, gamma, order = Fraction(rho), Fraction(beta), Fraction(gamma), Fraction(order)
+    tau = 1 + w * beta + (order if (w > 0 and L > 1) else 0)
+    clock = [Fraction(0)] * P
+    tile_end = []
+    for i in range(L * Wc):
+        b = i % P
+        clock[b] += tau
+        tile_end.append(clock[b])
+    publish = [max(tile_end[s * Wc:(s + 1) * Wc]) if Wc > 0 else Fraction(0) for s in range(L)]
+    A = publish[L - 1]
+    Wq = Wm * warps_cta
+    n_early = C * warps_cta + w * n_sm
+    n_eff = C * warps_cta + int(Fraction(w * n_sm) / gamma)
+    pool = Wq
+    open_at_A = False
+    if n_eff <= 0:
+        pool += (L - 1) * Wq
+    else:
+        wave = rho * max(n_early, n_sat) / n_sat
+        prev = Fraction(0)
+        for s in range(L - 1):
+            t = max(publish[s], prev)
+            left = Wq
+            while left > 0:
+                n = min(n_eff, left)
+                if t + wave > A:
+                    pool += n
+                    open_at_A = True
+                t += wave
+                left -= n
+            prev = t
+    n_tail = (C + n_sm) * warps_cta + w * n_sm
+    T = A
+    left = pool
+    while left > 0:                       # wave by wave: n warps streaming together take rho * max(n, n_sat) / n_sat
+        n = min(n_tail, left)
+        T += rho * max(n, n_sat) / n_sat
+        left -= n
+    return dict(publish=publish, T=T, pool=pool, open_at_A=open_at_A)
+
+
+# ----------------------------------------------------------------------------- tile-level readiness
+# Section III-C derives A_s from the position of a split's LAST tile in the global tile sequence (Eq. 9):
+# readiness is one number per split.  A kernel that publishes every tile lets a communication tile start
+# as soon as the compute tiles under ITS tokens are done.  The same construction as Eq. 9, applied to each
+# communication tile instead of each split:
+#   * inside a split the compute tiles run expert by expert, m-tile by m-tile (index (mu*g + p)*NT + n);
+#   * the rows of an expert are in token order (stable sort), so the tokens of the communication token-tile
+#     that ends at token t_hi sit in the last non-empty expert's rows up to about M_e * t_hi / T (its load
+#     taken as even over the tokens: exact for an always-active shared expert), i.e. in its m-tiles up to
+#     i = ceil(n_last * t_hi / T) - 1 of its n_last tiles; every earlier expert's tiles come before those;
+#   * the communication tile (token-tile j, column tile c) is therefore complete when compute tile
+#       idx(j, c) = ((S - n_last + i_j) * g + (g - 1)) * NT + n_hi(c)
+#     of its split has finished, at the end of wave floor((s*W_comp + idx) / P), one more than that in
+#     compute-wave units (Eq. 9 is the special case idx = W_comp - 1).
+# Not in the paper as an equation: this library's reading of "split-level dependency" for per-tile flags.
+
+def comm_tile_ready_index(tiles, g: int, M: int, D: int, N: int, L: int, T_N: int, T_Mc: int, T_Nc: int) -> list:
+    """idx(j, c) for every communication tile of a split, in the static map's order ct = j * n_col + c
+    (token-tiles rank-major: rank d owns a contiguous block of ceil(M/D) tokens)."""
+    tiles = [int(t) for t in tiles]
+    S = sum(tiles)
+    split_w = ceil_div(N, L)
+    NT = ceil_div(split_w, T_N)
+    n_col = ceil_div(split_w, T_Nc)
+    nz = [t for t in tiles if t > 0]
+    n_last = nz[-1] if nz else 0
+    blk = ceil_div(M, D)
+    out = []
+    for d in range(D):
+        own = owned_tokens(M, D, d)
+        for ti in range(ceil_div(own, T_Mc)):
+            t_hi = d * blk + min(own, (ti + 1) * T_Mc)
+            i_j = max(0, ceil_div(n_last * t_hi, M) - 1) if M > 0 else 0
+            mu = S - n_last + i_j
+            for c in range(n_col):
+                n_hi = ceil_div(min(split_w, (c + 1) * T_Nc), T_N) - 1
+                out.append((mu * g + (g - 1)) * NT + n_hi)
+    return out
+
+
+def makespan_tile_level(C: int, ready_idx, Wc: int, L: int, G: int, o_comp: int, o_comm: int, rho, slot_sms: int = 1):
+    """The static partition (Section III-A map: communication tile ct belongs to CTA ct mod C) with
+    tile-level readiness, wave by wave: wave v of split s (tiles vC .. vC+C-1) starts when all its tiles
+    are ready and the previous wave is served,
+        F_{s,v} = max(max_{ct < min(vC+C, W_comm)} a_{s,ct}, F_{s,v-1}) + rho,   T = F_{L-1, V-1},
+    a_{s,ct} = floor((s W_comp + idx(ct)) / P) + 1 (the maximum may run over all earlier tiles of the split
+    as well: their waves have been served by then).  rho exact (int scaled by 2^20, or Fraction).
+    Returns (T, Delta_comp, R, P) or None when P(C) <= 0."""
+    R = reservation(C, o_comm)
+    P = compute_capacity(C, G, o_comp, o_comm, slot_sms)
+    if P <= 0:
+        return None
+    Wm = len(ready_idx)
+    one = RHO_ONE if isinstance(rho, int) else 1
+    F = 0
+    for s in range(L):
+        top = -1                                   # largest idx among the tiles of this split seen so far
+        for v in range(ceil_div(Wm, C)):
+            top = max([top] + list(ready_idx[v * C:min(v * C + C, Wm)]))
+            a = ((s * Wc + top) // P + 1) * one
+            F = max(a, F) + rho
+    return F, ceil_div(Wc, P) * P - Wc, R, P
+
+
+def simulate_tile_level(C: int, ready_idx, Wc: int, L: int, P: int, rho: Fraction) -> dict:
+    """Event simulation of the static partition with per-tile flags, CTA by CTA (no waves): compute CTA b
+    takes global tiles b, b+P, ... (unit time each); communication CTA k walks its tiles k, k+C, ... of
+    split 0, then of split 1, ...; a tile starts when the compute tile idx(ct) of its split has finished and
+    the CTA is free, and takes rho."""
+    rho = Fraction(rho)
+    clock = [Fraction(0)] * P
+    tile_end = []
+    for i in range(L * Wc):
+        b = i % P
+        clock[b] += 1
+        tile_end.append(clock[b])
+    Wm = len(ready_idx)
+    worker = [Fraction(0)] * C
+    for s in range(L):
+        for ct in range(Wm):
+            k = ct % C
+            worker[k] = max(worker[k], tile_end[s * Wc + ready_idx[ct]]) + rho
+    return dict(T=max(worker) if Wm > 0 and L > 0 else Fraction(0))

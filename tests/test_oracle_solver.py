@@ -341,3 +341,190 @@ def test_drain_help_closed_forms():
             extra = (mL[0] - A_last) // rho_q * workers - Wm
             assert 0 <= extra + workers and mL[0] >= A_last + rho_q * sr.ceil_div(Wm, workers)
             assert mL[0] <= A_last + rho_q * sr.ceil_div(L * Wm, workers)
+
+
+# ----------------------------------------------------------------------------- co-resident family, tile-level readiness
+
+def _parse_family_golden(path):
+    cos, tiles = [], []
+    for line in open(path):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        kind, name, rest = line.split(None, 2)
+        parts = [p.split() for p in rest.split("|")]
+        if kind == "co":
+            a, t = parts
+            cos.append((name, [int(v) for v in a[:9]], Fraction(a[9]), int(a[10]), int(a[11]),
+                        Fraction(a[12]), Fraction(a[13]), Fraction(a[14]), Fraction(t[0])))
+        elif kind == "tile":
+            a, idx, gpu, pts = parts
+            tiles.append((name, [int(v) for v in a[0].split(",")], [int(v) for v in a[1:]],
+                          [int(v) for v in idx[0].split(",")], [int(v) for v in gpu[:4]], Fraction(gpu[4]),
+                          {int(k): Fraction(v) for k, v in (p.split("=") for p in pts)}))
+    return cos, tiles
+
+
+def _q(x):
+    v = Fraction(x) * sr.RHO_ONE
+    assert v.denominator == 1
+    return int(v)
+
+
+def test_co_resident_hand_worked_values(golden_dir):
+    cos, _ = _parse_family_golden(os.path.join(golden_dir, "rho_local_worked.txt"))
+    assert len(cos) >= 3
+    for name, (G, o_comp, o_comm, slot, C, w, Wc, Wm, L), rho, warps_cta, n_sat, beta, gamma, order, want in cos:
+        m = sr.makespan_co_resident(C, w, Wc, Wm, L, G, o_comp, o_comm, _q(rho), slot, warps_cta, n_sat,
+                                    _q(beta), _q(gamma), _q(order))
+        assert Fraction(m[0], sr.RHO_ONE) == want, (name, Fraction(m[0], sr.RHO_ONE))
+        P = sr.compute_capacity(C, G, o_comp, o_comm, slot)
+        sim = sr.simulate_co_resident(C, w, Wc, Wm, L, P, P * slot // o_comp, rho, warps_cta, n_sat, beta, gamma, order)
+        assert sim["T"] <= want
+
+
+def test_coupled_service_rate_properties():
+    rng = random.Random(31)
+    for _ in range(3000):
+        rho_q = rng.randint(1, 40 * sr.RHO_ONE)
+        n_sat = rng.randint(1, 2000)
+        N = rng.randint(1, 4000)
+        X = rng.randint(0, 50000)
+        t = sr.coupled_service(rho_q, X, N, n_sat)
+        # below saturation: Eq. 8 and Eq. 10 unchanged
+        if N <= n_sat:
+            assert t == rho_q * sr.ceil_div(X, N)
+        # never faster than the bytes at the bandwidth, never faster than one pass per wave ...
+        assert t * n_sat >= rho_q * X and t >= rho_q * sr.ceil_div(X, N)
+        # ... and within one (coupled) wave plus rounding of the larger of the two
+        assert t <= max(rho_q * sr.ceil_div(X, N), sr.ceil_div(rho_q * X, n_sat)) + sr.coupled_rho(rho_q, min(N, max(X, 1)), n_sat) + X // N + 1
+        # more work never takes less time
+        assert sr.coupled_service(rho_q, X + rng.randint(0, 500), N, n_sat) >= t
+    # saturated and whole waves: exactly the bytes at the bandwidth
+    assert sr.coupled_service(3 * sr.RHO_ONE, 4000, 2000, 1000) == 3 * sr.RHO_ONE * 4
+    assert sr.coupled_rho(5 * sr.RHO_ONE, 10, 20) == 5 * sr.RHO_ONE and sr.coupled_rho(5 * sr.RHO_ONE, 30, 20) == 15 * sr.RHO_ONE // 2
+
+
+def test_co_resident_model_reductions_and_simulation():
+    rng = random.Random(32)
+    n_exact = 0
+    for _ in range(1500):
+        G = rng.choice([4, 6, 10, 16, 148])
+        o_comp, slot = rng.choice([1, 2]), rng.choice([1, 2])
+        L = rng.choice([1, 2, 3, 4])
+        Wc, Wm = rng.randint(1, 400), rng.randint(1, 24)
+        rho = Fraction(rng.randint(1, 48), rng.choice([1, 2, 4]))
+        warps_cta = rng.choice([1, 4, 12])
+        C = rng.randint(1, G - 1)
+        P = sr.compute_capacity(C, G, o_comp, 1, slot)
+        # (a) no co-resident warp and no saturation: the drain-help recurrence, bit for bit
+        a = sr.makespan_co_resident(C, 0, Wc, Wm, L, G, o_comp, 1, _q(rho), slot, warps_cta, 10 ** 9, _q(Fraction(1, 16)),
+                                    _q(2), _q(Fraction(1, 32)))
+        b = sr.makespan_drain_help(C, Wc, Wm, L, G, o_comp, 1, _q(rho), slot)
+        assert a == b
+        if P <= 0:
+            continue
+        n_sm = P * slot // o_comp
+        w = rng.randint(0, 3)
+        n_sat = rng.choice([3, 17, 200, 10 ** 6])
+        beta, gamma, order = Fraction(rng.randint(0, 8), 64), Fraction(rng.randint(4, 16), 4), Fraction(rng.randint(0, 4), 32)
+        m = sr.makespan_co_resident(C, w, Wc, Wm, L, G, o_comp, 1, _q(rho), slot, warps_cta, n_sat, _q(beta), _q(gamma), _q(order))
+        tau = 1 + w * beta + (order if (w > 0 and L > 1) else 0)
+        n_tail = (C + n_sm) * warps_cta + w * n_sm
+        # (b) L = 1: one compute phase stretched by the co-resident warps, then every warp serves the only split
+        if L == 1:
+            assert m[0] == sr.ceil_div(Wc, P) * _q(tau) + sr.coupled_service(_q(rho), Wm * warps_cta, n_tail, n_sat)
+        # (c) the event simulation of the same schedule: the closed form never under-estimates it (up to the
+        # rounding of rho(N) to 2^-20), and equals it when no early wave is open at the end of the GEMM
+        sim = sr.simulate_co_resident(C, w, Wc, Wm, L, P, n_sm, rho, warps_cta, n_sat, beta, gamma, order)
+        T_model = Fraction(m[0], sr.RHO_ONE)
+        assert sim["T"] <= T_model + Fraction(L * Wm * warps_cta + 8, sr.RHO_ONE)
+        if not sim["open_at_A"]:
+            assert abs(sim["T"] - T_model) <= Fraction(L * Wm * warps_cta + 8, sr.RHO_ONE)
+            n_exact += 1
+        # (d) more co-resident warps never lengthen the tail's service and never shorten the compute phase
+        m2 = sr.makespan_co_resident(C, w + 1, Wc, Wm, L, G, o_comp, 1, _q(rho), slot, warps_cta, n_sat, _q(beta), _q(gamma), _q(order))
+        assert sr.ceil_div(L * Wc, P) * _q(tau) <= m[0] and m2[1:] == m[1:]
+    assert n_exact > 300
+
+
+def test_select_co_resident_is_the_lexicographic_minimum_and_honours_overrides():
+    rng = random.Random(33)
+    for _ in range(120):
+        G, slot = rng.choice([16, 108, 148]), rng.choice([1, 2])
+        Wc, Wm, L = rng.randint(1, 9000), rng.randint(1, 256), rng.choice([1, 2, 4])
+        rho_q = rng.randint(sr.RHO_ONE // 4, 30 * sr.RHO_ONE)
+        kw = dict(warps_cta=12, n_sat=rng.choice([200, 1030, 10 ** 6]), beta_q=rng.randint(0, sr.RHO_ONE // 16),
+                  gamma_q=rng.randint(sr.RHO_ONE, 4 * sr.RHO_ONE), order_q=rng.randint(0, sr.RHO_ONE // 16))
+        C_max, w_max, C_co = rng.randint(1, G), rng.randint(0, 3), rng.randint(1, 16)
+        try:
+            sel = sr.select_co_resident(Wc, Wm, L, G, 1, 1, C_max, rho_q, slot, w_max, C_co, **kw)
+        except ValueError:
+            assert sr.compute_capacity(1, G, 1, 1, slot) <= 0
+            continue
+        keys = []
+        for w in range(w_max + 1):
+            for C in range(1, (C_max if w == 0 else min(C_max, C_co)) + 1):
+                m = sr.makespan_co_resident(C, w, Wc, Wm, L, G, 1, 1, rho_q, slot, kw["warps_cta"], kw["n_sat"],
+                                            kw["beta_q"], kw["gamma_q"], kw["order_q"])
+                if m is not None:
+                    keys.append((m[0], m[1], w, C))
+        assert (sel["T_q"], sel["delta"], sel["co_warps"], sel["comm_ctas"]) == min(keys)
+        if sr.compute_capacity(2, G, 1, 1, slot) > 0:
+            f = sr.select_co_resident(Wc, Wm, L, G, 1, 1, C_max, rho_q, slot, w_max, C_co, force_comm_ctas=2,
+                                      force_co_warps=1, **kw)
+            assert f["comm_ctas"] == 2 and f["co_warps"] == min(1, w_max)
+
+
+def test_tile_level_readiness_hand_worked_values(golden_dir):
+    _, tiles = _parse_family_golden(os.path.join(golden_dir, "rho_local_worked.txt"))
+    assert len(tiles) >= 1
+    for name, counts, (g, M, D, N, L, T_N, T_Mc, T_Nc), idx, (G, o_comp, o_comm, slot), rho, pts in tiles:
+        got = sr.comm_tile_ready_index(counts, g, M, D, N, L, T_N, T_Mc, T_Nc)
+        assert got == idx, name
+        Wc = sr.w_comp(counts, g, N, L, T_N)
+        for C, want in pts.items():
+            m = sr.makespan_tile_level(C, got, Wc, L, G, o_comp, o_comm, rho, slot)
+            assert m[0] == want, (name, C)
+            assert sr.makespan_tile_level(C, got, Wc, L, G, o_comp, o_comm, _q(rho), slot)[0] == _q(want)
+
+
+def test_tile_level_readiness_properties():
+    rng = random.Random(34)
+    n_eq = 0
+    for _ in range(600):
+        E = rng.randint(1, 12)
+        counts = [rng.randint(0, 9) for _ in range(E)]
+        if sum(counts) == 0:
+            counts[rng.randrange(E)] = 1
+        g, D, L = rng.choice([1, 2]), rng.choice([1, 2, 4]), rng.choice([1, 2, 4])
+        T_N, T_Nc, T_Mc = rng.choice([64, 128, 256]), rng.choice([512, 1024]), 128
+        N = rng.choice([512, 1536, 2048])
+        M = rng.randint(1, 3000)
+        idx = sr.comm_tile_ready_index(counts, g, M, D, N, L, T_N, T_Mc, T_Nc)
+        Wc = sr.w_comp(counts, g, N, L, T_N)
+        Wm = sr.w_comm_gpu(M, D, N, L, T_Mc, T_Nc)
+        assert len(idx) == Wm and max(idx) == Wc - 1 and min(idx) >= 0     # the last tile waits for the whole split (Eq. 9)
+        n_col = sr.ceil_div(sr.ceil_div(N, L), T_Nc)
+        for c in range(n_col):                                             # later tokens are never ready earlier
+            col = idx[c::n_col]
+            assert all(a <= b for a, b in zip(col, col[1:]))
+        G = rng.choice([8, 20, 148])
+        rho = Fraction(rng.randint(1, 40), rng.choice([1, 2, 4]))
+        for C in rng.sample(range(1, G), min(4, G - 1)):
+            m = sr.makespan_tile_level(C, idx, Wc, L, G, 1, 1, rho)
+            ref = sr.makespan(C, Wc, Wm, L, G, 1, 1, rho)
+            assert m[0] <= ref[0] and m[1:] == (ref[1], ref[2], ref[3])    # never later than split-level readiness
+            # an event simulation CTA by CTA is never slower than the wave-by-wave recurrence ...
+            sim = sr.simulate_tile_level(C, idx, Wc, L, m[3], rho)
+            assert sim["T"] <= m[0]
+            # ... and equals it when every communication tile waits for the end of its split (Eq. 11 itself)
+            flat = [Wc - 1] * Wm
+            mf = sr.makespan_tile_level(C, flat, Wc, L, G, 1, 1, rho)
+            assert mf[0] == ref[0]
+            assert sr.simulate_tile_level(C, flat, Wc, L, m[3], rho)["T"] == ref[0]
+            n_eq += 1
+    assert n_eq > 1000
+    # an always-active last expert with one m-tile per communication token-tile: readiness steps through the tiles
+    idx = sr.comm_tile_ready_index([3, 4], 1, 512, 1, 256, 1, 256, 128, 1024)
+    assert idx == [3, 4, 5, 6]
