@@ -296,6 +296,92 @@ def calibrate(h, device, C_ref=32, tile=(128, 256)):
         "rows_ref": rho.rows_ref, "comm_cols_ref": rho.comm_cols_ref, "D_ref": rho.D_ref}}))
 
 
+# ----------------------------------------------------------------------------- per-CTA timeline
+# Reader of the records the instrumented build (libmoe_b200_timeline.so) writes; slot numbers as in
+# csrc/gemm2_combine.cu.
+
+TL = dict(begin=0, role=1, first_acc=2, mma_end=3, tiles=4, wait_operand=5, issue=6, wait_tmem=7, mma_cycles=8,
+          compute_end=9, cta_end=10, epi_wait=11, epi_work=12, producer_wait=13, comm_units=14, comm_wait_ns=15, co=16)
+
+
+def run_timeline(h, dw, step, occ, lim, args):
+    """One recorded fused launch (after warm-up launches): where the time of the compute CTAs goes, when the
+    splits complete and what the communication warps serve while the GEMM is still running."""
+    import numpy as np
+    import torch
+    B, w = dw.B, dw.w
+    slots = B.MOE_TIMELINE_SLOTS
+    n_words = (lim.G + 2) * slots + B.MOE_MAX_L
+    buf = torch.zeros(n_words, dtype=torch.int64, device=dw.x.device)
+    kw = dict(C_override=0, P_override=lim.G // occ.comp_slot_sms) if args.no_comm_ctas else {}
+    for _ in range(max(1, args.warmup)):
+        step(args.force_C, **kw)
+    torch.cuda.synchronize()
+    B.moe_set_timeline(h, buf, n_words * 8)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    plan, counts = step(args.force_C, ev_before=a, ev_after=b, **kw)
+    torch.cuda.synchronize()
+    B.moe_set_timeline(h, None, 0)
+    kernel_us = a.elapsed_time(b) * 1e3
+    pair = w.tile_m == 256
+    grid = (((plan.comm_ctas + 1) & ~1) + 2 * plan.P) if pair else plan.comm_ctas + plan.P
+    raw = buf.cpu().numpy().astype(np.uint64)
+    rec = raw[:grid * slots].reshape(grid, slots).astype(np.float64)
+    splits = raw[grid * slots:grid * slots + w.L].astype(np.float64)
+    t0 = rec[:, TL["begin"]][rec[:, TL["begin"]] > 0].min()
+    comp = rec[(rec[:, TL["role"]] == 1) & (rec[:, TL["tiles"]] > 0)]      # CTAs that issued MMAs (pair: the leaders)
+    allc = rec[rec[:, TL["role"]] == 1]
+
+    def rel(v):   # ns stamps -> us after the first CTA began
+        v = v[v > 0]
+        return {"min": float((v.min() - t0) / 1e3), "median": float((np.median(v) - t0) / 1e3),
+                "max": float((v.max() - t0) / 1e3)} if v.size else None
+
+    K = w.I // w.TP
+    num_kb = -(-K // 64)
+    kb = comp[:, TL["tiles"]] * num_kb
+    per_kb = lambda slot: float(np.median(comp[:, TL[slot]] / kb)) if comp.size else None
+    out = {
+        "timeline": w.name, "tile": f"{w.tile_m}x{w.tile_n}", "L": w.L, "C": plan.comm_ctas, "P": plan.P,
+        "co_warps": plan.co_warps, "kernel_us": kernel_us, "num_kb": num_kb,
+        "cta_begin_us": rel(rec[:, TL["begin"]]), "first_accumulator_us": rel(comp[:, TL["first_acc"]]),
+        "last_mma_us": rel(comp[:, TL["mma_end"]]), "compute_role_end_us": rel(allc[:, TL["compute_end"]]),
+        "cta_end_us": rel(rec[:, TL["cta_end"]]),
+        "split_complete_us": [float((t - t0) / 1e3) if t > 0 else None for t in splits],
+        "tiles_per_cta": {"min": float(comp[:, TL["tiles"]].min()), "max": float(comp[:, TL["tiles"]].max())} if comp.size else None,
+        "mma_thread_cycles_per_kblock": {"total": per_kb("mma_cycles"), "waiting_for_operands": per_kb("wait_operand"),
+                                         "issuing": per_kb("issue"), "waiting_for_accumulator_buffer": per_kb("wait_tmem")},
+        "epilogue_warp_cycles_per_tile": {
+            "waiting": float(np.median(allc[:, TL["epi_wait"]] / np.maximum(1, comp[:, TL["tiles"]].mean()))),
+            "working": float(np.median(allc[:, TL["epi_work"]] / np.maximum(1, comp[:, TL["tiles"]].mean())))} if allc.size else None,
+        "producer_wait_cycles_per_kblock": float(np.median(allc[:, TL["producer_wait"]]) / max(1.0, float(np.median(kb)))) if comp.size else None,
+    }
+    Q = w.k_tot * w.TP
+    slab = 1024
+    while slab > 8 and Q * slab * 2 > 8192:
+        slab //= 2
+    unit_bytes = Q * min(slab, -(-w.H // w.L)) * 2
+    if plan.co_warps > 0 and allc.size:
+        co = allc[:, TL["co"]:TL["co"] + 8 * plan.co_warps].reshape(-1, 8)
+        units = co[:, 2]
+        by_split = co[:, 4:8].sum(axis=0)
+        gemm_end = np.median(comp[:, TL["mma_end"]])
+        # units a warp served before the median compute CTA issued its last MMA, taking its service as even in time
+        span = np.maximum(1.0, co[:, 1] - co[:, 0])
+        early = np.clip((gemm_end - co[:, 0]) / span, 0.0, 1.0) * units
+        out["co_resident_warps"] = {
+            "warps": int(co.shape[0]), "units_total": float(units.sum()), "units_by_split": [float(v) for v in by_split[:w.L]],
+            "bytes_total": float(units.sum() * unit_bytes), "units_before_median_last_mma": float(early.sum()),
+            "bytes_before_median_last_mma": float(early.sum() * unit_bytes),
+            "first_unit_us": rel(co[:, 0]), "last_unit_us": rel(co[:, 1]),
+            "asleep_us_per_warp_median": float(np.median(co[:, 3]) / 1e3),
+            "gb_per_s_per_warp_while_serving": float(np.median(units * unit_bytes / span)),
+        }
+    out["units_all_splits"] = w.T * w.L * (-(-(-(-w.H // w.L)) // min(slab, -(-w.H // w.L))))
+    out["unit_bytes"] = unit_bytes
+    print(json.dumps(out))
+
+
 # ----------------------------------------------------------------------------- up-stream stage (next row)
 
 def time_gemm1(h, dw, torch, n_warm=3, n_samples=9, cpu_rows=0):
@@ -457,11 +543,23 @@ def main():
     ap.add_argument("--counts", default="host", choices=["host", "device"],
                     help="host: tile counts copied to the host, exact plan (default); device: no copy and no wait, "
                          "plan from the normalised-load estimate (Section III-E)")
+    ap.add_argument("--co-warps", type=int, default=-1,
+                    help="co-resident communication warps per compute CTA (-1: the selector decides)")
+    ap.add_argument("--no-comm-ctas", action="store_true",
+                    help="with --only fused: launch without any dedicated communication CTA (C = 0, every SM computes)")
     ap.add_argument("--drain-help", type=int, default=1, choices=[0, 1],
                     help="1 (default): compute CTAs help with the communication tail; 0: the paper's static partition")
+    ap.add_argument("--timeline", action="store_true",
+                    help="run the instrumented build (libmoe_b200_timeline.so, built on demand) and print where the "
+                         "time of one fused launch goes per CTA role; honours --force-C / --no-comm-ctas / --co-warps / --L / --tile")
     args = ap.parse_args()
     if args.impl == "reference":
         return reference_arm(args)
+    if args.timeline:
+        from paper_2609_07536_b200 import binding as B0
+        from paper_2609_07536_b200 import build as lib_build
+        lib_build.build(timeline=True)
+        B0.use_timeline_library()
 
     import numpy as np
     import torch
@@ -498,10 +596,15 @@ def main():
     if args.T:
         from dataclasses import replace
         w = replace(w, T=args.T, name=f"{w.name}_T{args.T}")
-    dw = DeviceWorkload(w, device, data=args.data if args.only else "seeded")
-    step, (occ, lim, rho) = make_stepper(h, dw, limits_override=dict(drain_help=args.drain_help))
+    dw = DeviceWorkload(w, device, data=args.data if (args.only or args.timeline) else "seeded")
+    step, (occ, lim, rho) = make_stepper(h, dw, limits_override=dict(drain_help=args.drain_help,
+                                                                      force_co_warps=args.co_warps))
     K, W = max(1, args.steps), max(3, args.warmup)
 
+    if args.timeline:
+        run_timeline(h, dw, step, occ, lim, args)
+        B.moe_destroy(h)
+        return
     if args.only == "gemm1":
         res = time_gemm1(h, dw, torch, n_warm=max(1, args.warmup), n_samples=K)
         print(json.dumps({"only": "gemm1", "workload": w.name, **res}))
@@ -515,12 +618,15 @@ def main():
             kw = dict(P_override=((lim.G - args.force_C) if args.force_C else lim.G) // occ.comp_slot_sms)
         elif args.only == "combine_only":
             kw = dict(C_override=args.force_C or lim.G)
+        elif args.no_comm_ctas:
+            kw = dict(C_override=0, P_override=lim.G // occ.comp_slot_sms)
         if args.only == "combine_only":   # Y must exist
             step(0, mode=B.MOE_MODE_GEMM_ONLY, P_override=lim.G // occ.comp_slot_sms)
         ts = time_fused(step, torch, (args.force_C if args.only == "fused" else (1 if args.only == "combine_only" else 0)),
                         args.warmup, K, mode=mode, **kw)
         med = statistics.median(ts)
-        print(json.dumps({"only": args.only, "workload": w.name, "force_C": args.force_C, "us": med,
+        print(json.dumps({"only": args.only, "workload": w.name, "force_C": 0 if args.no_comm_ctas else args.force_C,
+                          "co_warps": args.co_warps, "L": w.L, "tile": f"{w.tile_m}x{w.tile_n}", "us": med,
                           "min_us": min(ts), "tflops": dw.flops / med / 1e6, "combine_gbs": dw.combine_bytes / med / 1e3}))
         B.moe_destroy(h)
         return

@@ -96,6 +96,9 @@ typedef struct {
                                 of this library, not in the paper: with it the selector models the tail after
                                 the last compute wave as served by every SM);
                                 0: the paper's static partition and its recurrence exactly */
+    int32_t co_warps_max;    /* upper end of the legal set {0..co_warps_max} of co-resident communication warps
+                                per compute CTA (0: a kernel family without them) */
+    int32_t force_co_warps;  /* >= 0: use exactly this many (clamped to co_warps_max); < 0: the selector decides */
 } moe_sm_limits;
 
 /* Relative wave service rate (Eq. 13-15). */
@@ -121,7 +124,10 @@ typedef struct {
     int32_t mode;        /* MOE_MODE_* (plan_partition writes MOE_MODE_FUSED) */
     int32_t debug_withhold_tile; /* test hook: global tile whose readiness is never raised; -1 = none */
     int32_t drain_help;  /* copied from moe_sm_limits: compute CTAs help with the communication tail */
-    int32_t reserved;
+    int32_t co_warps;    /* co-resident communication warps per compute CTA (Section III-B with communication
+                            work sharing the SM of a compute CTA instead of reserving one): they serve split s
+                            while the CTA computes split s + 1.  Needs drain_help; the launch drops them when
+                            the shape leaves them no shared memory (see moe_gemm2_combine) */
 } moe_plan;
 
 /* Views into the routing workspace, all [device] int32. */
@@ -156,6 +162,20 @@ const char *moe_last_cuda_error(const moe_handle *h);
  * records MOE_DEV_TIMEOUT and leaves; the context stays usable.  The limit is counted from
  * the start of each CTA, so it bounds the whole launch as well. */
 int32_t moe_set_wait_limit_ns(moe_handle *h, uint64_t ns);
+
+/* Tracing aid (Section III-C characterises service rates by timing the two roles; this is the tool for
+ * it).  In a library built with -DMOE_TIMELINE=1 (python -m paper_2609_07536_b200.build --timeline, a
+ * separate libmoe_b200_timeline.so) every later moe_gemm2_combine launch on this handle records, per CTA,
+ * MOE_TIMELINE_SLOTS 64-bit words -- %globaltimer stamps (CTA begin, first accumulator, last MMA, end of
+ * the compute role, CTA end), cycle counters of the MMA-issuing thread (waiting for operands, issuing,
+ * waiting for an accumulator buffer), of one epilogue warp and of one producer, and what its communication
+ * warps served and when -- followed by one completion stamp per split, into timeline_dev [device, 8-byte
+ * aligned, at least (grid * MOE_TIMELINE_SLOTS + MOE_MAX_L) * 8 bytes, zero-filled by the caller; a buffer
+ * that is too small for a launch is left alone].  NULL switches recording off.  The normal library accepts
+ * only NULL (MOE_ERR_UNSUPPORTED otherwise): its kernels carry no instrumentation.  bench.py --timeline
+ * reads the records.  [host] */
+#define MOE_TIMELINE_SLOTS 32
+int32_t moe_set_timeline(moe_handle *h, void *timeline_dev, size_t bytes);
 
 /* Tile shape and residency of the GEMM2 kernel for (tile_m, tile_n), the communication tile,
  * the GPU limits and the stored service-rate constants (Section III-B, III-D, III-E).

@@ -32,7 +32,7 @@ EXPORTS = [
     "plan_partition", "plan_partition_estimate", "moe_time_plan_partition", "moe_gemm2_combine", "moe_get_status",
     "moe_clear_status",
     "moe_layer", "moe_calibrate_rho", "moe_host_arena_bytes", "moe_layer_host",
-    "moe_gemm1_workspace_bytes", "moe_gemm1_act", "moe_post_router_layer",
+    "moe_gemm1_workspace_bytes", "moe_gemm1_act", "moe_post_router_layer", "moe_set_timeline",
 ]
 
 
@@ -53,7 +53,7 @@ class moe_occupancy(C.Structure):
 
 class moe_sm_limits(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("G", "C_max", "force_comm_ctas", "selector_off", "default_C",
-                                                "drain_help")]
+                                                "drain_help", "co_warps_max", "force_co_warps")]
 
 
 class moe_rho(C.Structure):
@@ -64,7 +64,7 @@ class moe_rho(C.Structure):
 class moe_plan(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("comm_ctas", "R", "P", "W_comp", "W_comm", "delta")] + [
         ("pred_T_q", C.c_int64), ("rho_q", C.c_int64), ("mode", C.c_int32), ("debug_withhold_tile", C.c_int32),
-        ("drain_help", C.c_int32), ("reserved", C.c_int32)]
+        ("drain_help", C.c_int32), ("co_warps", C.c_int32)]
 
 
 class moe_routing(C.Structure):
@@ -77,18 +77,31 @@ class moe_status(C.Structure):
     _fields_ = [(n, C.c_uint32) for n in ("code", "detail", "where", "count")]
 
 
+TIMELINE_LIB_PATH = os.path.join(HERE, "libmoe_b200_timeline.so")
+MOE_TIMELINE_SLOTS = 32
+
 _lib = None
+_lib_path = LIB_PATH
+
+
+def use_timeline_library():
+    """Selects the instrumented build (libmoe_b200_timeline.so) for this process; must come before the
+    first call into the library."""
+    global _lib_path
+    if _lib is not None and _lib_path != TIMELINE_LIB_PATH:
+        raise RuntimeError("the library is already loaded")
+    _lib_path = TIMELINE_LIB_PATH
 
 
 def lib():
     """The loaded library.  Raises if it has not been built."""
     global _lib
     if _lib is None:
-        if not os.path.exists(LIB_PATH):
+        if not os.path.exists(_lib_path):
             raise ImportError(
-                f"{LIB_PATH} is missing: build it with `python -m paper_2609_07536_b200.build` "
-                "(this package has no fallback path)")
-        L = C.CDLL(LIB_PATH)
+                f"{_lib_path} is missing: build it with `python -m paper_2609_07536_b200.build"
+                f"{' --timeline' if _lib_path == TIMELINE_LIB_PATH else ''}` (this package has no fallback path)")
+        L = C.CDLL(_lib_path)
         vp, i32, u64 = C.c_void_p, C.c_int32, C.c_uint64
         P = C.POINTER
         L.moe_create.argtypes = [i32, P(vp)]
@@ -120,6 +133,7 @@ def lib():
         L.moe_gemm1_act.argtypes = [vp, vp, vp, P(moe_shape), i32, P(moe_routing), i32, vp, vp, vp, vp]
         L.moe_post_router_layer.argtypes = [vp, vp, vp, vp, vp, vp, P(moe_shape), i32, i32, P(moe_sm_limits),
                                             P(moe_routing), vp, vp, vp, P(vp), vp, vp, vp, P(moe_plan), vp]
+        L.moe_set_timeline.argtypes = [vp, vp, C.c_size_t]
         L.moe_host_arena_bytes.argtypes = [P(moe_shape), i32, i32, P(C.c_size_t)]
         L.moe_layer_host.argtypes = [vp, vp, vp, vp, vp, P(moe_shape), i32, i32, P(moe_sm_limits), vp,
                                      C.c_size_t, vp, vp, P(moe_plan), vp]
@@ -170,6 +184,11 @@ def moe_destroy(h):
 
 def moe_set_wait_limit_ns(h, ns: int):
     _check(lib().moe_set_wait_limit_ns(h, ns), "moe_set_wait_limit_ns")
+
+
+def moe_set_timeline(h, timeline_dev, nbytes: int):
+    """Timeline build only: later fused launches record per-CTA stamps into `timeline_dev` (None: off)."""
+    _check(lib().moe_set_timeline(h, _ptr(timeline_dev), nbytes), "moe_set_timeline", h)
 
 
 def moe_query_occupancy(h, tile_m: int, tile_n: int):

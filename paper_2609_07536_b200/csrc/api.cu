@@ -131,6 +131,19 @@ int32_t moe_set_wait_limit_ns(moe_handle *h, uint64_t ns)
     return MOE_OK;
 }
 
+int32_t moe_set_timeline(moe_handle *h, void *timeline_dev, size_t bytes)
+{
+    if (!h) return MOE_ERR_NULL;
+    if (timeline_dev && !fused_timeline_build()) {
+        snprintf(h->err, sizeof h->err, "moe_set_timeline: this library was built without -DMOE_TIMELINE=1");
+        return MOE_ERR_UNSUPPORTED;
+    }
+    if (timeline_dev && (reinterpret_cast<uintptr_t>(timeline_dev) & 7u)) return MOE_ERR_ALIGN;
+    h->timeline = static_cast<unsigned long long *>(timeline_dev);
+    h->timeline_bytes = timeline_dev ? bytes : 0;
+    return MOE_OK;
+}
+
 int32_t moe_query_occupancy(moe_handle *h, int32_t tile_m, int32_t tile_n, moe_occupancy *occ,
                             moe_sm_limits *limits, moe_rho *rho)
 {
@@ -155,6 +168,8 @@ int32_t moe_query_occupancy(moe_handle *h, int32_t tile_m, int32_t tile_n, moe_o
         limits->selector_off = 0;
         limits->default_C = 3;      // the fixed count of the upstream path (Section II-C)
         limits->drain_help = 1;
+        limits->co_warps_max = fused_co_warps_max();
+        limits->force_co_warps = -1;
     }
     if (rho) {
         // One-time service-rate characterisation of this kernel family on B200 (Eq. 13), one constant per
@@ -286,7 +301,11 @@ int32_t moe_gemm2_combine(moe_handle *h, const void *x_routed, const void *W2, c
     const bool pair = (occ->tile_m == 256);
     const int slot_sms = pair ? 2 : 1;
     if (occ->comp_slot_sms != slot_sms) return MOE_ERR_UNSUPPORTED;
-    if (mode != MOE_MODE_GEMM_ONLY && C < 1) return MOE_ERR_PLAN_INFEASIBLE;
+    // without a communication CTA somebody else has to serve the communication work: the compute CTAs, once
+    // their GEMM tiles are done (drain help)
+    if (mode != MOE_MODE_GEMM_ONLY && (C < 0 || (C < 1 && !(mode == MOE_MODE_FUSED && plan->drain_help))))
+        return MOE_ERR_PLAN_INFEASIBLE;
+    if (plan->co_warps < 0 || plan->co_warps > kCoWarpsMax) return MOE_ERR_PLAN_INFEASIBLE;
     if (mode != MOE_MODE_COMBINE_ONLY && Pc < 1) return MOE_ERR_PLAN_INFEASIBLE;
     if (mode == MOE_MODE_FUSED && (int64_t)plan->R * o_comm < C) return MOE_ERR_PLAN_INFEASIBLE;
     // every CTA must be resident at once: spinning communication CTAs may never keep a compute
@@ -311,7 +330,6 @@ int32_t moe_gemm2_combine(moe_handle *h, const void *x_routed, const void *W2, c
     p.S_dev = counts_on_device ? r->tiles + s->E_tot : nullptr;
     p.C = C; p.P = Pc; p.mode = mode; p.withhold = plan->debug_withhold_tile;
     p.drain_help = (mode == MOE_MODE_FUSED && plan->drain_help) ? 1 : 0;
-    p.tile_order = plan->drain_help ? 1 : 0;   // nothing waits for an early split then: x is read once
     p.tok_blk = (int32_t)ceil_div(s->T, s->EP);
     p.tok_tiles_per_rank = (int32_t)ceil_div(p.tok_blk, kCommTileM);
     p.comm_cols = (int32_t)ceil_div(p.split_w, kCommTileN);
@@ -344,6 +362,14 @@ int32_t moe_gemm2_combine(moe_handle *h, const void *x_routed, const void *W2, c
                     (reinterpret_cast<uintptr_t>(y_ws) & 31u) == 0) ? 1 : 0;
     p.status = status_dev;
     for (int d = 0; d < s->EP; ++d) p.out[d] = out[d];
+    // Co-resident communication warps need the dynamic hand-out (they pull from the queues), the aux region
+    // of shared memory (free only when the epilogue stores straight from registers) and units of at most 16
+    // rows; where one of these does not hold the launch runs without them (same result, bit for bit).
+    p.co_warps = plan->co_warps < fused_co_warps_max() ? plan->co_warps : fused_co_warps_max();
+    if (!p.drain_help || !p.wide_store || p.Q > 16) p.co_warps = 0;
+    // Tile sequence: split-major (the paper's) whenever something consumes a split while the next one is
+    // computed; m-tile-major across the splits (x is read from DRAM once) when nothing does
+    p.tile_order = (plan->drain_help && p.co_warps == 0) ? 1 : 0;
 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e;
@@ -393,7 +419,11 @@ int32_t moe_gemm2_combine(moe_handle *h, const void *x_routed, const void *W2, c
             return MOE_ERR_CUDA;
         }
     }
-    e = pair ? pair_launch(p, ((C + 1) & ~1) + 2 * Pc, st) : fused_launch(TN, p, C + Pc, st);
+    const int grid = pair ? ((C + 1) & ~1) + 2 * Pc : C + Pc;
+    p.timeline = nullptr;
+    if (h->timeline && h->timeline_bytes >= ((size_t)grid * kTimelineSlots + MOE_MAX_L) * sizeof(unsigned long long))
+        p.timeline = h->timeline;
+    e = pair ? pair_launch(p, grid, st) : fused_launch(TN, p, grid, st);
     if (e != cudaSuccess) return cuda_fail(h, e, "fused launch");
     return MOE_OK;
 }

@@ -26,6 +26,12 @@
 //   copy into its own double-buffered shared-memory stage (the readiness of the producing tiles is
 //   checked first: split counter, else per-tile flags with ld.acquire.gpu; bounded), sums the rows in
 //   fp32 in (j, p) order with the token's weights and stores bf16 into the owning rank's buffer.
+// Co-resident communication warps (Section III-B with o_comm > 1 in spirit: communication work that
+//   shares an SM with a compute CTA instead of reserving one): every compute CTA carries up to four
+//   extra warps (16-19) that run the same per-unit pipeline on stages of their own, take work from
+//   the front of the per-split queues and serve split s while the CTA's other warps compute split
+//   s + 1.  They wait for a whole split (no token of a split is complete before the last expert's
+//   tiles of that split are), not for single tiles.
 //
 // Every wait is bounded: after `wait_ns` the waiter records MOE_DEV_TIMEOUT and the CTA winds
 // down (pending bulk copies are drained, TMEM is released).
@@ -35,8 +41,35 @@
 #include "moe_internal.h"
 #include "sm100_device.cuh"
 
+// Timeline build (-DMOE_TIMELINE=1, a separate library): the kernels record per-CTA time stamps and cycle
+// counters into a caller-provided buffer (moe_set_timeline), kTimelineSlots 64-bit words per CTA followed by
+// one completion stamp per split.  In the normal build every TL(...) statement compiles to nothing.
+#ifndef MOE_TIMELINE
+#define MOE_TIMELINE 0
+#endif
+#if MOE_TIMELINE
+#define TL(...) do { __VA_ARGS__; } while (0)
+#define TL_DECL(...) __VA_ARGS__
+#else
+#define TL(...) do { } while (0)
+#define TL_DECL(...)
+#endif
+
 namespace moe {
 namespace {
+
+// slots of a CTA's timeline record (see bench.py --timeline for the reader)
+enum {
+    kTlBegin = 0, kTlRole = 1, kTlFirstAcc = 2, kTlMmaEnd = 3, kTlTiles = 4, kTlWaitOperand = 5, kTlIssue = 6,
+    kTlWaitTmem = 7, kTlMmaCycles = 8, kTlComputeEnd = 9, kTlCtaEnd = 10, kTlEpiWait = 11, kTlEpiWork = 12,
+    kTlProducerWait = 13, kTlCommUnits = 14, kTlCommWaitNs = 15, kTlCoWarp = 16   // 8 slots per co-resident warp
+};
+#if MOE_TIMELINE
+__device__ __forceinline__ void tl_put(const FusedParams &P, int slot, unsigned long long v)
+{
+    if (P.timeline) P.timeline[(size_t)blockIdx.x * kTimelineSlots + slot] = v;
+}
+#endif
 
 // --------------------------------------------------------------------------- shared memory
 
@@ -61,6 +94,7 @@ struct Control {
     uint32_t tmem_base;
     volatile uint32_t abort;
     unsigned long long comm_full[24];   // communication CTA: one barrier per warp and stage
+    unsigned long long co_full[8];      // co-resident communication warps: one barrier per warp and stage
 };
 
 // 32 KB after the control block, used by one role per CTA:
@@ -117,6 +151,12 @@ __device__ __forceinline__ bool wait_barrier_1t(uint32_t bar, uint32_t parity, C
         }
     }
     return true;
+}
+
+// Barrier of the 16 warps that compute (the co-resident communication warps never join it).
+__device__ __forceinline__ void sync_compute_warps()
+{
+    asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory");
 }
 
 struct Tile {
@@ -298,13 +338,12 @@ __device__ void compute_cta(const FusedParams &P, int W_comp, uint8_t *ring, Con
             mbar_init(smem_u32(&ctl->epi_done[i]), C::kEpiWarps);
             mbar_init(smem_u32(&ctl->pub_done[i]), 1);
         }
-        ctl->abort = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (warp == 1) tmem_alloc(smem_u32(&ctl->tmem_base), C::kTmemCols);
     tc_fence_before();
-    __syncthreads();
+    sync_compute_warps();
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
 
@@ -318,6 +357,7 @@ __device__ void compute_cta(const FusedParams &P, int W_comp, uint8_t *ring, Con
             uint32_t phase = 0;
             uint32_t armed = 0;  // bit s: stage s was handed to the TMA unit at least once
             bool ok = true;
+            TL_DECL(long long tl_pw = 0, tl_q;)
             // the m-tile table entries of the NEXT tile are fetched while this tile's k-blocks are issued, so
             // that the two dependent global loads never stall the stream of copies at a tile boundary
             Tile t = decode_tile(b, P, W_comp);
@@ -330,8 +370,10 @@ __device__ void compute_cta(const FusedParams &P, int W_comp, uint8_t *ring, Con
                 const int n0 = t.s * P.split_w + t.i_n * TN;
                 int kx = t.p * P.K;
                 for (int kb = 0; kb < P.num_kb; ++kb, kx += kBlockK) {
+                    TL(tl_q = clock64());
                     ok = wait_barrier_1t(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, deadline, P.status, (uint32_t)g, 10u);
                     if (!ok) break;
+                    TL(tl_pw += clock64() - tl_q);
                     const uint32_t full = smem_u32(&ctl->full[stage]);
                     const uint32_t a_dst = smem_u32(ring + stage * C::kStageBytes);
                     if (load_a) {
@@ -347,6 +389,7 @@ __device__ void compute_cta(const FusedParams &P, int W_comp, uint8_t *ring, Con
                 e = e_next;
                 row0 = row0_next;
             }
+            TL(if (load_a) tl_put(P, kTlProducerWait, (unsigned long long)tl_pw));
             if (!ok) {
                 // wind-down: let the copies already issued land before shared memory is released
                 // (bounded; a stage consumed meanwhile has completed its phase and passes at once)
@@ -367,16 +410,21 @@ __device__ void compute_cta(const FusedParams &P, int W_comp, uint8_t *ring, Con
             uint32_t phase = 0;
             int it = 0;
             bool ok = true;
+            TL_DECL(const long long tl_c0 = clock64(); long long tl_wf = 0, tl_wt = 0, tl_is = 0, tl_q;)
             for (int g = b; g < total_tiles && ok; g += P.P, ++it) {
                 const int a = it & 1;
                 const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+                TL(tl_q = clock64());
                 ok = wait_barrier_1t(smem_u32(&ctl->tmem_empty[a]), acc_phase ^ 1u, ctl, deadline, P.status, (uint32_t)g, 20u);
                 if (!ok) break;
+                TL(tl_wt += clock64() - tl_q);
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(a * TN);
                 for (int kb = 0; kb < P.num_kb; ++kb) {
+                    TL(tl_q = clock64());
                     ok = wait_barrier_1t(smem_u32(&ctl->full[stage]), phase, ctl, deadline, P.status, (uint32_t)g, 21u);
                     if (!ok) break;
+                    TL(tl_wf += clock64() - tl_q; tl_q = clock64());
                     tc_fence_after();
                     const uint32_t a_addr = smem_u32(ring + stage * C::kStageBytes);
                     const uint64_t a_desc = make_smem_desc(a_addr);
@@ -397,10 +445,15 @@ __device__ void compute_cta(const FusedParams &P, int W_comp, uint8_t *ring, Con
                                         k > 0 ? 1u : acc0);
                     }
                     tc_commit(smem_u32(&ctl->empty[stage]));   // stage reusable once these MMAs have read it
+                    TL(tl_is += clock64() - tl_q);
                     if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
                 }
                 if (ok) tc_commit(smem_u32(&ctl->tmem_full[a]));  // accumulator complete
+                TL(if (it == 0) tl_put(P, kTlFirstAcc, globaltimer_ns()));
             }
+            TL(tl_put(P, kTlMmaEnd, globaltimer_ns()); tl_put(P, kTlTiles, (unsigned long long)it);
+               tl_put(P, kTlWaitOperand, (unsigned long long)tl_wf); tl_put(P, kTlIssue, (unsigned long long)tl_is);
+               tl_put(P, kTlWaitTmem, (unsigned long long)tl_wt); tl_put(P, kTlMmaCycles, (unsigned long long)(clock64() - tl_c0)));
         }
         __syncwarp();
     } else if (warp >= 4 && warp < 4 + C::kEpiWarps) {
@@ -415,6 +468,7 @@ __device__ void compute_cta(const FusedParams &P, int W_comp, uint8_t *ring, Con
         // ahead and the row's flat assignment one tile ahead, so that these dependent global loads are
         // not in the way between an accumulator becoming ready and its first store.
         int valid = 0, f_row = 0, valid_n = 0, first_n = 0;
+        TL_DECL(long long tl_ew = 0, tl_ek = 0, tl_q;)
         if (b < total_tiles) {
             const int mu0 = decode_tile(b, P, W_comp).mu;
             const int mu1 = decode_tile(min(b + P.P, total_tiles - 1), P, W_comp).mu;
@@ -433,8 +487,10 @@ __device__ void compute_cta(const FusedParams &P, int W_comp, uint8_t *ring, Con
             const int valid_nn = __ldg(&P.mtile_valid[mu_nn]);
             const int first_nn = __ldg(&P.mtile_first_row[mu_nn]);
             const int f_row_n = (row_in_tile < valid_n) ? __ldg(&P.perm[first_n + row_in_tile]) : 0;
+            TL(tl_q = clock64());
             bool ok = wait_barrier(smem_u32(&ctl->tmem_full[a]), acc_phase, ctl, deadline, P.status, (uint32_t)g, 30u);
             ok = __all_sync(0xffffffffu, ok);
+            TL(tl_ew += clock64() - tl_q; tl_q = clock64());
             if (ok) {
                 tc_fence_after();
                 const int n0 = t.s * P.split_w + t.i_n * TN;
@@ -465,6 +521,7 @@ __device__ void compute_cta(const FusedParams &P, int W_comp, uint8_t *ring, Con
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&ctl->tmem_empty[a]));
+                TL(tl_ek += clock64() - tl_q);
             }
             // hand the tile to the publisher warp.  Its barrier is reused every other tile, so the warp
             // first makes sure that the tile two back has been published (it normally has, long ago).
@@ -479,6 +536,7 @@ __device__ void compute_cta(const FusedParams &P, int W_comp, uint8_t *ring, Con
             valid_n = valid_nn;
             first_n = first_nn;
         }
+        TL(if (warp == 4 && lane == 0) { tl_put(P, kTlEpiWait, (unsigned long long)tl_ew); tl_put(P, kTlEpiWork, (unsigned long long)tl_ek); });
     } else if (warp == 3) {
         // ---------------- publisher: one thread raises the readiness flag of every finished tile.  The
         // release costs a microsecond or more (it waits for the CTA's stores to be performed); here it
@@ -494,7 +552,12 @@ __device__ void compute_cta(const FusedParams &P, int W_comp, uint8_t *ring, Con
                 if (t.id != P.withhold) {
                     __threadfence();   // release: the epilogue warps' stores (observed through epi_done) come first
                     st_relaxed_u32(&P.flags[t.id], P.epoch);
+#if MOE_TIMELINE
+                    if (atomicAdd(&P.split_done[t.s], 1u) + 1u == (uint32_t)(W_comp * P.flag_parts) && P.timeline)
+                        P.timeline[(size_t)gridDim.x * kTimelineSlots + t.s] = globaltimer_ns();
+#else
                     red_relaxed_add_u32(&P.split_done[t.s], 1u);
+#endif
                 }
                 mbar_arrive(smem_u32(&ctl->pub_done[a]));
             }
@@ -503,7 +566,7 @@ __device__ void compute_cta(const FusedParams &P, int W_comp, uint8_t *ring, Con
     }
     // ---------------- teardown
     tc_fence_before();
-    __syncthreads();
+    sync_compute_warps();
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, C::kTmemCols);
@@ -553,14 +616,14 @@ __device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring
             mbar_init(smem_u32(&ctl->epi_done[i]), C::kEpiWarps);
             mbar_init(smem_u32(&ctl->pub_done[i]), 1);
         }
-        ctl->abort = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (warp == 1) tmem_alloc_pair(smem_u32(&ctl->tmem_base), C::kTmemCols);
     tc_fence_before();
-    __syncthreads();
-    cluster_sync_all();          // the peer's barriers exist before anything arrives on them
+    sync_compute_warps();
+    cluster_sync_all();          // the peer's barriers exist before anything arrives on them (the co-resident
+                                 // communication warps of both CTAs arrive on this cluster barrier too)
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
 
@@ -574,6 +637,7 @@ __device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring
             uint32_t phase = 0;
             uint32_t armed = 0;
             bool ok = true;
+            TL_DECL(long long tl_pw = 0, tl_q;)
             // next tile's table entries are fetched one tile ahead (see compute_cta)
             Tile t = decode_tile(b, P, W_comp);
             int e = __ldg(&P.mtile_expert[t.mu]);
@@ -586,8 +650,10 @@ __device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring
                 int kx = t.p * P.K;
                 for (int kb = 0; kb < P.num_kb; ++kb, kx += kBlockK) {
                     const uint32_t own_full = smem_u32(&ctl->full[stage]);
+                    TL(tl_q = clock64());
                     ok = wait_barrier_1t(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, deadline, P.status, (uint32_t)g, 10u);
                     if (!ok) break;
+                    TL(tl_pw += clock64() - tl_q);
                     const uint32_t leader_full = own_full & 0xFEFFFFFFu;   // same offset in the leader CTA (rank 0)
                     const uint32_t a_dst = smem_u32(ring + stage * C::kStageBytes);
                     if (load_a) {
@@ -603,6 +669,7 @@ __device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring
                 e = e_next;
                 row0 = row0_next;
             }
+            TL(if (load_a) tl_put(P, kTlProducerWait, (unsigned long long)tl_pw));
             if (!ok && leader_cta) {
                 // wind-down: let the copies already issued land before shared memory is released
                 const unsigned long long drain = globaltimer_ns() + 2000000ull;
@@ -622,16 +689,21 @@ __device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring
             uint32_t phase = 0;
             int it = 0;
             bool ok = true;
+            TL_DECL(const long long tl_c0 = clock64(); long long tl_wf = 0, tl_wt = 0, tl_is = 0, tl_q;)
             for (int g = b; g < total_tiles && ok; g += P.P, ++it) {
                 const int a = it & 1;
                 const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+                TL(tl_q = clock64());
                 ok = wait_barrier_1t(smem_u32(&ctl->tmem_empty[a]), acc_phase ^ 1u, ctl, deadline, P.status, (uint32_t)g, 20u);
                 if (!ok) break;
+                TL(tl_wt += clock64() - tl_q);
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(a * TN);
                 for (int kb = 0; kb < P.num_kb; ++kb) {
+                    TL(tl_q = clock64());
                     ok = wait_barrier_1t(smem_u32(&ctl->full[stage]), phase, ctl, deadline, P.status, (uint32_t)g, 21u);
                     if (!ok) break;
+                    TL(tl_wf += clock64() - tl_q; tl_q = clock64());
                     tc_fence_after();
                     const uint32_t a_addr = smem_u32(ring + stage * C::kStageBytes);
                     const uint64_t a_desc = make_smem_desc(a_addr);
@@ -648,11 +720,20 @@ __device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring
                             tc_mma_bf16_pair(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
                                              k > 0 ? 1u : acc0);
                     }
-                    tc_commit_pair(smem_u32(&ctl->empty[stage]));      // both CTAs may refill the stage
+                    const uint32_t empty_bar = smem_u32(&ctl->empty[stage]);
+                    tc_commit_pair(empty_bar, mapa_u32(empty_bar, 1u));   // both CTAs may refill the stage
+                    TL(tl_is += clock64() - tl_q);
                     if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
                 }
-                if (ok) tc_commit_pair(smem_u32(&ctl->tmem_full[a]));   // both epilogues may start
+                if (ok) {                                                   // both epilogues may start
+                    const uint32_t acc_bar = smem_u32(&ctl->tmem_full[a]);
+                    tc_commit_pair(acc_bar, mapa_u32(acc_bar, 1u));
+                }
+                TL(if (it == 0) tl_put(P, kTlFirstAcc, globaltimer_ns()));
             }
+            TL(tl_put(P, kTlMmaEnd, globaltimer_ns()); tl_put(P, kTlTiles, (unsigned long long)it);
+               tl_put(P, kTlWaitOperand, (unsigned long long)tl_wf); tl_put(P, kTlIssue, (unsigned long long)tl_is);
+               tl_put(P, kTlWaitTmem, (unsigned long long)tl_wt); tl_put(P, kTlMmaCycles, (unsigned long long)(clock64() - tl_c0)));
         }
         __syncwarp();
     } else if (warp >= 4 && warp < 4 + C::kEpiWarps) {
@@ -667,6 +748,7 @@ __device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring
         // ahead and the row's flat assignment one tile ahead, so that these dependent global loads are
         // not in the way between an accumulator becoming ready and its first store.
         int valid = 0, f_row = 0, valid_n = 0, first_n = 0;
+        TL_DECL(long long tl_ew = 0, tl_ek = 0, tl_q;)
         if (b < total_tiles) {
             const int mu0 = decode_tile(b, P, W_comp).mu;
             const int mu1 = decode_tile(min(b + P.P, total_tiles - 1), P, W_comp).mu;
@@ -685,7 +767,9 @@ __device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring
             const int valid_nn = __ldg(&P.mtile_valid[mu_nn]);
             const int first_nn = __ldg(&P.mtile_first_row[mu_nn]);
             const int f_row_n = (row_in_tile < valid_n) ? __ldg(&P.perm[first_n + row_in_tile]) : 0;
+            TL(tl_q = clock64());
             const bool ok = wait_barrier(smem_u32(&ctl->tmem_full[a]), acc_phase, ctl, deadline, P.status, (uint32_t)g, 30u);
+            TL(tl_ew += clock64() - tl_q; tl_q = clock64());
             if (ok) {
                 tc_fence_after();
                 const int n0 = t.s * P.split_w + t.i_n * TN;
@@ -714,6 +798,7 @@ __device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive_cluster_relaxed(mapa_u32(smem_u32(&ctl->tmem_empty[a]), 0u));
+                TL(tl_ek += clock64() - tl_q);
             }
             // hand the tile to the publisher warp (see compute_cta)
             bool ok2 = ok;
@@ -728,6 +813,7 @@ __device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring
             valid_n = valid_nn;
             first_n = first_nn;
         }
+        TL(if (warp == 4 && lane == 0) { tl_put(P, kTlEpiWait, (unsigned long long)tl_ew); tl_put(P, kTlEpiWork, (unsigned long long)tl_ek); });
     } else if (warp == 3) {
         // ---------------- publisher (both CTAs): raises this CTA's flag of every finished pair tile
         if (lane == 0) {
@@ -741,16 +827,22 @@ __device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring
                 if (t.id != P.withhold) {
                     __threadfence();
                     st_relaxed_u32(&P.flags[2 * t.id + (int)rank], P.epoch);
+#if MOE_TIMELINE
+                    if (atomicAdd(&P.split_done[t.s], 1u) + 1u == (uint32_t)(W_comp * P.flag_parts) && P.timeline)
+                        P.timeline[(size_t)gridDim.x * kTimelineSlots + t.s] = globaltimer_ns();
+#else
                     red_relaxed_add_u32(&P.split_done[t.s], 1u);
+#endif
                 }
                 mbar_arrive(smem_u32(&ctl->pub_done[a]));
             }
         }
         __syncwarp();
     }
-    // ---------------- teardown: nobody leaves while its peer may still touch its memory
+    // ---------------- teardown: nobody leaves while its peer may still touch its memory (the co-resident
+    // communication warps arrived on this cluster barrier right after the set-up one)
     tc_fence_before();
-    __syncthreads();
+    sync_compute_warps();
     cluster_sync_all();
     if (warp == 1) {
         tc_fence_after();
@@ -797,17 +889,47 @@ __device__ __forceinline__ void fma_bf16x8(float (&acc)[8], const uint4 &v, floa
     }
 }
 
-// Communication CTA.  Y is token-major: the k_tot * TP partial rows of one (token, split, column
-// slab) are one contiguous block (a "unit", at most 8 KB).  Twelve warps work independently; warp w
-// serves units w, w+12, ... of its CTA.  Each warp owns two 8 KB stages of shared memory and one
-// mbarrier per stage: it fetches a unit with ONE bulk asynchronous copy (global -> shared), and
-// while that copy is in flight it reduces the previous unit in fp32 in (j, p) order with the token's
-// weights and stores the bf16 result into the owning rank's buffer.  No warp waits on another one:
-// the issue latency of the copies and the memory latency overlap across the twelve warps.
+// Communication warp.  Y is token-major: the k_tot * TP partial rows of one (token, split, column
+// slab) are one contiguous block (a "unit", at most 8 KB).  Every communication warp works on its own:
+// it owns two 8 KB stages of shared memory and one mbarrier per stage, fetches a unit with ONE bulk
+// asynchronous copy (global -> shared), and while that copy is in flight it reduces the previous unit
+// in fp32 in (j, p) order with the token's weights and stores the bf16 result into the owning rank's
+// buffer.  No warp waits on another one: the issue latency of the copies and the memory latency
+// overlap across the warps of an SM.
+//
+// Who runs it (role):
+//   kRoleStatic      warp w of communication CTA c, static map: units w, w+12, ... of the communication
+//                    tiles c, c+C, ... of every split (the paper's map);
+//   kRoleFront       warp of a communication CTA, dynamic hand-out: ranges from the front of the
+//                    per-split queues, split 0 first; a unit waits for the tiles under it (flags);
+//   kRoleBack        warp of a compute CTA whose GEMM tiles are done (drain help): ranges from the back,
+//                    last split first;
+//   kRoleCoResident  extra warp of a compute CTA that is still computing: from the front, split 0
+//                    first, but only from splits that are complete (it sleeps on the split counter
+//                    instead of polling single tiles, so that it costs the computing warps nothing
+//                    while it has nothing to do).
 constexpr int kCommWarps = 12;
 constexpr int kCommUnitBytes = 8192;
 constexpr int kCommWarpBytes = 2 * kCommUnitBytes;
 static_assert(kCommWarps * kCommWarpBytes <= kStageBytesTotal, "communication stages exceed the ring");
+// Co-resident communication warps live in the aux region, which the epilogue leaves alone when it
+// stores straight from registers: two warps' stages (32 KB), then the per-row weights in compact
+// 16-float slots -- four for co-resident warps, twelve for the CTA's own warps once they turn to
+// communication (their usual 256-float slots would overlap the co-resident stages).  Needs Q <= 16.
+constexpr int kCoWarpsAux = 2;          // co-resident warps whose stages fit the aux region
+constexpr int kCoWeightFloats = 16;
+constexpr int kCoWeightsOffset = kCoWarpsAux * kCommWarpBytes;
+static_assert(kCoWeightsOffset + (kCoWarpsMax + kCommWarps) * kCoWeightFloats * 4 <= kAuxBytes,
+              "co-resident stages and weights exceed the aux region");
+
+enum { kRoleStatic = 0, kRoleFront = 1, kRoleBack = 2, kRoleCoResident = 3 };
+
+// what one communication warp owns
+struct CommWarpRes {
+    uint8_t *stages;              // 2 x kCommUnitBytes
+    unsigned long long *full;     // 2 mbarriers (initialised with count 1 at kernel start)
+    float *wq;                    // room for Q floats
+};
 
 struct CommUnit {
     int t, d, s, slab, wslab, ucols;
@@ -816,33 +938,29 @@ struct CommUnit {
     bool all_valid;   // every slot of the token has a source row
 };
 
+// `c`, `warp`: communication CTA and warp inside it (static map only).
 template <int TN>
-__device__ void comm_cta(const FusedParams &P, int W_comp, uint8_t *ring, Control *ctl, uint8_t *aux, int c, bool helper)
+__device__ void comm_warp(const FusedParams &P, int W_comp, Control *ctl, const CommWarpRes res, int role, int c, int warp,
+                          int tl_slot)
 {
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    (void)tl_slot;   // index of the warp's record in a timeline build
+    const int lane = threadIdx.x & 31;
     const bool wait_needed = (P.mode != MOE_MODE_COMBINE_ONLY);
-    const bool claiming = (P.drain_help != 0);   // work is handed out dynamically (queue per split) instead of by the static map
+    const bool helper = (role == kRoleBack);
     const unsigned long long deadline = globaltimer_ns() + P.wait_ns;
     // the wait for a copy only follows a readiness wait: it gets a later deadline so that the first
     // report names the wait that really ran out
     const unsigned long long deadline2 = deadline + P.wait_ns / 4 + 1000000ull;
 
-    if (threadIdx.x == 0) {
-        for (int i = 0; i < 2 * kCommWarps; ++i) mbar_init(smem_u32(&ctl->comm_full[i]), 1);
-        ctl->abort = 0u;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-    __syncthreads();
-    if (warp >= kCommWarps) return;
-    uint8_t *my_ring = ring + warp * kCommWarpBytes;
-    float *wq = reinterpret_cast<float *>(aux) + warp * 256;
+    TL_DECL(unsigned long long tl_first = 0, tl_last = 0, tl_sleep = 0; uint32_t tl_units = 0, tl_by_split[4] = {0u, 0u, 0u, 0u};)
+    uint8_t *my_ring = res.stages;
+    float *wq = res.wq;
+    const uint32_t full_s = smem_u32(res.full);
     const __nv_bfloat16 *Y = reinterpret_cast<const __nv_bfloat16 *>(P.Y);
 
     // reduce the unit sitting in stage `st` (its copy was issued one unit ago)
     auto consume = [&](const CommUnit &u, int st, uint32_t parity) -> bool {
-        bool ok = wait_barrier(smem_u32(&ctl->comm_full[2 * warp + st]), parity, ctl, deadline2, P.status,
-                               (uint32_t)u.t, 43u);
+        bool ok = wait_barrier(full_s + 8u * (uint32_t)st, parity, ctl, deadline2, P.status, (uint32_t)u.t, 43u);
         if (!ok) return false;
         const int n16 = u.ucols >> 3;
         const uint32_t row_bytes = (uint32_t)u.wslab * 2u;
@@ -925,6 +1043,7 @@ __device__ void comm_cta(const FusedParams &P, int W_comp, uint8_t *ring, Contro
             }
         }
         __syncwarp();   // all lanes are done with the stage (and with wq) before either is reused
+        TL(tl_last = globaltimer_ns(); if (tl_units == 0) tl_first = tl_last; ++tl_units; if (u.s < 4) ++tl_by_split[u.s]);
         return true;
     };
 
@@ -963,6 +1082,7 @@ __device__ void comm_cta(const FusedParams &P, int W_comp, uint8_t *ring, Contro
                     const int part = (P.flag_parts == 2) ? ((row - mu * P.tile_m) >> 7) : 0;
                     const int g = (u.s * W_comp + (mu * P.TP + p) * P.NTs + in0 + tn) * P.flag_parts + part;
                     uint32_t spins = 0;
+                    TL_DECL(const unsigned long long tl_f0 = globaltimer_ns();)
                     while (ld_acquire_u32(&P.flags[g]) != P.epoch) {
                         if ((++spins & 31u) == 0u && (ctl->abort || globaltimer_ns() > deadline)) {
                             report(P.status, MOE_DEV_TIMEOUT, (uint32_t)g, 40u);
@@ -971,6 +1091,7 @@ __device__ void comm_cta(const FusedParams &P, int W_comp, uint8_t *ring, Contro
                         }
                         __nanosleep(64);
                     }
+                    TL(tl_sleep += globaltimer_ns() - tl_f0);
                 }
                 if (__any_sync(0xffffffffu, failed)) {
                     // this warp gives up; the copy it still has in flight must land first
@@ -986,7 +1107,7 @@ __device__ void comm_cta(const FusedParams &P, int W_comp, uint8_t *ring, Contro
         // ---- issue this unit's copy, then reduce the previous unit while it is in flight
         const int st = n_mine & 1;
         if (lane == 0) {
-            const uint32_t full = smem_u32(&ctl->comm_full[2 * warp + st]);
+            const uint32_t full = full_s + 8u * (uint32_t)st;
             const uint32_t bytes = (uint32_t)(P.Q * u.wslab) * 2u;
             const __nv_bfloat16 *src = Y + ((size_t)u.t * P.L + u.s) * (size_t)P.Q * (size_t)P.split_w +
                                        ((size_t)u.slab * P.Q << P.slab_shift);
@@ -998,8 +1119,7 @@ __device__ void comm_cta(const FusedParams &P, int W_comp, uint8_t *ring, Contro
         if (prev.live && !consume(prev, (n_mine - 2) & 1, (uint32_t)((n_mine - 2) >> 1) & 1u)) {
             // the previous copy never landed (reported); wait for the one just issued, then leave
             const unsigned long long drain = globaltimer_ns() + 2000000ull;
-            while (!mbar_try_wait(smem_u32(&ctl->comm_full[2 * warp + st]), (uint32_t)((n_mine - 1) >> 1) & 1u) &&
-                   globaltimer_ns() < drain) {}
+            while (!mbar_try_wait(full_s + 8u * (uint32_t)st, (uint32_t)((n_mine - 1) >> 1) & 1u) && globaltimer_ns() < drain) {}
             prev.live = false;
             return false;
         }
@@ -1118,7 +1238,7 @@ __device__ void comm_cta(const FusedParams &P, int W_comp, uint8_t *ring, Contro
         return true;
     };
 
-    if (!claiming) {
+    if (role == kRoleStatic) {
         // the paper's static map: communication tile ct belongs to CTA ct mod C (Section III-A)
         for (int s = 0; s < P.L; ++s)
             for (int ct = c; ct < P.comm_tiles; ct += P.C)
@@ -1127,12 +1247,12 @@ __device__ void comm_cta(const FusedParams &P, int W_comp, uint8_t *ring, Contro
                     return;
                 }
     } else {
-        // Drain help: work is handed out dynamically, to warps.  Every split has a two-ended queue of
-        // its items in one 64-bit word (low half: items taken from the front, high half: from the back).
-        // Warps of the communication CTAs take from the front, split 0 first; warps of compute CTAs that
-        // have run out of GEMM tiles take from the back, last split first.  One atomic add claims a
-        // range; ranges shrink towards the end so that the last ones finish together.  The next claim is
-        // issued before the current range is served, which hides the latency of the atomic.
+        // Dynamic hand-out, to warps.  Every split has a two-ended queue of its items in one 64-bit word
+        // (low half: items taken from the front, high half: from the back).  Warps of the communication
+        // CTAs and co-resident warps take from the front, split 0 first; warps of compute CTAs that have
+        // run out of GEMM tiles take from the back, last split first.  One atomic add claims a range;
+        // ranges shrink towards the end so that the last ones finish together.  The next claim is issued
+        // before the current range is served, which hides the latency of the atomic.
         const uint32_t n_items = (uint32_t)P.T * (uint32_t)P.comm_cols;
         int s = helper ? P.L - 1 : 0;
         unsigned long long old = 0;
@@ -1146,8 +1266,48 @@ __device__ void comm_cta(const FusedParams &P, int W_comp, uint8_t *ring, Contro
                 old = atomicAdd(&P.queue[split], helper ? ((unsigned long long)chunk << 32) : (unsigned long long)chunk);
             }
         };
-        claim(s);
+        bool claimed = false;      // a claim on split s is outstanding
         while (s >= 0 && s < P.L) {
+            if (!claimed) {
+                if (role == kRoleCoResident && !((ready_mask >> s) & 1u)) {
+                    // A co-resident warp only takes work that can be served at once.  Inside a split the
+                    // tiles run expert by expert and a token needs tiles of all its experts, so hardly any
+                    // token is complete before the split is: wait for the whole split, asleep most of the time.
+                    uint32_t state = 0;   // 1: split complete, 2: split handed out already, 3: give up
+                    if (lane == 0) {
+                        if (ld_acquire_u32(&P.split_done[s]) >= (uint32_t)(W_comp * P.flag_parts)) state = 1;
+                        else {
+                            const unsigned long long q = *reinterpret_cast<volatile unsigned long long *>(&P.queue[s]);
+                            if ((uint32_t)q + (uint32_t)(q >> 32) >= n_items) state = 2;
+                            else if (ctl->abort) state = 3;
+                            else if (globaltimer_ns() > deadline) {
+                                report(P.status, MOE_DEV_TIMEOUT, (uint32_t)s, 44u);
+                                state = 3;
+                            }
+                        }
+                    }
+                    state = __shfl_sync(0xffffffffu, state, 0);
+                    if (state == 0) {
+                        TL_DECL(const unsigned long long tl_s0 = globaltimer_ns();)
+                        __nanosleep(2000);
+                        TL(tl_sleep += globaltimer_ns() - tl_s0);
+                        continue;
+                    }
+                    if (state == 2) {
+                        ++s;
+                        continue;
+                    }
+                    if (state == 3) {
+                        ctl->abort = 1u;
+                        break;
+                    }
+                    ready_mask |= 1u << s;
+                    // rows published through ordinary stores are read by the copy engine next
+                    asm volatile("fence.proxy.async;" ::: "memory");
+                }
+                claim(s);
+                claimed = true;
+            }
             const unsigned long long o = __shfl_sync(0xffffffffu, old, 0);
             const uint32_t ch = __shfl_sync(0xffffffffu, chunk, 0);
             const uint32_t f = (uint32_t)o, bk = (uint32_t)(o >> 32);
@@ -1163,11 +1323,12 @@ __device__ void comm_cta(const FusedParams &P, int W_comp, uint8_t *ring, Contro
             const int cur = s;
             if (i0 >= i1) {                      // this split is handed out: go on to the next one
                 s += helper ? -1 : 1;
-                if (s >= 0 && s < P.L) claim(s);
+                claimed = false;
                 continue;
             }
             claim(s);
-            if (ctl->abort) break;
+            // warp-uniform exit: the loop body holds full-mask collectives
+            if (__any_sync(0xffffffffu, ctl->abort != 0u)) break;
             if (!serve_items(cur, i0, i1)) {
                 ctl->abort = 1u;
                 return;
@@ -1175,6 +1336,67 @@ __device__ void comm_cta(const FusedParams &P, int W_comp, uint8_t *ring, Contro
         }
     }
     if (prev.live) consume(prev, (n_mine - 1) & 1, (uint32_t)((n_mine - 1) >> 1) & 1u);
+#if MOE_TIMELINE
+    if (lane == 0) {
+        if (role == kRoleCoResident) {
+            const int base = kTlCoWarp + 8 * tl_slot;
+            tl_put(P, base + 0, tl_first); tl_put(P, base + 1, tl_last); tl_put(P, base + 2, tl_units); tl_put(P, base + 3, tl_sleep);
+            for (int i = 0; i < 4; ++i) tl_put(P, base + 4 + i, tl_by_split[i]);
+        } else if (tl_slot == 0) {
+            tl_put(P, kTlCommUnits, tl_units);
+            tl_put(P, kTlCommWaitNs, tl_sleep);
+        }
+    }
+#endif
+}
+
+// The communication warps of a CTA whose only role is communication (dedicated communication CTA, or a
+// compute CTA that has run out of GEMM tiles): warps 0-11, stages in the operand ring.
+template <int TN>
+__device__ __forceinline__ void comm_cta(const FusedParams &P, int W_comp, uint8_t *ring, Control *ctl, uint8_t *aux, int role, int c)
+{
+    const int warp = threadIdx.x >> 5;
+    if (warp >= kCommWarps) return;
+    CommWarpRes res;
+    res.stages = ring + warp * kCommWarpBytes;
+    res.full = &ctl->comm_full[2 * warp];
+    res.wq = (role == kRoleBack && P.co_warps > 0)
+                 ? reinterpret_cast<float *>(aux + kCoWeightsOffset) + (kCoWarpsMax + warp) * kCoWeightFloats
+                 : reinterpret_cast<float *>(aux) + warp * 256;
+    comm_warp<TN>(P, W_comp, ctl, res, role, c, warp, warp);
+}
+
+// Co-resident communication warp `cw` of a compute CTA: stages and weights in the aux region (free when
+// the epilogue stores straight from registers, which the host checks before it asks for such warps).
+template <int TN>
+__device__ __forceinline__ void co_resident_warp(const FusedParams &P, int W_comp, Control *ctl, uint8_t *aux, int cw)
+{
+    CommWarpRes res;
+    res.stages = aux + cw * kCommWarpBytes;
+    res.full = &ctl->co_full[2 * cw];
+    res.wq = reinterpret_cast<float *>(aux + kCoWeightsOffset) + cw * kCoWeightFloats;
+    comm_warp<TN>(P, W_comp, ctl, res, kRoleCoResident, 0, 0, cw);
+}
+
+// Co-resident warp number of warp 16..19.  The four warp schedulers of an SM take warps by number modulo
+// four, and scheduler 1 holds the thread that issues the MMAs, which has to stay ahead of the tensor pipe:
+// warps 18 and 19 are used first, then 16, and 17 (scheduler 1) last.
+__device__ __forceinline__ int co_warp_number(int warp)
+{
+    return warp == 18 ? 0 : warp == 19 ? 1 : warp == 16 ? 2 : 3;
+}
+
+// Barriers of every communication stage the CTA may use, and the abort flag; before the first CTA-wide
+// barrier of the kernel.
+__device__ __forceinline__ void init_comm_barriers(Control *ctl)
+{
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < 2 * kCommWarps; ++i) mbar_init(smem_u32(&ctl->comm_full[i]), 1);
+        for (int i = 0; i < 2 * kCoWarpsMax; ++i) mbar_init(smem_u32(&ctl->co_full[i]), 1);
+        ctl->abort = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
 }
 
 // --------------------------------------------------------------------------- kernel
@@ -1187,7 +1409,7 @@ __device__ __forceinline__ int launch_w_comp(const FusedParams &P)
 }
 
 template <int TN>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kFusedThreads, 1)
 moe_gemm2_combine_kernel(const __grid_constant__ FusedParams P)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -1200,20 +1422,29 @@ moe_gemm2_combine_kernel(const __grid_constant__ FusedParams P)
         P.split_done_next[threadIdx.x] = 0u;
         P.queue_next[threadIdx.x] = 0ull;
     }
+    init_comm_barriers(ctl);
+    __syncthreads();          // the only barrier all 20 warps share
+    TL(if (threadIdx.x == 0) { tl_put(P, kTlBegin, globaltimer_ns()); tl_put(P, kTlRole, (int)blockIdx.x < P.C ? 0u : 1u); });
 
+    const int warp = threadIdx.x >> 5;
     const int W_comp = launch_w_comp(P);
-    if ((int)blockIdx.x < P.C)
-        comm_cta<TN>(P, W_comp, ring, ctl, aux, (int)blockIdx.x, false);
-    else {
+    if ((int)blockIdx.x < P.C) {
+        comm_cta<TN>(P, W_comp, ring, ctl, aux, P.drain_help ? kRoleFront : kRoleStatic, (int)blockIdx.x);
+    } else if (warp >= kThreads / 32) {
+        if (co_warp_number(warp) < P.co_warps) co_resident_warp<TN>(P, W_comp, ctl, aux, co_warp_number(warp));
+        return;
+    } else {
         compute_cta<TN>(P, W_comp, ring, ctl, aux, (int)blockIdx.x - P.C);
+        TL(if (threadIdx.x == 0) tl_put(P, kTlComputeEnd, globaltimer_ns()));
         // out of GEMM tiles: help with the communication that is left (all TMA and TMEM traffic is over)
-        if (P.drain_help && P.mode == MOE_MODE_FUSED && !ctl->abort) comm_cta<TN>(P, W_comp, ring, ctl, aux, 0, true);
+        if (P.drain_help && P.mode == MOE_MODE_FUSED && !ctl->abort) comm_cta<TN>(P, W_comp, ring, ctl, aux, kRoleBack, 0);
     }
+    TL(if (threadIdx.x == 0) tl_put(P, kTlCtaEnd, globaltimer_ns()));
 }
 
 // Pair kernel: launched with clusters of two CTAs.  Communication CTAs are single CTAs (blockIdx < C);
 // with an odd C the cluster-mate of the last one has no role; compute pairs start at the next even index.
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kFusedThreads, 1)
 moe_gemm2_combine_pair_kernel(const __grid_constant__ FusedParams P)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -1225,22 +1456,40 @@ moe_gemm2_combine_pair_kernel(const __grid_constant__ FusedParams P)
         P.split_done_next[threadIdx.x] = 0u;
         P.queue_next[threadIdx.x] = 0ull;
     }
+    init_comm_barriers(ctl);
+    __syncthreads();          // the only CTA-wide barrier all 20 warps share
+    TL(if (threadIdx.x == 0) { tl_put(P, kTlBegin, globaltimer_ns()); tl_put(P, kTlRole, (int)blockIdx.x < ((P.C + 1) & ~1) ? 0u : 1u); });
 
+    const int warp = threadIdx.x >> 5;
     const int c_even = (P.C + 1) & ~1;
     const int W_comp = launch_w_comp(P);
-    if ((int)blockIdx.x < P.C)
-        comm_cta<256>(P, W_comp, ring, ctl, aux, (int)blockIdx.x, false);
-    else if ((int)blockIdx.x < c_even) {
+    if ((int)blockIdx.x < P.C) {
+        comm_cta<256>(P, W_comp, ring, ctl, aux, P.drain_help ? kRoleFront : kRoleStatic, (int)blockIdx.x);
+    } else if ((int)blockIdx.x < c_even) {
         // odd C: the last communication CTA's cluster-mate cannot compute (no partner).  With dynamic work
         // distribution it serves communication work as well; under the static map it has no tile list.
-        if (P.drain_help && P.mode == MOE_MODE_FUSED) comm_cta<256>(P, W_comp, ring, ctl, aux, (int)blockIdx.x, false);
+        if (P.drain_help && P.mode == MOE_MODE_FUSED) comm_cta<256>(P, W_comp, ring, ctl, aux, kRoleFront, (int)blockIdx.x);
+    } else if (warp >= kThreads / 32) {
+        // The compute warps of both CTAs meet at two cluster barriers (set-up and teardown), and a cluster
+        // barrier counts every thread: these warps join the first, arrive at once on the second (they hold
+        // nothing a peer could touch) and pick its completion up when their own work is done.
+        cluster_sync_all();
+        cluster_arrive();
+        if (co_warp_number(warp) < P.co_warps) co_resident_warp<256>(P, W_comp, ctl, aux, co_warp_number(warp));
+        cluster_wait();
+        return;
     } else {
         compute_cta_pair(P, W_comp, ring, ctl, aux, ((int)blockIdx.x - c_even) >> 1);
-        if (P.drain_help && P.mode == MOE_MODE_FUSED && !ctl->abort) comm_cta<256>(P, W_comp, ring, ctl, aux, 0, true);
+        TL(if (threadIdx.x == 0) tl_put(P, kTlComputeEnd, globaltimer_ns()));
+        if (P.drain_help && P.mode == MOE_MODE_FUSED && !ctl->abort) comm_cta<256>(P, W_comp, ring, ctl, aux, kRoleBack, 0);
     }
+    TL(if (threadIdx.x == 0) tl_put(P, kTlCtaEnd, globaltimer_ns()));
 }
 
 }  // namespace
+
+int fused_co_warps_max() { return kCoWarpsAux; }
+bool fused_timeline_build() { return MOE_TIMELINE != 0; }
 
 size_t fused_smem_bytes(int) { return (size_t)kStageBytesTotal + 1024 + ((sizeof(Control) + 127) & ~(size_t)127) + kAuxBytes; }
 
@@ -1258,13 +1507,13 @@ cudaError_t fused_occupancy(int tile_n, int *blocks_per_sm)
     switch (tile_n) {
     case 64:
         if ((e = prepare<64>()) != cudaSuccess) return e;
-        return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, moe_gemm2_combine_kernel<64>, kThreads, sm);
+        return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, moe_gemm2_combine_kernel<64>, kFusedThreads, sm);
     case 128:
         if ((e = prepare<128>()) != cudaSuccess) return e;
-        return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, moe_gemm2_combine_kernel<128>, kThreads, sm);
+        return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, moe_gemm2_combine_kernel<128>, kFusedThreads, sm);
     case 256:
         if ((e = prepare<256>()) != cudaSuccess) return e;
-        return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, moe_gemm2_combine_kernel<256>, kThreads, sm);
+        return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, moe_gemm2_combine_kernel<256>, kFusedThreads, sm);
     }
     return cudaErrorInvalidValue;
 }
@@ -1274,14 +1523,14 @@ cudaError_t pair_occupancy(int *blocks_per_sm, int *max_clusters)
     const size_t sm = fused_smem_bytes(256);
     cudaError_t e = cudaFuncSetAttribute(moe_gemm2_combine_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
     if (e != cudaSuccess) return e;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, moe_gemm2_combine_pair_kernel, kThreads, sm);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, moe_gemm2_combine_pair_kernel, kFusedThreads, sm);
     if (e != cudaSuccess) return e;
     int dev = 0, n_sm = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(n_sm & ~1));
-    cfg.blockDim = dim3(kThreads);
+    cfg.blockDim = dim3(kFusedThreads);
     cfg.dynamicSmemBytes = sm;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -1297,7 +1546,7 @@ cudaError_t pair_launch(const FusedParams &p, int grid, cudaStream_t stream)
 {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
-    cfg.blockDim = dim3(kThreads);
+    cfg.blockDim = dim3(kFusedThreads);
     cfg.dynamicSmemBytes = fused_smem_bytes(256);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
@@ -1314,9 +1563,9 @@ cudaError_t fused_launch(int tile_n, const FusedParams &p, int grid, cudaStream_
 {
     const size_t sm = fused_smem_bytes(tile_n);
     switch (tile_n) {
-    case 64: moe_gemm2_combine_kernel<64><<<grid, kThreads, sm, stream>>>(p); break;
-    case 128: moe_gemm2_combine_kernel<128><<<grid, kThreads, sm, stream>>>(p); break;
-    case 256: moe_gemm2_combine_kernel<256><<<grid, kThreads, sm, stream>>>(p); break;
+    case 64: moe_gemm2_combine_kernel<64><<<grid, kFusedThreads, sm, stream>>>(p); break;
+    case 128: moe_gemm2_combine_kernel<128><<<grid, kFusedThreads, sm, stream>>>(p); break;
+    case 256: moe_gemm2_combine_kernel<256><<<grid, kFusedThreads, sm, stream>>>(p); break;
     default: return cudaErrorInvalidValue;
     }
     return cudaGetLastError();

@@ -12,7 +12,9 @@
 
 namespace moe {
 
-constexpr int kThreads = 512;          // threads of every CTA of the fused kernel
+constexpr int kThreads = 512;          // threads of a CTA's compute (or dedicated communication) role: 16 warps
+constexpr int kCoWarpsMax = 4;         // co-resident communication warps a compute CTA of the fused kernel may carry
+constexpr int kFusedThreads = kThreads + 32 * kCoWarpsMax;   // block size of the fused kernel
 constexpr int kBlockK = 64;            // bf16 elements per k-block: one 128-byte swizzle row
 constexpr int kUmmaK = 16;             // K of one tcgen05.mma.kind::f16 instruction
 constexpr int kMmaM = 128;             // M of the MMA (tile_m = 64 stores the first 64 rows only)
@@ -21,6 +23,7 @@ constexpr int kCommTileM = 128;        // T_M^comm
 constexpr int kCommTileN = 1024;       // T_N^comm
 constexpr int kRoutingChunk = 256;     // flat assignments handled by one warp while sorting
 constexpr uint64_t kDefaultWaitNs = 2000000000ull;
+constexpr int kTimelineSlots = 32;     // 64-bit words per CTA in a timeline buffer (timeline build only)
 
 // Parameters of one fused launch.  Passed by value (__grid_constant__): the two tensor maps
 // must sit in kernel parameter space, 64-byte aligned.
@@ -41,6 +44,7 @@ struct alignas(64) FusedParams {
     unsigned long long *queue;     // [L] drain help: items of the split handed out so far, front | back << 32
     unsigned long long *queue_next;  // [L] ... of the next launch, zeroed by this one
     uint32_t *status;              // 4 words
+    unsigned long long *timeline;  // timeline build: per-CTA records, then one stamp per split; else nullptr
     void *out[MOE_MAX_EP];
     unsigned long long wait_ns;
     long long R_pad;
@@ -50,6 +54,7 @@ struct alignas(64) FusedParams {
     int32_t tok_blk, tok_tiles_per_rank, comm_cols, comm_tiles;
     int32_t num_kb, last_ksteps;
     int32_t drain_help;                 // compute CTAs serve communication tiles once their GEMM tiles are done
+    int32_t co_warps;                   // co-resident communication warps per compute CTA (0..2)
     int32_t tile_order;                 // 0: split-major tile sequence (the paper's); 1: m-tile-major across splits
     int32_t flag_parts;                 // readiness flags per tile: 1, or 2 for a CTA-pair tile
     int32_t Q, slab_cols, slab_shift;   // Q = k_tot * TP rows per unit; slab_cols = 1 << slab_shift
@@ -70,6 +75,8 @@ struct moe_handle {
     int o_pair = 0;                                     // CTA-pair kernel: resident CTAs per SM
     int max_pairs = 0;                                  // ... and co-resident clusters of two
     void *counts_event = nullptr;                       // cudaEvent_t: "the tile counts have reached the host"
+    unsigned long long *timeline = nullptr;             // timeline build: where the next fused launch records
+    size_t timeline_bytes = 0;
 };
 
 namespace moe {
@@ -85,6 +92,8 @@ int32_t require_handle_device(moe_handle *h, const char *who);
 size_t fused_smem_bytes(int tile_n);
 cudaError_t fused_occupancy(int tile_n, int *blocks_per_sm);
 cudaError_t fused_launch(int tile_n, const FusedParams &p, int grid, cudaStream_t stream);
+int fused_co_warps_max();
+bool fused_timeline_build();   // the library was compiled with -DMOE_TIMELINE=1   // co-resident communication warps a compute CTA has shared memory for
 // CTA-pair kernel (256 x 256 tiles, clusters of two)
 cudaError_t pair_occupancy(int *blocks_per_sm, int *max_clusters);
 cudaError_t pair_launch(const FusedParams &p, int grid, cudaStream_t stream);

@@ -106,10 +106,18 @@ __device__ __forceinline__ uint32_t mapa_u32(uint32_t addr, uint32_t rank)
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
     return r;
 }
-__device__ __forceinline__ void cluster_sync_all()
+__device__ __forceinline__ void cluster_arrive()
 {
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait()
+{
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    cluster_arrive();
+    cluster_wait();
 }
 // Arrival that hands back an accumulator buffer.  Relaxed on purpose: what it orders are this warp's
 // TMEM reads, which tcgen05.wait::ld and tcgen05.fence::before_thread_sync have completed; a release
@@ -142,13 +150,13 @@ __device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t cols)
 {
     asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
 }
-// arrives on the barrier at the same shared-memory offset in both CTAs of the pair
-__device__ __forceinline__ void tc_commit_pair(uint32_t bar)
+// Arrives on the barrier at the same shared-memory offset in both CTAs of the pair once the MMAs issued
+// so far have completed: one commit per CTA (issued by the leader, rank 0; `peer_bar` is the address of
+// the same barrier in rank 1 as mapa gives it).  Both commits track the same preceding MMAs.
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar, uint32_t peer_bar)
 {
-    asm volatile(
-        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-        ::"r"(bar), "h"((uint16_t)3)
-        : "memory");
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(peer_bar) : "memory");
 }
 __device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
 {

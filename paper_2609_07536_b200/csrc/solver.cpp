@@ -272,7 +272,9 @@ extern "C" int32_t plan_partition(const int32_t *routed_tile_counts, int32_t n_e
     out->mode = MOE_MODE_FUSED;
     out->debug_withhold_tile = -1;
     out->drain_help = limits->drain_help != 0 ? 1 : 0;
-    out->reserved = 0;
+    out->co_warps = 0;
+    if (limits->drain_help != 0 && limits->co_warps_max > 0 && limits->force_co_warps > 0)
+        out->co_warps = limits->force_co_warps < limits->co_warps_max ? limits->force_co_warps : limits->co_warps_max;
     return MOE_OK;
 }
 

@@ -53,7 +53,7 @@ def build_routing(w: wl.Workload, topk_idx: np.ndarray, ws: B.Workspace = None):
 
 
 def run_layer(w: wl.Workload, topk_idx, topk_w, x, W2, force_C=0, mode=B.MOE_MODE_FUSED, ws=None,
-              withhold=-1, check_status=True, P_override=None, drain_help=None):
+              withhold=-1, check_status=True, P_override=None, drain_help=None, co_warps=0, C_override=None):
     """x, W2: bf16 torch tensors (CPU or CUDA).  Returns (list of EP outputs on CPU as float32,
     plan, workspace, S)."""
     h = handle()
@@ -63,12 +63,15 @@ def run_layer(w: wl.Workload, topk_idx, topk_w, x, W2, force_C=0, mode=B.MOE_MOD
     lim.force_comm_ctas = force_C
     if drain_help is not None:
         lim.drain_help = int(drain_help)
+    lim.force_co_warps = int(co_warps)
     tiles = ws.tile_counts[:shape.E_tot].tolist()
     plan = B.plan_partition(tiles, occ, lim, shape, rho)
     plan.mode = mode
     plan.debug_withhold_tile = withhold
     if P_override is not None:
         plan.P = P_override
+    if C_override is not None:
+        plan.comm_ctas = plan.R = C_override
     xd, Wd = x.cuda(), W2.cuda()
     wd = torch.from_numpy(np.ascontiguousarray(topk_w)).cuda() if topk_w.size else torch.zeros(1, device="cuda")
     for o in ws.out:

@@ -30,7 +30,7 @@ def test_every_declared_symbol_is_exported():
 def test_structs_match_header_sizes():
     assert ctypes.sizeof(B.moe_shape) == 32
     assert ctypes.sizeof(B.moe_occupancy) == 28
-    assert ctypes.sizeof(B.moe_sm_limits) == 24
+    assert ctypes.sizeof(B.moe_sm_limits) == 32
     assert ctypes.sizeof(B.moe_rho) == 40
     assert ctypes.sizeof(B.moe_plan) == 56
     assert ctypes.sizeof(B.moe_status) == 16

@@ -167,6 +167,50 @@ def test_drain_help_and_tile_families_change_nothing_but_time():
     assert np.max(np.abs(got - expect)) <= G.tolerance(expect)
 
 
+def test_co_resident_communication_warps_change_nothing_but_time():
+    # extra communication warps inside every compute CTA (they serve split s while the CTA computes split
+    # s + 1), with or without dedicated communication CTAs, in both kernels: same bits as the plain launch,
+    # and those bits are the oracle's result within the path's tolerance
+    w = replace(wl.GRANITE, name="co", T=2000, L=2)
+    idx, wt, _ = wl.make_routing(w)
+    x, W2 = wl.make_data(w)
+    base = None
+    for tile in ((128, 256), (256, 256), (128, 128)):
+        for co, C, C_override in ((0, 1, None), (1, 1, None), (2, 1, None), (2, 9, None), (2, 1, 0), (1, 1, 0)):
+            wt_ = replace(w, tile_m=tile[0], tile_n=tile[1])
+            P_override = (148 // (2 if tile[0] == 256 else 1)) if C_override == 0 else None
+            outs, plan, ws, S, st = G.run_layer(wt_, idx, wt, x, W2, force_C=C, drain_help=1, co_warps=co,
+                                                C_override=C_override, P_override=P_override)
+            assert st.code == 0 and plan.co_warps == co
+            bits = [torch.from_numpy(o).bfloat16().view(torch.int16).numpy() for o in outs]
+            if base is None:
+                base = bits
+            for a, b in zip(base, bits):
+                assert np.array_equal(a, b), (tile, co, C, C_override)
+    expect, _ = _oracle_tokens(w, idx, wt, x, W2)
+    got = np.concatenate([o[:len(G.tokens_of_rank(w.T, w.EP, d))] for d, o in enumerate(outs)])
+    assert np.max(np.abs(got - expect)) <= G.tolerance(expect)
+
+
+@pytest.mark.parametrize("kw", [
+    dict(T=777, E=5, k=2, H=1536, I=512, TP=2, EP=3, tile_m=128, tile_n=256, L=4),   # partial n-tile at the split end
+    dict(T=1030, E=70, k=2, H=512, I=256, TP=2, EP=8, tile_m=128, tile_n=128, L=8),  # empty experts, L = 8
+    dict(T=200, E=6, k=2, n_shared=2, H=256, I=128, TP=1, EP=1, tile_m=128, tile_n=64, L=2),  # shared experts
+    dict(T=900, E=9, k=4, H=1024, I=256, TP=4, EP=2, tile_m=256, tile_n=256, L=2),    # pair tiles, 16-row units
+    dict(T=333, E=12, k=3, H=264, I=80, tile_m=64, tile_n=64, EP=4, L=1),             # no room for them: dropped
+], ids=lambda kw: "-".join(f"{k}{v}" for k, v in kw.items()))
+def test_co_resident_warps_edge_shapes(kw):
+    base = dict(name="co_edge", routing_seed=5, data_seed=6, TP=1, EP=1, L=1)
+    base.update(kw)
+    w = replace(wl.TINY, **base)
+    _check_against_oracle(w, drain_help=1, co_warps=2)
+    _check_against_oracle(w, drain_help=1, co_warps=1, force_C=3)
+
+
+def test_dsv2lite_with_co_resident_warps_sampled():
+    _check_against_oracle(wl.DSV2L, n_random=96, co_warps=2)
+
+
 def test_pair_tiles_against_oracle():
     for kw in (dict(T=777, E=5, k=2, H=1536, I=512, TP=2, EP=3, L=4),      # partial n-tile at the split end
                dict(T=300, E=3, k=1, H=256, I=64, TP=1, EP=1, L=1),         # m-tiles with an empty second half
@@ -267,7 +311,16 @@ def test_argument_validation():
     occ, lim, rho = B.moe_query_occupancy(h, w.tile_m, w.tile_n)
     xd, Wd, wd = x.cuda(), W2.cuda(), torch.from_numpy(wt).cuda()
     args = lambda p, xx=xd: (h, xx, Wd, None, wd, shape, occ, ws.routing, S, p, ws.out, ws.y_ws, ws.flags_ws, ws.status)
-    bad = B.moe_plan.from_buffer_copy(plan); bad.comm_ctas = 0
+    # no communication CTA at all is only legal when the compute CTAs serve the communication work themselves
+    bad = B.moe_plan.from_buffer_copy(plan); bad.comm_ctas = 0; bad.R = 0; bad.drain_help = 0
+    with pytest.raises(B.MoeError) as e:
+        B.moe_gemm2_combine(*args(bad))
+    assert e.value.code == B.MOE_ERR_PLAN_INFEASIBLE
+    bad = B.moe_plan.from_buffer_copy(plan); bad.comm_ctas = -1
+    with pytest.raises(B.MoeError) as e:
+        B.moe_gemm2_combine(*args(bad))
+    assert e.value.code == B.MOE_ERR_PLAN_INFEASIBLE
+    bad = B.moe_plan.from_buffer_copy(plan); bad.co_warps = 5     # more co-resident warps than a CTA has
     with pytest.raises(B.MoeError) as e:
         B.moe_gemm2_combine(*args(bad))
     assert e.value.code == B.MOE_ERR_PLAN_INFEASIBLE

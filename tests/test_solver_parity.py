@@ -36,7 +36,7 @@ def _same(plan, sel):
     assert (plan.comm_ctas, plan.R, plan.P) == (sel["comm_ctas"], sel["R"], sel["P"])
     assert (plan.W_comp, plan.W_comm, plan.delta) == (sel["W_comp"], sel["W_comm"], sel["delta"])
     assert plan.pred_T_q == sel["T_q"] and plan.rho_q == sel["rho_q"]
-    assert plan.mode == B.MOE_MODE_FUSED and plan.debug_withhold_tile == -1 and plan.reserved == 0
+    assert plan.mode == B.MOE_MODE_FUSED and plan.debug_withhold_tile == -1 and plan.co_warps == 0
 
 
 def _rand_inputs(rng):
