@@ -327,8 +327,10 @@ def simulate_drain_help(C: int, Wc: int, Wm: int, L: int, P: int, helpers: int, 
 #   * the unit of communication capacity is a WARP.  A dedicated communication CTA is `warps_cta` warps;
 #     a compute CTA carries w co-resident communication warps (the second decision variable) and turns
 #     into `warps_cta` communication warps once its GEMM tiles are done (drain help);
-#   * a communication tile is `warps_cta` quanta, one per warp of a dedicated CTA, so that a dedicated CTA
-#     still serves a tile in rho compute waves (Eq. 10 with quanta and warps in place of tiles and CTAs);
+#   * a communication tile is handed out in `quanta_tile` pieces ("quanta": one per warp of a dedicated CTA
+#     under the static map, one per token of the tile under the kernels' dynamic hand-out); one warp serves a
+#     quantum in rho * warps_cta / quanta_tile, so that a dedicated CTA still serves a tile in rho compute
+#     waves (Eq. 10 with quanta and warps in place of tiles and CTAs);
 #   * bandwidth-coupled service rate: N warps streaming together are limited by HBM once N exceeds `n_sat`
 #     (the warp count whose aggregate demand equals the measured copy bandwidth); the time of one quantum is
 #     rho(N) = rho * max(N, n_sat) / n_sat (rounded up in fixed point);
@@ -353,16 +355,24 @@ def coupled_service(rho_q: int, quanta: int, n_workers: int, n_sat: int) -> int:
 
 
 def makespan_co_resident(C: int, w: int, Wc: int, Wm: int, L: int, G: int, o_comp: int, o_comm: int, rho_q: int,
-                         slot_sms: int, warps_cta: int, n_sat: int, beta_q: int, gamma_q: int, order_q: int):
-    """T(C, w) for the co-resident family with drain help, fixed point.  Returns
-    (T_q, Delta_comp, R, P) or None when P(C) <= 0."""
+                         slot_sms: int, warps_cta: int, n_sat: int, beta_q: int, gamma_q: int, order_q: int,
+                         quanta_tile: int = 0):
+    """T(C, w) for the co-resident family with drain help, fixed point.  `quanta_tile` = pieces a
+    communication tile is handed out in (0: one per warp of a dedicated CTA, `warps_cta`; the dynamic
+    hand-out of the kernels gives out single tokens of a tile, T_M^comm pieces): one warp serves one piece in
+    rho * warps_cta / quanta_tile (rounded down in fixed point), so that a dedicated CTA still serves a tile
+    in rho.  Returns (T_q, Delta_comp, R, P) or None when P(C) <= 0."""
     R = reservation(C, o_comm)
     P = compute_capacity(C, G, o_comp, o_comm, slot_sms)
     if P <= 0:
         return None
+    if quanta_tile > 0:
+        rho_q = rho_q * warps_cta // quanta_tile               # service time of one piece by one warp
+    else:
+        quanta_tile = warps_cta
     n_sm = P * slot_sms // o_comp                              # SMs that compute
     tau_q = RHO_ONE + w * beta_q + (order_q if (w > 0 and L > 1) else 0)     # one compute wave
-    Wq = Wm * warps_cta                                        # quanta per split
+    Wq = Wm * quanta_tile                                      # quanta per split
     n_early = C * warps_cta + w * n_sm                         # warps that serve while the GEMM runs
     n_eff = C * warps_cta + (w * n_sm * RHO_ONE) // gamma_q    # ... in dedicated-warp equivalents
     A_last = ceil_div(L * Wc, P) * tau_q
@@ -385,7 +395,7 @@ def makespan_co_resident(C: int, w: int, Wc: int, Wm: int, L: int, G: int, o_com
 def select_co_resident(Wc: int, Wm: int, L: int, G: int, o_comp: int, o_comm: int, C_max: int, rho_q: int,
                        slot_sms: int, w_max: int, C_co_max: int, warps_cta: int, n_sat: int, beta_q: int,
                        gamma_q: int, order_q: int, force_comm_ctas: int = 0, selector_off: bool = False,
-                       default_C: int = 3, force_co_warps: int = -1) -> dict:
+                       default_C: int = 3, force_co_warps: int = -1, quanta_tile: int = 0) -> dict:
     """Algorithm 1 over the product set: C in 1..C_max with w = 0, and C in 1..min(C_max, C_co_max) with
     w in 1..w_max (a one-time characterisation bounds the dedicated CTAs worth trying beside co-resident
     warps, as the paper's C <= 16 does for its family).  Lexicographic minimum of (T, Delta_comp, w, C).
@@ -402,7 +412,7 @@ def select_co_resident(Wc: int, Wm: int, L: int, G: int, o_comp: int, o_comm: in
     for w in ws:
         for C in (Cs0 if w == 0 else Cs1):
             m = makespan_co_resident(C, w, Wc, Wm, L, G, o_comp, o_comm, rho_q, slot_sms, warps_cta, n_sat,
-                                     beta_q, gamma_q, order_q)
+                                     beta_q, gamma_q, order_q, quanta_tile)
             if m is None:
                 continue
             key = (m[0], m[1], w, C)
@@ -414,7 +424,8 @@ def select_co_resident(Wc: int, Wm: int, L: int, G: int, o_comp: int, o_comm: in
 
 
 def simulate_co_resident(C: int, w: int, Wc: int, Wm: int, L: int, P: int, n_sm: int, rho: Fraction,
-                         warps_cta: int, n_sat: int, beta: Fraction, gamma: Fraction, order: Fraction) -> dict:
+                         warps_cta: int, n_sat: int, beta: Fraction, gamma: Fraction, order: Fraction,
+                         quanta_tile: int = 0) -> dict:
     """Event-by-event simulation of the schedule makespan_co_resident stands for (no closed form):
       * P compute slots take tiles round-robin, a tile takes tau = 1 + w*beta (+ order when w > 0 and L > 1);
       * while the GEMM runs, split s (once published, and after split s-1) is served in waves of at most
@@ -424,6 +435,10 @@ def simulate_co_resident(C: int, w: int, Wc: int, Wm: int, L: int, P: int, n_sm:
         which n warps stream together takes rho * max(n, n_sat) / n_sat.
     As with simulate_drain_help the closed form can only over-estimate (it counts an open wave in full)."""
     rho, beta, gamma, order = Fraction(rho), Fraction(beta), Fraction(gamma), Fraction(order)
+    if quanta_tile > 0:
+        rho = rho * warps_cta / quanta_tile        # one warp, one quantum
+    else:
+        quanta_tile = warps_cta
     tau = 1 + w * beta + (order if (w > 0 and L > 1) else 0)
     clock = [Fraction(0)] * P
     tile_end = []
@@ -433,7 +448,7 @@ def simulate_co_resident(C: int, w: int, Wc: int, Wm: int, L: int, P: int, n_sm:
         tile_end.append(clock[b])
     publish = [max(tile_end[s * Wc:(s + 1) * Wc]) if Wc > 0 else Fraction(0) for s in range(L)]
     A = publish[L - 1]
-    Wq = Wm * warps_cta
+    Wq = Wm * quanta_tile
     n_early = C * warps_cta + w * n_sm
     n_eff = C * warps_cta + int(Fraction(w * n_sm) / gamma)
     pool = Wq

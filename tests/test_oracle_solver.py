@@ -353,10 +353,11 @@ def _parse_family_golden(path):
             continue
         kind, name, rest = line.split(None, 2)
         parts = [p.split() for p in rest.split("|")]
-        if kind == "co":
+        if kind in ("co", "coq"):
             a, t = parts
             cos.append((name, [int(v) for v in a[:9]], Fraction(a[9]), int(a[10]), int(a[11]),
-                        Fraction(a[12]), Fraction(a[13]), Fraction(a[14]), Fraction(t[0])))
+                        Fraction(a[12]), Fraction(a[13]), Fraction(a[14]), Fraction(t[0]),
+                        int(a[15]) if kind == "coq" else 0))
         elif kind == "tile":
             a, idx, gpu, pts = parts
             tiles.append((name, [int(v) for v in a[0].split(",")], [int(v) for v in a[1:]],
@@ -373,13 +374,13 @@ def _q(x):
 
 def test_co_resident_hand_worked_values(golden_dir):
     cos, _ = _parse_family_golden(os.path.join(golden_dir, "rho_local_worked.txt"))
-    assert len(cos) >= 3
-    for name, (G, o_comp, o_comm, slot, C, w, Wc, Wm, L), rho, warps_cta, n_sat, beta, gamma, order, want in cos:
+    assert len(cos) >= 4
+    for name, (G, o_comp, o_comm, slot, C, w, Wc, Wm, L), rho, warps_cta, n_sat, beta, gamma, order, want, qt in cos:
         m = sr.makespan_co_resident(C, w, Wc, Wm, L, G, o_comp, o_comm, _q(rho), slot, warps_cta, n_sat,
-                                    _q(beta), _q(gamma), _q(order))
+                                    _q(beta), _q(gamma), _q(order), qt)
         assert Fraction(m[0], sr.RHO_ONE) == want, (name, Fraction(m[0], sr.RHO_ONE))
         P = sr.compute_capacity(C, G, o_comp, o_comm, slot)
-        sim = sr.simulate_co_resident(C, w, Wc, Wm, L, P, P * slot // o_comp, rho, warps_cta, n_sat, beta, gamma, order)
+        sim = sr.simulate_co_resident(C, w, Wc, Wm, L, P, P * slot // o_comp, rho, warps_cta, n_sat, beta, gamma, order, qt)
         assert sim["T"] <= want
 
 
@@ -428,22 +429,29 @@ def test_co_resident_model_reductions_and_simulation():
         w = rng.randint(0, 3)
         n_sat = rng.choice([3, 17, 200, 10 ** 6])
         beta, gamma, order = Fraction(rng.randint(0, 8), 64), Fraction(rng.randint(4, 16), 4), Fraction(rng.randint(0, 4), 32)
-        m = sr.makespan_co_resident(C, w, Wc, Wm, L, G, o_comp, 1, _q(rho), slot, warps_cta, n_sat, _q(beta), _q(gamma), _q(order))
+        qt = rng.choice([0, 0, warps_cta, 4 * warps_cta, 128])     # pieces a tile is handed out in (0: one per warp)
+        m = sr.makespan_co_resident(C, w, Wc, Wm, L, G, o_comp, 1, _q(rho), slot, warps_cta, n_sat, _q(beta), _q(gamma), _q(order), qt)
         tau = 1 + w * beta + (order if (w > 0 and L > 1) else 0)
         n_tail = (C + n_sm) * warps_cta + w * n_sm
+        rho_u = _q(rho) * warps_cta // qt if qt else _q(rho)
+        if qt in (0, warps_cta):          # one piece per warp of a dedicated CTA: the same model either way
+            assert m == sr.makespan_co_resident(C, w, Wc, Wm, L, G, o_comp, 1, _q(rho), slot, warps_cta, n_sat, _q(beta),
+                                                _q(gamma), _q(order), warps_cta - qt)
         # (b) L = 1: one compute phase stretched by the co-resident warps, then every warp serves the only split
         if L == 1:
-            assert m[0] == sr.ceil_div(Wc, P) * _q(tau) + sr.coupled_service(_q(rho), Wm * warps_cta, n_tail, n_sat)
+            assert m[0] == sr.ceil_div(Wc, P) * _q(tau) + sr.coupled_service(rho_u, Wm * (qt or warps_cta), n_tail, n_sat)
         # (c) the event simulation of the same schedule: the closed form never under-estimates it (up to the
         # rounding of rho(N) to 2^-20), and equals it when no early wave is open at the end of the GEMM
-        sim = sr.simulate_co_resident(C, w, Wc, Wm, L, P, n_sm, rho, warps_cta, n_sat, beta, gamma, order)
+        sim = sr.simulate_co_resident(C, w, Wc, Wm, L, P, n_sm, rho, warps_cta, n_sat, beta, gamma, order, qt)
         T_model = Fraction(m[0], sr.RHO_ONE)
-        assert sim["T"] <= T_model + Fraction(L * Wm * warps_cta + 8, sr.RHO_ONE)
-        if not sim["open_at_A"]:
-            assert abs(sim["T"] - T_model) <= Fraction(L * Wm * warps_cta + 8, sr.RHO_ONE)
-            n_exact += 1
+        slack = Fraction(L * Wm * (qt or warps_cta) + 8, sr.RHO_ONE)     # roundings of rho(N) and of rho per piece to 2^-20
+        if qt == 0 or (_q(rho) * warps_cta) % qt == 0:
+            assert sim["T"] <= T_model + slack
+            if not sim["open_at_A"]:
+                assert abs(sim["T"] - T_model) <= slack
+                n_exact += 1
         # (d) more co-resident warps never lengthen the tail's service and never shorten the compute phase
-        m2 = sr.makespan_co_resident(C, w + 1, Wc, Wm, L, G, o_comp, 1, _q(rho), slot, warps_cta, n_sat, _q(beta), _q(gamma), _q(order))
+        m2 = sr.makespan_co_resident(C, w + 1, Wc, Wm, L, G, o_comp, 1, _q(rho), slot, warps_cta, n_sat, _q(beta), _q(gamma), _q(order), qt)
         assert sr.ceil_div(L * Wc, P) * _q(tau) <= m[0] and m2[1:] == m[1:]
     assert n_exact > 300
 
