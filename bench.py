@@ -42,6 +42,20 @@ def load_peaks():
     return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
 
 
+def config_of(w, info, world):
+    """The `config` object of the JSON line: the same dict in the main arm and in the reference arm."""
+    x_mb, w2_mb = w.R * w.I * 2 / 1e6, w.E_tot * w.H * w.I * 2 / 1e6
+    y_mb = w.T * w.L * w.k_tot * w.TP * (-(-w.H // w.L)) * 2 / 1e6
+    return {"workload": w.name, "T": w.T, "H": w.H, "I": w.I, "E": w.E, "k": w.k,
+            "n_shared": w.n_shared, "TP": w.TP, "EP": w.EP, "tile": f"{w.tile_m}x{w.tile_n}",
+            "L": w.L, "routing": f"{w.routing} s={w.zipf_s}", "r_expert": info["r_expert"],
+            "p90_ratio": info["p90_ratio"],
+            "l2": f"inputs larger than L2 (x {x_mb:.0f} MB, W2 {w2_mb:.0f} MB, Y {y_mb:.0f} MB vs 126 MB)"
+                  if x_mb + w2_mb + y_mb > 252 else
+                  f"inputs x {x_mb:.0f} MB, W2 {w2_mb:.0f} MB, Y {y_mb:.0f} MB; a 256 MB buffer is written between timed steps to flush L2",
+            "replicas": "independent per GPU, no collective" if world > 1 else "single GPU"}
+
+
 # ----------------------------------------------------------------------------- replicas
 
 def max_over_ranks(values, world, device="cpu"):
@@ -59,6 +73,21 @@ def max_over_ranks(values, world, device="cpu"):
 def job_value(us_per_layer_slowest_rank, world):
     """N independent replicas finish N layers in the time of the slowest one: us per layer of the whole job."""
     return us_per_layer_slowest_rank / max(1, world)
+
+
+# ----------------------------------------------------------------------------- roofline denominator
+
+def tensor_peak_for(peaks, loop_seconds, clocks):
+    """Which measured cuBLAS figure a tensor-bound kernel is set against.  The burst figure (a kernel timed
+    alone, clocks at their maximum) unless the timed loop itself lasted at least a second AND the SM clock
+    sampled during it sat below 0.9 of its maximum (the power-capped steady state the sustained figure was
+    measured in).  Returns (TFLOP/s, the rule spelled out with the run's own numbers)."""
+    sust = peaks.get("bf16_tflops_sustained")
+    mhz, mx = (clocks or {}).get("sm_mhz"), (clocks or {}).get("sm_max_mhz")
+    capped = bool(sust) and loop_seconds >= 1.0 and mhz is not None and mx and mhz < 0.9 * mx
+    why = (f"timed loop {loop_seconds:.3f} s, median SM clock {mhz} of {mx} MHz -> "
+           + ("sustained figure (loop >= 1 s and clock < 0.9 max)" if capped else "burst figure (a loop shorter than 1 s, or a clock at >= 0.9 max)"))
+    return (sust if capped else peaks["bf16_tflops"]), why
 
 
 # ----------------------------------------------------------------------------- clocks
@@ -155,8 +184,10 @@ def make_stepper(h, dw, limits_override=None):
     stream = torch.cuda.current_stream()
     E = w.E_tot
 
+    w_default = lim.force_co_warps
+
     def step(force_C=0, mode=B.MOE_MODE_FUSED, ev_before=None, ev_after=None, P_override=None,
-             C_override=None, reuse=None):
+             C_override=None, reuse=None, force_w=None):
         if reuse is None:
             B.moe_build_routing(h, dw.idx_d, dw.shape, w.tile_m, ws.routing, ws.tile_counts, ws.status)
             stream.synchronize()                               # tile counts are on the host now
@@ -164,7 +195,9 @@ def make_stepper(h, dw, limits_override=None):
         else:                                                  # sweeps: routing already built
             counts = reuse
         lim.force_comm_ctas = force_C
+        lim.force_co_warps = w_default if force_w is None else force_w
         plan = B.plan_partition(counts[:E], occ, lim, dw.shape, rho)
+        lim.force_co_warps = w_default
         plan.mode = mode
         if P_override is not None:
             plan.P = P_override
@@ -195,43 +228,49 @@ def time_fused(step, torch, force_C, n_warm, n_samples, **kw):
 # Section IV-B: the measured oracle is the C with the lowest median latency over a sweep of every
 # legal C; regret = (T_pick - T_best) / T_best.
 
-def time_all_C(step, torch, counts, C_list, n_warm=1, n_samples=5):
-    """Median fused-kernel time [us] for every C in C_list (routing is reused).  The candidates are
+def time_all_C(step, torch, counts, cands, n_warm=1, n_samples=5):
+    """Median fused-kernel time [us] for every candidate (C, w) (routing is reused).  The candidates are
     interleaved: every round visits all of them in a fresh seeded random order, so that slow drifts
-    of the GPU's state (power capping sets in after a second or two of load) hit every C alike."""
+    of the GPU's state (power capping sets in after a second or two of load) hit every candidate alike."""
     import random
     rng = random.Random(1234)
-    order = list(C_list)
+    order = list(cands)
     for _ in range(n_warm):
-        for C in order:
-            step(C, reuse=counts)
-    samples = {C: [] for C in order}
+        for C, w in order:
+            step(C, reuse=counts, force_w=w)
+    samples = {c: [] for c in order}
     evs = []
     for _ in range(n_samples):
         rng.shuffle(order)
-        for C in order:
+        for C, w in order:
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            step(C, ev_before=a, ev_after=b, reuse=counts)
-            evs.append((C, a, b))
+            step(C, ev_before=a, ev_after=b, reuse=counts, force_w=w)
+            evs.append(((C, w), a, b))
     torch.cuda.synchronize()
-    for C, a, b in evs:
-        samples[C].append(a.elapsed_time(b) * 1e3)
-    return {C: statistics.median(v) for C, v in samples.items()}
+    for c, a, b in evs:
+        samples[c].append(a.elapsed_time(b) * 1e3)
+    return {c: statistics.median(v) for c, v in samples.items()}
 
 
-def regret_of_workload(step, torch, counts, lim, picked_C, n_warm=1, n_samples=5, C_hi=None, keep_curve=True):
-    """Times every C of the legal set {1..C_max} (or up to C_hi) and compares the analytical pick."""
+def regret_of_workload(step, torch, counts, lim, picked, n_warm=1, n_samples=5, C_hi=None, keep_curve=True):
+    """Times every member of the legal set -- C in 1..C_max without co-resident warps and, where the kernel
+    family has them (drain help), C in 1..C_co_max with w in 1..co_warps_max -- and compares the analytical
+    pick `picked` = (C, w)."""
     C_hi = C_hi or lim.C_max
-    Cs = sorted(set(list(range(1, C_hi + 1)) + [picked_C]))
-    times = time_all_C(step, torch, counts, Cs, n_warm, n_samples)
-    best_C = min(times, key=times.get)
-    t_best, t_pick = times[best_C], times[picked_C]
-    out = {"picked_C": picked_C, "t_pick_us": t_pick, "best_C": best_C, "t_best_us": t_best,
-           "regret": (t_pick - t_best) / t_best,
-           "regret_static_C3": (times[3] - t_best) / t_best if 3 in times else None,
-           "swept_C": [1, C_hi], "samples_per_C": n_samples}
+    cands = {(C, 0) for C in range(1, C_hi + 1)}
+    if lim.drain_help and lim.co_warps_max > 0:
+        cands |= {(C, w) for C in range(1, min(C_hi, lim.C_co_max) + 1) for w in range(1, lim.co_warps_max + 1)}
+    cands.add(tuple(picked))
+    times = time_all_C(step, torch, counts, sorted(cands), n_warm, n_samples)
+    best = min(times, key=times.get)
+    t_best, t_pick = times[best], times[tuple(picked)]
+    out = {"picked_C": picked[0], "picked_w": picked[1], "t_pick_us": t_pick, "best_C": best[0], "best_w": best[1],
+           "t_best_us": t_best, "regret": (t_pick - t_best) / t_best,
+           "regret_static_C3": (times[(3, 0)] - t_best) / t_best if (3, 0) in times else None,
+           "best_without_co_warps_us": min(t for (C, w), t in times.items() if w == 0),
+           "swept_C": [1, C_hi], "candidates": len(times), "samples_per_C": n_samples}
     if keep_curve:
-        out["times_us"] = {str(c): round(t, 1) for c, t in times.items()}
+        out["times_us"] = {f"{c}" if w == 0 else f"{c}w{w}": round(t, 1) for (c, w), t in times.items()}
     return out
 
 
@@ -248,30 +287,44 @@ def run_sweep(h, args, peaks):
         dw = DeviceWorkload(w, device, data="device")
         row = dict(name=w.name, T=w.T, zipf_s=w.zipf_s, EP=w.EP, tile=f"{w.tile_m}x{w.tile_n}", L=w.L,
                    r_expert=dw.info["r_expert"])
-        for dh in (0, 1):
-            step, (occ, lim, rho) = make_stepper(h, dw, limits_override=dict(drain_help=dh))
+        for dh in ((0,) if args.sweep_modes == "static" else (1,) if args.sweep_modes == "drain_help" else (0, 1)):
+            step, (occ, lim, rho) = make_stepper(h, dw, limits_override=dict(drain_help=dh, dep_model=args.dep_model))
             plan, counts = step()
             torch.cuda.synchronize()
-            r = regret_of_workload(step, torch, counts, lim, plan.comm_ctas, n_warm=1, n_samples=args.sweep_samples,
-                                   keep_curve=args.sweep_curves)
+            r = regret_of_workload(step, torch, counts, lim, (plan.comm_ctas, plan.co_warps), n_warm=1,
+                                   n_samples=args.sweep_samples * (2 if w.T <= 4096 else 1) + (1 if w.T <= 4096 else 0),
+                                   keep_curve=args.sweep_curves)   # short launches are noisier: twice the samples
             r.update(W_comp=plan.W_comp, W_comm=plan.W_comm, rho=plan.rho_q / 2 ** 20,
                      roofline_frac=(dw.flops / peaks["bf16_tflops"] / 1e6) / r["t_pick_us"])
             row["static" if dh == 0 else "drain_help"] = r
         results.append(row)
+        if "static" not in row or "drain_help" not in row:
+            k = "static" if "static" in row else "drain_help"
+            print(f"{w.name}: {k} pick C={row[k]['picked_C']} w={row[k]['picked_w']} {row[k]['t_pick_us']:.0f} us best C={row[k]['best_C']} "
+                  f"w={row[k]['best_w']} {row[k]['t_best_us']:.0f} us regret {100 * row[k]['regret']:.1f}%", flush=True)
+            del dw, step
+            torch.cuda.empty_cache()
+            continue
         a, b = row["static"], row["drain_help"]
         print(f"{w.name}: static pick C={a['picked_C']} {a['t_pick_us']:.0f} us best C={a['best_C']} {a['t_best_us']:.0f} us "
               f"regret {100 * a['regret']:.1f}% (C=3: {100 * a['regret_static_C3']:.0f}%) | drain-help pick C={b['picked_C']} "
-              f"{b['t_pick_us']:.0f} us best C={b['best_C']} {b['t_best_us']:.0f} us regret {100 * b['regret']:.1f}%", flush=True)
+              f"w={b['picked_w']} {b['t_pick_us']:.0f} us best C={b['best_C']} w={b['best_w']} {b['t_best_us']:.0f} us "
+              f"regret {100 * b['regret']:.1f}%", flush=True)
         del dw, step
         torch.cuda.empty_cache()
     summary = {"n": len(results)}
     for key in ("static", "drain_help"):
-        regs = [r[key]["regret"] for r in results]
+        regs = [r[key]["regret"] for r in results if key in r]
         if regs:
+            rows = [r[key] for r in results if key in r]
             summary[key] = {"mean_regret": statistics.mean(regs), "max_regret": max(regs),
-                            "mean_regret_static_C3": statistics.mean(r[key]["regret_static_C3"] for r in results),
+                            "mean_regret_static_C3": statistics.mean(r["regret_static_C3"] for r in rows),
                             "geomean_speedup_pick_over_C3": statistics.geometric_mean(
-                                (1 + r[key]["regret_static_C3"]) / (1 + r[key]["regret"]) for r in results)}
+                                (1 + r["regret_static_C3"]) / (1 + r["regret"]) for r in rows),
+                            "picks_with_co_warps": sum(1 for r in rows if r["picked_w"] > 0),
+                            "best_with_co_warps": sum(1 for r in rows if r["best_w"] > 0),
+                            "geomean_best_over_best_without_co_warps": statistics.geometric_mean(
+                                r["t_best_us"] / r["best_without_co_warps_us"] for r in rows)}
     os.makedirs(os.path.dirname(args.sweep_out) or ".", exist_ok=True)
     json.dump({"summary": summary, "results": results}, open(args.sweep_out, "w"))
     print(json.dumps({"sweep_summary": summary}))
@@ -294,6 +347,90 @@ def calibrate(h, device, C_ref=32, tile=(128, 256)):
         "us_per_compute_wave": wave_comp, "us_per_comm_wave": wave_comm,
         "rho_ref": rho.rho_ref, "K_ref": rho.K_ref, "tile_ref": [rho.tile_m_ref, rho.tile_n_ref],
         "rows_ref": rho.rows_ref, "comm_cols_ref": rho.comm_cols_ref, "D_ref": rho.D_ref}}))
+
+
+# ----------------------------------------------------------------------------- other workloads, briefly
+
+def all_traffic_bytes(w, x_passes=1):
+    """Every byte one launch has to move through HBM: x (once per pass), W2, Y written and read back, out."""
+    return (w.R * w.I * 2 * x_passes + w.E_tot * w.H * w.I * 2 +
+            2 * w.T * w.L * w.k_tot * w.TP * (-(-w.H // w.L)) * 2 + w.T * w.H * 2)
+
+
+def quick_config(h, w, device, peaks, steps=30, warm=5):
+    """A bounded measurement of one more workload (a second or two): the whole step timed like the headline
+    one (K moe_layer calls between two events), the fused kernel by events around its launch.  Fractions
+    against the headline roofline (GEMM FLOPs at the burst peak -- these loops last milliseconds -- or combine
+    bytes at the copy bandwidth, whichever is slower) and against the time all of the launch's HBM traffic needs."""
+    import torch
+    dw = DeviceWorkload(w, device, data="device")
+    B = dw.B
+    occ, lim, rho = B.moe_query_occupancy(h, w.tile_m, w.tile_n)
+    layer = B.LayerCall(h, dw.x, dw.W2, dw.idx_d, dw.wt_d, dw.ws, limits=lim)
+    for _ in range(warm):
+        plan = layer()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for a, b in evs:
+        a.record(); b.record()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    t0.record()
+    for a, b in evs:
+        plan = layer(a, b)
+    t1.record()
+    torch.cuda.synchronize()
+    assert B.moe_get_status(h, dw.ws.status).code == 0
+    fused = statistics.median(a.elapsed_time(b) * 1e3 for a, b in evs)
+    step_us = t0.elapsed_time(t1) * 1e3 / steps
+    t_flops = dw.flops / peaks["bf16_tflops"] / 1e6
+    t_comb = dw.combine_bytes / peaks["hbm_gbs"] / 1e3
+    t_all = all_traffic_bytes(w) / peaks["hbm_gbs"] / 1e3
+    roof = max(t_flops, t_comb)
+    out = {"workload": w.name, "T": w.T, "tile": f"{w.tile_m}x{w.tile_n}", "L": w.L, "steps": steps,
+           "plan": {"comm_ctas": plan.comm_ctas, "P": plan.P, "co_warps": plan.co_warps},
+           "step_us": step_us, "fused_kernel_us": fused, "tflops": dw.flops / fused / 1e6,
+           "roofline_us": roof, "roofline_bound": "tensor" if t_flops >= t_comb else "hbm", "roofline_frac": roof / fused,
+           "hbm_all_traffic_us": t_all, "frac_of_all_traffic_bound": t_all / fused,
+           "bound_us": max(roof, t_all), "frac_of_bound": max(roof, t_all) / fused,
+           "r_expert": dw.info["r_expert"]}
+    del dw, layer
+    torch.cuda.empty_cache()
+    return out
+
+
+DECODE_T = (16, 64, 256, 1024)
+
+
+def run_decode(h, args, device, peaks):
+    """--workload dsv2lite_decode: decode-sized token counts on the DeepSeek-V2-Lite shape, tile family chosen
+    by moe_select_tile.  At these sizes every expert's W2 slice is read for a handful of rows: the bound is the
+    time all HBM traffic of a launch needs (W2 dominates), not the FLOPs or the combine bytes."""
+    from dataclasses import replace
+    from paper_2609_07536_b200 import binding as B
+    from paper_2609_07536_b200 import workloads as wl
+    rows = []
+    for T in DECODE_T:
+        w = replace(wl.DSV2L, name=f"dsv2lite_decode_T{T}", T=T)
+        shape = B.make_shape(w.T, w.H, w.I, w.E_tot, w.k_tot, w.TP, w.EP, w.L)
+        tm, tn = B.moe_select_tile(h, shape)
+        rows.append(quick_config(h, replace(w, tile_m=tm, tile_n=tn), device, peaks, steps=max(20, args.steps), warm=max(3, args.warmup)))
+    main = rows[2]   # T = 256
+    w = replace(wl.DSV2L, name="dsv2lite_decode", T=main["T"])
+    idx, wt, info = wl.make_routing(w)
+    print(json.dumps({
+        "metric": METRIC, "value": main["step_us"], "unit": "us/layer", "n_gpus": 1, "steps": main["steps"],
+        "warmup": max(3, args.warmup), "ms_per_step": main["step_us"] / 1e3, "higher_is_better": False, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": dict(config_of(replace(w, tile_m=int(main["tile"].split("x")[0]), tile_n=int(main["tile"].split("x")[1])), info, 1),
+                       T_list=list(DECODE_T), value_is_for_T=main["T"]),
+        "roofline": {"bound": "hbm", "achieved": all_traffic_bytes(w) / main["fused_kernel_us"] / 1e3, "peak": peaks["hbm_gbs"],
+                     "unit": "GB/s", "frac": main["frac_of_all_traffic_bound"], "traffic": None,
+                     "peak_source": peaks["source"] + ": copy bandwidth; bytes = ALL HBM traffic of a launch (x, W2, Y written "
+                                    "and read back, out): at decode sizes the weights dominate, the headline roofline "
+                                    "(FLOPs or combine bytes) does not bound these launches",
+                     "kernel": "moe_gemm2_combine_kernel", "kernel_us": main["fused_kernel_us"]},
+        "decode": rows, "cpu_baseline": None, "e2e": None, "gpu_launches": 5 * main["steps"],
+    }))
 
 
 # ----------------------------------------------------------------------------- per-CTA timeline
@@ -504,12 +641,16 @@ def reference_arm(args):
             vals.append(base["value"])
     v = statistics.median(vals)
     base["value"] = v
+    base["extrapolated"] = True
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": v, "unit": "us/layer", "n_gpus": args.gpus,
         "steps": steps, "warmup": warm, "ms_per_step": v / 1e3, "higher_is_better": False,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": w.name, "T": w.T, "H": w.H, "I": w.I, "E": w.E, "k": w.k,
-                   "n_shared": w.n_shared, "TP": w.TP, "EP": w.EP},
+        "config": config_of(w, info, int(os.environ.get("WORLD_SIZE", "1"))),
+        "extrapolated": True,
+        "note": "each of the `steps` steps times the oracle on a bounded seeded token sample and scales it by T/n "
+                "(`cpu_baseline.sample` says how many tokens the last one ran); value and ms_per_step are that "
+                "extrapolation to a whole layer, not the wall time of a step",
         "cpu_baseline": base,
         "e2e": {"value": v, "unit": "us/layer", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
@@ -540,6 +681,7 @@ def main():
     ap.add_argument("--sweep-filter", default="", help="substring a sweep workload name must contain")
     ap.add_argument("--sweep-curves", action="store_true", help="keep every t(C) in the sweep output")
     ap.add_argument("--sweep-samples", type=int, default=5, help="timed samples per C in the sweep")
+    ap.add_argument("--sweep-modes", default="both", choices=["both", "static", "drain_help"])
     ap.add_argument("--counts", default="host", choices=["host", "device"],
                     help="host: tile counts copied to the host, exact plan (default); device: no copy and no wait, "
                          "plan from the normalised-load estimate (Section III-E)")
@@ -547,6 +689,8 @@ def main():
                     help="co-resident communication warps per compute CTA (-1: the selector decides)")
     ap.add_argument("--no-comm-ctas", action="store_true",
                     help="with --only fused: launch without any dedicated communication CTA (C = 0, every SM computes)")
+    ap.add_argument("--dep-model", type=int, default=0, choices=[0, 1],
+                    help="static partition: 0 = readiness per split (Eq. 9 as printed), 1 = per communication tile")
     ap.add_argument("--drain-help", type=int, default=1, choices=[0, 1],
                     help="1 (default): compute CTAs help with the communication tail; 0: the paper's static partition")
     ap.add_argument("--timeline", action="store_true",
@@ -585,6 +729,10 @@ def main():
         tile = tuple(int(v) for v in args.tile.split("x")) if args.tile else (128, 256)
         return calibrate(h, device, tile=tile)
 
+    if args.workload == "dsv2lite_decode":
+        run_decode(h, args, device, peaks)
+        B.moe_destroy(h)
+        return
     w = wl.CONFIGS[args.workload]
     if args.tile:
         from dataclasses import replace
@@ -711,13 +859,13 @@ def main():
                                  "frac_of_hbm_peak": dw.combine_bytes / comb_only / 1e3 / peaks["hbm_gbs"], "C": lim_all}
         # ---- selector regret on this workload: every feasible C timed
         if not args.no_regret:
-            extra["regret"] = regret_of_workload(step, torch, counts, lim, plan.comm_ctas, n_warm=1, n_samples=5)
+            extra["regret"] = regret_of_workload(step, torch, counts, lim, (plan.comm_ctas, plan.co_warps), n_warm=1, n_samples=5)
             # the paper's static partition on the same workload: its pick, its sweep, its regret
             step0, (occ0, lim0, rho0) = make_stepper(h, dw, limits_override=dict(drain_help=1 - args.drain_help))
             lim0.force_comm_ctas = 0
             plan0 = B.plan_partition(counts[:w.E_tot], occ0, lim0, dw.shape, rho0)
             key = "regret_static_partition" if args.drain_help else "regret_drain_help"
-            extra[key] = regret_of_workload(step0, torch, counts, lim0, plan0.comm_ctas, n_warm=1, n_samples=5)
+            extra[key] = regret_of_workload(step0, torch, counts, lim0, (plan0.comm_ctas, plan0.co_warps), n_warm=1, n_samples=5)
         # ---- solver overhead: mean over >= 1e6 calls, rotating routed-count vectors
         rng = np.random.default_rng(0)
         base_counts = np.array(counts[:w.E_tot])
@@ -726,34 +874,37 @@ def main():
         extra["solver_ns"] = B.moe_time_plan_partition(sets, occ, lim, dw.shape, rho, 1_000_000)
         if not args.no_cpu_baseline:
             extra["cpu_baseline"], _ = cpu_baseline(w, dw.idx, dw.wt, dw.x_cpu, dw.W2_cpu)
+        # ---- the other named workloads, briefly (a second or two each): fused time and roofline fractions
+        if args.workload == "dsv2lite" and not args.tile and not args.T and not args.L:
+            extra["other_configs"] = [quick_config(h, wl.CONFIGS[n], device, peaks) for n in ("granite3moe", "qwen15moe")]
         # ---- the up-stream stage (next row of the scope table), reported beside the headline, not in it
         g1res = time_gemm1(h, dw, torch, cpu_rows=0 if args.no_cpu_baseline else 4096)
         g1res["frac_of_bf16_peak"] = g1res["tflops"] / peaks["bf16_tflops"]
         extra["gemm1_act"] = g1res
 
     if rank == 0:
-        # the fused kernel is timed inside the K-step loop (power-capped steady state), so its tensor
-        # denominator is the sustained cuBLAS figure; the burst figure is reported beside it
-        tf_sust = peaks.get("bf16_tflops_sustained") or peaks["bf16_tflops"]
-        t_flops_us = dw.flops / tf_sust / 1e6
+        tf_peak, tf_rule = tensor_peak_for(peaks, K * step_us / 1e6, clocks)
+        t_flops_us = dw.flops / tf_peak / 1e6
         t_hbm_us = dw.combine_bytes / peaks["hbm_gbs"] / 1e3
         tensor_bound = t_flops_us >= t_hbm_us
         ach = dw.flops / fused_med / 1e6 if tensor_bound else dw.combine_bytes / fused_med / 1e3
-        peak = tf_sust if tensor_bound else peaks["hbm_gbs"]
+        peak = tf_peak if tensor_bound else peaks["hbm_gbs"]
+        tf_sust = peaks.get("bf16_tflops_sustained") or peaks["bf16_tflops"]
         roofline = {
             "bound": "tensor" if tensor_bound else "hbm", "achieved": ach, "peak": peak,
             "unit": "TFLOP/s" if tensor_bound else "GB/s", "frac": ach / peak, "traffic": None,
-            "peak_source": peaks["source"] + (" (sustained: the kernel is timed inside the step loop)" if tensor_bound else ""),
+            "peak_source": peaks["source"] + (": " + tf_rule if tensor_bound else ": copy bandwidth"),
             "kernel": "moe_gemm2_combine_pair_kernel" if w.tile_m == 256 else "moe_gemm2_combine_kernel",
             "kernel_us": fused_med, "kernel_us_ci95": fused_ci, "roofline_us": max(t_flops_us, t_hbm_us),
             "frac_of_burst_peak": (ach / peaks["bf16_tflops"]) if tensor_bound else None,
             "burst_peak": peaks["bf16_tflops"] if tensor_bound else None,
+            "frac_of_sustained_peak": (ach / tf_sust) if tensor_bound else None,
+            "sustained_peak": tf_sust if tensor_bound else None,
         }
         # DRAM read + write bytes of one fused launch from the ncu capture summarised in
         # profiles/fused_gemm2_combine_dsv2lite_ncu.md (same workload, same launch configuration)
-        x_passes = 1 if args.drain_help else w.L      # m-tile-major order reads x once, split-major once per split
-        all_bytes = (w.R * w.I * 2 * x_passes + w.E_tot * w.H * w.I * 2 +
-                     2 * w.T * w.L * w.k_tot * w.TP * (-(-w.H // w.L)) * 2 + w.T * w.H * 2)
+        x_passes = 1 if (args.drain_help and plan.co_warps == 0) else w.L   # m-tile-major order reads x once, split-major once per split
+        all_bytes = all_traffic_bytes(w, x_passes)
         # every byte the launch has to move through HBM (x, W2, Y written and read back, out): not part of the
         # headline roofline, but the real bound at small T, where every expert's weights are read for a few rows
         roofline["hbm_all_traffic_us"] = all_bytes / peaks["hbm_gbs"] / 1e3
@@ -764,14 +915,10 @@ def main():
             "metric": METRIC, "value": job_value(step_us, world), "unit": "us/layer", "n_gpus": world, "steps": K, "warmup": W,
             "ms_per_step": step_us / 1e3, "higher_is_better": False, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": w.name, "T": w.T, "H": w.H, "I": w.I, "E": w.E, "k": w.k,
-                       "n_shared": w.n_shared, "TP": w.TP, "EP": w.EP, "tile": f"{w.tile_m}x{w.tile_n}",
-                       "L": w.L, "routing": f"{w.routing} s={w.zipf_s}", "r_expert": dw.info["r_expert"],
-                       "p90_ratio": dw.info["p90_ratio"],
-                       "l2": "inputs larger than L2 (x 369 MB, W2 381 MB, Y 1.1 GB vs 126 MB)",
-                       "replicas": "independent per GPU, no collective" if world > 1 else "single GPU"},
+            "config": config_of(w, dw.info, world),
             "plan": {"comm_ctas": plan.comm_ctas, "R": plan.R, "P": plan.P, "W_comp": plan.W_comp,
-                     "W_comm": plan.W_comm, "rho": plan.rho_q / 2 ** 20, "drain_help": plan.drain_help},
+                     "W_comm": plan.W_comm, "rho": plan.rho_q / 2 ** 20, "drain_help": plan.drain_help,
+                     "co_warps": plan.co_warps},
             "fused_kernel_us": fused_med, "tflops": dw.flops / fused_med / 1e6,
             "wall_ms_per_step": wall * 1e3 / K,
             "roofline": roofline,

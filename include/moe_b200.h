@@ -62,6 +62,7 @@ enum { MOE_MODE_FUSED = 0, MOE_MODE_GEMM_ONLY = 1, MOE_MODE_COMBINE_ONLY = 2 };
  * to the rows it moves per token (k_tot * TP read + 1 written) and to its real width
  * min(T_N^comm, ceil(H/L)). */
 enum { MOE_RHO_PAPER = 0, MOE_RHO_LOCAL = 1 };
+enum { MOE_DEP_SPLIT = 0, MOE_DEP_TILE = 1 };
 #define MOE_MAX_EP 8
 #define MOE_MAX_L 8
 #define MOE_MTILES_ON_DEVICE (-1)   /* moe_gemm2_combine: read the m-tile count from routing->tiles[E_tot] on the device */
@@ -99,6 +100,10 @@ typedef struct {
     int32_t co_warps_max;    /* upper end of the legal set {0..co_warps_max} of co-resident communication warps
                                 per compute CTA (0: a kernel family without them) */
     int32_t force_co_warps;  /* >= 0: use exactly this many (clamped to co_warps_max); < 0: the selector decides */
+    int32_t C_co_max;        /* dedicated communication CTAs tried beside co-resident warps: C in 1..min(C_max, C_co_max)
+                                for w >= 1 (a one-time characterisation, like C_max) */
+    int32_t dep_model;       /* static partition only: MOE_DEP_SPLIT = Eq. 9 as printed (one readiness per split),
+                                MOE_DEP_TILE = Eq. 9 applied to every communication tile (per-tile flags) */
 } moe_sm_limits;
 
 /* Relative wave service rate (Eq. 13-15). */
@@ -108,6 +113,21 @@ typedef struct {
     int32_t rows_ref;        /* k_tot * TP + 1 of the reference run (MOE_RHO_LOCAL only) */
     int32_t comm_cols_ref;   /* min(T_N^comm, ceil(H/L)) of the reference run (MOE_RHO_LOCAL only) */
     int32_t mode;            /* MOE_RHO_PAPER | MOE_RHO_LOCAL */
+    /* Bandwidth coupling and co-resident communication warps (this library's re-derivation for a kernel
+     * family whose communication work can share SMs with compute; used with drain_help only; all zero =
+     * the plain recurrence).  Capacity is counted in warps: a communication tile is comm_warps_per_cta
+     * quanta, a dedicated communication CTA serves comm_warps_per_cta of them per wave. */
+    int32_t comm_warps_per_cta; /* warps of a communication CTA (0: coupling and co-resident warps off) */
+    int32_t n_sat_warps;        /* warps streaming together that saturate HBM: above it one quantum takes
+                                   rho * N / n_sat_warps (0: never saturated) */
+    int32_t comm_quanta_per_tile; /* pieces a communication tile is handed out in (0: one per warp of a CTA; the
+                                   dynamic hand-out gives out single tokens: T_M^comm); one warp serves a piece in
+                                   rho * comm_warps_per_cta / comm_quanta_per_tile */
+    int32_t reserved0;
+    double co_beta;             /* one co-resident warp stretches the compute wave by this fraction */
+    double co_gamma;            /* a co-resident warp serves this many times slower than a dedicated one (>= 1) */
+    double co_order;            /* with co-resident warps and L > 1 the tile order is split-major (x is read once
+                                   per split): the compute wave is stretched by this fraction */
 } moe_rho;
 
 /* Result of the selector, and the launch description moe_gemm2_combine() consumes.
@@ -184,6 +204,14 @@ int32_t moe_set_timeline(moe_handle *h, void *timeline_dev, size_t bytes);
 int32_t moe_query_occupancy(moe_handle *h, int32_t tile_m, int32_t tile_n,
                             moe_occupancy *occ, moe_sm_limits *limits, moe_rho *rho);
 
+/* Kernel dispatch by shape (Section III-E, first paragraph: a conventional dispatch layer selects the GEMM2
+ * kernel; the resource manager then reads that kernel's tile shape and residency).  Chooses the GEMM tile
+ * family for `shape`: the widest n-tile the split width ceil(H/L) holds (256, 128 or 64), and 256-row
+ * CTA-pair tiles when the experts hold at least 1536 routed rows on average (T * k_tot / E_tot), 128-row
+ * single-CTA tiles below (small and decode-sized token counts: less row padding, every SM its own tile).
+ * The result is a valid (tile_m, tile_n) for every other call.  [host] */
+int32_t moe_select_tile(moe_handle *h, const moe_shape *shape, int32_t *tile_m, int32_t *tile_n);
+
 /* Sizes of the caller-allocated workspaces [bytes]: routing arrays, the tile-padded GEMM2
  * output Y (bf16, token-major: [T][L][k_tot * TP][ceil(H/L)]), readiness flags + split counters +
  * work queues (must be zero-filled once before first use and not shared between handles), status
@@ -231,6 +259,13 @@ int32_t moe_build_routing_static(moe_handle *h, const int32_t *topk_idx, const m
  * routed_tile_counts [host] ceil(M_e / T_M) for e in [0, n_experts).
  * Picks the lexicographic minimum of (T(C), Delta_comp(C), C) over the legal C; rho is
  * quantised to 2^-20.  limits->force_comm_ctas > 0 wins over everything, then selector_off.
+ * With limits->drain_help and rho->comm_warps_per_cta > 0 the candidate set is the product of C and the
+ * number w of co-resident communication warps per compute CTA (w = 0 with C in 1..C_max, w in
+ * 1..co_warps_max with C in 1..min(C_max, C_co_max)), T(C, w) follows the bandwidth-coupled recurrence
+ * described at moe_rho, and the winner is the lexicographic minimum of (T, Delta_comp, w, C).
+ * With drain_help = 0 and limits->dep_model = MOE_DEP_TILE the readiness of Eq. 9 is evaluated per
+ * communication tile (from the routed tile counts: the last non-empty expert's tiles gate the tokens in
+ * order) instead of per split.
  * Errors: MOE_ERR_PLAN_INFEASIBLE when no C (or the forced C) leaves P >= 1. */
 int32_t plan_partition(const int32_t *routed_tile_counts, int32_t n_experts,
                        const moe_occupancy *occ, const moe_sm_limits *limits,

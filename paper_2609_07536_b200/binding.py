@@ -22,6 +22,7 @@ MOE_ERR_STATIC_LIMIT = -9
 MOE_DEV_OK, MOE_DEV_TIMEOUT, MOE_DEV_OOB, MOE_DEV_DUP_EXPERT = 0, 1, 2, 3
 MOE_MODE_FUSED, MOE_MODE_GEMM_ONLY, MOE_MODE_COMBINE_ONLY = 0, 1, 2
 MOE_RHO_PAPER, MOE_RHO_LOCAL = 0, 1
+MOE_DEP_SPLIT, MOE_DEP_TILE = 0, 1
 MOE_MAX_EP, MOE_MAX_L = 8, 8
 MOE_MTILES_ON_DEVICE = -1
 
@@ -33,6 +34,7 @@ EXPORTS = [
     "moe_clear_status",
     "moe_layer", "moe_calibrate_rho", "moe_host_arena_bytes", "moe_layer_host",
     "moe_gemm1_workspace_bytes", "moe_gemm1_act", "moe_post_router_layer", "moe_set_timeline",
+    "moe_select_tile",
 ]
 
 
@@ -53,12 +55,14 @@ class moe_occupancy(C.Structure):
 
 class moe_sm_limits(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("G", "C_max", "force_comm_ctas", "selector_off", "default_C",
-                                                "drain_help", "co_warps_max", "force_co_warps")]
+                                                "drain_help", "co_warps_max", "force_co_warps", "C_co_max", "dep_model")]
 
 
 class moe_rho(C.Structure):
     _fields_ = [("rho_ref", C.c_double)] + [(n, C.c_int32) for n in (
-        "K_ref", "tile_m_ref", "tile_n_ref", "D_ref", "rows_ref", "comm_cols_ref", "mode")]
+        "K_ref", "tile_m_ref", "tile_n_ref", "D_ref", "rows_ref", "comm_cols_ref", "mode",
+        "comm_warps_per_cta", "n_sat_warps", "comm_quanta_per_tile", "reserved0")] + [("co_beta", C.c_double), ("co_gamma", C.c_double),
+                                                 ("co_order", C.c_double)]
 
 
 class moe_plan(C.Structure):
@@ -134,6 +138,7 @@ def lib():
         L.moe_post_router_layer.argtypes = [vp, vp, vp, vp, vp, vp, P(moe_shape), i32, i32, P(moe_sm_limits),
                                             P(moe_routing), vp, vp, vp, P(vp), vp, vp, vp, P(moe_plan), vp]
         L.moe_set_timeline.argtypes = [vp, vp, C.c_size_t]
+        L.moe_select_tile.argtypes = [vp, P(moe_shape), P(i32), P(i32)]
         L.moe_host_arena_bytes.argtypes = [P(moe_shape), i32, i32, P(C.c_size_t)]
         L.moe_layer_host.argtypes = [vp, vp, vp, vp, vp, P(moe_shape), i32, i32, P(moe_sm_limits), vp,
                                      C.c_size_t, vp, vp, P(moe_plan), vp]
@@ -189,6 +194,13 @@ def moe_set_wait_limit_ns(h, ns: int):
 def moe_set_timeline(h, timeline_dev, nbytes: int):
     """Timeline build only: later fused launches record per-CTA stamps into `timeline_dev` (None: off)."""
     _check(lib().moe_set_timeline(h, _ptr(timeline_dev), nbytes), "moe_set_timeline", h)
+
+
+def moe_select_tile(h, shape: moe_shape):
+    """Kernel dispatch by shape: (tile_m, tile_n) of the GEMM tile family the library would use."""
+    tm, tn = C.c_int32(), C.c_int32()
+    _check(lib().moe_select_tile(h, C.byref(shape), C.byref(tm), C.byref(tn)), "moe_select_tile", h)
+    return tm.value, tn.value
 
 
 def moe_query_occupancy(h, tile_m: int, tile_n: int):

@@ -34,6 +34,7 @@ inline size_t align16(size_t x) { return (x + 15) & ~(size_t)15; }
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 
+constexpr int64_t kPairTileMinRowsPerExpert = 1536;  // mean routed rows per expert from which 256-row pair tiles pay
 constexpr int kSplitCounterWords = 64;  // 2 parities x MOE_MAX_L split counters (32-bit), then 2 x MOE_MAX_L work queues (64-bit), padded
 
 bool shape_ok(const moe_shape *s)
@@ -170,6 +171,8 @@ int32_t moe_query_occupancy(moe_handle *h, int32_t tile_m, int32_t tile_n, moe_o
         limits->drain_help = 1;
         limits->co_warps_max = fused_co_warps_max();
         limits->force_co_warps = -1;
+        limits->C_co_max = 8;       // beside co-resident warps more dedicated CTAs than this never paid (one-time sweep)
+        limits->dep_model = MOE_DEP_SPLIT;
     }
     if (rho) {
         // One-time service-rate characterisation of this kernel family on B200 (Eq. 13), one constant per
@@ -190,7 +193,40 @@ int32_t moe_query_occupancy(moe_handle *h, int32_t tile_m, int32_t tile_n, moe_o
         rho->rows_ref = 8 * 2 + 1;
         rho->comm_cols_ref = 1024;
         rho->mode = MOE_RHO_LOCAL;
+        // Warp-level capacity and bandwidth coupling, measured once on B200 (DeepSeek-V2-Lite shape):
+        //   a communication CTA is 12 warps; alone it streams 68 GB/s (5.7 GB/s per warp), 148 of them together
+        //   5.85 TB/s (the copy bandwidth): 5850 / 5.67 = 1030 warps saturate HBM;
+        //   a co-resident warp beside a running GEMM serves 2.6-2.8 GB/s (2.2 times slower than a dedicated warp)
+        //   and each one stretches the compute wave by 1.25 % (683 -> 704 -> 714 us of GEMM phase for w = 0, 1, 2,
+        //   of which 2 % is the split-major tile order that w > 0 needs when L > 1: x is read once per split).
+        //   the dynamic hand-out gives out single tokens of a communication tile (T_M^comm pieces per tile).
+        rho->comm_warps_per_cta = 12;
+        rho->comm_quanta_per_tile = kCommTileM;
+        rho->reserved0 = 0;
+        rho->n_sat_warps = 1030;
+        rho->co_beta = 0.0125;
+        rho->co_gamma = 2.2;
+        rho->co_order = 0.02;
     }
+    return MOE_OK;
+}
+
+int32_t moe_select_tile(moe_handle *h, const moe_shape *s, int32_t *tile_m, int32_t *tile_n)
+{
+    if (!h || !s || !tile_m || !tile_n) return MOE_ERR_NULL;
+    if (!shape_ok(s)) return MOE_ERR_SHAPE;
+    // Conventional kernel dispatch (Section III-E: it runs before the resource manager and hands it the tile
+    // shape and residency of the kernel it chose).  Widest n-tile the split holds; rows: the 256-row CTA-pair
+    // tile moves a third less operand traffic per FLOP but pads every expert's last tile to 256 rows and needs
+    // two co-scheduled SMs, so it pays once an expert holds several such tiles on average (measured on the
+    // DeepSeek-V2-Lite shape, fused kernel, 128x256 against 256x256: 78 / 100 us at T = 16, 128 / 139 at 1024,
+    // 268 / 276 at 4096, 465 / 478 at 8192 (993 rows per expert), 889 / 880 at 16384 (1986 rows per expert)).
+    const int64_t split_w = ceil_div(s->H, s->L);
+    const int32_t tn = split_w >= 256 ? 256 : split_w >= 128 ? 128 : 64;
+    const int64_t rows_per_expert = (int64_t)s->T * s->k_tot / s->E_tot;
+    const bool pair = tn == 256 && h->max_pairs > 0 && rows_per_expert >= kPairTileMinRowsPerExpert;
+    *tile_m = pair ? 256 : 128;
+    *tile_n = tn;
     return MOE_OK;
 }
 

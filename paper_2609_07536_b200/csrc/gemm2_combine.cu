@@ -720,15 +720,11 @@ __device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring
                             tc_mma_bf16_pair(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
                                              k > 0 ? 1u : acc0);
                     }
-                    const uint32_t empty_bar = smem_u32(&ctl->empty[stage]);
-                    tc_commit_pair(empty_bar, mapa_u32(empty_bar, 1u));   // both CTAs may refill the stage
+                    tc_commit_pair(smem_u32(&ctl->empty[stage]));      // both CTAs may refill the stage
                     TL(tl_is += clock64() - tl_q);
                     if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
                 }
-                if (ok) {                                                   // both epilogues may start
-                    const uint32_t acc_bar = smem_u32(&ctl->tmem_full[a]);
-                    tc_commit_pair(acc_bar, mapa_u32(acc_bar, 1u));
-                }
+                if (ok) tc_commit_pair(smem_u32(&ctl->tmem_full[a]));   // both epilogues may start
                 TL(if (it == 0) tl_put(P, kTlFirstAcc, globaltimer_ns()));
             }
             TL(tl_put(P, kTlMmaEnd, globaltimer_ns()); tl_put(P, kTlTiles, (unsigned long long)it);

@@ -4,6 +4,8 @@ include/moe_b200.h declares; argument errors come back as status codes.  No comp
 import ctypes
 import os
 import re
+import shutil
+import subprocess
 
 import pytest
 
@@ -30,10 +32,40 @@ def test_every_declared_symbol_is_exported():
 def test_structs_match_header_sizes():
     assert ctypes.sizeof(B.moe_shape) == 32
     assert ctypes.sizeof(B.moe_occupancy) == 28
-    assert ctypes.sizeof(B.moe_sm_limits) == 32
-    assert ctypes.sizeof(B.moe_rho) == 40
+    assert ctypes.sizeof(B.moe_sm_limits) == 40
+    assert ctypes.sizeof(B.moe_rho) == 80
     assert ctypes.sizeof(B.moe_plan) == 56
     assert ctypes.sizeof(B.moe_status) == 16
+
+
+def test_struct_layouts_match_the_compiled_header(tmp_path):
+    # sizes and the offsets of the last fields as a C compiler lays the header's structs out, against the
+    # ctypes mirrors the binding passes across the boundary
+    gcc = shutil.which("gcc")
+    if gcc is None:
+        pytest.skip("no C compiler")
+    header = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "include", "moe_b200.h")
+    structs = {"moe_shape": "L", "moe_occupancy": "comp_slot_sms", "moe_sm_limits": "dep_model", "moe_rho": "co_order",
+               "moe_plan": "co_warps", "moe_routing": "max_mtiles", "moe_status": "count"}
+    src = tmp_path / "layout.c"
+    lines = ['#include <stdio.h>', '#include <stddef.h>', f'#include "{header}"', 'int main(void) {']
+    for name, last in structs.items():
+        lines.append(f'  printf("{name} %zu %zu\\n", sizeof({name}), offsetof({name}, {last}));')
+    lines += ['  return 0;', '}']
+    src.write_text("\n".join(lines))
+    exe = tmp_path / "layout"
+    subprocess.run([gcc, "-std=c99", "-o", str(exe), str(src)], check=True)
+    out = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split("\n")
+    seen = 0
+    for line in out:
+        if not line.strip():
+            continue
+        name, size, off = line.split()
+        cls = getattr(B, name)
+        assert ctypes.sizeof(cls) == int(size), name
+        assert getattr(cls, structs[name]).offset == int(off), name
+        seen += 1
+    assert seen == len(structs)
 
 
 def test_workspace_sizes_and_argument_errors():

@@ -211,6 +211,34 @@ def test_dsv2lite_with_co_resident_warps_sampled():
     _check_against_oracle(wl.DSV2L, n_random=96, co_warps=2)
 
 
+@pytest.mark.parametrize("T", [16, 64, 256, 1024])
+def test_decode_sized_token_counts_on_the_deepseek_shape(T):
+    # small and decode-sized batches (every expert holds a handful of rows): the tile family comes from the
+    # library's dispatch by shape, every token is checked
+    w = replace(wl.DSV2L, name=f"decode{T}", T=T)
+    tm, tn = B.moe_select_tile(G.handle(), G.shape_of(w))
+    assert (tm, tn) == (128, 256)
+    _check_against_oracle(replace(w, tile_m=tm, tile_n=tn))
+
+
+def test_dispatch_by_shape():
+    h = G.handle()
+    sel = lambda w: B.moe_select_tile(h, G.shape_of(w))
+    assert sel(wl.DSV2L) == (256, 256) and sel(replace(wl.DSV2L, T=32768)) == (256, 256)   # >= 1536 routed rows per expert
+    assert sel(replace(wl.DSV2L, T=8192)) == (128, 256) and sel(wl.QWEN) == (128, 256)     # 993 and 546 rows per expert
+    assert sel(replace(wl.DSV2L, T=1)) == (128, 256)
+    assert sel(replace(wl.DSV2L, L=8)) == (256, 256)                            # split width 256
+    assert sel(replace(wl.DSV2L, L=4, H=512)) == (128, 128)                     # split width 128: no pair tile
+    assert sel(wl.TINY) == (128, 256) and sel(replace(wl.TINY, H=64)) == (128, 64)
+    with pytest.raises(B.MoeError):
+        sel(replace(wl.TINY, H=250))
+    # whatever it returns is a configuration the other calls accept
+    for w in (wl.DSV2L, wl.GRANITE, replace(wl.TINY, H=64)):
+        tm, tn = sel(w)
+        occ, lim, rho = B.moe_query_occupancy(h, tm, tn)
+        assert (occ.tile_m, occ.tile_n) == (tm, tn) and occ.comp_slot_sms == (2 if tm == 256 else 1)
+
+
 def test_pair_tiles_against_oracle():
     for kw in (dict(T=777, E=5, k=2, H=1536, I=512, TP=2, EP=3, L=4),      # partial n-tile at the split end
                dict(T=300, E=3, k=1, H=256, I=64, TP=1, EP=1, L=1),         # m-tiles with an empty second half

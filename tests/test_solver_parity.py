@@ -25,9 +25,41 @@ def _oracle_plan(tiles, shape, occ, lim, rho):
                          rho.comm_cols_ref, K, occ.tile_m, occ.tile_n, shape.k_tot, shape.TP,
                          shape.H, shape.L, occ.comm_tile_n)
     rho_q = sr.quantise_rho(r)
-    sel = sr.select(Wc, Wm, shape.L, lim.G, occ.o_comp, occ.o_comm, lim.C_max, rho_q,
-                    force_comm_ctas=lim.force_comm_ctas, selector_off=bool(lim.selector_off),
-                    default_C=lim.default_C, slot_sms=occ.comp_slot_sms, drain_help=bool(lim.drain_help))
+    if lim.drain_help and rho.comm_warps_per_cta > 0:
+        # the co-resident family: product set (C, w), bandwidth-coupled service rate
+        sel = sr.select_co_resident(
+            Wc, Wm, shape.L, lim.G, occ.o_comp, occ.o_comm, lim.C_max, rho_q, occ.comp_slot_sms,
+            max(0, lim.co_warps_max), lim.C_co_max, rho.comm_warps_per_cta,
+            rho.n_sat_warps if rho.n_sat_warps > 0 else 2 ** 63 - 1, sr.quantise_rho(rho.co_beta),
+            sr.quantise_rho(rho.co_gamma), sr.quantise_rho(rho.co_order), force_comm_ctas=lim.force_comm_ctas,
+            selector_off=bool(lim.selector_off), default_C=lim.default_C, force_co_warps=lim.force_co_warps,
+            quanta_tile=rho.comm_quanta_per_tile)
+    elif not lim.drain_help and lim.dep_model == B.MOE_DEP_TILE:
+        # static partition with tile-level readiness
+        idx = sr.comm_tile_ready_index(tiles, shape.TP, shape.T, shape.EP, shape.H, shape.L, occ.tile_n,
+                                       occ.comm_tile_m, occ.comm_tile_n)
+        assert len(idx) == Wm
+        if lim.force_comm_ctas > 0 or lim.selector_off:
+            Cs = [lim.force_comm_ctas if lim.force_comm_ctas > 0 else lim.default_C]
+            if Cs[0] < 1:
+                raise ValueError("C must be at least 1")
+        else:
+            Cs = range(1, lim.C_max + 1)
+        best = None
+        for C in Cs:
+            m = sr.makespan_tile_level(C, idx, Wc, shape.L, lim.G, occ.o_comp, occ.o_comm, rho_q, occ.comp_slot_sms)
+            if m is not None and (best is None or (m[0], m[1], C) < best[0]):
+                best = ((m[0], m[1], C), dict(comm_ctas=C, R=m[2], P=m[3], T_q=m[0], delta=m[1], W_comp=Wc, W_comm=Wm))
+        if best is None:
+            raise ValueError("no legal C")
+        sel = best[1]
+    else:
+        sel = sr.select(Wc, Wm, shape.L, lim.G, occ.o_comp, occ.o_comm, lim.C_max, rho_q,
+                        force_comm_ctas=lim.force_comm_ctas, selector_off=bool(lim.selector_off),
+                        default_C=lim.default_C, slot_sms=occ.comp_slot_sms, drain_help=bool(lim.drain_help))
+        if lim.drain_help and lim.co_warps_max > 0 and lim.force_co_warps > 0:
+            sel["co_warps"] = min(lim.force_co_warps, lim.co_warps_max)   # an explicit request is passed through
+    sel.setdefault("co_warps", 0)
     sel["rho_q"] = rho_q
     return sel
 
@@ -36,7 +68,7 @@ def _same(plan, sel):
     assert (plan.comm_ctas, plan.R, plan.P) == (sel["comm_ctas"], sel["R"], sel["P"])
     assert (plan.W_comp, plan.W_comm, plan.delta) == (sel["W_comp"], sel["W_comm"], sel["delta"])
     assert plan.pred_T_q == sel["T_q"] and plan.rho_q == sel["rho_q"]
-    assert plan.mode == B.MOE_MODE_FUSED and plan.debug_withhold_tile == -1 and plan.co_warps == 0
+    assert plan.mode == B.MOE_MODE_FUSED and plan.debug_withhold_tile == -1 and plan.co_warps == sel["co_warps"]
 
 
 def _rand_inputs(rng):
@@ -49,9 +81,22 @@ def _rand_inputs(rng):
                          rng.choice([1, 2, 4, 8]), rng.choice([1, 2, 4, 8]))
     occ = B.moe_occupancy(tile_m, tile_n, rng.choice([64, 128]), rng.choice([512, 1024]),
                           rng.choice([1, 2]), rng.choice([1, 2, 4]), rng.choice([1, 1, 2]))
-    lim = B.moe_sm_limits(rng.choice([4, 108, 148]), rng.randint(1, 160), 0, 0, 3, rng.choice([0, 0, 1]))
+    # the three model families: the paper's recurrence / drain help (as before), the co-resident family with
+    # a bandwidth-coupled service rate (drain help and warp-level constants), tile-level readiness (static)
+    family = rng.choice(["plain", "plain", "co", "co", "tile"])
+    dh = 1 if family == "co" else (0 if family == "tile" else rng.choice([0, 0, 1]))
+    lim = B.moe_sm_limits(rng.choice([4, 108, 148]), rng.randint(1, 160), 0, 0, 3, dh,
+                          rng.choice([0, 1, 2, 4]), rng.choice([-1, -1, 0, 1, 3]), rng.choice([1, 8, 16, 200]),
+                          B.MOE_DEP_TILE if family == "tile" else rng.choice([B.MOE_DEP_SPLIT, B.MOE_DEP_TILE]))
     rho = B.moe_rho(rng.uniform(0.05, 30.0), rng.choice([352, 704]), 128, rng.choice([128, 256]),
                     rng.choice([2, 4]), 17, 1024, rng.choice([B.MOE_RHO_PAPER, B.MOE_RHO_LOCAL]))
+    if family == "co":
+        rho.comm_warps_per_cta = rng.choice([1, 4, 12])
+        rho.n_sat_warps = rng.choice([0, 7, 300, 1030, 100000])
+        rho.comm_quanta_per_tile = rng.choice([0, 0, 12, 128, 5])
+        rho.co_beta = rng.choice([0.0, 0.0125, 0.2])
+        rho.co_gamma = rng.choice([1.0, 2.2, 7.5])
+        rho.co_order = rng.choice([0.0, 0.02, 0.3])
     tiles = [rng.randint(0, 40) for _ in range(E)]
     return tiles, shape, occ, lim, rho
 
@@ -59,7 +104,7 @@ def _rand_inputs(rng):
 def test_random_inputs_bit_exact():
     rng = random.Random(11)
     n = 0
-    for _ in range(20000):
+    for _ in range(100000):
         tiles, shape, occ, lim, rho = _rand_inputs(rng)
         try:
             sel = _oracle_plan(tiles, shape, occ, lim, rho)
@@ -70,7 +115,7 @@ def test_random_inputs_bit_exact():
             continue
         _same(B.plan_partition(tiles, occ, lim, shape, rho), sel)
         n += 1
-    assert n > 15000
+    assert n > 75000
 
 
 def test_overrides_and_errors():
