@@ -337,7 +337,10 @@ def simulate_drain_help(C: int, Wc: int, Wm: int, L: int, P: int, helpers: int, 
 #   * a co-resident warp shares its SM's issue slots and memory path with a running GEMM: it serves
 #     `gamma` times slower than a dedicated warp (N_eff counts it as 1/gamma warps), and every co-resident
 #     warp stretches the compute wave by `beta`; with more than one split they also force the split-major
-#     tile order (x is read once per split), which stretches the compute wave by `order`.
+#     tile order (x is read once per split), which stretches the compute wave by `order`;
+#   * without co-resident warps the kernels run the tiles m-tile-major across the splits (x is read once):
+#     no split is published before the last one, so for w = 0 every split becomes ready at A_{L-1} and all
+#     communication work is served after the GEMM (dedicated CTAs then only cost SMs).
 #   All four constants are fixed point (2^-20) except n_sat and warps_cta (integers).
 
 def coupled_rho(rho_q: int, n_workers: int, n_sat: int) -> int:
@@ -383,7 +386,8 @@ def makespan_co_resident(C: int, w: int, Wc: int, Wm: int, L: int, G: int, o_com
         q = q_wave * ceil_div(Wq, n_eff)
         F = 0
         for s in range(L - 1):                                 # Eq. 11 on splits 0..L-2
-            F = max(ceil_div((s + 1) * Wc, P) * tau_q, F) + q
+            A_s = ceil_div((s + 1) * Wc, P) * tau_q if w > 0 else A_last     # m-tile-major order: nothing is early
+            F = max(A_s, F) + q
         backlog = 0
         if F > A_last and q_wave > 0:
             backlog = min(ceil_div(F - A_last, q_wave) * n_eff, (L - 1) * Wq)
@@ -395,11 +399,16 @@ def makespan_co_resident(C: int, w: int, Wc: int, Wm: int, L: int, G: int, o_com
 def select_co_resident(Wc: int, Wm: int, L: int, G: int, o_comp: int, o_comm: int, C_max: int, rho_q: int,
                        slot_sms: int, w_max: int, C_co_max: int, warps_cta: int, n_sat: int, beta_q: int,
                        gamma_q: int, order_q: int, force_comm_ctas: int = 0, selector_off: bool = False,
-                       default_C: int = 3, force_co_warps: int = -1, quanta_tile: int = 0) -> dict:
+                       default_C: int = 3, force_co_warps: int = -1, quanta_tile: int = 0,
+                       co_min_waves: int = 0) -> dict:
     """Algorithm 1 over the product set: C in 1..C_max with w = 0, and C in 1..min(C_max, C_co_max) with
     w in 1..w_max (a one-time characterisation bounds the dedicated CTAs worth trying beside co-resident
-    warps, as the paper's C <= 16 does for its family).  Lexicographic minimum of (T, Delta_comp, w, C).
-    Overrides as in select(): a forced C / a forced w restrict the set to that value."""
+    warps, as the paper's C <= 16 does for its family).  A second characterisation constant bounds the
+    legal set from below: co-resident warps are only legal when the compute phase is at least
+    `co_min_waves` waves long, ceil(L * W_comp / P(C)) >= co_min_waves (on shorter launches their start-up
+    costs more than they can overlap, which a wave model does not see).  Lexicographic minimum of
+    (T, Delta_comp, w, C).  Overrides as in select(): a forced C / a forced w restrict the set to that value
+    (a forced w is not subject to co_min_waves)."""
     if force_comm_ctas > 0 or selector_off:
         Cs0 = Cs1 = [force_comm_ctas if force_comm_ctas > 0 else default_C]
         if Cs0[0] < 1:
@@ -414,6 +423,8 @@ def select_co_resident(Wc: int, Wm: int, L: int, G: int, o_comp: int, o_comm: in
             m = makespan_co_resident(C, w, Wc, Wm, L, G, o_comp, o_comm, rho_q, slot_sms, warps_cta, n_sat,
                                      beta_q, gamma_q, order_q, quanta_tile)
             if m is None:
+                continue
+            if w > 0 and force_co_warps < 0 and ceil_div(L * Wc, m[3]) < co_min_waves:
                 continue
             key = (m[0], m[1], w, C)
             if best is None or key < best[0]:
@@ -448,6 +459,8 @@ def simulate_co_resident(C: int, w: int, Wc: int, Wm: int, L: int, P: int, n_sm:
         tile_end.append(clock[b])
     publish = [max(tile_end[s * Wc:(s + 1) * Wc]) if Wc > 0 else Fraction(0) for s in range(L)]
     A = publish[L - 1]
+    if w == 0:
+        publish = [A] * L                  # m-tile-major order: every split completes with the last tile
     Wq = Wm * quanta_tile
     n_early = C * warps_cta + w * n_sm
     n_eff = C * warps_cta + int(Fraction(w * n_sm) / gamma)

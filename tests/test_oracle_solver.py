@@ -418,14 +418,20 @@ def test_co_resident_model_reductions_and_simulation():
         warps_cta = rng.choice([1, 4, 12])
         C = rng.randint(1, G - 1)
         P = sr.compute_capacity(C, G, o_comp, 1, slot)
-        # (a) no co-resident warp and no saturation: the drain-help recurrence, bit for bit
+        # (a) no co-resident warp: the tiles run m-tile-major, every split is published with the last tile, so the
+        # whole communication work is served after the GEMM by every warp -- a closed form; without saturation and
+        # with one split it is the drain-help recurrence bit for bit
         a = sr.makespan_co_resident(C, 0, Wc, Wm, L, G, o_comp, 1, _q(rho), slot, warps_cta, 10 ** 9, _q(Fraction(1, 16)),
                                     _q(2), _q(Fraction(1, 32)))
-        b = sr.makespan_drain_help(C, Wc, Wm, L, G, o_comp, 1, _q(rho), slot)
-        assert a == b
+        b = sr.makespan_drain_help(C, Wc, Wm, 1, G, o_comp, 1, _q(rho), slot)
         if P <= 0:
+            assert a is None and b is None
             continue
         n_sm = P * slot // o_comp
+        workers = (C + n_sm) * warps_cta
+        assert a[0] == sr.ceil_div(L * Wc, P) * sr.RHO_ONE + _q(rho) * sr.ceil_div(L * Wm * warps_cta, workers)
+        if L == 1:
+            assert a == b
         w = rng.randint(0, 3)
         n_sat = rng.choice([3, 17, 200, 10 ** 6])
         beta, gamma, order = Fraction(rng.randint(0, 8), 64), Fraction(rng.randint(4, 16), 4), Fraction(rng.randint(0, 4), 32)
@@ -478,6 +484,11 @@ def test_select_co_resident_is_the_lexicographic_minimum_and_honours_overrides()
                 if m is not None:
                     keys.append((m[0], m[1], w, C))
         assert (sel["T_q"], sel["delta"], sel["co_warps"], sel["comm_ctas"]) == min(keys)
+        # the lower end of the legal set: no co-resident warps on launches whose compute phase is short
+        thr = rng.randint(1, 200)
+        lim = sr.select_co_resident(Wc, Wm, L, G, 1, 1, C_max, rho_q, slot, w_max, C_co, co_min_waves=thr, **kw)
+        keys2 = [k for k in keys if k[2] == 0 or sr.ceil_div(L * Wc, sr.compute_capacity(k[3], G, 1, 1, slot)) >= thr]
+        assert (lim["T_q"], lim["delta"], lim["co_warps"], lim["comm_ctas"]) == min(keys2)
         if sr.compute_capacity(2, G, 1, 1, slot) > 0:
             f = sr.select_co_resident(Wc, Wm, L, G, 1, 1, C_max, rho_q, slot, w_max, C_co, force_comm_ctas=2,
                                       force_co_warps=1, **kw)
