@@ -104,6 +104,10 @@ typedef struct {
                                 for w >= 1 (a one-time characterisation, like C_max) */
     int32_t dep_model;       /* static partition only: MOE_DEP_SPLIT = Eq. 9 as printed (one readiness per split),
                                 MOE_DEP_TILE = Eq. 9 applied to every communication tile (per-tile flags) */
+    int32_t co_min_waves;    /* lower end of the legal set for co-resident warps: they are tried only when the compute
+                                phase is at least this many waves long, ceil(L * W_comp / P(C)) >= co_min_waves (a
+                                one-time characterisation: on short launches their start-up costs more than they can
+                                overlap); a forced w is not subject to it */
 } moe_sm_limits;
 
 /* Relative wave service rate (Eq. 13-15). */
@@ -307,6 +311,14 @@ int32_t moe_gemm2_combine(moe_handle *h, const void *x_routed, const void *W2,
                           const moe_routing *routing, int32_t n_mtiles, const moe_plan *plan,
                           void *const *out, void *y_ws, uint32_t *flags_ws,
                           uint32_t *status_dev, void *stream);
+
+/* The handle keeps, per flags workspace it has launched on, the launch epoch that marks a launch's readiness
+ * flags (host memory: a small table keyed by the workspace address, touched by every moe_gemm2_combine; this is
+ * why a handle serves one host thread at a time).  Call this before freeing a flags workspace, or before
+ * zero-filling it again, so that the entry goes away and a later workspace at the same address starts from
+ * epoch 0 with clean flags; flags_ws = NULL forgets every workspace.  A workspace must not be shared between
+ * handles, and one that is reused without this call must not have been modified by anybody else.  [host] */
+int32_t moe_release_workspace(moe_handle *h, const uint32_t *flags_ws);
 
 /* Copies the 4-word device status to the host (synchronises the stream).  Returns
  * MOE_ERR_DEVICE_STATUS when code != 0. */

@@ -34,7 +34,7 @@ EXPORTS = [
     "moe_clear_status",
     "moe_layer", "moe_calibrate_rho", "moe_host_arena_bytes", "moe_layer_host",
     "moe_gemm1_workspace_bytes", "moe_gemm1_act", "moe_post_router_layer", "moe_set_timeline",
-    "moe_select_tile",
+    "moe_select_tile", "moe_release_workspace",
 ]
 
 
@@ -55,7 +55,7 @@ class moe_occupancy(C.Structure):
 
 class moe_sm_limits(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("G", "C_max", "force_comm_ctas", "selector_off", "default_C",
-                                                "drain_help", "co_warps_max", "force_co_warps", "C_co_max", "dep_model")]
+                                                "drain_help", "co_warps_max", "force_co_warps", "C_co_max", "dep_model", "co_min_waves")]
 
 
 class moe_rho(C.Structure):
@@ -139,6 +139,7 @@ def lib():
                                             P(moe_routing), vp, vp, vp, P(vp), vp, vp, vp, P(moe_plan), vp]
         L.moe_set_timeline.argtypes = [vp, vp, C.c_size_t]
         L.moe_select_tile.argtypes = [vp, P(moe_shape), P(i32), P(i32)]
+        L.moe_release_workspace.argtypes = [vp, vp]
         L.moe_host_arena_bytes.argtypes = [P(moe_shape), i32, i32, P(C.c_size_t)]
         L.moe_layer_host.argtypes = [vp, vp, vp, vp, vp, P(moe_shape), i32, i32, P(moe_sm_limits), vp,
                                      C.c_size_t, vp, vp, P(moe_plan), vp]
@@ -288,6 +289,12 @@ def moe_get_status(h, status_dev, stream=None, check: bool = True) -> moe_status
         raise MoeError(rc, "moe_get_status",
                        f"device status code={st.code} detail={st.detail} where={st.where} count={st.count}")
     return st
+
+
+def moe_release_workspace(h, flags_ws=None):
+    """Forgets the launch epoch kept for `flags_ws` (None: for every workspace): call before freeing or
+    re-zeroing a flags workspace."""
+    _check(lib().moe_release_workspace(h, _ptr(flags_ws)), "moe_release_workspace", h)
 
 
 def moe_clear_status(h, status_dev, stream=None):

@@ -173,6 +173,7 @@ int32_t moe_query_occupancy(moe_handle *h, int32_t tile_m, int32_t tile_n, moe_o
         limits->force_co_warps = -1;
         limits->C_co_max = 8;       // beside co-resident warps more dedicated CTAs than this never paid (one-time sweep)
         limits->dep_model = MOE_DEP_SPLIT;
+        limits->co_min_waves = 24;  // below it co-resident warps lost 2-5 % in the sweep (T = 1024: 19 waves; T = 2048: 37)
     }
     if (rho) {
         // One-time service-rate characterisation of this kernel family on B200 (Eq. 13), one constant per
@@ -403,6 +404,9 @@ int32_t moe_gemm2_combine(moe_handle *h, const void *x_routed, const void *W2, c
     // rows; where one of these does not hold the launch runs without them (same result, bit for bit).
     p.co_warps = plan->co_warps < fused_co_warps_max() ? plan->co_warps : fused_co_warps_max();
     if (!p.drain_help || !p.wide_store || p.Q > 16) p.co_warps = 0;
+    // warps 16-19 of a compute CTA: co-resident communication warps, or -- when none is asked for -- a fourth
+    // epilogue column group (a third less epilogue work per warp: what bounds tiles with a short K)
+    p.epi_warps = (p.co_warps == 0 && p.wide_store) ? 16 : 12;
     // Tile sequence: split-major (the paper's) whenever something consumes a split while the next one is
     // computed; m-tile-major across the splits (x is read from DRAM once) when nothing does
     p.tile_order = (plan->drain_help && p.co_warps == 0) ? 1 : 0;
@@ -461,6 +465,14 @@ int32_t moe_gemm2_combine(moe_handle *h, const void *x_routed, const void *W2, c
         p.timeline = h->timeline;
     e = pair ? pair_launch(p, grid, st) : fused_launch(TN, p, grid, st);
     if (e != cudaSuccess) return cuda_fail(h, e, "fused launch");
+    return MOE_OK;
+}
+
+int32_t moe_release_workspace(moe_handle *h, const uint32_t *flags_ws)
+{
+    if (!h) return MOE_ERR_NULL;
+    if (flags_ws) h->epochs.erase(flags_ws);
+    else h->epochs.clear();
     return MOE_OK;
 }
 

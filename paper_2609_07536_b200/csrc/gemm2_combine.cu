@@ -80,8 +80,8 @@ struct Cfg {
     static constexpr int kStageBytes = kABytes + kBBytes;
     static constexpr int kStages = kStageBytesTotal / kStageBytes;  // 8 / 6 / 4
     static constexpr int kTmemCols = 2 * TN;                     // two accumulator buffers
-    static constexpr int kEpiWarps = 12;                          // warps 4..15: three column groups x four lane quarters
-    static constexpr int kColsPerGroup = ((TN / 32 + 2) / 3) * 32;  // 32-column rounds dealt to the groups: 96 / 64 / 32
+    // epilogue: warps 4..15 (three column groups x four TMEM lane quarters), plus warps 16..19 as a fourth
+    // column group when the launch carries no co-resident communication warps (FusedParams::epi_warps)
 };
 
 struct Control {
@@ -153,10 +153,16 @@ __device__ __forceinline__ bool wait_barrier_1t(uint32_t bar, uint32_t parity, C
     return true;
 }
 
-// Barrier of the 16 warps that compute (the co-resident communication warps never join it).
-__device__ __forceinline__ void sync_compute_warps()
+// Barrier of the warps that compute: 16, or all 20 when warps 16-19 serve as a fourth epilogue column group
+// (co-resident communication warps never join it).
+__device__ __forceinline__ void sync_compute_warps(const FusedParams &P)
 {
-    asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory");
+    asm volatile("bar.sync 1, %0;" ::"r"(kThreads + 32 * (P.epi_warps - 12)) : "memory");
+}
+// 32-column rounds of a TN-wide tile dealt to `groups` epilogue column groups (3 or 4)
+__device__ __forceinline__ int epi_cols_per_group(int tn, int groups)
+{
+    return ((tn / 32 + groups - 1) / groups) * 32;
 }
 
 struct Tile {
@@ -334,8 +340,8 @@ __device__ void compute_cta(const FusedParams &P, int W_comp, uint8_t *ring, Con
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&ctl->tmem_full[i]), 1);
-            mbar_init(smem_u32(&ctl->tmem_empty[i]), C::kEpiWarps);
-            mbar_init(smem_u32(&ctl->epi_done[i]), C::kEpiWarps);
+            mbar_init(smem_u32(&ctl->tmem_empty[i]), (uint32_t)P.epi_warps);
+            mbar_init(smem_u32(&ctl->epi_done[i]), (uint32_t)P.epi_warps);
             mbar_init(smem_u32(&ctl->pub_done[i]), 1);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -343,7 +349,7 @@ __device__ void compute_cta(const FusedParams &P, int W_comp, uint8_t *ring, Con
     }
     if (warp == 1) tmem_alloc(smem_u32(&ctl->tmem_base), C::kTmemCols);
     tc_fence_before();
-    sync_compute_warps();
+    sync_compute_warps(P);
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
 
@@ -456,12 +462,13 @@ __device__ void compute_cta(const FusedParams &P, int W_comp, uint8_t *ring, Con
                tl_put(P, kTlWaitTmem, (unsigned long long)tl_wt); tl_put(P, kTlMmaCycles, (unsigned long long)(clock64() - tl_c0)));
         }
         __syncwarp();
-    } else if (warp >= 4 && warp < 4 + C::kEpiWarps) {
+    } else if (warp >= 4 && warp < 4 + P.epi_warps) {
         // ---------------- epilogue: TMEM -> bf16 -> Y, then publish the tile
         const int q4 = warp & 3;                   // TMEM lane quarter this warp may read
         const int grp = (warp - 4) >> 2;           // column group of the tile
-        const int col_first = grp * C::kColsPerGroup;
-        const int n_cols = max(0, min(C::kColsPerGroup, TN - col_first));
+        const int cols_per_group = epi_cols_per_group(TN, P.epi_warps >> 2);
+        const int col_first = grp * cols_per_group;
+        const int n_cols = max(0, min(cols_per_group, TN - col_first));
         const int row_in_tile = q4 * 32 + lane;
         __nv_bfloat16 *Y = reinterpret_cast<__nv_bfloat16 *>(P.Y);
         // Row bookkeeping runs ahead of the accumulators: the m-tile table entries are fetched two tiles
@@ -566,7 +573,7 @@ __device__ void compute_cta(const FusedParams &P, int W_comp, uint8_t *ring, Con
     }
     // ---------------- teardown
     tc_fence_before();
-    sync_compute_warps();
+    sync_compute_warps(P);
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, C::kTmemCols);
@@ -591,8 +598,6 @@ struct PairCfg {
     static constexpr int kStageBytes = kABytes + kBBytes;               // 32 KB
     static constexpr int kStages = kStageBytesTotal / kStageBytes;      // 6
     static constexpr int kTmemCols = 2 * kTileN;                        // two accumulator buffers
-    static constexpr int kEpiWarps = 12;
-    static constexpr int kColsPerGroup = ((kTileN / 32 + 2) / 3) * 32;  // 96, 96, 64
 };
 
 __device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring, Control *ctl, uint8_t *aux, int b)
@@ -612,8 +617,8 @@ __device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&ctl->tmem_full[i]), 1);
-            mbar_init(smem_u32(&ctl->tmem_empty[i]), 2 * C::kEpiWarps);
-            mbar_init(smem_u32(&ctl->epi_done[i]), C::kEpiWarps);
+            mbar_init(smem_u32(&ctl->tmem_empty[i]), 2u * (uint32_t)P.epi_warps);
+            mbar_init(smem_u32(&ctl->epi_done[i]), (uint32_t)P.epi_warps);
             mbar_init(smem_u32(&ctl->pub_done[i]), 1);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -621,7 +626,7 @@ __device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring
     }
     if (warp == 1) tmem_alloc_pair(smem_u32(&ctl->tmem_base), C::kTmemCols);
     tc_fence_before();
-    sync_compute_warps();
+    sync_compute_warps(P);
     cluster_sync_all();          // the peer's barriers exist before anything arrives on them (the co-resident
                                  // communication warps of both CTAs arrive on this cluster barrier too)
     tc_fence_after();
@@ -732,12 +737,13 @@ __device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring
                tl_put(P, kTlWaitTmem, (unsigned long long)tl_wt); tl_put(P, kTlMmaCycles, (unsigned long long)(clock64() - tl_c0)));
         }
         __syncwarp();
-    } else if (warp >= 4 && warp < 4 + C::kEpiWarps) {
+    } else if (warp >= 4 && warp < 4 + P.epi_warps) {
         // ---------------- epilogue (both CTAs): own 128 rows of the pair tile
         const int q4 = warp & 3;
         const int grp = (warp - 4) >> 2;
-        const int col_first = grp * C::kColsPerGroup;
-        const int n_cols = max(0, min(C::kColsPerGroup, TN - col_first));
+        const int cols_per_group = epi_cols_per_group(TN, P.epi_warps >> 2);
+        const int col_first = grp * cols_per_group;
+        const int n_cols = max(0, min(cols_per_group, TN - col_first));
         const int row_in_tile = (int)rank * kMmaM + q4 * 32 + lane;
         __nv_bfloat16 *Y = reinterpret_cast<__nv_bfloat16 *>(P.Y);
         // Row bookkeeping runs ahead of the accumulators: the m-tile table entries are fetched two tiles
@@ -838,7 +844,7 @@ __device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring
     // ---------------- teardown: nobody leaves while its peer may still touch its memory (the co-resident
     // communication warps arrived on this cluster barrier right after the set-up one)
     tc_fence_before();
-    sync_compute_warps();
+    sync_compute_warps(P);
     cluster_sync_all();
     if (warp == 1) {
         tc_fence_after();
@@ -951,6 +957,7 @@ __device__ void comm_warp(const FusedParams &P, int W_comp, Control *ctl, const 
     TL_DECL(unsigned long long tl_first = 0, tl_last = 0, tl_sleep = 0; uint32_t tl_units = 0, tl_by_split[4] = {0u, 0u, 0u, 0u};)
     uint8_t *my_ring = res.stages;
     float *wq = res.wq;
+    const unsigned long long y_policy = l2_evict_first_policy();
     const uint32_t full_s = smem_u32(res.full);
     const __nv_bfloat16 *Y = reinterpret_cast<const __nv_bfloat16 *>(P.Y);
 
@@ -1108,7 +1115,7 @@ __device__ void comm_warp(const FusedParams &P, int W_comp, Control *ctl, const 
             const __nv_bfloat16 *src = Y + ((size_t)u.t * P.L + u.s) * (size_t)P.Q * (size_t)P.split_w +
                                        ((size_t)u.slab * P.Q << P.slab_shift);
             mbar_arrive_expect_tx(full, bytes);
-            bulk_load(smem_u32(my_ring + st * kCommUnitBytes), src, bytes, full);
+            bulk_load_once(smem_u32(my_ring + st * kCommUnitBytes), src, bytes, full, y_policy);   // Y is read once
         }
         __syncwarp();
         ++n_mine;
@@ -1426,7 +1433,7 @@ moe_gemm2_combine_kernel(const __grid_constant__ FusedParams P)
     const int W_comp = launch_w_comp(P);
     if ((int)blockIdx.x < P.C) {
         comm_cta<TN>(P, W_comp, ring, ctl, aux, P.drain_help ? kRoleFront : kRoleStatic, (int)blockIdx.x);
-    } else if (warp >= kThreads / 32) {
+    } else if (warp >= kThreads / 32 && P.epi_warps == 12) {
         if (co_warp_number(warp) < P.co_warps) co_resident_warp<TN>(P, W_comp, ctl, aux, co_warp_number(warp));
         return;
     } else {
@@ -1465,7 +1472,7 @@ moe_gemm2_combine_pair_kernel(const __grid_constant__ FusedParams P)
         // odd C: the last communication CTA's cluster-mate cannot compute (no partner).  With dynamic work
         // distribution it serves communication work as well; under the static map it has no tile list.
         if (P.drain_help && P.mode == MOE_MODE_FUSED) comm_cta<256>(P, W_comp, ring, ctl, aux, kRoleFront, (int)blockIdx.x);
-    } else if (warp >= kThreads / 32) {
+    } else if (warp >= kThreads / 32 && P.epi_warps == 12) {
         // The compute warps of both CTAs meet at two cluster barriers (set-up and teardown), and a cluster
         // barrier counts every thread: these warps join the first, arrive at once on the second (they hold
         // nothing a peer could touch) and pick its completion up when their own work is done.

@@ -161,7 +161,8 @@ inline bool evaluate_co(int32_t C, int32_t w, int64_t Wc, int64_t Wm, int32_t L,
         const int64_t q = q_wave * ceil_div64(Wq, n_eff);
         int64_t F = 0;
         for (int32_t s = 0; s + 1 < L; ++s) {
-            const int64_t A = ceil_div64((int64_t)(s + 1) * Wc, P) * tau_q;
+            // without co-resident warps the tiles run m-tile-major: no split is published before the last
+            const int64_t A = w > 0 ? ceil_div64((int64_t)(s + 1) * Wc, P) * tau_q : A_last;
             F = (A > F ? A : F) + q;
         }
         backlog = 0;
@@ -372,6 +373,8 @@ extern "C" int32_t plan_partition(const int32_t *routed_tile_counts, int32_t n_e
                 for (int32_t C = C_lo; C <= C_hi; ++C) {
                     Candidate c;
                     if (!evaluate_co(C, w, Wc, Wm, L, G, o_comp, o_comm, slot, rho_q, m, &c)) break;   // P only falls
+                    // lower end of the legal set: co-resident warps need a compute phase of co_min_waves waves
+                    if (w > 0 && limits->force_co_warps < 0 && ceil_div64((int64_t)L * Wc, c.P) < limits->co_min_waves) continue;
                     if (!have || c.T_q < best.T_q || (c.T_q == best.T_q && c.delta < best.delta)) {
                         best = c;
                         best_w = w;
@@ -409,6 +412,8 @@ extern "C" int32_t plan_partition(const int32_t *routed_tile_counts, int32_t n_e
                 }
                 const int64_t A_last = qa[L - 1] * tau_q;
                 if (have && A_last + lb_tail > best.T_q) break;     // A_last only grows with C: nothing further can win
+                // lower end of the legal set: co-resident warps need a compute phase of co_min_waves waves
+                if (w > 0 && limits->force_co_warps < 0 && qa[L - 1] < limits->co_min_waves) continue;
                 const int64_t n_early = (int64_t)C * m.warps_cta + w * n_sm;
                 const int64_t n_eff = (int64_t)C * m.warps_cta + co_eff;
                 int64_t backlog;
@@ -421,7 +426,7 @@ extern "C" int32_t plan_partition(const int32_t *routed_tile_counts, int32_t n_e
                         const int64_t q = q_wave * ceil_div64(Wq, n_eff);
                         int64_t F = 0;
                         for (int32_t s = 0; s + 1 < L; ++s) {
-                            const int64_t A = qa[s] * tau_q;
+                            const int64_t A = w > 0 ? qa[s] * tau_q : A_last;   // m-tile-major order: nothing is early
                             F = (A > F ? A : F) + q;
                         }
                         if (F > A_last) {

@@ -32,7 +32,7 @@ def test_every_declared_symbol_is_exported():
 def test_structs_match_header_sizes():
     assert ctypes.sizeof(B.moe_shape) == 32
     assert ctypes.sizeof(B.moe_occupancy) == 28
-    assert ctypes.sizeof(B.moe_sm_limits) == 40
+    assert ctypes.sizeof(B.moe_sm_limits) == 44
     assert ctypes.sizeof(B.moe_rho) == 80
     assert ctypes.sizeof(B.moe_plan) == 56
     assert ctypes.sizeof(B.moe_status) == 16
@@ -45,7 +45,7 @@ def test_struct_layouts_match_the_compiled_header(tmp_path):
     if gcc is None:
         pytest.skip("no C compiler")
     header = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "include", "moe_b200.h")
-    structs = {"moe_shape": "L", "moe_occupancy": "comp_slot_sms", "moe_sm_limits": "dep_model", "moe_rho": "co_order",
+    structs = {"moe_shape": "L", "moe_occupancy": "comp_slot_sms", "moe_sm_limits": "co_min_waves", "moe_rho": "co_order",
                "moe_plan": "co_warps", "moe_routing": "max_mtiles", "moe_status": "count"}
     src = tmp_path / "layout.c"
     lines = ['#include <stdio.h>', '#include <stddef.h>', f'#include "{header}"', 'int main(void) {']

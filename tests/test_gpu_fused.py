@@ -297,6 +297,23 @@ def test_gemm_only_then_combine_only_equals_fused():
         assert np.array_equal(a, b, equal_nan=True)
 
 
+def test_a_released_and_rezeroed_flags_workspace_starts_over():
+    # the handle keeps the launch epoch of every flags workspace; after moe_release_workspace and a fresh
+    # zero-fill the same buffer is a new workspace (epoch 1 again) and gives the same bits
+    h = G.handle()
+    w = replace(wl.GRANITE, name="release", T=900)
+    idx, wt, _ = wl.make_routing(w)
+    x, W2 = wl.make_data(w)
+    first, plan, ws, S, st = G.run_layer(w, idx, wt, x, W2)
+    first = [o.copy() for o in first]
+    G.run_layer(w, idx, wt, x, W2, ws=ws)                     # epoch 2 on the same workspace
+    B.moe_release_workspace(h, ws.flags_ws)
+    ws.flags_ws.zero_()
+    again, *_ = G.run_layer(w, idx, wt, x, W2, ws=ws)
+    for a, b in zip(first, again):
+        assert np.array_equal(a, b, equal_nan=True)
+
+
 def test_bounded_wait_reports_a_timeout_and_the_context_survives():
     h = G.handle()
     w = replace(wl.TINY, name="withhold", T=512, E=4, k=2, H=256, I=128, TP=1, EP=1, tile_m=128, tile_n=128)

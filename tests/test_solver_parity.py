@@ -33,7 +33,7 @@ def _oracle_plan(tiles, shape, occ, lim, rho):
             rho.n_sat_warps if rho.n_sat_warps > 0 else 2 ** 63 - 1, sr.quantise_rho(rho.co_beta),
             sr.quantise_rho(rho.co_gamma), sr.quantise_rho(rho.co_order), force_comm_ctas=lim.force_comm_ctas,
             selector_off=bool(lim.selector_off), default_C=lim.default_C, force_co_warps=lim.force_co_warps,
-            quanta_tile=rho.comm_quanta_per_tile)
+            quanta_tile=rho.comm_quanta_per_tile, co_min_waves=lim.co_min_waves)
     elif not lim.drain_help and lim.dep_model == B.MOE_DEP_TILE:
         # static partition with tile-level readiness
         idx = sr.comm_tile_ready_index(tiles, shape.TP, shape.T, shape.EP, shape.H, shape.L, occ.tile_n,
@@ -87,7 +87,8 @@ def _rand_inputs(rng):
     dh = 1 if family == "co" else (0 if family == "tile" else rng.choice([0, 0, 1]))
     lim = B.moe_sm_limits(rng.choice([4, 108, 148]), rng.randint(1, 160), 0, 0, 3, dh,
                           rng.choice([0, 1, 2, 4]), rng.choice([-1, -1, 0, 1, 3]), rng.choice([1, 8, 16, 200]),
-                          B.MOE_DEP_TILE if family == "tile" else rng.choice([B.MOE_DEP_SPLIT, B.MOE_DEP_TILE]))
+                          B.MOE_DEP_TILE if family == "tile" else rng.choice([B.MOE_DEP_SPLIT, B.MOE_DEP_TILE]),
+                          rng.choice([0, 0, 5, 24, 300]))
     rho = B.moe_rho(rng.uniform(0.05, 30.0), rng.choice([352, 704]), 128, rng.choice([128, 256]),
                     rng.choice([2, 4]), 17, 1024, rng.choice([B.MOE_RHO_PAPER, B.MOE_RHO_LOCAL]))
     if family == "co":
