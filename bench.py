@@ -29,8 +29,8 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "fused GEMM2+combine us/layer (whole step: routing build + analytical plan + fused kernel)"
-# workload -> (dram__bytes_read.sum + dram__bytes_write.sum of one fused launch, (tile_m, tile_n, L) it was captured at)
-NCU_TRAFFIC_BYTES = {"dsv2lite": (1819238000 + 1139128000, (256, 256, 2))}
+# workload -> (dram__bytes_read.sum + dram__bytes_write.sum of one fused launch, (tile_m, tile_n, L, co_warps) it was captured at)
+NCU_TRAFFIC_BYTES = {"dsv2lite": (2218184000 + 1095459000, (256, 256, 2, 2))}
 
 
 def load_peaks():
@@ -693,6 +693,10 @@ def main():
                     help="static partition: 0 = readiness per split (Eq. 9 as printed), 1 = per communication tile")
     ap.add_argument("--drain-help", type=int, default=1, choices=[0, 1],
                     help="1 (default): compute CTAs help with the communication tail; 0: the paper's static partition")
+    ap.add_argument("--probe", type=int, default=0,
+                    help="with --timeline: time GEMM-only launches with part of the data movement left out (bits: 1 = no W2 "
+                         "tile on every second k-block, 2 = no W2 tile at all, 4 = no Y stores); results are garbage, only "
+                         "the time means something")
     ap.add_argument("--timeline", action="store_true",
                     help="run the instrumented build (libmoe_b200_timeline.so, built on demand) and print where the "
                          "time of one fused launch goes per CTA role; honours --force-C / --no-comm-ctas / --co-warps / --L / --tile")
@@ -749,6 +753,16 @@ def main():
                                                                       force_co_warps=args.co_warps))
     K, W = max(1, args.steps), max(3, args.warmup)
 
+    if args.timeline and args.probe:
+        res = {}
+        for bits in (0, args.probe):
+            B.moe_set_probe(h, bits)
+            ts = time_fused(step, torch, 0, 3, 9, mode=B.MOE_MODE_GEMM_ONLY, P_override=lim.G // occ.comp_slot_sms)
+            res["gemm_only_us" if bits == 0 else f"gemm_only_us_probe_{bits}"] = statistics.median(ts)
+        B.moe_set_probe(h, 0)
+        print(json.dumps({"probe": args.probe, "workload": w.name, "tile": f"{w.tile_m}x{w.tile_n}", **res}))
+        B.moe_destroy(h)
+        return
     if args.timeline:
         run_timeline(h, dw, step, occ, lim, args)
         B.moe_destroy(h)
@@ -908,7 +922,7 @@ def main():
         # every byte the launch has to move through HBM (x, W2, Y written and read back, out): not part of the
         # headline roofline, but the real bound at small T, where every expert's weights are read for a few rows
         roofline["hbm_all_traffic_us"] = all_bytes / peaks["hbm_gbs"] / 1e3
-        if w.name in NCU_TRAFFIC_BYTES and (w.tile_m, w.tile_n, w.L) == NCU_TRAFFIC_BYTES[w.name][1]:
+        if w.name in NCU_TRAFFIC_BYTES and (w.tile_m, w.tile_n, w.L, plan.co_warps) == NCU_TRAFFIC_BYTES[w.name][1]:
             roofline["traffic"] = NCU_TRAFFIC_BYTES[w.name][0]
             roofline["traffic_algorithmic"] = all_bytes
         line = {

@@ -200,6 +200,14 @@ int32_t moe_set_wait_limit_ns(moe_handle *h, uint64_t ns);
  * reads the records.  [host] */
 #define MOE_TIMELINE_SLOTS 32
 int32_t moe_set_timeline(moe_handle *h, void *timeline_dev, size_t bytes);
+/* Timeline build only: later fused launches on this handle leave out part of their data movement, so that its
+ * cost shows in the launch time (the outputs of such a launch are garbage by construction; never for a result
+ * that is used).  Bits: MOE_PROBE_SKIP_ODD_W2 (the W2 tile of every second k-block is not loaded: a quarter
+ * less operand traffic), MOE_PROBE_SKIP_ALL_W2 (no W2 tile is loaded: half the operand traffic),
+ * MOE_PROBE_SKIP_Y_STORES (the epilogue converts but does not store: no Y write traffic; GEMM-only launches).
+ * 0 switches the probes off; the normal library accepts only 0 (MOE_ERR_UNSUPPORTED otherwise).  [host] */
+enum { MOE_PROBE_SKIP_ODD_W2 = 1, MOE_PROBE_SKIP_ALL_W2 = 2, MOE_PROBE_SKIP_Y_STORES = 4 };
+int32_t moe_set_probe(moe_handle *h, uint32_t probe_bits);
 
 /* Tile shape and residency of the GEMM2 kernel for (tile_m, tile_n), the communication tile,
  * the GPU limits and the stored service-rate constants (Section III-B, III-D, III-E).

@@ -34,7 +34,7 @@ EXPORTS = [
     "moe_clear_status",
     "moe_layer", "moe_calibrate_rho", "moe_host_arena_bytes", "moe_layer_host",
     "moe_gemm1_workspace_bytes", "moe_gemm1_act", "moe_post_router_layer", "moe_set_timeline",
-    "moe_select_tile", "moe_release_workspace",
+    "moe_select_tile", "moe_release_workspace", "moe_set_probe",
 ]
 
 
@@ -140,6 +140,7 @@ def lib():
         L.moe_set_timeline.argtypes = [vp, vp, C.c_size_t]
         L.moe_select_tile.argtypes = [vp, P(moe_shape), P(i32), P(i32)]
         L.moe_release_workspace.argtypes = [vp, vp]
+        L.moe_set_probe.argtypes = [vp, C.c_uint32]
         L.moe_host_arena_bytes.argtypes = [P(moe_shape), i32, i32, P(C.c_size_t)]
         L.moe_layer_host.argtypes = [vp, vp, vp, vp, vp, P(moe_shape), i32, i32, P(moe_sm_limits), vp,
                                      C.c_size_t, vp, vp, P(moe_plan), vp]
@@ -202,6 +203,11 @@ def moe_select_tile(h, shape: moe_shape):
     tm, tn = C.c_int32(), C.c_int32()
     _check(lib().moe_select_tile(h, C.byref(shape), C.byref(tm), C.byref(tn)), "moe_select_tile", h)
     return tm.value, tn.value
+
+
+def moe_set_probe(h, probe_bits: int):
+    """Timeline build only: leave out part of the data movement of later fused launches (garbage results)."""
+    _check(lib().moe_set_probe(h, probe_bits), "moe_set_probe", h)
 
 
 def moe_query_occupancy(h, tile_m: int, tile_n: int):

@@ -145,6 +145,18 @@ int32_t moe_set_timeline(moe_handle *h, void *timeline_dev, size_t bytes)
     return MOE_OK;
 }
 
+int32_t moe_set_probe(moe_handle *h, uint32_t probe_bits)
+{
+    if (!h) return MOE_ERR_NULL;
+    if (probe_bits && !fused_timeline_build()) {
+        snprintf(h->err, sizeof h->err, "moe_set_probe: this library was built without -DMOE_TIMELINE=1");
+        return MOE_ERR_UNSUPPORTED;
+    }
+    if (probe_bits & ~7u) return MOE_ERR_SHAPE;
+    h->probe = probe_bits;
+    return MOE_OK;
+}
+
 int32_t moe_query_occupancy(moe_handle *h, int32_t tile_m, int32_t tile_n, moe_occupancy *occ,
                             moe_sm_limits *limits, moe_rho *rho)
 {
@@ -463,6 +475,7 @@ int32_t moe_gemm2_combine(moe_handle *h, const void *x_routed, const void *W2, c
     p.timeline = nullptr;
     if (h->timeline && h->timeline_bytes >= ((size_t)grid * kTimelineSlots + MOE_MAX_L) * sizeof(unsigned long long))
         p.timeline = h->timeline;
+    p.probe = h->probe;
     e = pair ? pair_launch(p, grid, st) : fused_launch(TN, p, grid, st);
     if (e != cudaSuccess) return cuda_fail(h, e, "fused launch");
     return MOE_OK;

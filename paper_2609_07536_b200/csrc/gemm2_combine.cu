@@ -69,7 +69,13 @@ __device__ __forceinline__ void tl_put(const FusedParams &P, int slot, unsigned 
 {
     if (P.timeline) P.timeline[(size_t)blockIdx.x * kTimelineSlots + slot] = v;
 }
+// Probes of the timeline build (moe_set_probe): parts of the launch's data movement are left out so that their
+// cost shows in the launch time.  The results of a probed launch are garbage by construction.
+#define MOE_PROBE(bit) ((P.probe & (bit)) != 0)
+#else
+#define MOE_PROBE(bit) false
 #endif
+enum { kProbeSkipOddW2 = 1, kProbeSkipAllW2 = 2, kProbeSkipYStores = 4 };
 
 // --------------------------------------------------------------------------- shared memory
 
@@ -244,7 +250,7 @@ __device__ __forceinline__ void store_accumulator_rows(const FusedParams &P, uin
 __device__ __forceinline__ void emit_wide(const FusedParams &P, const uint32_t (&r)[32], int col, bool row_ok,
                                           __nv_bfloat16 *ybase, int q, int n0, int col_end, int cis0)
 {
-    if (!row_ok) return;
+    if (!row_ok || MOE_PROBE(kProbeSkipYStores)) return;
     const int cis = cis0 + col;
     const int slab = cis >> P.slab_shift;
     const int wslab = min(P.slab_cols, P.split_w - (slab << P.slab_shift));
@@ -382,10 +388,11 @@ __device__ void compute_cta(const FusedParams &P, int W_comp, uint8_t *ring, Con
                     TL(tl_pw += clock64() - tl_q);
                     const uint32_t full = smem_u32(&ctl->full[stage]);
                     const uint32_t a_dst = smem_u32(ring + stage * C::kStageBytes);
+                    const bool skip_b = MOE_PROBE(kProbeSkipAllW2) || (MOE_PROBE(kProbeSkipOddW2) && (kb & 1));
                     if (load_a) {
-                        mbar_arrive_expect_tx(full, (uint32_t)C::kStageBytes);
+                        mbar_arrive_expect_tx(full, (uint32_t)(skip_b ? C::kABytes : C::kStageBytes));
                         tma_load_2d(a_dst, &P.tmA, full, kx, row0);
-                    } else {
+                    } else if (!skip_b) {
                         tma_load_3d(a_dst + C::kABytes, &P.tmB, full, kx, n0, e);
                     }
                     armed |= 1u << stage;
@@ -661,10 +668,11 @@ __device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring
                     TL(tl_pw += clock64() - tl_q);
                     const uint32_t leader_full = own_full & 0xFEFFFFFFu;   // same offset in the leader CTA (rank 0)
                     const uint32_t a_dst = smem_u32(ring + stage * C::kStageBytes);
+                    const bool skip_b = MOE_PROBE(kProbeSkipAllW2) || (MOE_PROBE(kProbeSkipOddW2) && (kb & 1));
                     if (load_a) {
-                        if (leader_cta) mbar_arrive_expect_tx(own_full, 2u * (uint32_t)C::kStageBytes);
+                        if (leader_cta) mbar_arrive_expect_tx(own_full, 2u * (uint32_t)(skip_b ? C::kABytes : C::kStageBytes));
                         tma_load_2d_pair(a_dst, &P.tmA, leader_full, kx, row0);
-                    } else {
+                    } else if (!skip_b) {
                         tma_load_3d_pair(a_dst + C::kABytes, &P.tmB, leader_full, kx, n0, e);
                     }
                     armed |= 1u << stage;

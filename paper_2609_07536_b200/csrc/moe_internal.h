@@ -45,6 +45,7 @@ struct alignas(64) FusedParams {
     unsigned long long *queue_next;  // [L] ... of the next launch, zeroed by this one
     uint32_t *status;              // 4 words
     unsigned long long *timeline;  // timeline build: per-CTA records, then one stamp per split; else nullptr
+    uint32_t probe;                // timeline build: parts of the data movement left out (moe_set_probe); else 0
     void *out[MOE_MAX_EP];
     unsigned long long wait_ns;
     long long R_pad;
@@ -79,6 +80,7 @@ struct moe_handle {
     void *counts_event = nullptr;                       // cudaEvent_t: "the tile counts have reached the host"
     unsigned long long *timeline = nullptr;             // timeline build: where the next fused launch records
     size_t timeline_bytes = 0;
+    uint32_t probe = 0;                                 // timeline build: moe_set_probe bits for the next launches
 };
 
 namespace moe {
