@@ -346,6 +346,32 @@ def test_bounded_wait_reports_a_timeout_and_the_context_survives():
     assert np.max(np.abs(outs[0][:w.T] - expect)) <= G.tolerance(expect)
 
 
+def test_bounded_wait_with_co_resident_warps_winds_down_cleanly():
+    # a split that never completes (one readiness flag withheld): the co-resident warps that sleep on its counter
+    # and the communication CTAs that poll the tile give up at the limit, the launch returns, the context lives
+    h = G.handle()
+    w = replace(wl.TINY, name="withhold_co", T=512, E=4, k=2, H=512, I=128, TP=1, EP=1, tile_m=128, tile_n=128, L=2)
+    idx, wt, _ = wl.make_routing(w)
+    x, W2 = wl.make_data(w)
+    r = rr.build_routing(idx, w.E_tot, w.tile_m)
+    g_withheld = ((r["S"] - 1) * w.TP + 0) * (w.H // w.L // w.tile_n) + 0      # split 0, last m-tile, n-tile 0
+    B.moe_set_wait_limit_ns(h, 20_000_000)
+    try:
+        for tile in ((128, 128), (256, 256)):
+            wt_ = replace(w, tile_m=tile[0], tile_n=tile[1])
+            gw = g_withheld if tile[0] == 128 else 0
+            outs, plan, ws, S, st = G.run_layer(wt_, idx, wt, x, W2, force_C=2, withhold=gw, check_status=False,
+                                                drain_help=1, co_warps=2)
+            assert plan.co_warps == 2
+            assert st.code == B.MOE_DEV_TIMEOUT and st.where in (40, 44)
+            outs, plan, ws, S, st = G.run_layer(wt_, idx, wt, x, W2, ws=ws, drain_help=1, co_warps=2)
+            assert st.code == 0
+            expect, _ = _oracle_tokens(wt_, idx, wt, x, W2)
+            assert np.max(np.abs(outs[0][:w.T] - expect)) <= G.tolerance(expect)
+    finally:
+        B.moe_set_wait_limit_ns(h, 2_000_000_000)
+
+
 def test_argument_validation():
     h = G.handle()
     w = wl.TINY
