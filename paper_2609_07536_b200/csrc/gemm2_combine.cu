@@ -328,6 +328,133 @@ __device__ __forceinline__ void store_accumulator_rows_staged(const FusedParams 
     }
 }
 
+// --------------------------------------------------------------------------- epilogue and publisher roles
+//
+// Shared by the one-CTA and the CTA-pair compute roles (kPair: this CTA is rank `rank` of a pair and owns rows
+// rank * 128 ... of the 256-row tile; the accumulator buffer is handed back on the leader's barrier; the tile is
+// published in two parts, one flag per CTA).
+
+// Epilogue, one warp: TMEM -> bf16 -> Y for the warp's TMEM lane quarter and column group of every tile of
+// this CTA, then the hand-over to the publisher warp.
+template <int TN, bool kPair>
+__device__ __forceinline__ void epilogue_role(const FusedParams &P, int W_comp, Control *ctl, uint8_t *aux, int b,
+                                              uint32_t tmem_base, unsigned long long deadline, int rank)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int total_tiles = P.L * W_comp;
+    const int q4 = warp & 3;                   // TMEM lane quarter this warp may read
+    const int grp = (warp - 4) >> 2;           // column group of the tile
+    const int cols_per_group = epi_cols_per_group(TN, P.epi_warps >> 2);
+    const int col_first = grp * cols_per_group;
+    const int n_cols = max(0, min(cols_per_group, TN - col_first));
+    const int row_in_tile = (kPair ? rank * kMmaM : 0) + q4 * 32 + lane;
+    __nv_bfloat16 *Y = reinterpret_cast<__nv_bfloat16 *>(P.Y);
+    // Row bookkeeping runs ahead of the accumulators: the m-tile table entries are fetched two tiles
+    // ahead and the row's flat assignment one tile ahead, so that these dependent global loads are
+    // not in the way between an accumulator becoming ready and its first store.
+    int valid = 0, f_row = 0, valid_n = 0, first_n = 0;
+    TL_DECL(long long tl_ew = 0, tl_ek = 0, tl_q;)
+    if (b < total_tiles) {
+        const int mu0 = decode_tile(b, P, W_comp).mu;
+        const int mu1 = decode_tile(min(b + P.P, total_tiles - 1), P, W_comp).mu;
+        valid = __ldg(&P.mtile_valid[mu0]);
+        const int first0 = __ldg(&P.mtile_first_row[mu0]);
+        valid_n = __ldg(&P.mtile_valid[mu1]);
+        first_n = __ldg(&P.mtile_first_row[mu1]);
+        if (row_in_tile < valid) f_row = __ldg(&P.perm[first0 + row_in_tile]);
+    }
+    int it = 0;
+    for (int g = b; g < total_tiles; g += P.P, ++it) {
+        const Tile t = decode_tile(g, P, W_comp);
+        const int a = it & 1;
+        const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+        const int mu_nn = decode_tile(min(g + 2 * P.P, total_tiles - 1), P, W_comp).mu;
+        const int valid_nn = __ldg(&P.mtile_valid[mu_nn]);
+        const int first_nn = __ldg(&P.mtile_first_row[mu_nn]);
+        const int f_row_n = (row_in_tile < valid_n) ? __ldg(&P.perm[first_n + row_in_tile]) : 0;
+        TL(tl_q = clock64());
+        bool ok = wait_barrier(smem_u32(&ctl->tmem_full[a]), acc_phase, ctl, deadline, P.status, (uint32_t)g, 30u);
+        TL(tl_ew += clock64() - tl_q; tl_q = clock64());
+        if (ok) {
+            tc_fence_after();
+            const int n0 = t.s * P.split_w + t.i_n * TN;
+            const int col_end = min(P.H, (t.s + 1) * P.split_w);
+            const bool row_ok = row_in_tile < valid;
+            // destination of this thread's row: the routed row belongs to flat assignment
+            // f = (token, slot); Y is token-major so that the combine reads one contiguous block
+            __nv_bfloat16 *ybase = Y;
+            int q = 0;
+            if (row_ok) {
+                const int f = f_row;
+                const int tok = f / P.k_tot;
+                q = (f - tok * P.k_tot) * P.TP + t.p;
+                ybase = Y + ((size_t)tok * P.L + t.s) * (size_t)P.Q * (size_t)P.split_w;
+            }
+            const uint32_t taddr = tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(a * TN);
+            if (P.wide_store)
+                store_accumulator_rows_wide(P, taddr, col_first, n_cols, row_ok, ybase, q, n0, col_end, n0 - t.s * P.split_w);
+            else if (P.slab_cols >= 32)
+                store_accumulator_rows_staged(P, taddr, col_first, n_cols, row_ok, ybase, q, n0, col_end,
+                                              n0 - t.s * P.split_w, reinterpret_cast<EpiStage *>(aux) + (warp - 4));
+            else
+                store_accumulator_rows(P, taddr, col_first, n_cols, row_ok, ybase, q, n0, col_end, n0 - t.s * P.split_w);
+            // the accumulator buffer (this CTA's half of it) may be overwritten by the MMA of the tile after next
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {
+                if (kPair) mbar_arrive_cluster_relaxed(mapa_u32(smem_u32(&ctl->tmem_empty[a]), 0u));   // the leader's barrier
+                else mbar_arrive(smem_u32(&ctl->tmem_empty[a]));
+            }
+            TL(tl_ek += clock64() - tl_q);
+        }
+        // hand the tile to the publisher warp.  Its barrier is reused every other tile, so the warp
+        // first makes sure that the tile two back has been published (it normally has, long ago).
+        if (ok && it >= 2)
+            ok = wait_barrier(smem_u32(&ctl->pub_done[a]), (uint32_t)((it - 2) >> 1) & 1u, ctl, deadline, P.status,
+                              (uint32_t)g, 31u);
+        if (!ok) break;
+        __syncwarp();   // the lanes' stores are ordered before lane 0's arrival
+        if (lane == 0) mbar_arrive(smem_u32(&ctl->epi_done[a]));
+        valid = valid_n;
+        f_row = f_row_n;
+        valid_n = valid_nn;
+        first_n = first_nn;
+    }
+    TL(if (warp == 4 && lane == 0) { tl_put(P, kTlEpiWait, (unsigned long long)tl_ew); tl_put(P, kTlEpiWork, (unsigned long long)tl_ek); });
+}
+
+// Publisher, one thread of warp 3: raises the readiness flag of every finished tile.  The release costs a
+// microsecond or more (it waits for the CTA's stores to be performed); here it is off the path of the epilogue
+// warps, which go straight on to the next accumulator.
+template <bool kPair>
+__device__ __forceinline__ void publisher_role(const FusedParams &P, int W_comp, Control *ctl, int b,
+                                               unsigned long long deadline, int rank)
+{
+    const int total_tiles = P.L * W_comp;
+    if ((threadIdx.x & 31) == 0) {
+        int it = 0;
+        for (int g = b; g < total_tiles; g += P.P, ++it) {
+            const int a = it & 1;
+            if (!wait_barrier_1t(smem_u32(&ctl->epi_done[a]), (uint32_t)(it >> 1) & 1u, ctl, deadline, P.status,
+                                 (uint32_t)g, 32u))
+                break;
+            const Tile t = decode_tile(g, P, W_comp);
+            if (t.id != P.withhold) {
+                __threadfence();   // release: the epilogue warps' stores (observed through epi_done) come first
+                st_relaxed_u32(&P.flags[kPair ? 2 * t.id + rank : t.id], P.epoch);
+#if MOE_TIMELINE
+                if (atomicAdd(&P.split_done[t.s], 1u) + 1u == (uint32_t)(W_comp * P.flag_parts) && P.timeline)
+                    P.timeline[(size_t)gridDim.x * kTimelineSlots + t.s] = globaltimer_ns();
+#else
+                red_relaxed_add_u32(&P.split_done[t.s], 1u);
+#endif
+            }
+            mbar_arrive(smem_u32(&ctl->pub_done[a]));
+        }
+    }
+    __syncwarp();
+}
+
 // --------------------------------------------------------------------------- compute CTA
 
 template <int TN>
@@ -470,113 +597,9 @@ __device__ void compute_cta(const FusedParams &P, int W_comp, uint8_t *ring, Con
         }
         __syncwarp();
     } else if (warp >= 4 && warp < 4 + P.epi_warps) {
-        // ---------------- epilogue: TMEM -> bf16 -> Y, then publish the tile
-        const int q4 = warp & 3;                   // TMEM lane quarter this warp may read
-        const int grp = (warp - 4) >> 2;           // column group of the tile
-        const int cols_per_group = epi_cols_per_group(TN, P.epi_warps >> 2);
-        const int col_first = grp * cols_per_group;
-        const int n_cols = max(0, min(cols_per_group, TN - col_first));
-        const int row_in_tile = q4 * 32 + lane;
-        __nv_bfloat16 *Y = reinterpret_cast<__nv_bfloat16 *>(P.Y);
-        // Row bookkeeping runs ahead of the accumulators: the m-tile table entries are fetched two tiles
-        // ahead and the row's flat assignment one tile ahead, so that these dependent global loads are
-        // not in the way between an accumulator becoming ready and its first store.
-        int valid = 0, f_row = 0, valid_n = 0, first_n = 0;
-        TL_DECL(long long tl_ew = 0, tl_ek = 0, tl_q;)
-        if (b < total_tiles) {
-            const int mu0 = decode_tile(b, P, W_comp).mu;
-            const int mu1 = decode_tile(min(b + P.P, total_tiles - 1), P, W_comp).mu;
-            valid = __ldg(&P.mtile_valid[mu0]);
-            const int first0 = __ldg(&P.mtile_first_row[mu0]);
-            valid_n = __ldg(&P.mtile_valid[mu1]);
-            first_n = __ldg(&P.mtile_first_row[mu1]);
-            if (row_in_tile < valid) f_row = __ldg(&P.perm[first0 + row_in_tile]);
-        }
-        int it = 0;
-        for (int g = b; g < total_tiles; g += P.P, ++it) {
-            const Tile t = decode_tile(g, P, W_comp);
-            const int a = it & 1;
-            const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
-            const int mu_nn = decode_tile(min(g + 2 * P.P, total_tiles - 1), P, W_comp).mu;
-            const int valid_nn = __ldg(&P.mtile_valid[mu_nn]);
-            const int first_nn = __ldg(&P.mtile_first_row[mu_nn]);
-            const int f_row_n = (row_in_tile < valid_n) ? __ldg(&P.perm[first_n + row_in_tile]) : 0;
-            TL(tl_q = clock64());
-            bool ok = wait_barrier(smem_u32(&ctl->tmem_full[a]), acc_phase, ctl, deadline, P.status, (uint32_t)g, 30u);
-            ok = __all_sync(0xffffffffu, ok);
-            TL(tl_ew += clock64() - tl_q; tl_q = clock64());
-            if (ok) {
-                tc_fence_after();
-                const int n0 = t.s * P.split_w + t.i_n * TN;
-                const int col_end = min(P.H, (t.s + 1) * P.split_w);
-                const bool row_ok = row_in_tile < valid;
-                // destination of this thread's row: the routed row belongs to flat assignment
-                // f = (token, slot); Y is token-major so that the combine reads one contiguous block
-                __nv_bfloat16 *ybase = Y;
-                int q = 0;
-                if (row_ok) {
-                    const int f = f_row;
-                    const int tok = f / P.k_tot;
-                    q = (f - tok * P.k_tot) * P.TP + t.p;
-                    ybase = Y + ((size_t)tok * P.L + t.s) * (size_t)P.Q * (size_t)P.split_w;
-                }
-                if (P.wide_store)
-                    store_accumulator_rows_wide(P, tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(a * TN), col_first,
-                                                n_cols, row_ok, ybase, q, n0, col_end, n0 - t.s * P.split_w);
-                else if (P.slab_cols >= 32)
-                    store_accumulator_rows_staged(
-                        P, tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(a * TN), col_first, n_cols, row_ok,
-                        ybase, q, n0, col_end, n0 - t.s * P.split_w, reinterpret_cast<EpiStage *>(aux) + (warp - 4));
-                else
-                    store_accumulator_rows(P, tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(a * TN),
-                                                            col_first, n_cols, row_ok, ybase, q, n0, col_end,
-                                                            n0 - t.s * P.split_w);
-                // the accumulator buffer may be overwritten by the MMA of the tile after next
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&ctl->tmem_empty[a]));
-                TL(tl_ek += clock64() - tl_q);
-            }
-            // hand the tile to the publisher warp.  Its barrier is reused every other tile, so the warp
-            // first makes sure that the tile two back has been published (it normally has, long ago).
-            if (ok && it >= 2)
-                ok = wait_barrier(smem_u32(&ctl->pub_done[a]), (uint32_t)((it - 2) >> 1) & 1u, ctl, deadline, P.status,
-                                  (uint32_t)g, 31u);
-            if (!ok) break;
-            __syncwarp();   // the lanes' stores are ordered before lane 0's arrival
-            if (lane == 0) mbar_arrive(smem_u32(&ctl->epi_done[a]));
-            valid = valid_n;
-            f_row = f_row_n;
-            valid_n = valid_nn;
-            first_n = first_nn;
-        }
-        TL(if (warp == 4 && lane == 0) { tl_put(P, kTlEpiWait, (unsigned long long)tl_ew); tl_put(P, kTlEpiWork, (unsigned long long)tl_ek); });
+        epilogue_role<TN, false>(P, W_comp, ctl, aux, b, tmem_base, deadline, 0);
     } else if (warp == 3) {
-        // ---------------- publisher: one thread raises the readiness flag of every finished tile.  The
-        // release costs a microsecond or more (it waits for the CTA's stores to be performed); here it
-        // is off the path of the epilogue warps, which go straight on to the next accumulator.
-        if (lane == 0) {
-            int it = 0;
-            for (int g = b; g < total_tiles; g += P.P, ++it) {
-                const int a = it & 1;
-                if (!wait_barrier_1t(smem_u32(&ctl->epi_done[a]), (uint32_t)(it >> 1) & 1u, ctl, deadline, P.status,
-                                     (uint32_t)g, 32u))
-                    break;
-                const Tile t = decode_tile(g, P, W_comp);
-                if (t.id != P.withhold) {
-                    __threadfence();   // release: the epilogue warps' stores (observed through epi_done) come first
-                    st_relaxed_u32(&P.flags[t.id], P.epoch);
-#if MOE_TIMELINE
-                    if (atomicAdd(&P.split_done[t.s], 1u) + 1u == (uint32_t)(W_comp * P.flag_parts) && P.timeline)
-                        P.timeline[(size_t)gridDim.x * kTimelineSlots + t.s] = globaltimer_ns();
-#else
-                    red_relaxed_add_u32(&P.split_done[t.s], 1u);
-#endif
-                }
-                mbar_arrive(smem_u32(&ctl->pub_done[a]));
-            }
-        }
-        __syncwarp();
+        publisher_role<false>(P, W_comp, ctl, b, deadline, 0);
     }
     // ---------------- teardown
     tc_fence_before();
@@ -746,108 +769,9 @@ __device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring
         }
         __syncwarp();
     } else if (warp >= 4 && warp < 4 + P.epi_warps) {
-        // ---------------- epilogue (both CTAs): own 128 rows of the pair tile
-        const int q4 = warp & 3;
-        const int grp = (warp - 4) >> 2;
-        const int cols_per_group = epi_cols_per_group(TN, P.epi_warps >> 2);
-        const int col_first = grp * cols_per_group;
-        const int n_cols = max(0, min(cols_per_group, TN - col_first));
-        const int row_in_tile = (int)rank * kMmaM + q4 * 32 + lane;
-        __nv_bfloat16 *Y = reinterpret_cast<__nv_bfloat16 *>(P.Y);
-        // Row bookkeeping runs ahead of the accumulators: the m-tile table entries are fetched two tiles
-        // ahead and the row's flat assignment one tile ahead, so that these dependent global loads are
-        // not in the way between an accumulator becoming ready and its first store.
-        int valid = 0, f_row = 0, valid_n = 0, first_n = 0;
-        TL_DECL(long long tl_ew = 0, tl_ek = 0, tl_q;)
-        if (b < total_tiles) {
-            const int mu0 = decode_tile(b, P, W_comp).mu;
-            const int mu1 = decode_tile(min(b + P.P, total_tiles - 1), P, W_comp).mu;
-            valid = __ldg(&P.mtile_valid[mu0]);
-            const int first0 = __ldg(&P.mtile_first_row[mu0]);
-            valid_n = __ldg(&P.mtile_valid[mu1]);
-            first_n = __ldg(&P.mtile_first_row[mu1]);
-            if (row_in_tile < valid) f_row = __ldg(&P.perm[first0 + row_in_tile]);
-        }
-        int it = 0;
-        for (int g = b; g < total_tiles; g += P.P, ++it) {
-            const Tile t = decode_tile(g, P, W_comp);
-            const int a = it & 1;
-            const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
-            const int mu_nn = decode_tile(min(g + 2 * P.P, total_tiles - 1), P, W_comp).mu;
-            const int valid_nn = __ldg(&P.mtile_valid[mu_nn]);
-            const int first_nn = __ldg(&P.mtile_first_row[mu_nn]);
-            const int f_row_n = (row_in_tile < valid_n) ? __ldg(&P.perm[first_n + row_in_tile]) : 0;
-            TL(tl_q = clock64());
-            const bool ok = wait_barrier(smem_u32(&ctl->tmem_full[a]), acc_phase, ctl, deadline, P.status, (uint32_t)g, 30u);
-            TL(tl_ew += clock64() - tl_q; tl_q = clock64());
-            if (ok) {
-                tc_fence_after();
-                const int n0 = t.s * P.split_w + t.i_n * TN;
-                const int col_end = min(P.H, (t.s + 1) * P.split_w);
-                const bool row_ok = row_in_tile < valid;
-                __nv_bfloat16 *ybase = Y;
-                int q = 0;
-                if (row_ok) {
-                    const int f = f_row;
-                    const int tok = f / P.k_tot;
-                    q = (f - tok * P.k_tot) * P.TP + t.p;
-                    ybase = Y + ((size_t)tok * P.L + t.s) * (size_t)P.Q * (size_t)P.split_w;
-                }
-                if (P.wide_store)
-                    store_accumulator_rows_wide(P, tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(a * TN), col_first,
-                                                n_cols, row_ok, ybase, q, n0, col_end, n0 - t.s * P.split_w);
-                else if (P.slab_cols >= 32)
-                    store_accumulator_rows_staged(
-                        P, tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(a * TN), col_first, n_cols, row_ok,
-                        ybase, q, n0, col_end, n0 - t.s * P.split_w, reinterpret_cast<EpiStage *>(aux) + (warp - 4));
-                else
-                    store_accumulator_rows(P, tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(a * TN),
-                                                            col_first, n_cols, row_ok, ybase, q, n0, col_end,
-                                                            n0 - t.s * P.split_w);
-                // this CTA's half of the accumulator buffer is drained: tell the leader's MMA warp
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive_cluster_relaxed(mapa_u32(smem_u32(&ctl->tmem_empty[a]), 0u));
-                TL(tl_ek += clock64() - tl_q);
-            }
-            // hand the tile to the publisher warp (see compute_cta)
-            bool ok2 = ok;
-            if (ok2 && it >= 2)
-                ok2 = wait_barrier(smem_u32(&ctl->pub_done[a]), (uint32_t)((it - 2) >> 1) & 1u, ctl, deadline, P.status,
-                                   (uint32_t)g, 31u);
-            if (!ok2) break;
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&ctl->epi_done[a]));
-            valid = valid_n;
-            f_row = f_row_n;
-            valid_n = valid_nn;
-            first_n = first_nn;
-        }
-        TL(if (warp == 4 && lane == 0) { tl_put(P, kTlEpiWait, (unsigned long long)tl_ew); tl_put(P, kTlEpiWork, (unsigned long long)tl_ek); });
+        epilogue_role<TN, true>(P, W_comp, ctl, aux, b, tmem_base, deadline, (int)rank);
     } else if (warp == 3) {
-        // ---------------- publisher (both CTAs): raises this CTA's flag of every finished pair tile
-        if (lane == 0) {
-            int it = 0;
-            for (int g = b; g < total_tiles; g += P.P, ++it) {
-                const int a = it & 1;
-                if (!wait_barrier_1t(smem_u32(&ctl->epi_done[a]), (uint32_t)(it >> 1) & 1u, ctl, deadline, P.status,
-                                     (uint32_t)g, 32u))
-                    break;
-                const Tile t = decode_tile(g, P, W_comp);
-                if (t.id != P.withhold) {
-                    __threadfence();
-                    st_relaxed_u32(&P.flags[2 * t.id + (int)rank], P.epoch);
-#if MOE_TIMELINE
-                    if (atomicAdd(&P.split_done[t.s], 1u) + 1u == (uint32_t)(W_comp * P.flag_parts) && P.timeline)
-                        P.timeline[(size_t)gridDim.x * kTimelineSlots + t.s] = globaltimer_ns();
-#else
-                    red_relaxed_add_u32(&P.split_done[t.s], 1u);
-#endif
-                }
-                mbar_arrive(smem_u32(&ctl->pub_done[a]));
-            }
-        }
-        __syncwarp();
+        publisher_role<true>(P, W_comp, ctl, b, deadline, (int)rank);
     }
     // ---------------- teardown: nobody leaves while its peer may still touch its memory (the co-resident
     // communication warps arrived on this cluster barrier right after the set-up one)
