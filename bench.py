@@ -438,7 +438,8 @@ def run_decode(h, args, device, peaks):
 # csrc/gemm2_combine.cu.
 
 TL = dict(begin=0, role=1, first_acc=2, mma_end=3, tiles=4, wait_operand=5, issue=6, wait_tmem=7, mma_cycles=8,
-          compute_end=9, cta_end=10, epi_wait=11, epi_work=12, producer_wait=13, comm_units=14, comm_wait_ns=15, co=16)
+          compute_end=9, cta_end=10, epi_wait=11, epi_work=12, producer_wait=13, comm_units=14, comm_wait_ns=15, co=16,
+          pub_wait=32, pub_fence=33, epi_pub_wait=34)
 
 
 def run_timeline(h, dw, step, occ, lim, args):
@@ -491,6 +492,10 @@ def run_timeline(h, dw, step, occ, lim, args):
         "epilogue_warp_cycles_per_tile": {
             "waiting": float(np.median(allc[:, TL["epi_wait"]] / np.maximum(1, comp[:, TL["tiles"]].mean()))),
             "working": float(np.median(allc[:, TL["epi_work"]] / np.maximum(1, comp[:, TL["tiles"]].mean())))} if allc.size else None,
+        "publisher_cycles_per_tile": {
+            "waiting_for_the_epilogue": float(np.median(allc[:, TL["pub_wait"]]) / max(1.0, float(comp[:, TL["tiles"]].mean()))),
+            "fence_and_flag": float(np.median(allc[:, TL["pub_fence"]]) / max(1.0, float(comp[:, TL["tiles"]].mean()))),
+            "epilogue_warp_waiting_for_the_publisher": float(np.median(allc[:, TL["epi_pub_wait"]]) / max(1.0, float(comp[:, TL["tiles"]].mean())))} if allc.size else None,
         "producer_wait_cycles_per_kblock": float(np.median(allc[:, TL["producer_wait"]]) / max(1.0, float(np.median(kb)))) if comp.size else None,
     }
     Q = w.k_tot * w.TP

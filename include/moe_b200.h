@@ -198,7 +198,7 @@ int32_t moe_set_wait_limit_ns(moe_handle *h, uint64_t ns);
  * that is too small for a launch is left alone].  NULL switches recording off.  The normal library accepts
  * only NULL (MOE_ERR_UNSUPPORTED otherwise): its kernels carry no instrumentation.  bench.py --timeline
  * reads the records.  [host] */
-#define MOE_TIMELINE_SLOTS 32
+#define MOE_TIMELINE_SLOTS 40
 int32_t moe_set_timeline(moe_handle *h, void *timeline_dev, size_t bytes);
 /* Timeline build only: later fused launches on this handle leave out part of their data movement, so that its
  * cost shows in the launch time (the outputs of such a launch are garbage by construction; never for a result

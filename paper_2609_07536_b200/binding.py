@@ -82,7 +82,7 @@ class moe_status(C.Structure):
 
 
 TIMELINE_LIB_PATH = os.path.join(HERE, "libmoe_b200_timeline.so")
-MOE_TIMELINE_SLOTS = 32
+MOE_TIMELINE_SLOTS = 40
 
 _lib = None
 _lib_path = LIB_PATH

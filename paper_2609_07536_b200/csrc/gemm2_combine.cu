@@ -62,7 +62,8 @@ namespace {
 enum {
     kTlBegin = 0, kTlRole = 1, kTlFirstAcc = 2, kTlMmaEnd = 3, kTlTiles = 4, kTlWaitOperand = 5, kTlIssue = 6,
     kTlWaitTmem = 7, kTlMmaCycles = 8, kTlComputeEnd = 9, kTlCtaEnd = 10, kTlEpiWait = 11, kTlEpiWork = 12,
-    kTlProducerWait = 13, kTlCommUnits = 14, kTlCommWaitNs = 15, kTlCoWarp = 16   // 8 slots per co-resident warp
+    kTlProducerWait = 13, kTlCommUnits = 14, kTlCommWaitNs = 15, kTlCoWarp = 16,  // 8 slots per co-resident warp (16..31)
+    kTlPubWait = 32, kTlPubFence = 33, kTlEpiPubWait = 34
 };
 #if MOE_TIMELINE
 __device__ __forceinline__ void tl_put(const FusedParams &P, int slot, unsigned long long v)
@@ -90,13 +91,17 @@ struct Cfg {
     // column group when the launch carries no co-resident communication warps (FusedParams::epi_warps)
 };
 
+// Tiles a CTA may have stored but not yet published: the publisher's release fence takes thousands of cycles,
+// and one fence covers every tile whose epilogue is over by then.
+constexpr int kPubSlots = 4;
+
 struct Control {
     unsigned long long full[8];
     unsigned long long empty[8];
     unsigned long long tmem_full[2];
     unsigned long long tmem_empty[2];
-    unsigned long long epi_done[2];     // every epilogue warp has stored its rows of the tile (per accumulator buffer)
-    unsigned long long pub_done[2];     // the publisher warp has raised that tile's flag
+    unsigned long long epi_done[kPubSlots];   // every epilogue warp has stored its rows of the tile (tile number mod kPubSlots)
+    unsigned long long pub_done[kPubSlots];   // the publisher warp has raised that tile's flag
     uint32_t tmem_base;
     volatile uint32_t abort;
     unsigned long long comm_full[24];   // communication CTA: one barrier per warp and stage
@@ -353,7 +358,7 @@ __device__ __forceinline__ void epilogue_role(const FusedParams &P, int W_comp, 
     // ahead and the row's flat assignment one tile ahead, so that these dependent global loads are
     // not in the way between an accumulator becoming ready and its first store.
     int valid = 0, f_row = 0, valid_n = 0, first_n = 0;
-    TL_DECL(long long tl_ew = 0, tl_ek = 0, tl_q;)
+    TL_DECL(long long tl_ew = 0, tl_ek = 0, tl_ep = 0, tl_q;)
     if (b < total_tiles) {
         const int mu0 = decode_tile(b, P, W_comp).mu;
         const int mu1 = decode_tile(min(b + P.P, total_tiles - 1), P, W_comp).mu;
@@ -407,25 +412,31 @@ __device__ __forceinline__ void epilogue_role(const FusedParams &P, int W_comp, 
             }
             TL(tl_ek += clock64() - tl_q);
         }
-        // hand the tile to the publisher warp.  Its barrier is reused every other tile, so the warp
-        // first makes sure that the tile two back has been published (it normally has, long ago).
-        if (ok && it >= 2)
-            ok = wait_barrier(smem_u32(&ctl->pub_done[a]), (uint32_t)((it - 2) >> 1) & 1u, ctl, deadline, P.status,
-                              (uint32_t)g, 31u);
+        // hand the tile to the publisher warp.  Its barrier is reused every kPubSlots tiles, so the warp first
+        // makes sure that the tile kPubSlots back has been published (it normally has, long ago).
+        const int slot = it & (kPubSlots - 1);
+        TL(tl_q = clock64());
+        if (ok && it >= kPubSlots)
+            ok = wait_barrier(smem_u32(&ctl->pub_done[slot]), (uint32_t)((it - kPubSlots) / kPubSlots) & 1u, ctl, deadline,
+                              P.status, (uint32_t)g, 31u);
+        TL(tl_ep += clock64() - tl_q);
         if (!ok) break;
         __syncwarp();   // the lanes' stores are ordered before lane 0's arrival
-        if (lane == 0) mbar_arrive(smem_u32(&ctl->epi_done[a]));
+        if (lane == 0) mbar_arrive(smem_u32(&ctl->epi_done[slot]));
         valid = valid_n;
         f_row = f_row_n;
         valid_n = valid_nn;
         first_n = first_nn;
     }
-    TL(if (warp == 4 && lane == 0) { tl_put(P, kTlEpiWait, (unsigned long long)tl_ew); tl_put(P, kTlEpiWork, (unsigned long long)tl_ek); });
+    TL(if (warp == 4 && lane == 0) { tl_put(P, kTlEpiWait, (unsigned long long)tl_ew); tl_put(P, kTlEpiWork, (unsigned long long)tl_ek);
+                                      tl_put(P, kTlEpiPubWait, (unsigned long long)tl_ep); });
 }
 
-// Publisher, one thread of warp 3: raises the readiness flag of every finished tile.  The release costs a
-// microsecond or more (it waits for the CTA's stores to be performed); here it is off the path of the epilogue
-// warps, which go straight on to the next accumulator.
+// Publisher, one thread of warp 3: raises the readiness flag of every finished tile.  The release costs
+// microseconds (the fence waits until the CTA's stores to Y have been performed: 2800 cycles per tile at the
+// DeepSeek shape, 4900 at the Granite shape, where a tile's four k-blocks take less than that); here it is off
+// the path of the epilogue warps, which go straight on to the next accumulator, and one fence covers every tile
+// whose epilogue has finished by then (up to kPubSlots).
 template <bool kPair>
 __device__ __forceinline__ void publisher_role(const FusedParams &P, int W_comp, Control *ctl, int b,
                                                unsigned long long deadline, int rank)
@@ -433,24 +444,36 @@ __device__ __forceinline__ void publisher_role(const FusedParams &P, int W_comp,
     const int total_tiles = P.L * W_comp;
     if ((threadIdx.x & 31) == 0) {
         int it = 0;
-        for (int g = b; g < total_tiles; g += P.P, ++it) {
-            const int a = it & 1;
-            if (!wait_barrier_1t(smem_u32(&ctl->epi_done[a]), (uint32_t)(it >> 1) & 1u, ctl, deadline, P.status,
-                                 (uint32_t)g, 32u))
+        TL_DECL(long long tl_pw = 0, tl_pf = 0, tl_q;)
+        for (int g = b; g < total_tiles;) {
+            TL(tl_q = clock64());
+            if (!wait_barrier_1t(smem_u32(&ctl->epi_done[it & (kPubSlots - 1)]), (uint32_t)(it / kPubSlots) & 1u, ctl,
+                                 deadline, P.status, (uint32_t)g, 32u))
                 break;
-            const Tile t = decode_tile(g, P, W_comp);
-            if (t.id != P.withhold) {
-                __threadfence();   // release: the epilogue warps' stores (observed through epi_done) come first
-                st_relaxed_u32(&P.flags[kPair ? 2 * t.id + rank : t.id], P.epoch);
+            TL(tl_pw += clock64() - tl_q; tl_q = clock64());
+            // the following tiles too, as far as their epilogues are already over (waiting for more of them before
+            // the fence was measured: no gain)
+            int n = 1;
+            while (n < kPubSlots && g + n * P.P < total_tiles &&
+                   mbar_test_wait(smem_u32(&ctl->epi_done[(it + n) & (kPubSlots - 1)]), (uint32_t)((it + n) / kPubSlots) & 1u))
+                ++n;
+            fence_acq_rel_gpu();   // release: the epilogue warps' stores (observed through epi_done) come first
+            for (int j = 0; j < n; ++j, ++it, g += P.P) {
+                const Tile t = decode_tile(g, P, W_comp);
+                if (t.id != P.withhold) {
+                    st_relaxed_u32(&P.flags[kPair ? 2 * t.id + rank : t.id], P.epoch);
 #if MOE_TIMELINE
-                if (atomicAdd(&P.split_done[t.s], 1u) + 1u == (uint32_t)(W_comp * P.flag_parts) && P.timeline)
-                    P.timeline[(size_t)gridDim.x * kTimelineSlots + t.s] = globaltimer_ns();
+                    if (atomicAdd(&P.split_done[t.s], 1u) + 1u == (uint32_t)(W_comp * P.flag_parts) && P.timeline)
+                        P.timeline[(size_t)gridDim.x * kTimelineSlots + t.s] = globaltimer_ns();
 #else
-                red_relaxed_add_u32(&P.split_done[t.s], 1u);
+                    red_relaxed_add_u32(&P.split_done[t.s], 1u);
 #endif
+                }
+                mbar_arrive(smem_u32(&ctl->pub_done[it & (kPubSlots - 1)]));
             }
-            mbar_arrive(smem_u32(&ctl->pub_done[a]));
+            TL(tl_pf += clock64() - tl_q);
         }
+        TL(tl_put(P, kTlPubWait, (unsigned long long)tl_pw); tl_put(P, kTlPubFence, (unsigned long long)tl_pf));
     }
     __syncwarp();
 }
@@ -474,6 +497,8 @@ __device__ void compute_cta(const FusedParams &P, int W_comp, uint8_t *ring, Con
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&ctl->tmem_full[i]), 1);
             mbar_init(smem_u32(&ctl->tmem_empty[i]), (uint32_t)P.epi_warps);
+        }
+        for (int i = 0; i < kPubSlots; ++i) {
             mbar_init(smem_u32(&ctl->epi_done[i]), (uint32_t)P.epi_warps);
             mbar_init(smem_u32(&ctl->pub_done[i]), 1);
         }
@@ -648,6 +673,8 @@ __device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&ctl->tmem_full[i]), 1);
             mbar_init(smem_u32(&ctl->tmem_empty[i]), 2u * (uint32_t)P.epi_warps);
+        }
+        for (int i = 0; i < kPubSlots; ++i) {
             mbar_init(smem_u32(&ctl->epi_done[i]), (uint32_t)P.epi_warps);
             mbar_init(smem_u32(&ctl->pub_done[i]), 1);
         }

@@ -23,7 +23,7 @@ constexpr int kCommTileM = 128;        // T_M^comm
 constexpr int kCommTileN = 1024;       // T_N^comm
 constexpr int kRoutingChunk = 256;     // flat assignments handled by one warp while sorting
 constexpr uint64_t kDefaultWaitNs = 2000000000ull;
-constexpr int kTimelineSlots = 32;     // 64-bit words per CTA in a timeline buffer (timeline build only)
+constexpr int kTimelineSlots = 40;     // 64-bit words per CTA in a timeline buffer (timeline build only)
 
 // Parameters of one fused launch.  Passed by value (__grid_constant__): the two tensor maps
 // must sit in kernel parameter space, 64-byte aligned.
