@@ -442,35 +442,45 @@ int32_t moe_gemm2_combine(moe_handle *h, const void *x_routed, const void *W2, c
     p.queue_next = reinterpret_cast<unsigned long long *>(flags_ws + 2 * MOE_MAX_L) + ((ep + 1u) & 1u) * MOE_MAX_L;
     p.flags = flags_ws + kSplitCounterWords;
 
-    // tensor maps (Section II-A operands): x_routed [R, I] and W2 [E_tot, H, I], k contiguous
-    EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(h->encode_tiled);
-    const cuuint64_t R = (cuuint64_t)s->T * s->k_tot;
-    {
-        cuuint64_t dims[2] = {(cuuint64_t)s->I, R};
-        cuuint64_t strides[1] = {(cuuint64_t)s->I * 2};
-        cuuint32_t box[2] = {(cuuint32_t)kBlockK, (cuuint32_t)kMmaM};
-        cuuint32_t es[2] = {1, 1};
-        CUresult cr = encode(&p.tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(x_routed), dims,
-                             strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-        if (cr != CUDA_SUCCESS) {
-            snprintf(h->err, sizeof h->err, "cuTensorMapEncodeTiled(x_routed) failed: %d", (int)cr);
-            return MOE_ERR_CUDA;
+    // tensor maps (Section II-A operands): x_routed [R, I] and W2 [E_tot, H, I], k contiguous.  Encoding the two
+    // maps costs microseconds of host time between the wait for the tile counts and the launch: the handle
+    // keeps the last pair and reuses it while buffers, sizes and tile family stay the same (a loop of steps).
+    const TensorMapKey key = {x_routed, W2, s->T, s->k_tot, s->I, s->H, s->E_tot, pair ? TN / 2 : TN};
+    if (!h->tm_valid || memcmp(&h->tm_key, &key, sizeof key) != 0) {
+        EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(h->encode_tiled);
+        const cuuint64_t R = (cuuint64_t)s->T * s->k_tot;
+        h->tm_valid = false;
+        {
+            cuuint64_t dims[2] = {(cuuint64_t)s->I, R};
+            cuuint64_t strides[1] = {(cuuint64_t)s->I * 2};
+            cuuint32_t box[2] = {(cuuint32_t)kBlockK, (cuuint32_t)kMmaM};
+            cuuint32_t es[2] = {1, 1};
+            CUresult cr = encode(&h->tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(x_routed), dims,
+                                 strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (cr != CUDA_SUCCESS) {
+                snprintf(h->err, sizeof h->err, "cuTensorMapEncodeTiled(x_routed) failed: %d", (int)cr);
+                return MOE_ERR_CUDA;
+            }
         }
-    }
-    {
-        cuuint64_t dims[3] = {(cuuint64_t)s->I, (cuuint64_t)s->H, (cuuint64_t)s->E_tot};
-        cuuint64_t strides[2] = {(cuuint64_t)s->I * 2, (cuuint64_t)s->H * s->I * 2};
-        cuuint32_t box[3] = {(cuuint32_t)kBlockK, (cuuint32_t)(pair ? TN / 2 : TN), 1};   // a pair CTA loads half the rows
-        cuuint32_t es[3] = {1, 1, 1};
-        CUresult cr = encode(&p.tmB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(W2), dims, strides,
-                             box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-        if (cr != CUDA_SUCCESS) {
-            snprintf(h->err, sizeof h->err, "cuTensorMapEncodeTiled(W2) failed: %d", (int)cr);
-            return MOE_ERR_CUDA;
+        {
+            cuuint64_t dims[3] = {(cuuint64_t)s->I, (cuuint64_t)s->H, (cuuint64_t)s->E_tot};
+            cuuint64_t strides[2] = {(cuuint64_t)s->I * 2, (cuuint64_t)s->H * s->I * 2};
+            cuuint32_t box[3] = {(cuuint32_t)kBlockK, (cuuint32_t)(pair ? TN / 2 : TN), 1};   // a pair CTA loads half the rows
+            cuuint32_t es[3] = {1, 1, 1};
+            CUresult cr = encode(&h->tmB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(W2), dims, strides,
+                                 box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (cr != CUDA_SUCCESS) {
+                snprintf(h->err, sizeof h->err, "cuTensorMapEncodeTiled(W2) failed: %d", (int)cr);
+                return MOE_ERR_CUDA;
+            }
         }
+        h->tm_key = key;
+        h->tm_valid = true;
     }
+    p.tmA = h->tmA;
+    p.tmB = h->tmB;
     const int grid = pair ? ((C + 1) & ~1) + 2 * Pc : C + Pc;
     p.timeline = nullptr;
     if (h->timeline && h->timeline_bytes >= ((size_t)grid * kTimelineSlots + MOE_MAX_L) * sizeof(unsigned long long))

@@ -67,6 +67,14 @@ struct alignas(64) FusedParams {
 
 }  // namespace moe
 
+namespace moe {
+// what the two operand tensor maps of the fused kernel depend on
+struct TensorMapKey {
+    const void *x, *w2;
+    int32_t T, k_tot, I, H, E_tot, box_n;
+};
+}  // namespace moe
+
 struct moe_handle {
     int device = 0;
     int G = 0;
@@ -81,6 +89,9 @@ struct moe_handle {
     unsigned long long *timeline = nullptr;             // timeline build: where the next fused launch records
     size_t timeline_bytes = 0;
     uint32_t probe = 0;                                 // timeline build: moe_set_probe bits for the next launches
+    CUtensorMap tmA, tmB;                               // last encoded operand tensor maps of the fused kernel ...
+    moe::TensorMapKey tm_key = {};                      // ... and what they were encoded for
+    bool tm_valid = false;
 };
 
 namespace moe {
