@@ -893,6 +893,24 @@ def main():
         extra["solver_ns"] = B.moe_time_plan_partition(sets, occ, lim, dw.shape, rho, 1_000_000)
         if not args.no_cpu_baseline:
             extra["cpu_baseline"], _ = cpu_baseline(w, dw.idx, dw.wt, dw.x_cpu, dw.W2_cpu)
+        # ---- context: the library GEMM (cuBLAS through torch.matmul) on a dense problem with the same FLOPs and the
+        # same contraction length K = I / TP: [R * TP, K] x [K, H].  Not part of the operator: it says what a dense
+        # GEMM without routing, padding, scattered stores and flags reaches at this K on this GPU.
+        a_ = torch.randn((w.R * w.TP, w.I // w.TP), device=device, dtype=torch.bfloat16)
+        b_ = torch.randn((w.H, w.I // w.TP), device=device, dtype=torch.bfloat16)
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(9)]
+        for _ in range(2):
+            c_ = a_ @ b_.t()
+        for ea, eb in evs:
+            ea.record(); c_ = a_ @ b_.t(); eb.record()
+        torch.cuda.synchronize()
+        cub = statistics.median(ea.elapsed_time(eb) * 1e3 for ea, eb in evs)
+        extra["context_cublas_same_flops"] = {
+            "shape": [w.R * w.TP, w.H, w.I // w.TP], "us": cub, "tflops": dw.flops / cub / 1e6,
+            "gemm_only_over_cublas": cub / extra["gemm_only"]["us"],
+            "what": "torch.matmul (cuBLAS) on a dense bf16 GEMM of the same FLOPs and K, timed alone; context, not a target"}
+        del a_, b_, c_
+        torch.cuda.empty_cache()
         # ---- the other named workloads, briefly (a second or two each): fused time and roofline fractions
         if args.workload == "dsv2lite" and not args.tile and not args.T and not args.L:
             extra["other_configs"] = [quick_config(h, wl.CONFIGS[n], device, peaks) for n in ("granite3moe", "qwen15moe")]
