@@ -15,9 +15,10 @@
 //               W2 tile (tile_n rows x 64 k) of every k-block, into a ring of 128B-swizzled stages;
 //   warp 1      MMA issuer (one thread): tcgen05.mma (M = 128, N = tile_n, K = 16, bf16 -> fp32) into one
 //               of two TMEM accumulator buffers; tcgen05.commit frees stages / publishes the tile;
-//   warps 4-15  epilogue: tcgen05.ld -> bf16 -> Y (three column groups x four TMEM lane quarters);
-//   warp 3      publisher (one thread): once the twelve epilogue warps have stored a tile, release fence,
-//               then the tile's readiness flag and the split counter.
+//   warps 4-15  epilogue: tcgen05.ld -> bf16 -> Y (three column groups x four TMEM lane quarters; warps 16-19
+//               are a fourth column group when the launch carries no co-resident communication warp);
+//   warp 3      publisher (one thread): once the epilogue warps have stored a tile, release fence, then the
+//               tile's readiness flag and the split counter (one fence for all tiles stored by then).
 // Compute CTA pair (256 x 256 tiles): the same roles in both CTAs of a cluster of two; one
 //   tcgen05.mma.cta_group::2 spans both SMs, each CTA loads only its own operand halves.
 // Y is token-major: the epilogue scatters each accumulator row to its (token, slot, shard) place, so
@@ -27,8 +28,8 @@
 //   checked first: split counter, else per-tile flags with ld.acquire.gpu; bounded), sums the rows in
 //   fp32 in (j, p) order with the token's weights and stores bf16 into the owning rank's buffer.
 // Co-resident communication warps (Section III-B with o_comm > 1 in spirit: communication work that
-//   shares an SM with a compute CTA instead of reserving one): every compute CTA carries up to four
-//   extra warps (16-19) that run the same per-unit pipeline on stages of their own, take work from
+//   shares an SM with a compute CTA instead of reserving one): a compute CTA may carry extra warps
+//   (of 16-19; two have stages) that run the same per-unit pipeline on stages of their own, take work from
 //   the front of the per-split queues and serve split s while the CTA's other warps compute split
 //   s + 1.  They wait for a whole split (no token of a split is complete before the last expert's
 //   tiles of that split are), not for single tiles.
