@@ -429,7 +429,8 @@ def run_decode(h, args, device, peaks):
                                     "and read back, out): at decode sizes the weights dominate, the headline roofline "
                                     "(FLOPs or combine bytes) does not bound these launches",
                      "kernel": "moe_gemm2_combine_kernel", "kernel_us": main["fused_kernel_us"]},
-        "decode": rows, "cpu_baseline": None, "e2e": None, "gpu_launches": 5 * main["steps"],
+        "decode": rows, "cpu_baseline": None, "e2e": None,
+        "gpu_launches": 2 * main["steps"],      # one routing launch (single-CTA build at these sizes) + the fused launch
     }))
 
 

@@ -4,7 +4,7 @@
 // ceil(M_e / T_M) tiles along the token dimension; Eq. 16: their sum S.
 // The routed rows are the flat assignments f = t * k_tot + j in a *stable* order by expert.
 //
-// Four small launches (the data is a few hundred KB):
+// Four small launches (the data is a few hundred KB; one launch of one CTA for small batches, routing_small):
 //   1. hist          every warp histograms its own contiguous chunk of assignments;
 //   2. scan_columns  one CTA per expert: exclusive prefix of that expert's histogram column over
 //                    the warps (the per-(warp, expert) bases) and the expert's count;
@@ -170,6 +170,108 @@ routing_scatter(const int32_t *__restrict__ topk_idx, int R, int E_tot, int tile
     }
 }
 
+// The same four steps in ONE launch of one CTA, for small and decode-sized batches (at most 32 chunks of
+// 256 assignments, at most 256 experts): the per-warp histograms live in shared memory, the steps are
+// separated by CTA barriers instead of launch boundaries.  Same arithmetic, same outputs, bit for bit; four
+// launches cost ~30 us of which the work is a few microseconds at these sizes.
+constexpr int kSmallWarps = 32;
+constexpr int kSmallMaxExperts = 256;
+__global__ void __launch_bounds__(kSmallWarps * 32)
+routing_small(const int32_t *__restrict__ topk_idx, int R, int k_tot, int E_tot, int tile_m, int n_warps, int max_mtiles,
+              int32_t *__restrict__ counts, int32_t *__restrict__ offsets, int32_t *__restrict__ tiles,
+              int32_t *__restrict__ tile_offsets, int32_t *__restrict__ mtile_expert,
+              int32_t *__restrict__ mtile_first_row, int32_t *__restrict__ mtile_valid, int32_t *__restrict__ perm,
+              int32_t *__restrict__ inv_perm, int32_t *__restrict__ pad_row, uint32_t *status)
+{
+    extern __shared__ int32_t sm[];
+    int32_t *whist = sm;                                   // [kSmallWarps][E_tot]
+    int32_t *s_cnt = sm + kSmallWarps * E_tot, *s_off = s_cnt + (E_tot + 1), *s_toff = s_off + (E_tot + 1);
+    const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    int32_t *h = whist + w * E_tot;
+    // 1. per-warp histograms of the warp's chunk
+    for (int e = lane; e < E_tot; e += 32) h[e] = 0;
+    __syncwarp();
+    const int begin = w * kRoutingChunk;
+    const int end = w < n_warps ? min(R, begin + kRoutingChunk) : begin;
+    for (int f = begin + lane; f < end; f += 32) {
+        const int e = topk_idx[f];
+        if (e < 0 || e >= E_tot) {
+            report(status, MOE_DEV_OOB, (uint32_t)f, 1u);
+            continue;
+        }
+        atomicAdd(&h[e], 1);
+        const int t = f / k_tot, j = f - t * k_tot;
+        for (int jj = 0; jj < j; ++jj)
+            if (topk_idx[t * k_tot + jj] == e) report(status, MOE_DEV_DUP_EXPERT, (uint32_t)t, 1u);
+    }
+    __syncthreads();
+    // 2. per expert: exclusive prefix of its histogram column over the warps, and its count
+    for (int e = threadIdx.x; e < E_tot; e += blockDim.x) {
+        int base = 0;
+        for (int ww = 0; ww < n_warps; ++ww) {
+            const int c = whist[ww * E_tot + e];
+            whist[ww * E_tot + e] = base;
+            base += c;
+        }
+        s_cnt[e] = base;
+        counts[e] = base;
+    }
+    __syncthreads();
+    // 3. offsets, tiles per expert and their prefix, the m-tile table
+    if (threadIdx.x == 0) {
+        int off = 0, toff = 0;
+        for (int e = 0; e < E_tot; ++e) {
+            s_off[e] = off;
+            s_toff[e] = toff;
+            off += s_cnt[e];
+            toff += (s_cnt[e] + tile_m - 1) / tile_m;
+        }
+        s_off[E_tot] = off;
+        s_toff[E_tot] = toff;
+        if (toff > max_mtiles) report(status, MOE_DEV_OOB, (uint32_t)toff, 2u);
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e <= E_tot; e += blockDim.x) {
+        offsets[e] = s_off[e];
+        tile_offsets[e] = s_toff[e];
+        tiles[e] = (e < E_tot) ? s_toff[e + 1] - s_toff[e] : s_toff[E_tot];
+    }
+    const int S = min(s_toff[E_tot], max_mtiles);
+    for (int mu = threadIdx.x; mu < S; mu += blockDim.x) {
+        int lo = 0, hi = E_tot - 1;          // largest e with tile_offsets[e] <= mu
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (s_toff[mid] <= mu) lo = mid; else hi = mid - 1;
+        }
+        const int e = lo, i = mu - s_toff[e];
+        mtile_expert[mu] = e;
+        mtile_first_row[mu] = s_off[e] + i * tile_m;
+        mtile_valid[mu] = min(tile_m, s_cnt[e] - i * tile_m);
+    }
+    // 4. stable scatter of the warp's chunk: h[e] becomes the next free row of expert e for this warp
+    for (int e = lane; e < E_tot; e += 32) h[e] += s_off[e];
+    __syncwarp();
+    for (int f0 = begin; f0 < end; f0 += 32) {
+        const int f = f0 + lane;
+        const bool in = f < end;
+        int e = in ? topk_idx[f] : -1;
+        const bool ok = in && e >= 0 && e < E_tot;
+        const unsigned active = __ballot_sync(0xffffffffu, ok);
+        if (in && !ok) { inv_perm[f] = -1; pad_row[f] = -1; }
+        if (ok) {
+            const unsigned same = __match_any_sync(active, e);
+            const int rank = __popc(same & ((1u << lane) - 1u));
+            const int r = h[e] + rank;
+            __syncwarp(active);
+            if (rank == 0) h[e] += __popc(same);
+            perm[r] = f;
+            inv_perm[f] = r;
+            pad_row[f] = tile_m * s_toff[e] + (r - s_off[e]);
+        }
+        __syncwarp();
+    }
+}
+
 }  // namespace
 
 cudaError_t routing_launch(const int32_t *topk_idx, const moe_shape &s, int tile_m,
@@ -177,6 +279,13 @@ cudaError_t routing_launch(const int32_t *topk_idx, const moe_shape &s, int tile
 {
     const int R = s.T * s.k_tot;
     const int n_warps = (R + kRoutingChunk - 1) / kRoutingChunk;
+    if (n_warps <= kSmallWarps && s.E_tot <= kSmallMaxExperts) {
+        const size_t sm = ((size_t)kSmallWarps * s.E_tot + 3 * (size_t)(s.E_tot + 1)) * sizeof(int32_t);
+        routing_small<<<1, kSmallWarps * 32, sm, stream>>>(
+            topk_idx, R, s.k_tot, s.E_tot, tile_m, n_warps, r.max_mtiles, r.counts, r.offsets, r.tiles, r.tile_offsets,
+            r.mtile_expert, r.mtile_first_row, r.mtile_valid, r.perm, r.inv_perm, r.pad_row, status);
+        return cudaGetLastError();
+    }
     const int blocks = (n_warps + kWarpsPerBlock - 1) / kWarpsPerBlock;
     const size_t sh = (size_t)kWarpsPerBlock * s.E_tot * sizeof(int32_t);
     if (blocks > 0)
