@@ -357,7 +357,7 @@ def all_traffic_bytes(w, x_passes=1):
             2 * w.T * w.L * w.k_tot * w.TP * (-(-w.H // w.L)) * 2 + w.T * w.H * 2)
 
 
-def quick_config(h, w, device, peaks, steps=30, warm=5):
+def quick_config(h, w, device, peaks, steps=30, warm=5, counts_on_device_too=False):
     """A bounded measurement of one more workload (a second or two): the whole step timed like the headline
     one (K moe_layer calls between two events), the fused kernel by events around its launch.  Fractions
     against the headline roofline (GEMM FLOPs at the burst peak -- these loops last milliseconds -- or combine
@@ -393,6 +393,21 @@ def quick_config(h, w, device, peaks, steps=30, warm=5):
            "hbm_all_traffic_us": t_all, "frac_of_all_traffic_bound": t_all / fused,
            "bound_us": max(roof, t_all), "frac_of_bound": max(roof, t_all) / fused,
            "r_expert": dw.info["r_expert"]}
+    if counts_on_device_too:
+        # the same step with the routed counts left on the device (Section III-E: no copy, no host wait; the plan
+        # comes from the normalised-load estimate and the kernel reads the tile count itself)
+        layer2 = B.LayerCall(h, dw.x, dw.W2, dw.idx_d, dw.wt_d, dw.ws, limits=lim, counts_on_device=True)
+        for _ in range(warm):
+            layer2()
+        torch.cuda.synchronize()
+        t0.record()
+        for _ in range(steps):
+            layer2()
+        t1.record()
+        torch.cuda.synchronize()
+        assert B.moe_get_status(h, dw.ws.status).code == 0
+        out["step_us_counts_on_device"] = t0.elapsed_time(t1) * 1e3 / steps
+        del layer2
     del dw, layer
     torch.cuda.empty_cache()
     return out
@@ -413,7 +428,8 @@ def run_decode(h, args, device, peaks):
         w = replace(wl.DSV2L, name=f"dsv2lite_decode_T{T}", T=T)
         shape = B.make_shape(w.T, w.H, w.I, w.E_tot, w.k_tot, w.TP, w.EP, w.L)
         tm, tn = B.moe_select_tile(h, shape)
-        rows.append(quick_config(h, replace(w, tile_m=tm, tile_n=tn), device, peaks, steps=max(20, args.steps), warm=max(3, args.warmup)))
+        rows.append(quick_config(h, replace(w, tile_m=tm, tile_n=tn), device, peaks, steps=max(20, args.steps), warm=max(3, args.warmup),
+                                 counts_on_device_too=True))
     main = rows[2]   # T = 256
     w = replace(wl.DSV2L, name="dsv2lite_decode", T=main["T"])
     idx, wt, info = wl.make_routing(w)
