@@ -535,3 +535,33 @@ def test_random_small_shapes_against_the_oracle():
         _check_against_oracle(w, **kw)
         n_done += 1
     assert n_done >= 25
+
+
+def test_random_small_shapes_with_co_resident_warps_against_the_oracle():
+    # the same fuzz with co-resident communication warps asked for (the launch drops them where the shape has no
+    # room for them), with and without dedicated communication CTAs; every token checked
+    rng = np.random.default_rng(2025)
+    n_done = 0
+    for case in range(30):
+        tile_m, tile_n = [(64, 64), (128, 64), (128, 128), (128, 256), (256, 256)][int(rng.integers(5))]
+        TP = int(rng.choice([1, 2, 4]))
+        K = int(rng.choice([16, 64, 80, 128, 208]))
+        L = int(rng.choice([1, 2, 2, 4]))
+        H = int(rng.choice([64, 128, 256, 320, 512])) * L
+        E = int(rng.integers(1, 20))
+        k = int(rng.integers(1, min(E, 4) + 1))
+        n_shared = int(rng.choice([0, 0, 1, 2]))
+        T = int(rng.choice([1, 7, 65, 200, 513, 900, 1500]))
+        EP = int(rng.choice([1, 2, 3, 4]))
+        w = replace(wl.TINY, name=f"cofuzz{case}", T=T, H=H, I=K * TP, E=E, k=k, n_shared=n_shared, TP=TP, EP=EP, L=L,
+                    tile_m=tile_m, tile_n=tile_n, routing="zipf" if rng.random() < 0.5 else "uniform",
+                    zipf_s=1.0, target_r_expert=0.0, routing_seed=300 + case, data_seed=400 + case)
+        kw = dict(drain_help=1, co_warps=int(rng.choice([1, 2])))
+        r = rng.random()
+        if r < 0.35:
+            kw["force_C"] = int(rng.choice([1, 2, 5, 33]))
+        elif r < 0.6:      # no dedicated communication CTA at all: every SM computes
+            kw.update(force_C=1, C_override=0, P_override=148 // (2 if tile_m == 256 else 1))
+        _check_against_oracle(w, **kw)
+        n_done += 1
+    assert n_done >= 25
