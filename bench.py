@@ -357,6 +357,12 @@ def all_traffic_bytes(w, x_passes=1):
             2 * w.T * w.L * w.k_tot * w.TP * (-(-w.H // w.L)) * 2 + w.T * w.H * 2)
 
 
+def routing_launches(R):
+    """Launches of one routing build: one (a single CTA, or a single cluster) up to 128 chunks of 256 assignments,
+    four (histogram, column scan, finalize, scatter) beyond."""
+    return 1 if (R + 255) // 256 <= 128 else 4
+
+
 def quick_config(h, w, device, peaks, steps=30, warm=5, counts_on_device_too=False):
     """A bounded measurement of one more workload (a second or two): the whole step timed like the headline
     one (K moe_layer calls between two events), the fused kernel by events around its launch.  Fractions
@@ -978,7 +984,7 @@ def main():
             "roofline": roofline,
             "e2e": {"value": job_value(e2e_us, world), "unit": "us/layer", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": Ke},
-            "gpu_launches": 5 * K,
+            "gpu_launches": (routing_launches(w.T * w.k) + 1) * K,
             "clocks": clocks,
             "paper_context": {"hardware": "4xA100-SXM4-40GB", "mean_regret": 0.0322, "solver_us": 0.157,
                               "geomean_speedup_over_comet": 2.528},

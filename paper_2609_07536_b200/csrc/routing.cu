@@ -4,7 +4,11 @@
 // ceil(M_e / T_M) tiles along the token dimension; Eq. 16: their sum S.
 // The routed rows are the flat assignments f = t * k_tot + j in a *stable* order by expert.
 //
-// Four small launches (the data is a few hundred KB; one launch of one CTA for small batches, routing_small):
+// Three launch shapes, the same arithmetic and the same outputs bit for bit:
+//   routing_small    up to 32 chunks of 256 assignments: one launch of one CTA;
+//   routing_cluster  up to 128 chunks: one launch of one cluster of 8 CTAs, totals exchanged in
+//                    distributed shared memory;
+//   otherwise four small launches over the whole GPU:
 //   1. hist          every warp histograms its own contiguous chunk of assignments;
 //   2. scan_columns  one CTA per expert: exclusive prefix of that expert's histogram column over
 //                    the warps (the per-(warp, expert) bases) and the expert's count;
@@ -13,6 +17,8 @@
 //                    match_any gives each lane its rank among equal experts -> stable.
 
 #include "moe_internal.h"
+
+#include <cooperative_groups.h>
 
 namespace moe {
 namespace {
@@ -272,6 +278,167 @@ routing_small(const int32_t *__restrict__ topk_idx, int R, int k_tot, int E_tot,
     }
 }
 
+// The four steps in ONE launch of one thread-block cluster, for the batches between the single-CTA kernel
+// and the sizes where the whole GPU pays: CTA r of the cluster owns a contiguous run of chunks and keeps
+// their histograms in its own shared memory; the per-expert totals of the CTAs are exchanged through
+// distributed shared memory (the only step that crosses CTAs), the launch boundaries become one cluster
+// barrier.  Same arithmetic and outputs as the other two paths, bit for bit.
+// Measured on B200: against the four launches, 8 CTAs win ~10 us at 128 chunks and lose ~12 us at 512.
+constexpr int kClusterCtas = 8;
+constexpr int kClusterMaxChunks = 128;
+constexpr size_t kClusterMaxSmem = 200 * 1024;
+__global__ void __launch_bounds__(kSmallWarps * 32)
+routing_cluster(const int32_t *__restrict__ topk_idx, int R, int k_tot, int E_tot, int tile_m, int n_chunks, int max_mtiles,
+                int32_t *__restrict__ counts, int32_t *__restrict__ offsets, int32_t *__restrict__ tiles,
+                int32_t *__restrict__ tile_offsets, int32_t *__restrict__ mtile_expert,
+                int32_t *__restrict__ mtile_first_row, int32_t *__restrict__ mtile_valid, int32_t *__restrict__ perm,
+                int32_t *__restrict__ inv_perm, int32_t *__restrict__ pad_row, uint32_t *status)
+{
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int nb = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
+    const int cpc = (n_chunks + nb - 1) / nb;                       // chunks per CTA, a contiguous run
+    const int c_lo = min(n_chunks, rank * cpc), c_n = min(n_chunks, c_lo + cpc) - c_lo;
+    extern __shared__ int32_t sm[];
+    int32_t *whist = sm;                                            // [cpc][E_tot]
+    int32_t *s_tot = sm + (size_t)cpc * E_tot;                      // this CTA's rows per expert (read by the others)
+    int32_t *s_base = s_tot + E_tot;                                // rows per expert in the CTAs before this one
+    int32_t *s_cnt = s_base + E_tot, *s_off = s_cnt + (E_tot + 1), *s_toff = s_off + (E_tot + 1);
+    const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // 1. histogram of every chunk of this CTA (by the warp that will scatter it)
+    for (int lc = w; lc < c_n; lc += kSmallWarps) {
+        int32_t *h = whist + (size_t)lc * E_tot;
+        for (int e = lane; e < E_tot; e += 32) h[e] = 0;
+        __syncwarp();
+        const int begin = (c_lo + lc) * kRoutingChunk, end = min(R, begin + kRoutingChunk);
+        for (int f = begin + lane; f < end; f += 32) {
+            const int e = topk_idx[f];
+            if (e < 0 || e >= E_tot) {
+                report(status, MOE_DEV_OOB, (uint32_t)f, 1u);
+                continue;
+            }
+            atomicAdd(&h[e], 1);
+            const int t = f / k_tot, j = f - t * k_tot;
+            for (int jj = 0; jj < j; ++jj)
+                if (topk_idx[t * k_tot + jj] == e) report(status, MOE_DEV_DUP_EXPERT, (uint32_t)t, 1u);
+        }
+    }
+    __syncthreads();
+    // 2. per expert: exclusive prefix over this CTA's chunks, and the CTA's total
+    for (int e = threadIdx.x; e < E_tot; e += blockDim.x) {
+        int base = 0;
+        for (int lc = 0; lc < c_n; ++lc) {
+            const int v = whist[(size_t)lc * E_tot + e];
+            whist[(size_t)lc * E_tot + e] = base;
+            base += v;
+        }
+        s_tot[e] = base;
+    }
+    cluster.sync();
+    for (int e = threadIdx.x; e < E_tot; e += blockDim.x) {
+        int before = 0, total = 0;
+        for (int j = 0; j < nb; ++j) {
+            const int v = cluster.map_shared_rank(s_tot, j)[e];
+            if (j < rank) before += v;
+            total += v;
+        }
+        s_base[e] = before;
+        s_cnt[e] = total;
+        if (rank == 0) counts[e] = total;
+    }
+    __syncthreads();
+    // 3. offsets, tiles per expert and their prefix (every CTA, for its own scatter), the m-tile table
+    if (threadIdx.x == 0) {
+        int off = 0, toff = 0;
+        for (int e = 0; e < E_tot; ++e) {
+            s_off[e] = off;
+            s_toff[e] = toff;
+            off += s_cnt[e];
+            toff += (s_cnt[e] + tile_m - 1) / tile_m;
+        }
+        s_off[E_tot] = off;
+        s_toff[E_tot] = toff;
+        if (rank == 0 && toff > max_mtiles) report(status, MOE_DEV_OOB, (uint32_t)toff, 2u);
+    }
+    __syncthreads();
+    if (rank == 0)
+        for (int e = threadIdx.x; e <= E_tot; e += blockDim.x) {
+            offsets[e] = s_off[e];
+            tile_offsets[e] = s_toff[e];
+            tiles[e] = (e < E_tot) ? s_toff[e + 1] - s_toff[e] : s_toff[E_tot];
+        }
+    const int S = min(s_toff[E_tot], max_mtiles);
+    for (int mu = rank * blockDim.x + threadIdx.x; mu < S; mu += nb * blockDim.x) {
+        int lo = 0, hi = E_tot - 1;          // largest e with tile_offsets[e] <= mu
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (s_toff[mid] <= mu) lo = mid; else hi = mid - 1;
+        }
+        const int e = lo, i = mu - s_toff[e];
+        mtile_expert[mu] = e;
+        mtile_first_row[mu] = s_off[e] + i * tile_m;
+        mtile_valid[mu] = min(tile_m, s_cnt[e] - i * tile_m);
+    }
+    // 4. stable scatter, chunk by chunk: h[e] becomes the next free row of expert e for this chunk
+    for (int lc = w; lc < c_n; lc += kSmallWarps) {
+        int32_t *h = whist + (size_t)lc * E_tot;
+        for (int e = lane; e < E_tot; e += 32) h[e] += s_off[e] + s_base[e];
+        __syncwarp();
+        const int begin = (c_lo + lc) * kRoutingChunk, end = min(R, begin + kRoutingChunk);
+        for (int f0 = begin; f0 < end; f0 += 32) {
+            const int f = f0 + lane;
+            const bool in = f < end;
+            int e = in ? topk_idx[f] : -1;
+            const bool ok = in && e >= 0 && e < E_tot;
+            const unsigned active = __ballot_sync(0xffffffffu, ok);
+            if (in && !ok) { inv_perm[f] = -1; pad_row[f] = -1; }
+            if (ok) {
+                const unsigned same = __match_any_sync(active, e);
+                const int rk = __popc(same & ((1u << lane) - 1u));
+                const int r = h[e] + rk;
+                __syncwarp(active);
+                if (rk == 0) h[e] += __popc(same);
+                perm[r] = f;
+                inv_perm[f] = r;
+                pad_row[f] = tile_m * s_toff[e] + (r - s_off[e]);
+            }
+            __syncwarp();
+        }
+    }
+    cluster.sync();   // no CTA leaves while another may still read its totals
+}
+
+size_t routing_cluster_smem(int n_chunks, int E_tot)
+{
+    const int cpc = (n_chunks + kClusterCtas - 1) / kClusterCtas;
+    return ((size_t)cpc * E_tot + 2 * (size_t)E_tot + 3 * (size_t)(E_tot + 1)) * sizeof(int32_t);
+}
+
+cudaError_t routing_cluster_launch(const int32_t *topk_idx, const moe_shape &s, int tile_m, int R, int n_chunks,
+                                   const moe_routing &r, uint32_t *status, cudaStream_t stream)
+{
+    const size_t sm = routing_cluster_smem(n_chunks, s.E_tot);
+    cudaError_t e = cudaSuccess;
+    if (sm > 48 * 1024)
+        e = cudaFuncSetAttribute(routing_cluster, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kClusterMaxSmem);
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(kClusterCtas);
+    cfg.blockDim = dim3(kSmallWarps * 32);
+    cfg.dynamicSmemBytes = sm;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = kClusterCtas;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, routing_cluster, topk_idx, R, (int)s.k_tot, (int)s.E_tot, tile_m, n_chunks,
+                              (int)r.max_mtiles, r.counts, r.offsets, r.tiles, r.tile_offsets, r.mtile_expert,
+                              r.mtile_first_row, r.mtile_valid, r.perm, r.inv_perm, r.pad_row, status);
+}
+
 }  // namespace
 
 cudaError_t routing_launch(const int32_t *topk_idx, const moe_shape &s, int tile_m,
@@ -286,6 +453,8 @@ cudaError_t routing_launch(const int32_t *topk_idx, const moe_shape &s, int tile
             r.mtile_expert, r.mtile_first_row, r.mtile_valid, r.perm, r.inv_perm, r.pad_row, status);
         return cudaGetLastError();
     }
+    if (n_warps <= kClusterMaxChunks && routing_cluster_smem(n_warps, s.E_tot) <= kClusterMaxSmem)
+        return routing_cluster_launch(topk_idx, s, tile_m, R, n_warps, r, status, stream);
     const int blocks = (n_warps + kWarpsPerBlock - 1) / kWarpsPerBlock;
     const size_t sh = (size_t)kWarpsPerBlock * s.E_tot * sizeof(int32_t);
     if (blocks > 0)

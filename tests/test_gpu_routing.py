@@ -53,6 +53,29 @@ def test_adversarial():
     _compare(big, idx)
 
 
+def test_batches_of_the_cluster_launch():
+    """33 to 128 chunks of 256 assignments go through one cluster of 8 CTAs: uneven chunk runs (a CTA with
+    fewer chunks, a CTA with none), a ragged last chunk, one hot expert, bad ids reported."""
+    from dataclasses import replace
+    rng = np.random.default_rng(3)
+    for T, E, k, tm in ((2817, 40, 3, 128),      # 8451 assignments: 34 chunks, CTA 7 of 8 gets none
+                        (9003, 66, 1, 64),       # 36 chunks, the last one ragged
+                        (4099, 256, 8, 256),     # 129 chunks: the first size of the four-launch path
+                        (4000, 200, 8, 128)):    # 125 chunks, many experts
+        w = replace(wl.TINY, T=T, E=E, k=k, tile_m=tm, tile_n=256 if tm == 256 else 64)
+        idx = np.stack([rng.choice(E, k, replace=False) for _ in range(T)]).astype(np.int32)
+        _compare(w, idx)
+    w = replace(wl.TINY, T=10000, E=9, k=1, tile_m=64)
+    _compare(w, np.full((10000, 1), 4, dtype=np.int32))
+    idx = rng.integers(0, 9, size=(10000, 1)).astype(np.int32)
+    bad = idx.copy()
+    bad[9000, 0] = -3
+    ws, _, S = G.build_routing(w, bad)
+    st = B.moe_get_status(G.handle(), ws.status, check=False)
+    assert st.code == B.MOE_DEV_OOB and st.detail == 9000
+    _compare(w, idx)
+
+
 def test_bad_ids_are_reported_not_fatal():
     from dataclasses import replace
     w = replace(wl.TINY, T=64, E=8, k=2)
