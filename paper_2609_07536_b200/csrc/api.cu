@@ -7,6 +7,9 @@
 
 #include "moe_internal.h"
 
+#include <atomic>
+#include <chrono>
+
 namespace moe {
 
 int32_t cuda_fail(moe_handle *h, cudaError_t e, const char *what)
@@ -112,6 +115,19 @@ int32_t moe_create(int32_t device, moe_handle **out)
         return MOE_ERR_CUDA;
     }
     h->counts_event = ev;
+    // the count mailbox: a few KB of pinned host memory that the GPU addresses directly.  Without it (the
+    // allocation or the mapping refused) the whole-step calls copy the counts and synchronise instead.
+    void *mail = nullptr, *mail_dev = nullptr;
+    if (cudaHostAlloc(&mail, (size_t)kMailInts * sizeof(int32_t), cudaHostAllocMapped | cudaHostAllocPortable) == cudaSuccess) {
+        memset(mail, 0, (size_t)kMailInts * sizeof(int32_t));
+        if (cudaHostGetDevicePointer(&mail_dev, mail, 0) == cudaSuccess && mail_dev) {
+            h->mail_host = static_cast<int32_t *>(mail);
+            h->mail_dev = static_cast<int32_t *>(mail_dev);
+        } else {
+            cudaFreeHost(mail);
+        }
+    }
+    (void)cudaGetLastError();
     *out = h;
     return MOE_OK;
 }
@@ -119,6 +135,7 @@ int32_t moe_create(int32_t device, moe_handle **out)
 int32_t moe_destroy(moe_handle *h)
 {
     if (h && h->counts_event) cudaEventDestroy(static_cast<cudaEvent_t>(h->counts_event));
+    if (h && h->mail_host) cudaFreeHost(h->mail_host);
     delete h;
     return MOE_OK;
 }
@@ -309,7 +326,7 @@ int32_t moe_build_routing(moe_handle *h, const int32_t *topk_idx, const moe_shap
     if (r->max_mtiles < max_mtiles_of(s, tile_m)) return MOE_ERR_SHAPE;
     if (const int32_t rc = require_handle_device(h, "moe_build_routing")) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    cudaError_t e = routing_launch(topk_idx, *s, tile_m, *r, status_dev, st);
+    cudaError_t e = routing_launch(topk_idx, *s, tile_m, *r, status_dev, nullptr, 0u, st);
     if (e != cudaSuccess) return cuda_fail(h, e, "routing launch");
     if (tile_counts_host) {
         e = cudaMemcpyAsync(tile_counts_host, r->tiles, (size_t)(s->E_tot + 1) * 4, cudaMemcpyDeviceToHost, st);
@@ -317,6 +334,72 @@ int32_t moe_build_routing(moe_handle *h, const int32_t *topk_idx, const moe_shap
     }
     return MOE_OK;
 }
+
+}  // extern "C"
+
+namespace {
+
+// Routing build of the whole-step calls.  With the handle's mailbox the kernel that finishes the counts stores
+// them into host memory itself and `*seq` is the number to wait for (wait_counts); without it, the plain
+// build with its copy, and `*seq` = 0.
+int32_t build_routing_mailed(moe_handle *h, const int32_t *topk_idx, const moe_shape *s, int32_t tile_m, const moe_routing *r,
+                             int32_t *tile_counts_host, uint32_t *status_dev, cudaStream_t st, uint32_t *seq)
+{
+    *seq = 0;
+    if (!tile_counts_host || !h->mail_dev)
+        return moe_build_routing(h, topk_idx, s, tile_m, r, tile_counts_host, status_dev, st);
+    if (!s || !r || !status_dev) return MOE_ERR_NULL;
+    if (!shape_ok(s)) return MOE_ERR_SHAPE;
+    if (!tile_m_ok(tile_m)) return MOE_ERR_UNSUPPORTED;
+    if (s->T > 0 && !topk_idx) return MOE_ERR_NULL;
+    if (r->max_mtiles < max_mtiles_of(s, tile_m)) return MOE_ERR_SHAPE;
+    if (const int32_t rc = require_handle_device(h, "moe_build_routing")) return rc;
+    if (++h->mail_seq == 0u) h->mail_seq = 1u;
+    const cudaError_t e = routing_launch(topk_idx, *s, tile_m, *r, status_dev, h->mail_dev, h->mail_seq, st);
+    if (e != cudaSuccess) return cuda_fail(h, e, "routing launch");
+    *seq = h->mail_seq;
+    return MOE_OK;
+}
+
+// Waits until the counts of build `seq` are on the host and copies them to tile_counts_host (E_tot + 1 ints).
+// seq = 0: they come by the stream's copy: `fallback_event` if given (recorded behind that copy), else the stream.
+int32_t wait_counts(moe_handle *h, uint32_t seq, int32_t E_tot, int32_t *tile_counts_host, cudaStream_t st, cudaEvent_t fallback_event)
+{
+    if (seq == 0u) {
+        const cudaError_t e = fallback_event ? cudaEventSynchronize(fallback_event) : cudaStreamSynchronize(st);
+        return e == cudaSuccess ? MOE_OK : cuda_fail(h, e, "tile counts wait");
+    }
+    volatile uint32_t *word = reinterpret_cast<volatile uint32_t *>(h->mail_host);
+    const auto t0 = std::chrono::steady_clock::now();
+    uint32_t spins = 0;
+    while (*word != seq) {
+        if ((++spins & 2047u) == 0u) {
+            // the kernels finished or failed without the word arriving?
+            const cudaError_t q = cudaStreamQuery(st);
+            if (q != cudaErrorNotReady) {
+                if (*word == seq) break;
+                if (q != cudaSuccess) return cuda_fail(h, q, "routing build");
+                snprintf(h->err, sizeof h->err, "the routing build finished without delivering the tile counts");
+                return MOE_ERR_CUDA;
+            }
+            const double waited = std::chrono::duration<double>(std::chrono::steady_clock::now() - t0).count();
+            if (waited > 2.0 + 2e-9 * (double)h->wait_ns) {
+                snprintf(h->err, sizeof h->err, "no tile counts from the routing build after %.1f s", waited);
+                return MOE_ERR_CUDA;
+            }
+        }
+#if defined(__x86_64__) || defined(__i386__)
+        __builtin_ia32_pause();
+#endif
+    }
+    std::atomic_thread_fence(std::memory_order_acquire);
+    memcpy(tile_counts_host, h->mail_host + kMailCountsAt, (size_t)(E_tot + 1) * sizeof(int32_t));
+    return MOE_OK;
+}
+
+}  // namespace
+
+extern "C" {
 
 int32_t moe_gemm2_combine(moe_handle *h, const void *x_routed, const void *W2, const int32_t *topk_idx,
                           const float *topk_w, const moe_shape *s, const moe_occupancy *occ,
@@ -528,11 +611,14 @@ int32_t moe_layer(moe_handle *h, const void *x_routed, const void *W2, const int
 {
     if (!h || !s || !routing) return MOE_ERR_NULL;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    int32_t rc = moe_build_routing(h, topk_idx, s, tile_m, routing, tile_counts_pinned, status_dev, st);
+    uint32_t seq = 0;
+    int32_t rc = build_routing_mailed(h, topk_idx, s, tile_m, routing, tile_counts_pinned, status_dev, st, &seq);
     if (rc != MOE_OK) return rc;
     if (tile_counts_pinned) {
-        cudaError_t e = cudaStreamSynchronize(st);       // the tile counts are on the host now
-        if (e != cudaSuccess) return cuda_fail(h, e, "tile counts sync");
+        // the counts reach the host while the routing build is still scattering: planning and the fused
+        // launch below are queued behind it without a gap
+        rc = wait_counts(h, seq, s->E_tot, tile_counts_pinned, st, nullptr);
+        if (rc != MOE_OK) return rc;
     }
     moe_occupancy occ;
     moe_sm_limits lim;
@@ -563,11 +649,12 @@ int32_t moe_post_router_layer(moe_handle *h, const void *hidden, const void *W1,
 {
     if (!h || !s || !routing) return MOE_ERR_NULL;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    int32_t rc = moe_build_routing(h, topk_idx, s, tile_m, routing, tile_counts_pinned, status_dev, st);
+    uint32_t seq = 0;
+    int32_t rc = build_routing_mailed(h, topk_idx, s, tile_m, routing, tile_counts_pinned, status_dev, st, &seq);
     if (rc != MOE_OK) return rc;
     // GEMM1 reads the m-tile count on the device, so it is launched before the host waits for the counts:
     // the wait and the planning are hidden behind it
-    if (tile_counts_pinned && h->counts_event) cudaEventRecord(static_cast<cudaEvent_t>(h->counts_event), st);
+    if (tile_counts_pinned && seq == 0u && h->counts_event) cudaEventRecord(static_cast<cudaEvent_t>(h->counts_event), st);
     rc = moe_gemm1_act(h, hidden, W1, s, tile_m, routing, MOE_MTILES_ON_DEVICE, h_routed_ws, x_routed_ws, status_dev, st);
     if (rc != MOE_OK) return rc;
     moe_occupancy occ;
@@ -581,9 +668,9 @@ int32_t moe_post_router_layer(moe_handle *h, const void *hidden, const void *W1,
     if (tile_counts_pinned) {
         // the copy of the counts was queued right after the routing kernels, before GEMM1: wait for it alone
         cudaEvent_t counts_ready = static_cast<cudaEvent_t>(h->counts_event);
-        if (!counts_ready) return MOE_ERR_CUDA;
-        cudaError_t e = cudaEventSynchronize(counts_ready);
-        if (e != cudaSuccess) return cuda_fail(h, e, "tile counts wait");
+        if (seq == 0u && !counts_ready) return MOE_ERR_CUDA;
+        rc = wait_counts(h, seq, s->E_tot, tile_counts_pinned, st, counts_ready);
+        if (rc != MOE_OK) return rc;
         rc = plan_partition(tile_counts_pinned, s->E_tot, &occ, &lim, s, &rho, &plan);
         n_mtiles = tile_counts_pinned[s->E_tot];
     } else {

@@ -21,6 +21,8 @@ constexpr int kMmaM = 128;             // M of the MMA (tile_m = 64 stores the f
 constexpr int kStageBytesTotal = 192 * 1024;  // operand ring, all stages together
 constexpr int kCommTileM = 128;        // T_M^comm
 constexpr int kCommTileN = 1024;       // T_N^comm
+constexpr int kMailCountsAt = 32;      // the handle's count mailbox: word 0 = sequence number, counts from here on
+constexpr int kMailInts = kMailCountsAt + 1024 + 1 + 31;
 constexpr int kRoutingChunk = 256;     // flat assignments handled by one warp while sorting
 constexpr uint64_t kDefaultWaitNs = 2000000000ull;
 constexpr int kTimelineSlots = 40;     // 64-bit words per CTA in a timeline buffer (timeline build only)
@@ -85,6 +87,13 @@ struct moe_handle {
     int o_comp[3] = {0, 0, 0};                          // tile_n = 64, 128, 256
     int o_pair = 0;                                     // CTA-pair kernel: resident CTAs per SM
     int max_pairs = 0;                                  // ... and co-resident clusters of two
+    // Mailbox for the routed-tile counts (Section III-E: the manager reads them on the host): pinned host
+    // memory the GPU writes directly.  The routing kernel stores tiles[0..E_tot) and S at
+    // mail[kMailCountsAt...] and then the call's sequence number at mail[0]; the whole-step calls poll that
+    // word instead of queueing a copy and synchronising the stream.
+    int32_t *mail_host = nullptr;
+    int32_t *mail_dev = nullptr;                        // the same memory as the GPU addresses it
+    uint32_t mail_seq = 0;
     void *counts_event = nullptr;                       // cudaEvent_t: "the tile counts have reached the host"
     unsigned long long *timeline = nullptr;             // timeline build: where the next fused launch records
     size_t timeline_bytes = 0;
@@ -113,7 +122,8 @@ bool fused_timeline_build();   // the library was compiled with -DMOE_TIMELINE=1
 cudaError_t pair_occupancy(int *blocks_per_sm, int *max_clusters);
 cudaError_t pair_launch(const FusedParams &p, int grid, cudaStream_t stream);
 // routing kernels (routing.cu)
-cudaError_t routing_launch(const int32_t *topk_idx, const moe_shape &s, int tile_m,
-                           const moe_routing &r, uint32_t *status, cudaStream_t stream);
+// mail / mail_seq: see moe_handle::mail_host (nullptr: the counts are not mailed)
+cudaError_t routing_launch(const int32_t *topk_idx, const moe_shape &s, int tile_m, const moe_routing &r, uint32_t *status,
+                           int32_t *mail, uint32_t mail_seq, cudaStream_t stream);
 
 }  // namespace moe

@@ -24,6 +24,30 @@ namespace moe {
 namespace {
 
 constexpr int kWarpsPerBlock = 8;
+constexpr int kPerLane = kRoutingChunk / 32;   // assignments of a chunk held by one lane
+static_assert(kRoutingChunk % 32 == 0, "a chunk is a whole number of warp-wide rows");
+
+// The four launches of the large path are chained with programmatic stream serialization: a launch may be
+// set up while its predecessor still runs, and waits here, first thing, until the predecessor's writes are
+// visible.  Without that launch attribute this returns at once.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// launch `kernel` so that it may be set up before the previous kernel on the stream has finished
+template <typename... KArgs, typename... Args>
+cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 
 __device__ __forceinline__ void report(uint32_t *status, uint32_t code, uint32_t detail, uint32_t where)
 {
@@ -34,6 +58,137 @@ __device__ __forceinline__ void report(uint32_t *status, uint32_t code, uint32_t
     atomicAdd(&status[3], 1u);
 }
 
+// ---- the three steps every path runs on a chunk, one warp per chunk --------------------------------------
+//
+// Slot i of lane l is flat assignment begin + 32 i + l.  The ids of a chunk are fetched with independent
+// loads, all in flight together: a loop with one dependent load per 32 assignments spent its time on
+// memory latency (8 round trips per chunk and pass).
+
+// expert ids of the chunk (-1 past the end)
+__device__ __forceinline__ void chunk_load(const int32_t *__restrict__ topk_idx, int begin, int end, int lane, int (&e)[kPerLane])
+{
+#pragma unroll
+    for (int i = 0; i < kPerLane; ++i) {
+        const int f = begin + 32 * i + lane;
+        e[i] = f < end ? __ldg(topk_idx + f) : -1;
+    }
+}
+
+// histogram of the chunk into h[E_tot] (shared memory, zeroed by the caller); bad ids and an expert chosen
+// twice by one token are reported and left out / kept, as the scatter does
+__device__ __forceinline__ void chunk_hist(const int32_t *__restrict__ topk_idx, int begin, int end, int lane, int k_tot,
+                                           int E_tot, const int (&e)[kPerLane], int32_t *h, uint32_t *status)
+{
+#pragma unroll
+    for (int i = 0; i < kPerLane; ++i) {
+        const int f = begin + 32 * i + lane;
+        if (f >= end) continue;
+        if (e[i] < 0 || e[i] >= E_tot) {
+            report(status, MOE_DEV_OOB, (uint32_t)f, 1u);
+            continue;
+        }
+        atomicAdd(&h[e[i]], 1);
+        // the same expert twice inside one token?
+        const int t = f / k_tot, j = f - t * k_tot;
+        for (int jj = 0; jj < j; ++jj)
+            if (__ldg(topk_idx + t * k_tot + jj) == e[i]) report(status, MOE_DEV_DUP_EXPERT, (uint32_t)t, 1u);
+    }
+}
+
+// stable scatter of the chunk: run[e] is the next free routed row of expert e for this chunk; match_any
+// gives each lane its rank among the lanes of the row with the same expert.  off / toff: exclusive prefixes
+// of the per-expert rows and m-tiles.
+__device__ __forceinline__ void chunk_scatter(int begin, int end, int lane, int E_tot, int tile_m, const int (&e)[kPerLane],
+                                              int32_t *run, const int32_t *off, const int32_t *toff,
+                                              int32_t *__restrict__ perm, int32_t *__restrict__ inv_perm,
+                                              int32_t *__restrict__ pad_row)
+{
+#pragma unroll
+    for (int i = 0; i < kPerLane; ++i) {
+        if (begin + 32 * i >= end) break;     // warp-uniform
+        const int f = begin + 32 * i + lane;
+        const bool in = f < end;
+        const int ex = e[i];
+        const bool ok = in && ex >= 0 && ex < E_tot;
+        const unsigned active = __ballot_sync(0xffffffffu, ok);
+        if (in && !ok) { inv_perm[f] = -1; pad_row[f] = -1; }
+        if (ok) {
+            const unsigned same = __match_any_sync(active, ex);
+            const int rank = __popc(same & ((1u << lane) - 1u));
+            const int r = run[ex] + rank;
+            __syncwarp(active);
+            if (rank == 0) run[ex] += __popc(same);
+            perm[r] = f;
+            inv_perm[f] = r;
+            pad_row[f] = tile_m * toff[ex] + (r - off[ex]);
+        }
+        __syncwarp();
+    }
+}
+
+// One warp: exclusive prefixes over the experts of the rows (s_off) and of the m-tiles ceil(rows / tile_m)
+// (s_toff), totals in entry E_tot (Eq. 5, Eq. 16), 32 experts per step.
+__device__ __forceinline__ void expert_prefix(const int32_t *s_cnt, int32_t *s_off, int32_t *s_toff, int E_tot, int tile_m, int lane)
+{
+    int off = 0, toff = 0;
+    for (int e0 = 0; e0 < E_tot; e0 += 32) {
+        const int e = e0 + lane;
+        const int c = e < E_tot ? s_cnt[e] : 0;
+        const int tl = (c + tile_m - 1) / tile_m;
+        int ic = c, it = tl;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int uc = __shfl_up_sync(0xffffffffu, ic, d), ut = __shfl_up_sync(0xffffffffu, it, d);
+            if (lane >= d) { ic += uc; it += ut; }
+        }
+        if (e < E_tot) {
+            s_off[e] = off + ic - c;
+            s_toff[e] = toff + it - tl;
+        }
+        off += __shfl_sync(0xffffffffu, ic, 31);
+        toff += __shfl_sync(0xffffffffu, it, 31);
+    }
+    if (lane == 0) {
+        s_off[E_tot] = off;
+        s_toff[E_tot] = toff;
+    }
+}
+
+// The tile counts for the host, written straight into host memory the GPU can address (`mail`, or nullptr):
+// the word at mail[0] takes `seq` once tiles[0..E_tot) and S sit at mail[kMailCountsAt...].  A host that polls
+// the word has the counts while the scatter still runs and needs neither a copy nor a stream synchronisation.
+// Called by every thread of one CTA, after the prefixes are complete.
+__device__ __forceinline__ void mail_counts(int32_t *mail, uint32_t seq, const int32_t *s_toff, int E_tot)
+{
+    if (!mail) return;
+    for (int x = threadIdx.x; x <= E_tot; x += blockDim.x)
+        mail[kMailCountsAt + x] = (x < E_tot) ? s_toff[x + 1] - s_toff[x] : s_toff[E_tot];
+    __threadfence_system();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence_system();
+        *reinterpret_cast<volatile uint32_t *>(mail) = seq;
+    }
+}
+
+// m-tile table entry mu: the expert is found by bisection in the tile prefix
+__device__ __forceinline__ void mtile_entry(int mu, int E_tot, int tile_m, const int32_t *s_cnt, const int32_t *s_off,
+                                            const int32_t *s_toff, int32_t *__restrict__ mtile_expert,
+                                            int32_t *__restrict__ mtile_first_row, int32_t *__restrict__ mtile_valid)
+{
+    int lo = 0, hi = E_tot - 1;          // largest e with tile_offsets[e] <= mu
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (s_toff[mid] <= mu) lo = mid; else hi = mid - 1;
+    }
+    const int e = lo, i = mu - s_toff[e];
+    mtile_expert[mu] = e;
+    mtile_first_row[mu] = s_off[e] + i * tile_m;
+    mtile_valid[mu] = min(tile_m, s_cnt[e] - i * tile_m);
+}
+
+// ---- large batches: four launches over the whole GPU -------------------------------------------------------
+
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 routing_hist(const int32_t *__restrict__ topk_idx, int R, int k_tot, int E_tot, int n_warps,
              int32_t *__restrict__ whist, uint32_t *status)
@@ -41,27 +196,16 @@ routing_hist(const int32_t *__restrict__ topk_idx, int R, int k_tot, int E_tot, 
     extern __shared__ int32_t sh[];
     const int warp_in_block = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int w = blockIdx.x * kWarpsPerBlock + warp_in_block;
+    if (w >= n_warps) return;
     int32_t *h = sh + warp_in_block * E_tot;
-    for (int e = lane; e < E_tot; e += 32) h[e] = 0;
+    const int begin = w * kRoutingChunk, end = min(R, begin + kRoutingChunk);
+    int e[kPerLane];
+    chunk_load(topk_idx, begin, end, lane, e);
+    for (int x = lane; x < E_tot; x += 32) h[x] = 0;
     __syncwarp();
-    if (w < n_warps) {
-        const int begin = w * kRoutingChunk;
-        const int end = min(R, begin + kRoutingChunk);
-        for (int f = begin + lane; f < end; f += 32) {
-            const int e = topk_idx[f];
-            if (e < 0 || e >= E_tot) {
-                report(status, MOE_DEV_OOB, (uint32_t)f, 1u);
-                continue;
-            }
-            atomicAdd(&h[e], 1);
-            // the same expert twice inside one token?
-            const int t = f / k_tot, j = f - t * k_tot;
-            for (int jj = 0; jj < j; ++jj)
-                if (topk_idx[t * k_tot + jj] == e) report(status, MOE_DEV_DUP_EXPERT, (uint32_t)t, 1u);
-        }
-        __syncwarp();
-        for (int e = lane; e < E_tot; e += 32) whist[(size_t)w * E_tot + e] = h[e];
-    }
+    chunk_hist(topk_idx, begin, end, lane, k_tot, E_tot, e, h, status);
+    __syncwarp();
+    for (int x = lane; x < E_tot; x += 32) whist[(size_t)w * E_tot + x] = h[x];
 }
 
 // Per expert (one CTA each): counts[e], and whist[.][e] turned into an exclusive prefix over the
@@ -71,6 +215,7 @@ __global__ void __launch_bounds__(kScanThreads)
 routing_scan_columns(int E_tot, int n_warps, int32_t *__restrict__ whist, int32_t *__restrict__ counts)
 {
     __shared__ int warp_sum[kScanThreads / 32];
+    grid_dependency_wait();
     const int e = blockIdx.x, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const int chunk = (n_warps + kScanThreads - 1) / kScanThreads;
     const int w_lo = min(n_warps, tid * chunk), w_hi = min(n_warps, w_lo + chunk);
@@ -94,52 +239,35 @@ routing_scan_columns(int E_tot, int n_warps, int32_t *__restrict__ whist, int32_
     if (tid == kScanThreads - 1) counts[e] = base;
 }
 
-// Offsets, tile counts and the m-tile table from the per-expert counts (one CTA; the prefix over the
-// experts is serial but runs in shared memory).  Dynamic shared memory: 3 * (E_tot + 1) ints.
+// Offsets, tile counts and the m-tile table from the per-expert counts (one CTA).
+// Dynamic shared memory: 3 * (E_tot + 1) ints.
 __global__ void __launch_bounds__(1024)
 routing_finalize(int E_tot, int tile_m, int max_mtiles, const int32_t *__restrict__ counts,
                  int32_t *__restrict__ offsets, int32_t *__restrict__ tiles, int32_t *__restrict__ tile_offsets,
                  int32_t *__restrict__ mtile_expert, int32_t *__restrict__ mtile_first_row,
-                 int32_t *__restrict__ mtile_valid, uint32_t *status)
+                 int32_t *__restrict__ mtile_valid, uint32_t *status, int32_t *mail, uint32_t mail_seq)
 {
     extern __shared__ int32_t fin[];
+    grid_dependency_wait();
     int32_t *s_cnt = fin, *s_off = fin + (E_tot + 1), *s_toff = fin + 2 * (E_tot + 1);
     for (int e = threadIdx.x; e < E_tot; e += blockDim.x) s_cnt[e] = counts[e];
     __syncthreads();
-    if (threadIdx.x == 0) {
-        int off = 0, toff = 0;
-        for (int e = 0; e < E_tot; ++e) {
-            s_off[e] = off;
-            s_toff[e] = toff;
-            off += s_cnt[e];
-            toff += (s_cnt[e] + tile_m - 1) / tile_m;
-        }
-        s_off[E_tot] = off;
-        s_toff[E_tot] = toff;
-        if (toff > max_mtiles) report(status, MOE_DEV_OOB, (uint32_t)toff, 2u);
-    }
+    if (threadIdx.x < 32) expert_prefix(s_cnt, s_off, s_toff, E_tot, tile_m, threadIdx.x);
     __syncthreads();
+    mail_counts(mail, mail_seq, s_toff, E_tot);
+    if (threadIdx.x == 0 && s_toff[E_tot] > max_mtiles) report(status, MOE_DEV_OOB, (uint32_t)s_toff[E_tot], 2u);
     for (int e = threadIdx.x; e <= E_tot; e += blockDim.x) {
         offsets[e] = s_off[e];
         tile_offsets[e] = s_toff[e];
         // S rides behind the per-expert tile counts for the host copy
         tiles[e] = (e < E_tot) ? s_toff[e + 1] - s_toff[e] : s_toff[E_tot];
     }
-    // m-tile table, one thread per m-tile: the expert is found by bisection in the tile prefix
     const int S = min(s_toff[E_tot], max_mtiles);
-    for (int mu = threadIdx.x; mu < S; mu += blockDim.x) {
-        int lo = 0, hi = E_tot - 1;          // largest e with tile_offsets[e] <= mu
-        while (lo < hi) {
-            const int mid = (lo + hi + 1) >> 1;
-            if (s_toff[mid] <= mu) lo = mid; else hi = mid - 1;
-        }
-        const int e = lo, i = mu - s_toff[e];
-        mtile_expert[mu] = e;
-        mtile_first_row[mu] = s_off[e] + i * tile_m;
-        mtile_valid[mu] = min(tile_m, s_cnt[e] - i * tile_m);
-    }
+    for (int mu = threadIdx.x; mu < S; mu += blockDim.x)
+        mtile_entry(mu, E_tot, tile_m, s_cnt, s_off, s_toff, mtile_expert, mtile_first_row, mtile_valid);
 }
 
+// Dynamic shared memory: (kWarpsPerBlock * E_tot + 2 * (E_tot + 1)) ints.
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 routing_scatter(const int32_t *__restrict__ topk_idx, int R, int E_tot, int tile_m, int n_warps,
                 const int32_t *__restrict__ whist, const int32_t *__restrict__ offsets,
@@ -149,155 +277,106 @@ routing_scatter(const int32_t *__restrict__ topk_idx, int R, int E_tot, int tile
     extern __shared__ int32_t sh[];
     const int warp_in_block = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int w = blockIdx.x * kWarpsPerBlock + warp_in_block;
+    const int begin = min(R, w * kRoutingChunk), end = w < n_warps ? min(R, begin + kRoutingChunk) : begin;
+    // the ids do not depend on the launches before this one: fetch them before waiting
+    int e[kPerLane];
+    chunk_load(topk_idx, begin, end, lane, e);
+    grid_dependency_wait();
+    int32_t *s_off = sh + kWarpsPerBlock * E_tot, *s_toff = s_off + (E_tot + 1);
+    for (int x = threadIdx.x; x <= E_tot; x += blockDim.x) {
+        s_off[x] = offsets[x];
+        s_toff[x] = tile_offsets[x];
+    }
+    __syncthreads();
     if (w >= n_warps) return;
     int32_t *run = sh + warp_in_block * E_tot;  // next free row per expert, for this warp
-    for (int e = lane; e < E_tot; e += 32) run[e] = offsets[e] + whist[(size_t)w * E_tot + e];
+    for (int x = lane; x < E_tot; x += 32) run[x] = s_off[x] + whist[(size_t)w * E_tot + x];
     __syncwarp();
-    const int begin = w * kRoutingChunk;
-    const int end = min(R, begin + kRoutingChunk);
-    for (int f0 = begin; f0 < end; f0 += 32) {
-        const int f = f0 + lane;
-        const bool in = f < end;
-        int e = in ? topk_idx[f] : -1;
-        const bool ok = in && e >= 0 && e < E_tot;
-        const unsigned active = __ballot_sync(0xffffffffu, ok);
-        if (in && !ok) { inv_perm[f] = -1; pad_row[f] = -1; }
-        if (ok) {
-            const unsigned same = __match_any_sync(active, e);
-            const int rank = __popc(same & ((1u << lane) - 1u));
-            const int r = run[e] + rank;
-            __syncwarp(active);
-            if (rank == 0) run[e] += __popc(same);
-            perm[r] = f;
-            inv_perm[f] = r;
-            pad_row[f] = tile_m * tile_offsets[e] + (r - offsets[e]);
-        }
-        __syncwarp();
-    }
+    chunk_scatter(begin, end, lane, E_tot, tile_m, e, run, s_off, s_toff, perm, inv_perm, pad_row);
 }
 
-// The same four steps in ONE launch of one CTA, for small and decode-sized batches (at most 32 chunks of
-// 256 assignments, at most 256 experts): the per-warp histograms live in shared memory, the steps are
-// separated by CTA barriers instead of launch boundaries.  Same arithmetic, same outputs, bit for bit; four
-// launches cost ~30 us of which the work is a few microseconds at these sizes.
+// ---- small batches: the same steps in ONE launch of one CTA ------------------------------------------------
+//
+// At most 32 chunks (8192 assignments), one per warp; the per-chunk histograms live in shared memory, the ids
+// of a chunk stay in its warp's registers from the histogram to the scatter, the steps are separated by CTA
+// barriers instead of launch boundaries.  Same arithmetic, same outputs, bit for bit; four launches cost
+// ~30 us of which the work is a few microseconds at these sizes.
 constexpr int kSmallWarps = 32;
-constexpr int kSmallMaxExperts = 256;
+constexpr size_t kSmallMaxSmem = 200 * 1024;
 __global__ void __launch_bounds__(kSmallWarps * 32)
-routing_small(const int32_t *__restrict__ topk_idx, int R, int k_tot, int E_tot, int tile_m, int n_warps, int max_mtiles,
+routing_small(const int32_t *__restrict__ topk_idx, int R, int k_tot, int E_tot, int tile_m, int n_chunks, int max_mtiles,
               int32_t *__restrict__ counts, int32_t *__restrict__ offsets, int32_t *__restrict__ tiles,
               int32_t *__restrict__ tile_offsets, int32_t *__restrict__ mtile_expert,
               int32_t *__restrict__ mtile_first_row, int32_t *__restrict__ mtile_valid, int32_t *__restrict__ perm,
-              int32_t *__restrict__ inv_perm, int32_t *__restrict__ pad_row, uint32_t *status)
+              int32_t *__restrict__ inv_perm, int32_t *__restrict__ pad_row, uint32_t *status, int32_t *mail,
+              uint32_t mail_seq)
 {
     extern __shared__ int32_t sm[];
     int32_t *whist = sm;                                   // [kSmallWarps][E_tot]
     int32_t *s_cnt = sm + kSmallWarps * E_tot, *s_off = s_cnt + (E_tot + 1), *s_toff = s_off + (E_tot + 1);
     const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
     int32_t *h = whist + w * E_tot;
-    // 1. per-warp histograms of the warp's chunk
-    for (int e = lane; e < E_tot; e += 32) h[e] = 0;
+    const int begin = min(R, w * kRoutingChunk), end = w < n_chunks ? min(R, begin + kRoutingChunk) : begin;
+    // 1. histogram of the warp's chunk
+    int e[kPerLane];
+    chunk_load(topk_idx, begin, end, lane, e);
+    for (int x = lane; x < E_tot; x += 32) h[x] = 0;
     __syncwarp();
-    const int begin = w * kRoutingChunk;
-    const int end = w < n_warps ? min(R, begin + kRoutingChunk) : begin;
-    for (int f = begin + lane; f < end; f += 32) {
-        const int e = topk_idx[f];
-        if (e < 0 || e >= E_tot) {
-            report(status, MOE_DEV_OOB, (uint32_t)f, 1u);
-            continue;
-        }
-        atomicAdd(&h[e], 1);
-        const int t = f / k_tot, j = f - t * k_tot;
-        for (int jj = 0; jj < j; ++jj)
-            if (topk_idx[t * k_tot + jj] == e) report(status, MOE_DEV_DUP_EXPERT, (uint32_t)t, 1u);
-    }
+    chunk_hist(topk_idx, begin, end, lane, k_tot, E_tot, e, h, status);
     __syncthreads();
-    // 2. per expert: exclusive prefix of its histogram column over the warps, and its count
-    for (int e = threadIdx.x; e < E_tot; e += blockDim.x) {
+    // 2. per expert: exclusive prefix of its histogram column over the chunks, and its count
+    for (int x = threadIdx.x; x < E_tot; x += blockDim.x) {
         int base = 0;
-        for (int ww = 0; ww < n_warps; ++ww) {
-            const int c = whist[ww * E_tot + e];
-            whist[ww * E_tot + e] = base;
-            base += c;
+        for (int c = 0; c < n_chunks; ++c) {
+            const int v = whist[c * E_tot + x];
+            whist[c * E_tot + x] = base;
+            base += v;
         }
-        s_cnt[e] = base;
-        counts[e] = base;
+        s_cnt[x] = base;
+        counts[x] = base;
     }
     __syncthreads();
     // 3. offsets, tiles per expert and their prefix, the m-tile table
-    if (threadIdx.x == 0) {
-        int off = 0, toff = 0;
-        for (int e = 0; e < E_tot; ++e) {
-            s_off[e] = off;
-            s_toff[e] = toff;
-            off += s_cnt[e];
-            toff += (s_cnt[e] + tile_m - 1) / tile_m;
-        }
-        s_off[E_tot] = off;
-        s_toff[E_tot] = toff;
-        if (toff > max_mtiles) report(status, MOE_DEV_OOB, (uint32_t)toff, 2u);
-    }
+    if (w == 0) expert_prefix(s_cnt, s_off, s_toff, E_tot, tile_m, lane);
     __syncthreads();
-    for (int e = threadIdx.x; e <= E_tot; e += blockDim.x) {
-        offsets[e] = s_off[e];
-        tile_offsets[e] = s_toff[e];
-        tiles[e] = (e < E_tot) ? s_toff[e + 1] - s_toff[e] : s_toff[E_tot];
+    mail_counts(mail, mail_seq, s_toff, E_tot);
+    if (threadIdx.x == 0 && s_toff[E_tot] > max_mtiles) report(status, MOE_DEV_OOB, (uint32_t)s_toff[E_tot], 2u);
+    for (int x = threadIdx.x; x <= E_tot; x += blockDim.x) {
+        offsets[x] = s_off[x];
+        tile_offsets[x] = s_toff[x];
+        tiles[x] = (x < E_tot) ? s_toff[x + 1] - s_toff[x] : s_toff[E_tot];
     }
     const int S = min(s_toff[E_tot], max_mtiles);
-    for (int mu = threadIdx.x; mu < S; mu += blockDim.x) {
-        int lo = 0, hi = E_tot - 1;          // largest e with tile_offsets[e] <= mu
-        while (lo < hi) {
-            const int mid = (lo + hi + 1) >> 1;
-            if (s_toff[mid] <= mu) lo = mid; else hi = mid - 1;
-        }
-        const int e = lo, i = mu - s_toff[e];
-        mtile_expert[mu] = e;
-        mtile_first_row[mu] = s_off[e] + i * tile_m;
-        mtile_valid[mu] = min(tile_m, s_cnt[e] - i * tile_m);
-    }
-    // 4. stable scatter of the warp's chunk: h[e] becomes the next free row of expert e for this warp
-    for (int e = lane; e < E_tot; e += 32) h[e] += s_off[e];
+    for (int mu = threadIdx.x; mu < S; mu += blockDim.x)
+        mtile_entry(mu, E_tot, tile_m, s_cnt, s_off, s_toff, mtile_expert, mtile_first_row, mtile_valid);
+    // 4. stable scatter of the warp's chunk: h[x] becomes the next free row of expert x for this chunk
+    for (int x = lane; x < E_tot; x += 32) h[x] += s_off[x];
     __syncwarp();
-    for (int f0 = begin; f0 < end; f0 += 32) {
-        const int f = f0 + lane;
-        const bool in = f < end;
-        int e = in ? topk_idx[f] : -1;
-        const bool ok = in && e >= 0 && e < E_tot;
-        const unsigned active = __ballot_sync(0xffffffffu, ok);
-        if (in && !ok) { inv_perm[f] = -1; pad_row[f] = -1; }
-        if (ok) {
-            const unsigned same = __match_any_sync(active, e);
-            const int rank = __popc(same & ((1u << lane) - 1u));
-            const int r = h[e] + rank;
-            __syncwarp(active);
-            if (rank == 0) h[e] += __popc(same);
-            perm[r] = f;
-            inv_perm[f] = r;
-            pad_row[f] = tile_m * s_toff[e] + (r - s_off[e]);
-        }
-        __syncwarp();
-    }
+    chunk_scatter(begin, end, lane, E_tot, tile_m, e, h, s_off, s_toff, perm, inv_perm, pad_row);
 }
 
-// The four steps in ONE launch of one thread-block cluster, for the batches between the single-CTA kernel
-// and the sizes where the whole GPU pays: CTA r of the cluster owns a contiguous run of chunks and keeps
-// their histograms in its own shared memory; the per-expert totals of the CTAs are exchanged through
-// distributed shared memory (the only step that crosses CTAs), the launch boundaries become one cluster
-// barrier.  Same arithmetic and outputs as the other two paths, bit for bit.
-// Measured on B200: against the four launches, 8 CTAs win ~10 us at 128 chunks and lose ~12 us at 512.
+// ---- medium batches: ONE launch of one thread-block cluster ------------------------------------------------
+//
+// CTA r of the cluster owns a contiguous run of chunks, one per warp, and keeps their histograms in its own
+// shared memory; the per-expert totals of the CTAs are exchanged through distributed shared memory (the only
+// step that crosses CTAs), the launch boundaries become one cluster barrier.  Same outputs as the other two
+// paths, bit for bit.  Measured on B200 against the four launches: 8 CTAs win ~10 us at 128 chunks and
+// lose ~12 us at 512; a single CTA is 2x slower than four launches at 128 chunks.
 constexpr int kClusterCtas = 8;
 constexpr int kClusterMaxChunks = 128;
-constexpr size_t kClusterMaxSmem = 200 * 1024;
+static_assert(kClusterMaxChunks <= kClusterCtas * kSmallWarps, "one chunk per warp");
 __global__ void __launch_bounds__(kSmallWarps * 32)
 routing_cluster(const int32_t *__restrict__ topk_idx, int R, int k_tot, int E_tot, int tile_m, int n_chunks, int max_mtiles,
                 int32_t *__restrict__ counts, int32_t *__restrict__ offsets, int32_t *__restrict__ tiles,
                 int32_t *__restrict__ tile_offsets, int32_t *__restrict__ mtile_expert,
                 int32_t *__restrict__ mtile_first_row, int32_t *__restrict__ mtile_valid, int32_t *__restrict__ perm,
-                int32_t *__restrict__ inv_perm, int32_t *__restrict__ pad_row, uint32_t *status)
+                int32_t *__restrict__ inv_perm, int32_t *__restrict__ pad_row, uint32_t *status, int32_t *mail,
+                uint32_t mail_seq)
 {
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
     const int nb = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
-    const int cpc = (n_chunks + nb - 1) / nb;                       // chunks per CTA, a contiguous run
+    const int cpc = (n_chunks + nb - 1) / nb;                       // chunks per CTA (<= 32), a contiguous run
     const int c_lo = min(n_chunks, rank * cpc), c_n = min(n_chunks, c_lo + cpc) - c_lo;
     extern __shared__ int32_t sm[];
     int32_t *whist = sm;                                            // [cpc][E_tot]
@@ -305,105 +384,61 @@ routing_cluster(const int32_t *__restrict__ topk_idx, int R, int k_tot, int E_to
     int32_t *s_base = s_tot + E_tot;                                // rows per expert in the CTAs before this one
     int32_t *s_cnt = s_base + E_tot, *s_off = s_cnt + (E_tot + 1), *s_toff = s_off + (E_tot + 1);
     const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    // 1. histogram of every chunk of this CTA (by the warp that will scatter it)
-    for (int lc = w; lc < c_n; lc += kSmallWarps) {
-        int32_t *h = whist + (size_t)lc * E_tot;
-        for (int e = lane; e < E_tot; e += 32) h[e] = 0;
+    const bool mine = w < c_n;                                      // this warp has a chunk
+    int32_t *h = whist + (size_t)(mine ? w : 0) * E_tot;
+    const int begin = min(R, (c_lo + w) * kRoutingChunk), end = mine ? min(R, begin + kRoutingChunk) : begin;
+    // 1. histogram of the warp's chunk
+    int e[kPerLane];
+    chunk_load(topk_idx, begin, end, lane, e);
+    if (mine) {
+        for (int x = lane; x < E_tot; x += 32) h[x] = 0;
         __syncwarp();
-        const int begin = (c_lo + lc) * kRoutingChunk, end = min(R, begin + kRoutingChunk);
-        for (int f = begin + lane; f < end; f += 32) {
-            const int e = topk_idx[f];
-            if (e < 0 || e >= E_tot) {
-                report(status, MOE_DEV_OOB, (uint32_t)f, 1u);
-                continue;
-            }
-            atomicAdd(&h[e], 1);
-            const int t = f / k_tot, j = f - t * k_tot;
-            for (int jj = 0; jj < j; ++jj)
-                if (topk_idx[t * k_tot + jj] == e) report(status, MOE_DEV_DUP_EXPERT, (uint32_t)t, 1u);
-        }
+        chunk_hist(topk_idx, begin, end, lane, k_tot, E_tot, e, h, status);
     }
     __syncthreads();
-    // 2. per expert: exclusive prefix over this CTA's chunks, and the CTA's total
-    for (int e = threadIdx.x; e < E_tot; e += blockDim.x) {
+    // 2. per expert: exclusive prefix over this CTA's chunks, the CTA's total; then the totals of all CTAs
+    for (int x = threadIdx.x; x < E_tot; x += blockDim.x) {
         int base = 0;
         for (int lc = 0; lc < c_n; ++lc) {
-            const int v = whist[(size_t)lc * E_tot + e];
-            whist[(size_t)lc * E_tot + e] = base;
+            const int v = whist[(size_t)lc * E_tot + x];
+            whist[(size_t)lc * E_tot + x] = base;
             base += v;
         }
-        s_tot[e] = base;
+        s_tot[x] = base;
     }
     cluster.sync();
-    for (int e = threadIdx.x; e < E_tot; e += blockDim.x) {
+    for (int x = threadIdx.x; x < E_tot; x += blockDim.x) {
         int before = 0, total = 0;
         for (int j = 0; j < nb; ++j) {
-            const int v = cluster.map_shared_rank(s_tot, j)[e];
+            const int v = cluster.map_shared_rank(s_tot, j)[x];
             if (j < rank) before += v;
             total += v;
         }
-        s_base[e] = before;
-        s_cnt[e] = total;
-        if (rank == 0) counts[e] = total;
+        s_base[x] = before;
+        s_cnt[x] = total;
+        if (rank == 0) counts[x] = total;
     }
     __syncthreads();
     // 3. offsets, tiles per expert and their prefix (every CTA, for its own scatter), the m-tile table
-    if (threadIdx.x == 0) {
-        int off = 0, toff = 0;
-        for (int e = 0; e < E_tot; ++e) {
-            s_off[e] = off;
-            s_toff[e] = toff;
-            off += s_cnt[e];
-            toff += (s_cnt[e] + tile_m - 1) / tile_m;
-        }
-        s_off[E_tot] = off;
-        s_toff[E_tot] = toff;
-        if (rank == 0 && toff > max_mtiles) report(status, MOE_DEV_OOB, (uint32_t)toff, 2u);
-    }
+    if (w == 0) expert_prefix(s_cnt, s_off, s_toff, E_tot, tile_m, lane);
     __syncthreads();
-    if (rank == 0)
-        for (int e = threadIdx.x; e <= E_tot; e += blockDim.x) {
-            offsets[e] = s_off[e];
-            tile_offsets[e] = s_toff[e];
-            tiles[e] = (e < E_tot) ? s_toff[e + 1] - s_toff[e] : s_toff[E_tot];
+    if (rank == 0) {
+        mail_counts(mail, mail_seq, s_toff, E_tot);
+        if (threadIdx.x == 0 && s_toff[E_tot] > max_mtiles) report(status, MOE_DEV_OOB, (uint32_t)s_toff[E_tot], 2u);
+        for (int x = threadIdx.x; x <= E_tot; x += blockDim.x) {
+            offsets[x] = s_off[x];
+            tile_offsets[x] = s_toff[x];
+            tiles[x] = (x < E_tot) ? s_toff[x + 1] - s_toff[x] : s_toff[E_tot];
         }
-    const int S = min(s_toff[E_tot], max_mtiles);
-    for (int mu = rank * blockDim.x + threadIdx.x; mu < S; mu += nb * blockDim.x) {
-        int lo = 0, hi = E_tot - 1;          // largest e with tile_offsets[e] <= mu
-        while (lo < hi) {
-            const int mid = (lo + hi + 1) >> 1;
-            if (s_toff[mid] <= mu) lo = mid; else hi = mid - 1;
-        }
-        const int e = lo, i = mu - s_toff[e];
-        mtile_expert[mu] = e;
-        mtile_first_row[mu] = s_off[e] + i * tile_m;
-        mtile_valid[mu] = min(tile_m, s_cnt[e] - i * tile_m);
     }
-    // 4. stable scatter, chunk by chunk: h[e] becomes the next free row of expert e for this chunk
-    for (int lc = w; lc < c_n; lc += kSmallWarps) {
-        int32_t *h = whist + (size_t)lc * E_tot;
-        for (int e = lane; e < E_tot; e += 32) h[e] += s_off[e] + s_base[e];
+    const int S = min(s_toff[E_tot], max_mtiles);
+    for (int mu = rank * blockDim.x + threadIdx.x; mu < S; mu += nb * blockDim.x)
+        mtile_entry(mu, E_tot, tile_m, s_cnt, s_off, s_toff, mtile_expert, mtile_first_row, mtile_valid);
+    // 4. stable scatter of the warp's chunk: h[x] becomes the next free row of expert x for this chunk
+    if (mine) {
+        for (int x = lane; x < E_tot; x += 32) h[x] += s_off[x] + s_base[x];
         __syncwarp();
-        const int begin = (c_lo + lc) * kRoutingChunk, end = min(R, begin + kRoutingChunk);
-        for (int f0 = begin; f0 < end; f0 += 32) {
-            const int f = f0 + lane;
-            const bool in = f < end;
-            int e = in ? topk_idx[f] : -1;
-            const bool ok = in && e >= 0 && e < E_tot;
-            const unsigned active = __ballot_sync(0xffffffffu, ok);
-            if (in && !ok) { inv_perm[f] = -1; pad_row[f] = -1; }
-            if (ok) {
-                const unsigned same = __match_any_sync(active, e);
-                const int rk = __popc(same & ((1u << lane) - 1u));
-                const int r = h[e] + rk;
-                __syncwarp(active);
-                if (rk == 0) h[e] += __popc(same);
-                perm[r] = f;
-                inv_perm[f] = r;
-                pad_row[f] = tile_m * s_toff[e] + (r - s_off[e]);
-            }
-            __syncwarp();
-        }
+        chunk_scatter(begin, end, lane, E_tot, tile_m, e, h, s_off, s_toff, perm, inv_perm, pad_row);
     }
     cluster.sync();   // no CTA leaves while another may still read its totals
 }
@@ -415,13 +450,13 @@ size_t routing_cluster_smem(int n_chunks, int E_tot)
 }
 
 cudaError_t routing_cluster_launch(const int32_t *topk_idx, const moe_shape &s, int tile_m, int R, int n_chunks,
-                                   const moe_routing &r, uint32_t *status, cudaStream_t stream)
+                                   const moe_routing &r, uint32_t *status, int32_t *mail, uint32_t mail_seq, cudaStream_t stream)
 {
     const size_t sm = routing_cluster_smem(n_chunks, s.E_tot);
-    cudaError_t e = cudaSuccess;
-    if (sm > 48 * 1024)
-        e = cudaFuncSetAttribute(routing_cluster, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kClusterMaxSmem);
-    if (e != cudaSuccess) return e;
+    if (sm > 48 * 1024) {
+        const cudaError_t e = cudaFuncSetAttribute(routing_cluster, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmallMaxSmem);
+        if (e != cudaSuccess) return e;
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(kClusterCtas);
     cfg.blockDim = dim3(kSmallWarps * 32);
@@ -436,39 +471,54 @@ cudaError_t routing_cluster_launch(const int32_t *topk_idx, const moe_shape &s, 
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, routing_cluster, topk_idx, R, (int)s.k_tot, (int)s.E_tot, tile_m, n_chunks,
                               (int)r.max_mtiles, r.counts, r.offsets, r.tiles, r.tile_offsets, r.mtile_expert,
-                              r.mtile_first_row, r.mtile_valid, r.perm, r.inv_perm, r.pad_row, status);
+                              r.mtile_first_row, r.mtile_valid, r.perm, r.inv_perm, r.pad_row, status, mail, mail_seq);
+}
+
+// the four launches; `scratch`: n_chunks * E_tot ints that need not start at any value
+cudaError_t routing_four_launches(const int32_t *topk_idx, const moe_shape &s, int tile_m, int R, int n_chunks,
+                                  const moe_routing &r, int32_t *scratch, uint32_t *status, int32_t *mail, uint32_t mail_seq,
+                                  cudaStream_t stream)
+{
+    const int blocks = (n_chunks + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    const int E = (int)s.E_tot;
+    const size_t sh_hist = (size_t)kWarpsPerBlock * E * sizeof(int32_t);
+    const size_t sh_scat = sh_hist + 2 * (size_t)(E + 1) * sizeof(int32_t);
+    if (blocks > 0)
+        routing_hist<<<blocks, kWarpsPerBlock * 32, sh_hist, stream>>>(topk_idx, R, s.k_tot, E, n_chunks, scratch, status);
+    cudaError_t e = launch_chained(routing_scan_columns, dim3(E), dim3(kScanThreads), 0, stream, E, n_chunks, scratch, r.counts);
+    if (e != cudaSuccess) return e;
+    e = launch_chained(routing_finalize, dim3(1), dim3(1024), 3 * (size_t)(E + 1) * sizeof(int32_t), stream, E, tile_m,
+                       (int)r.max_mtiles, r.counts, r.offsets, r.tiles, r.tile_offsets, r.mtile_expert, r.mtile_first_row,
+                       r.mtile_valid, status, mail, mail_seq);
+    if (e != cudaSuccess) return e;
+    if (blocks > 0)
+        e = launch_chained(routing_scatter, dim3(blocks), dim3(kWarpsPerBlock * 32), sh_scat, stream, topk_idx, R, E, tile_m,
+                           n_chunks, scratch, r.offsets, r.tile_offsets, r.perm, r.inv_perm, r.pad_row);
+    if (e != cudaSuccess) return e;
+    return cudaGetLastError();
 }
 
 }  // namespace
 
-cudaError_t routing_launch(const int32_t *topk_idx, const moe_shape &s, int tile_m,
-                           const moe_routing &r, uint32_t *status, cudaStream_t stream)
+cudaError_t routing_launch(const int32_t *topk_idx, const moe_shape &s, int tile_m, const moe_routing &r, uint32_t *status,
+                           int32_t *mail, uint32_t mail_seq, cudaStream_t stream)
 {
     const int R = s.T * s.k_tot;
-    const int n_warps = (R + kRoutingChunk - 1) / kRoutingChunk;
-    if (n_warps <= kSmallWarps && s.E_tot <= kSmallMaxExperts) {
-        const size_t sm = ((size_t)kSmallWarps * s.E_tot + 3 * (size_t)(s.E_tot + 1)) * sizeof(int32_t);
-        routing_small<<<1, kSmallWarps * 32, sm, stream>>>(
-            topk_idx, R, s.k_tot, s.E_tot, tile_m, n_warps, r.max_mtiles, r.counts, r.offsets, r.tiles, r.tile_offsets,
-            r.mtile_expert, r.mtile_first_row, r.mtile_valid, r.perm, r.inv_perm, r.pad_row, status);
+    const int n_chunks = (R + kRoutingChunk - 1) / kRoutingChunk;
+    const size_t sm_small = ((size_t)kSmallWarps * s.E_tot + 3 * (size_t)(s.E_tot + 1)) * sizeof(int32_t);
+    if (n_chunks <= kSmallWarps && sm_small <= kSmallMaxSmem) {
+        if (sm_small > 48 * 1024) {
+            const cudaError_t e = cudaFuncSetAttribute(routing_small, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmallMaxSmem);
+            if (e != cudaSuccess) return e;
+        }
+        routing_small<<<1, kSmallWarps * 32, sm_small, stream>>>(
+            topk_idx, R, s.k_tot, s.E_tot, tile_m, n_chunks, r.max_mtiles, r.counts, r.offsets, r.tiles, r.tile_offsets,
+            r.mtile_expert, r.mtile_first_row, r.mtile_valid, r.perm, r.inv_perm, r.pad_row, status, mail, mail_seq);
         return cudaGetLastError();
     }
-    if (n_warps <= kClusterMaxChunks && routing_cluster_smem(n_warps, s.E_tot) <= kClusterMaxSmem)
-        return routing_cluster_launch(topk_idx, s, tile_m, R, n_warps, r, status, stream);
-    const int blocks = (n_warps + kWarpsPerBlock - 1) / kWarpsPerBlock;
-    const size_t sh = (size_t)kWarpsPerBlock * s.E_tot * sizeof(int32_t);
-    if (blocks > 0)
-        routing_hist<<<blocks, kWarpsPerBlock * 32, sh, stream>>>(topk_idx, R, s.k_tot, s.E_tot, n_warps,
-                                                                  r.scratch, status);
-    routing_scan_columns<<<s.E_tot, kScanThreads, 0, stream>>>(s.E_tot, n_warps, r.scratch, r.counts);
-    routing_finalize<<<1, 1024, 3 * (size_t)(s.E_tot + 1) * sizeof(int32_t), stream>>>(
-        s.E_tot, tile_m, r.max_mtiles, r.counts, r.offsets, r.tiles, r.tile_offsets, r.mtile_expert,
-        r.mtile_first_row, r.mtile_valid, status);
-    if (blocks > 0)
-        routing_scatter<<<blocks, kWarpsPerBlock * 32, sh, stream>>>(
-            topk_idx, R, s.E_tot, tile_m, n_warps, r.scratch, r.offsets, r.tile_offsets, r.perm,
-            r.inv_perm, r.pad_row);
-    return cudaGetLastError();
+    if (n_chunks <= kClusterMaxChunks && routing_cluster_smem(n_chunks, s.E_tot) <= kSmallMaxSmem)
+        return routing_cluster_launch(topk_idx, s, tile_m, R, n_chunks, r, status, mail, mail_seq, stream);
+    return routing_four_launches(topk_idx, s, tile_m, R, n_chunks, r, r.scratch, status, mail, mail_seq, stream);
 }
 
 }  // namespace moe
@@ -542,20 +592,7 @@ extern "C" int32_t moe_build_routing_static(moe_handle *h, const int32_t *topk_i
     // The array keeps whatever the previous call left in it.  Nothing has to start at zero: the
     // histogram pass overwrites every (warp, expert) entry the later passes read.
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const int iR = (int)R, nw = (int)n_warps;
-    const int blocks = (nw + kWarpsPerBlock - 1) / kWarpsPerBlock;
-    const size_t sh = (size_t)kWarpsPerBlock * s->E_tot * sizeof(int32_t);
-    if (blocks > 0)
-        routing_hist<<<blocks, kWarpsPerBlock * 32, sh, st>>>(topk_idx, iR, s->k_tot, s->E_tot, nw, scratch, status_dev);
-    routing_scan_columns<<<s->E_tot, kScanThreads, 0, st>>>(s->E_tot, nw, scratch, r->counts);
-    routing_finalize<<<1, 1024, 3 * (size_t)(s->E_tot + 1) * sizeof(int32_t), st>>>(
-        s->E_tot, tile_m, r->max_mtiles, r->counts, r->offsets, r->tiles, r->tile_offsets, r->mtile_expert,
-        r->mtile_first_row, r->mtile_valid, status_dev);
-    if (blocks > 0)
-        routing_scatter<<<blocks, kWarpsPerBlock * 32, sh, st>>>(topk_idx, iR, s->E_tot, tile_m, nw, scratch,
-                                                                r->offsets, r->tile_offsets, r->perm,
-                                                                r->inv_perm, r->pad_row);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = routing_four_launches(topk_idx, *s, tile_m, (int)R, (int)n_warps, *r, scratch, status_dev, nullptr, 0u, st);
     if (e != cudaSuccess) return cuda_fail(h, e, "static routing launch");
     if (tile_counts_host) {
         e = cudaMemcpyAsync(tile_counts_host, r->tiles, (size_t)(s->E_tot + 1) * 4, cudaMemcpyDeviceToHost, st);

@@ -455,6 +455,39 @@ def test_single_call_layer_matches_the_stepwise_path():
         assert np.array_equal(a, o.float().cpu().numpy(), equal_nan=True)
 
 
+@pytest.mark.parametrize("T", [40, 3000, 12000], ids=["one_cta", "cluster", "four_launches"])
+def test_whole_step_call_gets_the_counts_of_every_routing_build(T):
+    # Section III-E: the manager reads the routed-tile counts on the host between dispatch and launch.  The
+    # whole-step call has them written into host memory by the routing kernel and waits for a sequence
+    # number; three launch shapes of the routing build (k_tot = 3: 120, 9000 and 36000 assignments), changing
+    # routings call after call, counts and outputs against the references every time.
+    from oracle import routing_ref as rr
+    h = G.handle()
+    w = replace(wl.TINY, name="mailed", T=T, E=24, k=3, H=256, I=64, tile_m=128, tile_n=128, EP=2, TP=1, L=2)
+    x, W2 = wl.make_data(w)
+    xd, Wd = x.cuda(), W2.cuda()
+    ws = None
+    for rep in range(3):
+        wr = replace(w, routing="zipf" if rep else "uniform", zipf_s=1.2, routing_seed=7 + rep)
+        idx, wt, _ = wl.make_routing(wr)
+        ref_outs, plan, ws, S, st = G.run_layer(w, idx, wt, x, W2, ws=ws)
+        ref_outs = [o.copy() for o in ref_outs]
+        ref = rr.build_routing(idx, w.E_tot, w.tile_m)
+        for o in ws.out:
+            o.fill_(float("nan"))
+        ws.tile_counts.fill_(-7)
+        idx_d, wt_d = torch.from_numpy(idx).cuda(), torch.from_numpy(wt).cuda()
+        p2 = B.moe_layer(h, xd, Wd, idx_d, wt_d, ws)
+        # the counts are on the host when the call returns, before any synchronisation by the caller
+        assert ws.tile_counts[:w.E_tot].tolist() == ref["tiles"].tolist(), rep
+        assert int(ws.tile_counts[w.E_tot]) == ref["S"], rep
+        torch.cuda.synchronize()
+        assert B.moe_get_status(h, ws.status).code == 0
+        assert (p2.comm_ctas, p2.P, p2.W_comp) == (plan.comm_ctas, plan.P, plan.W_comp)
+        for a, o in zip(ref_outs, ws.out):
+            assert np.array_equal(a, o.float().cpu().numpy(), equal_nan=True), rep
+
+
 @pytest.mark.parametrize("tile", [(128, 256), (256, 256)], ids=["128x256", "pair"])
 def test_counts_left_on_the_device_give_the_same_bits(tile):
     # Section III-E: no copy of the routed counts and no wait; the plan comes from the normalised-load
