@@ -465,6 +465,30 @@ TL = dict(begin=0, role=1, first_acc=2, mma_end=3, tiles=4, wait_operand=5, issu
           pub_wait=32, pub_fence=33, epi_pub_wait=34)
 
 
+def gemm_only_mma_record(h, dw, step, occ, lim):
+    """One recorded GEMM-only launch on all SMs: cycles of the MMA-issuing thread per k-block and the SM clock
+    the launch ran at (those cycles over the time they took)."""
+    import numpy as np
+    import torch
+    B, w = dw.B, dw.w
+    slots = B.MOE_TIMELINE_SLOTS
+    n_words = (lim.G + 2) * slots + B.MOE_MAX_L
+    buf = torch.zeros(n_words, dtype=torch.int64, device=dw.x.device)
+    B.moe_set_timeline(h, buf, n_words * 8)
+    step(0, mode=B.MOE_MODE_GEMM_ONLY, P_override=lim.G // occ.comp_slot_sms)
+    torch.cuda.synchronize()
+    B.moe_set_timeline(h, None, 0)
+    rec = buf.cpu().numpy().astype(np.uint64)[:lim.G * slots].reshape(lim.G, slots).astype(np.float64)
+    comp = rec[rec[:, TL["tiles"]] > 0]
+    if not comp.size:
+        return None
+    kb = comp[:, TL["tiles"]] * (-(-(w.I // w.TP) // 64))
+    med = lambda v: float(np.median(v))
+    return {"cycles_per_kblock": med(comp[:, TL["mma_cycles"]] / kb), "waiting_for_operands": med(comp[:, TL["wait_operand"]] / kb),
+            "issuing": med(comp[:, TL["issue"]] / kb), "waiting_for_accumulator_buffer": med(comp[:, TL["wait_tmem"]] / kb),
+            "sm_clock_ghz": med(comp[:, TL["mma_cycles"]] / np.maximum(1.0, comp[:, TL["mma_end"]] - comp[:, TL["begin"]]))}
+
+
 def run_timeline(h, dw, step, occ, lim, args):
     """One recorded fused launch (after warm-up launches): where the time of the compute CTAs goes, when the
     splits complete and what the communication warps serve while the GEMM is still running."""
@@ -520,6 +544,8 @@ def run_timeline(h, dw, step, occ, lim, args):
             "fence_and_flag": float(np.median(allc[:, TL["pub_fence"]]) / max(1.0, float(comp[:, TL["tiles"]].mean()))),
             "epilogue_warp_waiting_for_the_publisher": float(np.median(allc[:, TL["epi_pub_wait"]]) / max(1.0, float(comp[:, TL["tiles"]].mean())))} if allc.size else None,
         "producer_wait_cycles_per_kblock": float(np.median(allc[:, TL["producer_wait"]]) / max(1.0, float(np.median(kb)))) if comp.size else None,
+        # the SM clock the launch really ran at: cycles of the MMA thread's loop over the time it took
+        "sm_clock_ghz_during_gemm": float(np.median(comp[:, TL["mma_cycles"]] / np.maximum(1.0, comp[:, TL["mma_end"]] - comp[:, TL["begin"]]))) if comp.size else None,
     }
     Q = w.k_tot * w.TP
     slab = 1024
@@ -723,7 +749,7 @@ def main():
                     help="1 (default): compute CTAs help with the communication tail; 0: the paper's static partition")
     ap.add_argument("--probe", type=int, default=0,
                     help="with --timeline: time GEMM-only launches with part of the data movement left out (bits: 1 = no W2 "
-                         "tile on every second k-block, 2 = no W2 tile at all, 4 = no Y stores); results are garbage, only "
+                         "tile on every second k-block, 2 = no W2 tile at all, 4 = no Y stores, 8 = no x tile on pair tiles, 16 = pair tiles: MMAs issued without operand barriers, 32 = pair tiles: the MMA-issuing thread idles 200 cycles per k-block); results are garbage, only "
                          "the time means something")
     ap.add_argument("--timeline", action="store_true",
                     help="run the instrumented build (libmoe_b200_timeline.so, built on demand) and print where the "
@@ -787,6 +813,7 @@ def main():
             B.moe_set_probe(h, bits)
             ts = time_fused(step, torch, 0, 3, 9, mode=B.MOE_MODE_GEMM_ONLY, P_override=lim.G // occ.comp_slot_sms)
             res["gemm_only_us" if bits == 0 else f"gemm_only_us_probe_{bits}"] = statistics.median(ts)
+            res["mma_thread" if bits == 0 else f"mma_thread_probe_{bits}"] = gemm_only_mma_record(h, dw, step, occ, lim)
         B.moe_set_probe(h, 0)
         print(json.dumps({"probe": args.probe, "workload": w.name, "tile": f"{w.tile_m}x{w.tile_n}", **res}))
         B.moe_destroy(h)

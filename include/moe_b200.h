@@ -207,9 +207,16 @@ int32_t moe_set_timeline(moe_handle *h, void *timeline_dev, size_t bytes);
  * cost shows in the launch time (the outputs of such a launch are garbage by construction; never for a result
  * that is used).  Bits: MOE_PROBE_SKIP_ODD_W2 (the W2 tile of every second k-block is not loaded: a quarter
  * less operand traffic), MOE_PROBE_SKIP_ALL_W2 (no W2 tile is loaded: half the operand traffic),
- * MOE_PROBE_SKIP_Y_STORES (the epilogue converts but does not store: no Y write traffic; GEMM-only launches).
+ * MOE_PROBE_SKIP_Y_STORES (the epilogue converts but does not store: no Y write traffic; GEMM-only launches),
+ * MOE_PROBE_SKIP_X (256-row pair tiles: no x_routed tile is loaded; with MOE_PROBE_SKIP_ALL_W2 the MMAs run on
+ * whatever shared memory holds and the launch time is that of MMA issue and epilogue alone),
+ * MOE_PROBE_FREE_RUN_MMA (256-row pair tiles: no loads, no operand barriers, no per-k-block commit: the rate at
+ * which the tensor pipe takes the MMAs when nothing but the accumulator hand-over gates them),
+ * MOE_PROBE_SLOW_ISSUER (256-row pair tiles: the thread that issues the MMAs idles 200 cycles per k-block;
+ * what the launch loses shows how little the tensor pipe buffers ahead of that thread).
  * 0 switches the probes off; the normal library accepts only 0 (MOE_ERR_UNSUPPORTED otherwise).  [host] */
-enum { MOE_PROBE_SKIP_ODD_W2 = 1, MOE_PROBE_SKIP_ALL_W2 = 2, MOE_PROBE_SKIP_Y_STORES = 4 };
+enum { MOE_PROBE_SKIP_ODD_W2 = 1, MOE_PROBE_SKIP_ALL_W2 = 2, MOE_PROBE_SKIP_Y_STORES = 4, MOE_PROBE_SKIP_X = 8,
+       MOE_PROBE_FREE_RUN_MMA = 16, MOE_PROBE_SLOW_ISSUER = 32 };
 int32_t moe_set_probe(moe_handle *h, uint32_t probe_bits);
 
 /* Tile shape and residency of the GEMM2 kernel for (tile_m, tile_n), the communication tile,

@@ -169,7 +169,7 @@ int32_t moe_set_probe(moe_handle *h, uint32_t probe_bits)
         snprintf(h->err, sizeof h->err, "moe_set_probe: this library was built without -DMOE_TIMELINE=1");
         return MOE_ERR_UNSUPPORTED;
     }
-    if (probe_bits & ~7u) return MOE_ERR_SHAPE;
+    if (probe_bits & ~63u) return MOE_ERR_SHAPE;
     h->probe = probe_bits;
     return MOE_OK;
 }

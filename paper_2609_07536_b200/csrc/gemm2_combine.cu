@@ -77,7 +77,7 @@ __device__ __forceinline__ void tl_put(const FusedParams &P, int slot, unsigned 
 #else
 #define MOE_PROBE(bit) false
 #endif
-enum { kProbeSkipOddW2 = 1, kProbeSkipAllW2 = 2, kProbeSkipYStores = 4 };
+enum { kProbeSkipOddW2 = 1, kProbeSkipAllW2 = 2, kProbeSkipYStores = 4, kProbeSkipX = 8, kProbeFreeRunMma = 16, kProbeSlowIssuer = 32 };
 
 // --------------------------------------------------------------------------- shared memory
 
@@ -569,9 +569,16 @@ __device__ void compute_cta(const FusedParams &P, int W_comp, uint8_t *ring, Con
         }
         __syncwarp();
     } else if (warp == 1) {
-        // ---------------- MMA issuer: one thread runs the whole loop
+        // ---------------- MMA issuer: one thread runs the whole loop, kept as short as it can be (the tensor
+        // pipe buffers little ahead of the MMA it executes, see compute_cta_pair): a whole k-block (four MMAs
+        // and the commit) is one statement with 32-bit descriptor arithmetic, addresses advance by additions,
+        // the barrier's first test is inline.
         if (lane == 0) {
             constexpr uint32_t idesc = make_idesc(kMmaM, TN);
+            constexpr uint32_t kLoStage = (uint32_t)(C::kStageBytes >> 4), kLoB = (uint32_t)(C::kABytes >> 4);
+            const uint32_t lo0 = smem_desc_lo(smem_u32(ring));
+            const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
+            uint32_t a_lo = lo0, full_bar = full0, empty_bar = empty0;
             int stage = 0;
             uint32_t phase = 0;
             int it = 0;
@@ -588,31 +595,33 @@ __device__ void compute_cta(const FusedParams &P, int W_comp, uint8_t *ring, Con
                 const uint32_t d_tmem = tmem_base + (uint32_t)(a * TN);
                 for (int kb = 0; kb < P.num_kb; ++kb) {
                     TL(tl_q = clock64());
-                    ok = wait_barrier_1t(smem_u32(&ctl->full[stage]), phase, ctl, deadline, P.status, (uint32_t)g, 21u);
-                    if (!ok) break;
+                    if (!mbar_try_wait(full_bar, phase)) {
+                        ok = wait_barrier_1t(full_bar, phase, ctl, deadline, P.status, (uint32_t)g, 21u);
+                        if (!ok) break;
+                    }
                     TL(tl_wf += clock64() - tl_q; tl_q = clock64());
                     tc_fence_after();
-                    const uint32_t a_addr = smem_u32(ring + stage * C::kStageBytes);
-                    const uint64_t a_desc = make_smem_desc(a_addr);
-                    const uint64_t b_desc = make_smem_desc(a_addr + C::kABytes);
-                    const int ksteps = (kb == P.num_kb - 1) ? P.last_ksteps : (kBlockK / kUmmaK);
-                    // advancing K by 16 bf16 = 32 bytes inside the swizzle row: +2 in the address field.
-                    // The full k-block is written out: the issuing thread has to stay ahead of the tensor
-                    // pipe, and the rolled loop (variable trip count, 64-bit adds) costs it twice the cycles.
-                    const uint32_t acc0 = kb > 0 ? 1u : 0u;
-                    if (ksteps == kBlockK / kUmmaK) {
-                        tc_mma_bf16(d_tmem, a_desc, b_desc, idesc, acc0);
-                        tc_mma_bf16(d_tmem, a_desc + 2ull, b_desc + 2ull, idesc, 1u);
-                        tc_mma_bf16(d_tmem, a_desc + 4ull, b_desc + 4ull, idesc, 1u);
-                        tc_mma_bf16(d_tmem, a_desc + 6ull, b_desc + 6ull, idesc, 1u);
+                    // advancing K by 16 bf16 = 32 bytes inside the swizzle row: +2 in the address field
+                    if (kb < P.num_kb - 1 || P.last_ksteps == kBlockK / kUmmaK) {
+                        tc_kblock_bf16(d_tmem, a_lo, a_lo + kLoB, idesc, kb > 0 ? 1u : 0u, empty_bar);
                     } else {
-                        for (int k = 0; k < ksteps; ++k)
+                        const uint64_t a_desc = ((uint64_t)kSmemDescHi << 32) | a_lo, b_desc = a_desc + kLoB;
+                        for (int k = 0; k < P.last_ksteps; ++k)
                             tc_mma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
-                                        k > 0 ? 1u : acc0);
+                                        (k > 0 || kb > 0) ? 1u : 0u);
+                        tc_commit(empty_bar);   // stage reusable once these MMAs have read it
                     }
-                    tc_commit(smem_u32(&ctl->empty[stage]));   // stage reusable once these MMAs have read it
                     TL(tl_is += clock64() - tl_q);
-                    if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+                    a_lo += kLoStage;
+                    full_bar += 8u;
+                    empty_bar += 8u;
+                    if (++stage == C::kStages) {
+                        stage = 0;
+                        phase ^= 1u;
+                        a_lo = lo0;
+                        full_bar = full0;
+                        empty_bar = empty0;
+                    }
                 }
                 if (ok) tc_commit(smem_u32(&ctl->tmem_full[a]));  // accumulator complete
                 TL(if (it == 0) tl_put(P, kTlFirstAcc, globaltimer_ns()));
@@ -695,7 +704,7 @@ __device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring
         // rows; both complete on the leader's full barrier.  Two issuing threads halve the serial issue
         // latency per k-block.  One thread per warp runs the whole loop; the others park below.
         const bool load_a = (warp == 0);
-        if (lane == 0 && b < total_tiles) {
+        if (lane == 0 && b < total_tiles && !MOE_PROBE(kProbeFreeRunMma)) {
             int stage = 0;
             uint32_t phase = 0;
             uint32_t armed = 0;
@@ -721,8 +730,10 @@ __device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring
                     const uint32_t a_dst = smem_u32(ring + stage * C::kStageBytes);
                     const bool skip_b = MOE_PROBE(kProbeSkipAllW2) || (MOE_PROBE(kProbeSkipOddW2) && (kb & 1));
                     if (load_a) {
-                        if (leader_cta) mbar_arrive_expect_tx(own_full, 2u * (uint32_t)(skip_b ? C::kABytes : C::kStageBytes));
-                        tma_load_2d_pair(a_dst, &P.tmA, leader_full, kx, row0);
+                        const bool skip_a = MOE_PROBE(kProbeSkipX);
+                        if (leader_cta)
+                            mbar_arrive_expect_tx(own_full, 2u * (uint32_t)((skip_b ? 0 : C::kStageBytes - C::kABytes) + (skip_a ? 0 : C::kABytes)));
+                        if (!skip_a) tma_load_2d_pair(a_dst, &P.tmA, leader_full, kx, row0);
                     } else if (!skip_b) {
                         tma_load_3d_pair(a_dst + C::kABytes, &P.tmB, leader_full, kx, n0, e);
                     }
@@ -746,9 +757,17 @@ __device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring
         }
         __syncwarp();
     } else if (warp == 1 && leader_cta) {
-        // ---------------- MMA issuer (leader CTA only): one thread runs the whole loop
+        // ---------------- MMA issuer (leader CTA only): one thread runs the whole loop, and that loop is kept
+        // as short as it can be.  The tensor pipe buffers little ahead of the MMA it executes: with 200 idle
+        // cycles of this thread per k-block a launch takes 130 cycles per k-block longer (bench.py --timeline
+        // --probe 32).  A whole k-block (four MMAs and the commit) is one statement with 32-bit descriptor
+        // arithmetic; addresses advance by additions; the barrier's first test is inline.
         if (lane == 0) {
             constexpr uint32_t idesc = make_idesc(2 * kMmaM, TN);
+            constexpr uint32_t kLoStage = (uint32_t)(C::kStageBytes >> 4), kLoB = (uint32_t)(C::kABytes >> 4);
+            const uint32_t lo0 = smem_desc_lo(smem_u32(ring));
+            const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
+            uint32_t a_lo = lo0, full_bar = full0, empty_bar = empty0;
             int stage = 0;
             uint32_t phase = 0;
             int it = 0;
@@ -765,28 +784,37 @@ __device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring
                 const uint32_t d_tmem = tmem_base + (uint32_t)(a * TN);
                 for (int kb = 0; kb < P.num_kb; ++kb) {
                     TL(tl_q = clock64());
-                    ok = wait_barrier_1t(smem_u32(&ctl->full[stage]), phase, ctl, deadline, P.status, (uint32_t)g, 21u);
-                    if (!ok) break;
+                    if (!MOE_PROBE(kProbeFreeRunMma) && !mbar_try_wait(full_bar, phase)) {
+                        ok = wait_barrier_1t(full_bar, phase, ctl, deadline, P.status, (uint32_t)g, 21u);
+                        if (!ok) break;
+                    }
                     TL(tl_wf += clock64() - tl_q; tl_q = clock64());
                     tc_fence_after();
-                    const uint32_t a_addr = smem_u32(ring + stage * C::kStageBytes);
-                    const uint64_t a_desc = make_smem_desc(a_addr);
-                    const uint64_t b_desc = make_smem_desc(a_addr + C::kABytes);
-                    const int ksteps = (kb == P.num_kb - 1) ? P.last_ksteps : (kBlockK / kUmmaK);
-                    const uint32_t acc0 = kb > 0 ? 1u : 0u;
-                    if (ksteps == kBlockK / kUmmaK) {   // written out: see compute_cta
-                        tc_mma_bf16_pair(d_tmem, a_desc, b_desc, idesc, acc0);
-                        tc_mma_bf16_pair(d_tmem, a_desc + 2ull, b_desc + 2ull, idesc, 1u);
-                        tc_mma_bf16_pair(d_tmem, a_desc + 4ull, b_desc + 4ull, idesc, 1u);
-                        tc_mma_bf16_pair(d_tmem, a_desc + 6ull, b_desc + 6ull, idesc, 1u);
+                    if (MOE_PROBE(kProbeSlowIssuer)) {   // 200 cycles in which this thread issues nothing
+                        const long long until = clock64() + 200;
+                        while (clock64() < until) {}
+                    }
+                    if ((kb < P.num_kb - 1 || P.last_ksteps == kBlockK / kUmmaK) && !MOE_PROBE(kProbeFreeRunMma)) {
+                        tc_kblock_bf16_pair(d_tmem, a_lo, a_lo + kLoB, idesc, kb > 0 ? 1u : 0u, empty_bar);
                     } else {
+                        const uint64_t a_desc = ((uint64_t)kSmemDescHi << 32) | a_lo, b_desc = a_desc + kLoB;
+                        const int ksteps = (kb == P.num_kb - 1) ? P.last_ksteps : (kBlockK / kUmmaK);
                         for (int k = 0; k < ksteps; ++k)
                             tc_mma_bf16_pair(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
-                                             k > 0 ? 1u : acc0);
+                                             (k > 0 || kb > 0) ? 1u : 0u);
+                        if (!MOE_PROBE(kProbeFreeRunMma)) tc_commit_pair(empty_bar);      // both CTAs may refill the stage
                     }
-                    tc_commit_pair(smem_u32(&ctl->empty[stage]));      // both CTAs may refill the stage
                     TL(tl_is += clock64() - tl_q);
-                    if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+                    a_lo += kLoStage;
+                    full_bar += 8u;
+                    empty_bar += 8u;
+                    if (++stage == C::kStages) {
+                        stage = 0;
+                        phase ^= 1u;
+                        a_lo = lo0;
+                        full_bar = full0;
+                        empty_bar = empty0;
+                    }
                 }
                 if (ok) tc_commit_pair(smem_u32(&ctl->tmem_full[a]));   // both epilogues may start
                 TL(if (it == 0) tl_put(P, kTlFirstAcc, globaltimer_ns()));

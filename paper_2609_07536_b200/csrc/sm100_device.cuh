@@ -199,6 +199,72 @@ __device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_des
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// One whole k-block of a pair tile in one statement: four MMAs (K = 16 each, 32 bytes further along the
+// swizzle row every time) and the commit that hands the stage back to both CTAs.  The thread that issues
+// the MMAs is on the critical path of the tensor pipe (the pipe buffers hardly any MMA ahead), so the
+// descriptors are kept as their low words (start address field and the constant leading offset) and
+// glued to the constant high word here instead of being rebuilt with 64-bit arithmetic per MMA.
+constexpr uint32_t kSmemDescHi = (uint32_t)(1024 >> 4) | (1u << 14) | (2u << 29);   // stride offset, version, SWIZZLE_128B
+__device__ __forceinline__ uint32_t smem_desc_lo(uint32_t smem_addr) { return ((smem_addr & 0x3FFFFu) >> 4) | (1u << 16); }
+__device__ __forceinline__ void tc_kblock_bf16_pair(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t accumulate,
+                                                    uint32_t empty_bar)
+{
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t.reg .b64 da, db;\n\t.reg .b32 al, bl;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "setp.eq.b32 q, %4, %4;\n\t"
+        "mov.b64 da, {%1, %6};\n\t"
+        "mov.b64 db, {%2, %6};\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %3, p;\n\t"
+        "add.u32 al, %1, 2;\n\t"
+        "add.u32 bl, %2, 2;\n\t"
+        "mov.b64 da, {al, %6};\n\t"
+        "mov.b64 db, {bl, %6};\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %3, q;\n\t"
+        "add.u32 al, %1, 4;\n\t"
+        "add.u32 bl, %2, 4;\n\t"
+        "mov.b64 da, {al, %6};\n\t"
+        "mov.b64 db, {bl, %6};\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %3, q;\n\t"
+        "add.u32 al, %1, 6;\n\t"
+        "add.u32 bl, %2, 6;\n\t"
+        "mov.b64 da, {al, %6};\n\t"
+        "mov.b64 db, {bl, %6};\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %3, q;\n\t"
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%5], %7;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(empty_bar), "r"(kSmemDescHi), "h"((uint16_t)3)
+        : "memory");
+}
+// the same for a tile computed by one CTA (cta_group::1): four MMAs and the commit on this CTA's barrier
+__device__ __forceinline__ void tc_kblock_bf16(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t accumulate,
+                                               uint32_t empty_bar)
+{
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t.reg .b64 da, db;\n\t.reg .b32 al, bl;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "setp.eq.b32 q, %4, %4;\n\t"
+        "mov.b64 da, {%1, %6};\n\t"
+        "mov.b64 db, {%2, %6};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t"
+        "add.u32 al, %1, 2;\n\t"
+        "add.u32 bl, %2, 2;\n\t"
+        "mov.b64 da, {al, %6};\n\t"
+        "mov.b64 db, {bl, %6};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, q;\n\t"
+        "add.u32 al, %1, 4;\n\t"
+        "add.u32 bl, %2, 4;\n\t"
+        "mov.b64 da, {al, %6};\n\t"
+        "mov.b64 db, {bl, %6};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, q;\n\t"
+        "add.u32 al, %1, 6;\n\t"
+        "add.u32 bl, %2, 6;\n\t"
+        "mov.b64 da, {al, %6};\n\t"
+        "mov.b64 db, {bl, %6};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, q;\n\t"
+        "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%5];\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(empty_bar), "r"(kSmemDescHi)
+        : "memory");
+}
 // 32 lanes x 32 consecutive fp32 columns: thread i reads TMEM lane (base lane + i)
 __device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32])
 {
