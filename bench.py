@@ -462,7 +462,7 @@ def run_decode(h, args, device, peaks):
 
 TL = dict(begin=0, role=1, first_acc=2, mma_end=3, tiles=4, wait_operand=5, issue=6, wait_tmem=7, mma_cycles=8,
           compute_end=9, cta_end=10, epi_wait=11, epi_work=12, producer_wait=13, comm_units=14, comm_wait_ns=15, co=16,
-          pub_wait=32, pub_fence=33, epi_pub_wait=34)
+          pub_wait=32, pub_fence=33, epi_pub_wait=34, stage_late=35)
 
 
 def gemm_only_mma_record(h, dw, step, occ, lim):
@@ -486,7 +486,8 @@ def gemm_only_mma_record(h, dw, step, occ, lim):
     med = lambda v: float(np.median(v))
     return {"cycles_per_kblock": med(comp[:, TL["mma_cycles"]] / kb), "waiting_for_operands": med(comp[:, TL["wait_operand"]] / kb),
             "issuing": med(comp[:, TL["issue"]] / kb), "waiting_for_accumulator_buffer": med(comp[:, TL["wait_tmem"]] / kb),
-            "sm_clock_ghz": med(comp[:, TL["mma_cycles"]] / np.maximum(1.0, comp[:, TL["mma_end"]] - comp[:, TL["begin"]]))}
+            "sm_clock_ghz": med(comp[:, TL["mma_cycles"]] / np.maximum(1.0, comp[:, TL["mma_end"]] - comp[:, TL["begin"]])),
+            "share_of_kblocks_whose_stage_was_not_ready": med(comp[:, TL["stage_late"]] / kb) if w.tile_m == 256 else None}
 
 
 def run_timeline(h, dw, step, occ, lim, args):

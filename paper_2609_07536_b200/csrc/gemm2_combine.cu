@@ -64,7 +64,8 @@ enum {
     kTlBegin = 0, kTlRole = 1, kTlFirstAcc = 2, kTlMmaEnd = 3, kTlTiles = 4, kTlWaitOperand = 5, kTlIssue = 6,
     kTlWaitTmem = 7, kTlMmaCycles = 8, kTlComputeEnd = 9, kTlCtaEnd = 10, kTlEpiWait = 11, kTlEpiWork = 12,
     kTlProducerWait = 13, kTlCommUnits = 14, kTlCommWaitNs = 15, kTlCoWarp = 16,  // 8 slots per co-resident warp (16..31)
-    kTlPubWait = 32, kTlPubFence = 33, kTlEpiPubWait = 34
+    kTlPubWait = 32, kTlPubFence = 33, kTlEpiPubWait = 34,
+    kTlStageLate = 35   // pair tiles: k-blocks whose operand stage was not complete when the MMA thread first looked
 };
 #if MOE_TIMELINE
 __device__ __forceinline__ void tl_put(const FusedParams &P, int slot, unsigned long long v)
@@ -569,11 +570,11 @@ __device__ void compute_cta(const FusedParams &P, int W_comp, uint8_t *ring, Con
         }
         __syncwarp();
     } else if (warp == 1) {
-        // ---------------- MMA issuer: one thread runs the whole loop, kept as short as it can be (the tensor
-        // pipe buffers little ahead of the MMA it executes, see compute_cta_pair): a whole k-block (four MMAs
-        // and the commit) is one statement with 32-bit descriptor arithmetic, addresses advance by additions,
-        // the barrier's first test is inline.
-        if (lane == 0) {
+        // ---------------- MMA issuer: the whole warp runs the loop, converged, one elected lane issues; the loop
+        // is as short as it can be and its operands are warp-uniform (both for the reasons given in
+        // compute_cta_pair): a whole k-block (four MMAs and the commit) is one statement with 32-bit descriptor
+        // arithmetic, addresses advance by additions, the barrier's first look is the non-suspending test.
+        {
             constexpr uint32_t idesc = make_idesc(kMmaM, TN);
             constexpr uint32_t kLoStage = (uint32_t)(C::kStageBytes >> 4), kLoB = (uint32_t)(C::kABytes >> 4);
             const uint32_t lo0 = smem_desc_lo(smem_u32(ring));
@@ -588,28 +589,33 @@ __device__ void compute_cta(const FusedParams &P, int W_comp, uint8_t *ring, Con
                 const int a = it & 1;
                 const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
                 TL(tl_q = clock64());
-                ok = wait_barrier_1t(smem_u32(&ctl->tmem_empty[a]), acc_phase ^ 1u, ctl, deadline, P.status, (uint32_t)g, 20u);
-                if (!ok) break;
+                if (!__all_sync(0xffffffffu, mbar_test_wait(smem_u32(&ctl->tmem_empty[a]), acc_phase ^ 1u))) {
+                    // (every lane polls; the vote keeps `ok`, and with it the loop, provably warp-uniform)
+                    ok = __all_sync(0xffffffffu, wait_barrier_1t(smem_u32(&ctl->tmem_empty[a]), acc_phase ^ 1u, ctl, deadline, P.status, (uint32_t)g, 20u));
+                    if (!ok) break;
+                }
                 TL(tl_wt += clock64() - tl_q);
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(a * TN);
                 for (int kb = 0; kb < P.num_kb; ++kb) {
                     TL(tl_q = clock64());
-                    if (!mbar_try_wait(full_bar, phase)) {
-                        ok = wait_barrier_1t(full_bar, phase, ctl, deadline, P.status, (uint32_t)g, 21u);
+                    if (!__all_sync(0xffffffffu, mbar_test_wait(full_bar, phase))) {
+                        ok = __all_sync(0xffffffffu, wait_barrier_1t(full_bar, phase, ctl, deadline, P.status, (uint32_t)g, 21u));
                         if (!ok) break;
                     }
                     TL(tl_wf += clock64() - tl_q; tl_q = clock64());
                     tc_fence_after();
                     // advancing K by 16 bf16 = 32 bytes inside the swizzle row: +2 in the address field
-                    if (kb < P.num_kb - 1 || P.last_ksteps == kBlockK / kUmmaK) {
-                        tc_kblock_bf16(d_tmem, a_lo, a_lo + kLoB, idesc, kb > 0 ? 1u : 0u, empty_bar);
-                    } else {
-                        const uint64_t a_desc = ((uint64_t)kSmemDescHi << 32) | a_lo, b_desc = a_desc + kLoB;
-                        for (int k = 0; k < P.last_ksteps; ++k)
-                            tc_mma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
-                                        (k > 0 || kb > 0) ? 1u : 0u);
-                        tc_commit(empty_bar);   // stage reusable once these MMAs have read it
+                    if (elect_one_sync()) {
+                        if (kb < P.num_kb - 1 || P.last_ksteps == kBlockK / kUmmaK) {
+                            tc_kblock_bf16(d_tmem, a_lo, a_lo + kLoB, idesc, kb > 0 ? 1u : 0u, empty_bar);
+                        } else {
+                            const uint64_t a_desc = ((uint64_t)kSmemDescHi << 32) | a_lo, b_desc = a_desc + kLoB;
+                            for (int k = 0; k < P.last_ksteps; ++k)
+                                tc_mma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
+                                            (k > 0 || kb > 0) ? 1u : 0u);
+                            tc_commit(empty_bar);   // stage reusable once these MMAs have read it
+                        }
                     }
                     TL(tl_is += clock64() - tl_q);
                     a_lo += kLoStage;
@@ -623,12 +629,14 @@ __device__ void compute_cta(const FusedParams &P, int W_comp, uint8_t *ring, Con
                         empty_bar = empty0;
                     }
                 }
-                if (ok) tc_commit(smem_u32(&ctl->tmem_full[a]));  // accumulator complete
-                TL(if (it == 0) tl_put(P, kTlFirstAcc, globaltimer_ns()));
+                __syncwarp();
+                if (ok && elect_one_sync()) tc_commit(smem_u32(&ctl->tmem_full[a]));  // accumulator complete
+                TL(if (it == 0 && lane == 0) tl_put(P, kTlFirstAcc, globaltimer_ns()));
             }
-            TL(tl_put(P, kTlMmaEnd, globaltimer_ns()); tl_put(P, kTlTiles, (unsigned long long)it);
-               tl_put(P, kTlWaitOperand, (unsigned long long)tl_wf); tl_put(P, kTlIssue, (unsigned long long)tl_is);
-               tl_put(P, kTlWaitTmem, (unsigned long long)tl_wt); tl_put(P, kTlMmaCycles, (unsigned long long)(clock64() - tl_c0)));
+            TL(if (lane == 0) {
+                   tl_put(P, kTlMmaEnd, globaltimer_ns()); tl_put(P, kTlTiles, (unsigned long long)it);
+                   tl_put(P, kTlWaitOperand, (unsigned long long)tl_wf); tl_put(P, kTlIssue, (unsigned long long)tl_is);
+                   tl_put(P, kTlWaitTmem, (unsigned long long)tl_wt); tl_put(P, kTlMmaCycles, (unsigned long long)(clock64() - tl_c0)); });
         }
         __syncwarp();
     } else if (warp >= 4 && warp < 4 + P.epi_warps) {
@@ -757,12 +765,16 @@ __device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring
         }
         __syncwarp();
     } else if (warp == 1 && leader_cta) {
-        // ---------------- MMA issuer (leader CTA only): one thread runs the whole loop, and that loop is kept
-        // as short as it can be.  The tensor pipe buffers little ahead of the MMA it executes: with 200 idle
-        // cycles of this thread per k-block a launch takes 130 cycles per k-block longer (bench.py --timeline
-        // --probe 32).  A whole k-block (four MMAs and the commit) is one statement with 32-bit descriptor
-        // arithmetic; addresses advance by additions; the barrier's first test is inline.
-        if (lane == 0) {
+        // ---------------- MMA issuer (leader CTA only).  The whole warp runs the loop, converged, and one elected
+        // lane issues.  Two measured facts shape it.  (1) The tensor pipe buffers little ahead of the MMA it
+        // executes: 200 idle cycles of the issuer per k-block cost a launch 130 cycles per k-block
+        // (bench.py --timeline --probe 32), so the loop is as short as it can be: a whole k-block (four MMAs and
+        // the commit) is one statement with 32-bit descriptor arithmetic, addresses advance by additions, the
+        // barrier's first look is the non-suspending test.  (2) tcgen05.mma takes its descriptors and addresses
+        // from uniform registers: when a single thread ran this loop inside `if (lane == 0)` every operand was
+        // moved over from ordinary registers, MMA by MMA; with warp-uniform values in warp-uniform control flow
+        // and elect.sync around the issue the GEMM phase is 6 % faster.
+        {
             constexpr uint32_t idesc = make_idesc(2 * kMmaM, TN);
             constexpr uint32_t kLoStage = (uint32_t)(C::kStageBytes >> 4), kLoB = (uint32_t)(C::kABytes >> 4);
             const uint32_t lo0 = smem_desc_lo(smem_u32(ring));
@@ -772,37 +784,43 @@ __device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring
             uint32_t phase = 0;
             int it = 0;
             bool ok = true;
-            TL_DECL(const long long tl_c0 = clock64(); long long tl_wf = 0, tl_wt = 0, tl_is = 0, tl_q;)
+            TL_DECL(const long long tl_c0 = clock64(); long long tl_wf = 0, tl_wt = 0, tl_is = 0, tl_q; unsigned long long tl_late = 0;)
             for (int g = b; g < total_tiles && ok; g += P.P, ++it) {
                 const int a = it & 1;
                 const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
                 TL(tl_q = clock64());
-                ok = wait_barrier_1t(smem_u32(&ctl->tmem_empty[a]), acc_phase ^ 1u, ctl, deadline, P.status, (uint32_t)g, 20u);
-                if (!ok) break;
+                if (!__all_sync(0xffffffffu, mbar_test_wait(smem_u32(&ctl->tmem_empty[a]), acc_phase ^ 1u))) {
+                    // (every lane polls; the vote keeps `ok`, and with it the loop, provably warp-uniform)
+                    ok = __all_sync(0xffffffffu, wait_barrier_1t(smem_u32(&ctl->tmem_empty[a]), acc_phase ^ 1u, ctl, deadline, P.status, (uint32_t)g, 20u));
+                    if (!ok) break;
+                }
                 TL(tl_wt += clock64() - tl_q);
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(a * TN);
                 for (int kb = 0; kb < P.num_kb; ++kb) {
                     TL(tl_q = clock64());
-                    if (!MOE_PROBE(kProbeFreeRunMma) && !mbar_try_wait(full_bar, phase)) {
-                        ok = wait_barrier_1t(full_bar, phase, ctl, deadline, P.status, (uint32_t)g, 21u);
+                    if (!MOE_PROBE(kProbeFreeRunMma) && !__all_sync(0xffffffffu, mbar_test_wait(full_bar, phase))) {
+                        TL(++tl_late);
+                        ok = __all_sync(0xffffffffu, wait_barrier_1t(full_bar, phase, ctl, deadline, P.status, (uint32_t)g, 21u));
                         if (!ok) break;
                     }
                     TL(tl_wf += clock64() - tl_q; tl_q = clock64());
                     tc_fence_after();
-                    if (MOE_PROBE(kProbeSlowIssuer)) {   // 200 cycles in which this thread issues nothing
+                    if (MOE_PROBE(kProbeSlowIssuer)) {   // 200 cycles in which nothing is issued
                         const long long until = clock64() + 200;
                         while (clock64() < until) {}
                     }
-                    if ((kb < P.num_kb - 1 || P.last_ksteps == kBlockK / kUmmaK) && !MOE_PROBE(kProbeFreeRunMma)) {
-                        tc_kblock_bf16_pair(d_tmem, a_lo, a_lo + kLoB, idesc, kb > 0 ? 1u : 0u, empty_bar);
-                    } else {
-                        const uint64_t a_desc = ((uint64_t)kSmemDescHi << 32) | a_lo, b_desc = a_desc + kLoB;
-                        const int ksteps = (kb == P.num_kb - 1) ? P.last_ksteps : (kBlockK / kUmmaK);
-                        for (int k = 0; k < ksteps; ++k)
-                            tc_mma_bf16_pair(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
-                                             (k > 0 || kb > 0) ? 1u : 0u);
-                        if (!MOE_PROBE(kProbeFreeRunMma)) tc_commit_pair(empty_bar);      // both CTAs may refill the stage
+                    if (elect_one_sync()) {
+                        if ((kb < P.num_kb - 1 || P.last_ksteps == kBlockK / kUmmaK) && !MOE_PROBE(kProbeFreeRunMma)) {
+                            tc_kblock_bf16_pair(d_tmem, a_lo, a_lo + kLoB, idesc, kb > 0 ? 1u : 0u, empty_bar);
+                        } else {
+                            const uint64_t a_desc = ((uint64_t)kSmemDescHi << 32) | a_lo, b_desc = a_desc + kLoB;
+                            const int ksteps = (kb == P.num_kb - 1) ? P.last_ksteps : (kBlockK / kUmmaK);
+                            for (int k = 0; k < ksteps; ++k)
+                                tc_mma_bf16_pair(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
+                                                 (k > 0 || kb > 0) ? 1u : 0u);
+                            if (!MOE_PROBE(kProbeFreeRunMma)) tc_commit_pair(empty_bar);      // both CTAs may refill the stage
+                        }
                     }
                     TL(tl_is += clock64() - tl_q);
                     a_lo += kLoStage;
@@ -816,12 +834,15 @@ __device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring
                         empty_bar = empty0;
                     }
                 }
-                if (ok) tc_commit_pair(smem_u32(&ctl->tmem_full[a]));   // both epilogues may start
-                TL(if (it == 0) tl_put(P, kTlFirstAcc, globaltimer_ns()));
+                __syncwarp();
+                if (ok && elect_one_sync()) tc_commit_pair(smem_u32(&ctl->tmem_full[a]));   // both epilogues may start
+                TL(if (it == 0 && lane == 0) tl_put(P, kTlFirstAcc, globaltimer_ns()));
             }
-            TL(tl_put(P, kTlMmaEnd, globaltimer_ns()); tl_put(P, kTlTiles, (unsigned long long)it);
-               tl_put(P, kTlWaitOperand, (unsigned long long)tl_wf); tl_put(P, kTlIssue, (unsigned long long)tl_is);
-               tl_put(P, kTlWaitTmem, (unsigned long long)tl_wt); tl_put(P, kTlMmaCycles, (unsigned long long)(clock64() - tl_c0)));
+            TL(if (lane == 0) {
+                   tl_put(P, kTlMmaEnd, globaltimer_ns()); tl_put(P, kTlTiles, (unsigned long long)it);
+                   tl_put(P, kTlWaitOperand, (unsigned long long)tl_wf); tl_put(P, kTlIssue, (unsigned long long)tl_is);
+                   tl_put(P, kTlWaitTmem, (unsigned long long)tl_wt); tl_put(P, kTlMmaCycles, (unsigned long long)(clock64() - tl_c0));
+                   tl_put(P, kTlStageLate, tl_late); });
         }
         __syncwarp();
     } else if (warp >= 4 && warp < 4 + P.epi_warps) {

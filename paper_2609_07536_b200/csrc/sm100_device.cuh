@@ -199,6 +199,17 @@ __device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_des
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// true in exactly one lane of a converged warp
+__device__ __forceinline__ bool elect_one_sync()
+{
+    uint32_t pred;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "elect.sync _|p, 0xffffffff;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(pred));
+    return pred != 0;
+}
 // One whole k-block of a pair tile in one statement: four MMAs (K = 16 each, 32 bytes further along the
 // swizzle row every time) and the commit that hands the stage back to both CTAs.  The thread that issues
 // the MMAs is on the critical path of the tensor pipe (the pipe buffers hardly any MMA ahead), so the
