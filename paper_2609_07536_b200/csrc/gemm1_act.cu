@@ -194,42 +194,60 @@ moe_gemm1_act_kernel(const __grid_constant__ G1Params P)
         }
         __syncwarp();
     } else if (warp == 1) {
-        // ---------------- MMA issuer
-        if (lane == 0) {
+        // ---------------- MMA issuer: the whole warp runs the loop, converged, and one elected lane issues.
+        // tcgen05.mma takes its descriptors and addresses from uniform registers, and the tensor pipe buffers
+        // little ahead of the MMA it executes: warp-uniform values in warp-uniform control flow spare a move per
+        // operand and MMA, a whole k-block (four MMAs and the commit) is one statement with 32-bit descriptor
+        // arithmetic, addresses advance by additions, the barrier's first look is the non-suspending test.
+        {
             constexpr uint32_t idesc = make_idesc(kMmaM, 2 * kG1TileN);
+            constexpr uint32_t kLoStage = (uint32_t)(kG1StageBytes >> 4), kLoB = (uint32_t)(kG1ABytes >> 4);
+            const uint32_t lo0 = smem_desc_lo(smem_u32(ring));
+            const uint32_t full0 = smem_u32(&ctl->full[0]), empty0 = smem_u32(&ctl->empty[0]);
+            uint32_t a_lo = lo0, full_bar = full0, empty_bar = empty0;
             int stage = 0, it = 0;
             uint32_t phase = 0;
             bool ok = true;
             for (int g = b; g < total_tiles && ok; g += stride, ++it) {
                 const int a = it & 1;
-                ok = g1_wait(smem_u32(&ctl->tmem_empty[a]), ((uint32_t)(it >> 1) & 1u) ^ 1u, ctl, deadline, P.status,
-                             (uint32_t)g, 51u);
-                if (!ok) break;
+                const uint32_t acc_parity = ((uint32_t)(it >> 1) & 1u) ^ 1u;
+                if (!__all_sync(0xffffffffu, mbar_test_wait(smem_u32(&ctl->tmem_empty[a]), acc_parity))) {
+                    // (every lane polls; the vote keeps `ok`, and with it the loop, provably warp-uniform)
+                    ok = __all_sync(0xffffffffu, g1_wait(smem_u32(&ctl->tmem_empty[a]), acc_parity, ctl, deadline, P.status, (uint32_t)g, 51u));
+                    if (!ok) break;
+                }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(a * 2 * kG1TileN);
                 for (int kb = 0; kb < P.num_kb; ++kb) {
-                    ok = g1_wait(smem_u32(&ctl->full[stage]), phase, ctl, deadline, P.status, (uint32_t)g, 52u);
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint32_t a_addr = smem_u32(ring + stage * kG1StageBytes);
-                    const uint64_t a_desc = make_smem_desc(a_addr);
-                    const uint64_t b_desc = make_smem_desc(a_addr + kG1ABytes);
-                    const int ksteps = (kb == P.num_kb - 1) ? P.last_ksteps : (kBlockK / kUmmaK);
-                    const uint32_t acc0 = kb > 0 ? 1u : 0u;
-                    if (ksteps == kBlockK / kUmmaK) {
-                        tc_mma_bf16(d_tmem, a_desc, b_desc, idesc, acc0);
-                        tc_mma_bf16(d_tmem, a_desc + 2ull, b_desc + 2ull, idesc, 1u);
-                        tc_mma_bf16(d_tmem, a_desc + 4ull, b_desc + 4ull, idesc, 1u);
-                        tc_mma_bf16(d_tmem, a_desc + 6ull, b_desc + 6ull, idesc, 1u);
-                    } else {
-                        for (int k = 0; k < ksteps; ++k)
-                            tc_mma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
-                                        k > 0 ? 1u : acc0);
+                    if (!__all_sync(0xffffffffu, mbar_test_wait(full_bar, phase))) {
+                        ok = __all_sync(0xffffffffu, g1_wait(full_bar, phase, ctl, deadline, P.status, (uint32_t)g, 52u));
+                        if (!ok) break;
                     }
-                    tc_commit(smem_u32(&ctl->empty[stage]));
-                    if (++stage == kG1Stages) { stage = 0; phase ^= 1u; }
+                    tc_fence_after();
+                    if (elect_one_sync()) {
+                        if (kb < P.num_kb - 1 || P.last_ksteps == kBlockK / kUmmaK) {
+                            tc_kblock_bf16(d_tmem, a_lo, a_lo + kLoB, idesc, kb > 0 ? 1u : 0u, empty_bar);
+                        } else {
+                            const uint64_t a_desc = ((uint64_t)kSmemDescHi << 32) | a_lo, b_desc = a_desc + kLoB;
+                            for (int k = 0; k < P.last_ksteps; ++k)
+                                tc_mma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
+                                            (k > 0 || kb > 0) ? 1u : 0u);
+                            tc_commit(empty_bar);
+                        }
+                    }
+                    a_lo += kLoStage;
+                    full_bar += 8u;
+                    empty_bar += 8u;
+                    if (++stage == kG1Stages) {
+                        stage = 0;
+                        phase ^= 1u;
+                        a_lo = lo0;
+                        full_bar = full0;
+                        empty_bar = empty0;
+                    }
                 }
-                if (ok) tc_commit(smem_u32(&ctl->tmem_full[a]));
+                __syncwarp();
+                if (ok && elect_one_sync()) tc_commit(smem_u32(&ctl->tmem_full[a]));
             }
         }
         __syncwarp();
