@@ -253,27 +253,46 @@ __device__ __forceinline__ void store_accumulator_rows(const FusedParams &P, uin
 // per 32-column group, straight from registers.  Needs every 16-column group whole and 32-byte aligned
 // (FusedParams::wide_store).  No shared memory and no intra-warp hand-over: this is the fastest of the
 // three when the epilogue is what limits a short-K tile.
-// one 32-column group of this thread's row: bf16, two 32-byte stores
-__device__ __forceinline__ void emit_wide(const FusedParams &P, const uint32_t (&r)[32], int col, bool row_ok,
-                                          __nv_bfloat16 *ybase, int q, int n0, int col_end, int cis0)
+// One 32-column group of every lane's row: bf16, 256-bit stores, with the stores of two neighbouring lanes
+// joined: lanes 2k and 2k+1 swap half of their rows' data, so that one store instruction covers 64 contiguous bytes of a row (one request of two
+// sectors instead of two requests of one) -- half as many write requests from the SM for the same bytes,
+// which is what matters when the epilogue has time to spare and the requests compete with the operand
+// stream (long K).  No shared memory.  The whole warp runs this, also lanes without a valid row.
+__device__ __forceinline__ void emit_wide_joined(const FusedParams &P, const uint32_t (&r)[32], int col, bool row_ok,
+                                                 __nv_bfloat16 *ybase, int q, int n0, int col_end, int cis0)
 {
-    if (!row_ok || MOE_PROBE(kProbeSkipYStores)) return;
+    const int lane = threadIdx.x & 31;
+    const bool odd = lane & 1;
     const int cis = cis0 + col;
     const int slab = cis >> P.slab_shift;
     const int wslab = min(P.slab_cols, P.split_w - (slab << P.slab_shift));
     __nv_bfloat16 *dst = ybase + ((size_t)slab * P.Q << P.slab_shift) + (size_t)q * wslab + (cis & (P.slab_cols - 1));
+    if (!row_ok || MOE_PROBE(kProbeSkipYStores)) dst = nullptr;
+    uint32_t w[16];
 #pragma unroll
-    for (int v = 0; v < 2; ++v) {
-        if (n0 + col + v * 16 < col_end) {
-            uint32_t w[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[v * 16 + 2 * i]), __uint_as_float(r[v * 16 + 2 * i + 1]));
-                w[i] = *reinterpret_cast<uint32_t *>(&h);
-            }
-            st_global_v8(dst + v * 16, w);
-        }
+    for (int i = 0; i < 16; ++i) {
+        __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
+        w[i] = *reinterpret_cast<uint32_t *>(&h);
     }
+    // what the neighbour stores for this lane's row: the even lane hands over columns 16..31, the odd one 0..15
+    uint32_t other[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) other[i] = __shfl_xor_sync(0xffffffffu, odd ? w[i] : w[8 + i], 1);
+    const unsigned long long mine = reinterpret_cast<unsigned long long>(dst);
+    const unsigned long long theirs = __shfl_xor_sync(0xffffffffu, mine, 1);
+    // first instruction: the even lane's row (even lane: its columns 0..15; odd lane: the even lane's 16..31);
+    // second instruction: the odd lane's row (even lane: the odd lane's 0..15; odd lane: its own 16..31)
+    __nv_bfloat16 *p1 = reinterpret_cast<__nv_bfloat16 *>(odd ? theirs : mine);
+    __nv_bfloat16 *p2 = reinterpret_cast<__nv_bfloat16 *>(odd ? mine : theirs);
+    const int c1 = n0 + col + (odd ? 16 : 0);
+    uint32_t d1[8], d2[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        d1[i] = odd ? other[i] : w[i];
+        d2[i] = odd ? w[8 + i] : other[i];
+    }
+    if (p1 != nullptr && c1 < col_end) st_global_v8(p1 + (odd ? 16 : 0), d1);
+    if (p2 != nullptr && c1 < col_end) st_global_v8(p2 + (odd ? 16 : 0), d2);
 }
 __device__ __forceinline__ void store_accumulator_rows_wide(const FusedParams &P, uint32_t taddr, int col_first, int n_cols, bool row_ok,
                                                             __nv_bfloat16 *ybase, int q, int n0, int col_end, int cis0)
@@ -284,7 +303,7 @@ __device__ __forceinline__ void store_accumulator_rows_wide(const FusedParams &P
         uint32_t r[32];
         tmem_ld_32x32(taddr + (uint32_t)(col_first + cc), r);
         tmem_ld_wait(r);
-        emit_wide(P, r, col_first + cc, row_ok, ybase, q, n0, col_end, cis0);
+        emit_wide_joined(P, r, col_first + cc, row_ok, ybase, q, n0, col_end, cis0);
     }
 }
 
@@ -544,10 +563,14 @@ __device__ void compute_cta(const FusedParams &P, int W_comp, uint8_t *ring, Con
                     const uint32_t a_dst = smem_u32(ring + stage * C::kStageBytes);
                     const bool skip_b = MOE_PROBE(kProbeSkipAllW2) || (MOE_PROBE(kProbeSkipOddW2) && (kb & 1));
                     if (load_a) {
-                        mbar_arrive_expect_tx(full, (uint32_t)(skip_b ? C::kABytes : C::kStageBytes));
+                        mbar_arrive_expect_tx(full, (uint32_t)C::kStageBytes);
                         tma_load_2d(a_dst, &P.tmA, full, kx, row0);
                     } else if (!skip_b) {
                         tma_load_3d(a_dst + C::kABytes, &P.tmB, full, kx, n0, e);
+                    } else {
+                        // a probe that leaves the copy out completes its bytes by hand: this producer stays in
+                        // the barrier's dependency chain, or the other one could lap it
+                        mbar_complete_tx_cluster(mapa_u32(full, cluster_ctarank()), (uint32_t)(C::kStageBytes - C::kABytes));
                     }
                     armed |= 1u << stage;
                     if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
@@ -737,13 +760,16 @@ __device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring
                     const uint32_t leader_full = own_full & 0xFEFFFFFFu;   // same offset in the leader CTA (rank 0)
                     const uint32_t a_dst = smem_u32(ring + stage * C::kStageBytes);
                     const bool skip_b = MOE_PROBE(kProbeSkipAllW2) || (MOE_PROBE(kProbeSkipOddW2) && (kb & 1));
+                    // (a probe that leaves a copy out completes its bytes by hand: every producer stays in the
+                    // barrier's dependency chain, or the leader's could lap the others)
                     if (load_a) {
-                        const bool skip_a = MOE_PROBE(kProbeSkipX);
-                        if (leader_cta)
-                            mbar_arrive_expect_tx(own_full, 2u * (uint32_t)((skip_b ? 0 : C::kStageBytes - C::kABytes) + (skip_a ? 0 : C::kABytes)));
-                        if (!skip_a) tma_load_2d_pair(a_dst, &P.tmA, leader_full, kx, row0);
+                        if (leader_cta) mbar_arrive_expect_tx(own_full, 2u * (uint32_t)C::kStageBytes);
+                        if (!MOE_PROBE(kProbeSkipX)) tma_load_2d_pair(a_dst, &P.tmA, leader_full, kx, row0);
+                        else mbar_complete_tx_cluster(mapa_u32(own_full, 0u), (uint32_t)C::kABytes);
                     } else if (!skip_b) {
                         tma_load_3d_pair(a_dst + C::kABytes, &P.tmB, leader_full, kx, n0, e);
+                    } else {
+                        mbar_complete_tx_cluster(mapa_u32(own_full, 0u), (uint32_t)(C::kStageBytes - C::kABytes));
                     }
                     armed |= 1u << stage;
                     if (++stage == C::kStages) { stage = 0; phase ^= 1u; }

@@ -199,6 +199,12 @@ __device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_des
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// the transaction-count half of a copy's completion, by hand (shared::cluster address of the barrier): used where
+// a probe leaves a copy out but its issuer has to stay part of the barrier's dependency chain
+__device__ __forceinline__ void mbar_complete_tx_cluster(uint32_t bar_cluster, uint32_t bytes)
+{
+    asm volatile("mbarrier.complete_tx.relaxed.cluster.shared::cluster.b64 [%0], %1;" ::"r"(bar_cluster), "r"(bytes) : "memory");
+}
 // true in exactly one lane of a converged warp
 __device__ __forceinline__ bool elect_one_sync()
 {
