@@ -249,15 +249,14 @@ __device__ __forceinline__ void store_accumulator_rows(const FusedParams &P, uin
     }
 }
 
-// Same job with 256-bit stores: every lane writes 32 bytes (one full sector) of its own row, twice
-// per 32-column group, straight from registers.  Needs every 16-column group whole and 32-byte aligned
-// (FusedParams::wide_store).  No shared memory and no intra-warp hand-over: this is the fastest of the
-// three when the epilogue is what limits a short-K tile.
-// One 32-column group of every lane's row: bf16, 256-bit stores, with the stores of two neighbouring lanes
-// joined: lanes 2k and 2k+1 swap half of their rows' data, so that one store instruction covers 64 contiguous bytes of a row (one request of two
-// sectors instead of two requests of one) -- half as many write requests from the SM for the same bytes,
-// which is what matters when the epilogue has time to spare and the requests compete with the operand
-// stream (long K).  No shared memory.  The whole warp runs this, also lanes without a valid row.
+// Same job with 256-bit stores straight from registers (no shared memory).  Needs every 16-column group whole
+// and 32-byte aligned (FusedParams::wide_store).
+// One 32-column group of every lane's row, bf16.  The stores of two neighbouring lanes are joined: lanes 2k and
+// 2k+1 swap half of their rows' data, so that one store instruction covers 64 contiguous bytes of a row (one
+// request of two sectors instead of two requests of one sector).  Half as many write requests from the SM for
+// the same bytes: the GEMM phase gets 2 % shorter where K is long (the requests compete with the operand stream)
+// and 10 % where it is short (K = 256: the epilogue bounds the tile).  The whole warp runs this, also lanes
+// without a valid row.
 __device__ __forceinline__ void emit_wide_joined(const FusedParams &P, const uint32_t (&r)[32], int col, bool row_ok,
                                                  __nv_bfloat16 *ybase, int q, int n0, int col_end, int cis0)
 {
