@@ -209,14 +209,14 @@ int32_t moe_query_occupancy(moe_handle *h, int32_t tile_m, int32_t tile_n, moe_o
         // GEMM tile shape (Section III-E: every kernel choice brings its own).  Reference run: DeepSeek-V2-
         // Lite shape, T = 4096, uniform routing, TP = 2, EP = 2, L = 2, K = 704; each role alone on its
         // share of the SMs at C = 32: time per communication wave / time per compute wave.
-        //   128x256: 66.8 us / 6.10 us ; 256x256 (CTA pair): 65.8 / 5.31 ; 128x128: 95.5 / 4.55
+        //   128x256: 70.8 us / 5.88 us ; 256x256 (CTA pair): 71.0 / 4.75 ; 128x128: 70.6 / 3.97
         rho->K_ref = 704;
         rho->tile_m_ref = tile_m;
         rho->tile_n_ref = tile_n;
-        if (tile_m == 256) rho->rho_ref = 12.39;
-        else if (tile_n == 256) rho->rho_ref = 10.94;
-        else if (tile_n == 128) rho->rho_ref = 20.99;
-        else rho->rho_ref = 20.99 * 2.0;          // 64-wide tiles: Eq. 14 tile-area scaling from 128x128
+        if (tile_m == 256) rho->rho_ref = 14.96;
+        else if (tile_n == 256) rho->rho_ref = 12.04;
+        else if (tile_n == 128) rho->rho_ref = 17.80;
+        else rho->rho_ref = 17.80 * 2.0;          // 64-wide tiles: Eq. 14 tile-area scaling from 128x128
         if (tile_m == 64) rho->rho_ref *= 1.0;     // a 64-row tile still occupies a 128-row MMA: same wave time
         if (tile_n == 64) { rho->tile_n_ref = 64; }
         rho->D_ref = 2;
