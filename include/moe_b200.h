@@ -107,7 +107,9 @@ typedef struct {
     int32_t co_min_waves;    /* lower end of the legal set for co-resident warps: they are tried only when the compute
                                 phase is at least this many waves long, ceil(L * W_comp / P(C)) >= co_min_waves (a
                                 one-time characterisation: on short launches their start-up costs more than they can
-                                overlap); a forced w is not subject to it */
+                                overlap; moe_query_occupancy returns INT32_MAX for the 256-row CTA-pair tiles, where
+                                a co-resident warp costs the seventh operand stage and never paid); a forced w is not
+                                subject to it */
 } moe_sm_limits;
 
 /* Relative wave service rate (Eq. 13-15). */

@@ -1,5 +1,7 @@
 // Host side of the C ABI: handle, workspace layout, argument validation, tensor maps, launches.
 
+#include <climits>
+#include <cstdint>
 #include <cstring>
 #include <new>
 
@@ -71,6 +73,11 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
 }  // namespace moe
 
 using namespace moe;
+
+#ifndef MOE_PAIR_SEVENTH_STAGE
+#define MOE_PAIR_SEVENTH_STAGE 1
+#endif
+static constexpr bool kPairSeventhStage = MOE_PAIR_SEVENTH_STAGE != 0;
 
 extern "C" {
 
@@ -202,7 +209,12 @@ int32_t moe_query_occupancy(moe_handle *h, int32_t tile_m, int32_t tile_n, moe_o
         limits->force_co_warps = -1;
         limits->C_co_max = 8;       // beside co-resident warps more dedicated CTAs than this never paid (one-time sweep)
         limits->dep_model = MOE_DEP_SPLIT;
-        limits->co_min_waves = 24;  // below it co-resident warps lost 2-5 % in the sweep (T = 1024: 19 waves; T = 2048: 37)
+        // Lower end of the co-resident family's legal set (one-time sweep).  One-CTA tiles: below 24 compute waves
+        // co-resident warps lost 2-5 % (T = 1024: 19 waves; T = 2048: 37).  CTA-pair tiles: a co-resident warp takes
+        // the shared memory of the seventh operand stage, and with seven stages for w = 0 the best w > 0 candidate
+        // never beat the best w = 0 one at any size of the sweep (1.00-1.05 of it): the family is not offered (a
+        // forced w is still honoured).
+        limits->co_min_waves = (tile_m == 256) ? INT32_MAX : 24;
     }
     if (rho) {
         // One-time service-rate characterisation of this kernel family on B200 (Eq. 13), one constant per
@@ -502,6 +514,8 @@ int32_t moe_gemm2_combine(moe_handle *h, const void *x_routed, const void *W2, c
     // warps 16-19 of a compute CTA: co-resident communication warps, or -- when none is asked for -- a fourth
     // epilogue column group (a third less epilogue work per warp: what bounds tiles with a short K)
     p.epi_warps = (p.co_warps == 0 && p.wide_store) ? 16 : 12;
+    // CTA-pair kernel: with the aux region free during the GEMM it becomes a seventh operand stage
+    p.pair_stages = (pair && p.co_warps == 0 && p.wide_store && kPairSeventhStage) ? 7 : 6;
     // Tile sequence: split-major (the paper's) whenever something consumes a split while the next one is
     // computed; m-tile-major across the splits (x is read from DRAM once) when nothing does
     p.tile_order = (plan->drain_help && p.co_warps == 0) ? 1 : 0;

@@ -691,7 +691,7 @@ struct PairCfg {
     static constexpr int kABytes = kMmaM * kBlockK * 2;                 // 16 KB: this CTA's 128 rows
     static constexpr int kBBytes = (kTileN / 2) * kBlockK * 2;          // 16 KB: this CTA's 128 W2 rows
     static constexpr int kStageBytes = kABytes + kBBytes;               // 32 KB
-    static constexpr int kStages = kStageBytesTotal / kStageBytes;      // 6
+    // kStageBytesTotal / kStageBytes = 6 stages; a seventh lies in the aux region when that is free (FusedParams::pair_stages)
     static constexpr int kTmemCols = 2 * kTileN;                        // two accumulator buffers
 };
 
@@ -703,10 +703,11 @@ __device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring
     const uint32_t rank = cluster_ctarank();
     const bool leader_cta = (rank == 0);
     const int total_tiles = P.L * W_comp;
+    const int n_stages = P.pair_stages;   // 6, or 7 with the aux region as one more stage
     const unsigned long long deadline = globaltimer_ns() + P.wait_ns;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < C::kStages; ++i) {
+        for (int i = 0; i < n_stages; ++i) {
             mbar_init(smem_u32(&ctl->full[i]), 1);
             mbar_init(smem_u32(&ctl->empty[i]), 1);
         }
@@ -771,7 +772,7 @@ __device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring
                         mbar_complete_tx_cluster(mapa_u32(own_full, 0u), (uint32_t)(C::kStageBytes - C::kABytes));
                     }
                     armed |= 1u << stage;
-                    if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+                    if (++stage == n_stages) { stage = 0; phase ^= 1u; }
                 }
                 t = t_next;
                 e = e_next;
@@ -781,7 +782,7 @@ __device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring
             if (!ok && leader_cta) {
                 // wind-down: let the copies already issued land before shared memory is released
                 const unsigned long long drain = globaltimer_ns() + 2000000ull;
-                for (int sidx = 0; sidx < C::kStages; ++sidx) {
+                for (int sidx = 0; sidx < n_stages; ++sidx) {
                     if (!(armed & (1u << sidx))) continue;
                     const uint32_t par = (sidx < stage) ? phase : (phase ^ 1u);
                     while (!mbar_try_wait(smem_u32(&ctl->full[sidx]), par) && globaltimer_ns() < drain) {}
@@ -851,7 +852,7 @@ __device__ void compute_cta_pair(const FusedParams &P, int W_comp, uint8_t *ring
                     a_lo += kLoStage;
                     full_bar += 8u;
                     empty_bar += 8u;
-                    if (++stage == C::kStages) {
+                    if (++stage == n_stages) {
                         stage = 0;
                         phase ^= 1u;
                         a_lo = lo0;
@@ -955,6 +956,8 @@ static_assert(kCommWarps * kCommWarpBytes <= kStageBytesTotal, "communication st
 constexpr int kCoWarpsAux = 2;          // co-resident warps whose stages fit the aux region
 constexpr int kCoWeightFloats = 16;
 constexpr int kCoWeightsOffset = kCoWarpsAux * kCommWarpBytes;
+static_assert(PairCfg::kStageBytes + ((sizeof(Control) + 127) & ~(size_t)127) <= kAuxBytes + ((sizeof(Control) + 127) & ~(size_t)127) &&
+              12 * 256 * 4 <= PairCfg::kStageBytes, "a seventh pair stage plus the control block exceed the allocation");
 static_assert(kCoWeightsOffset + (kCoWarpsMax + kCommWarps) * kCoWeightFloats * 4 <= kAuxBytes,
               "co-resident stages and weights exceed the aux region");
 
@@ -1486,8 +1489,14 @@ moe_gemm2_combine_pair_kernel(const __grid_constant__ FusedParams P)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    Control *ctl = reinterpret_cast<Control *>(ring + kStageBytesTotal);
-    uint8_t *aux = reinterpret_cast<uint8_t *>(ring + kStageBytesTotal + ((sizeof(Control) + 127) & ~(size_t)127));
+    // Layout: six operand stages, the control block, the aux region -- or, when nothing needs the aux region
+    // while the GEMM runs (256-bit epilogue stores, no co-resident communication warp), seven stages and the
+    // control block; the seventh stage then serves as the aux region of the communication role, which only
+    // starts after the CTA's last MMA (drain help) or never computes (communication CTA).
+    const bool seven = (P.pair_stages == 7);
+    Control *ctl = reinterpret_cast<Control *>(ring + kStageBytesTotal + (seven ? PairCfg::kStageBytes : 0));
+    uint8_t *aux = seven ? ring + kStageBytesTotal
+                         : reinterpret_cast<uint8_t *>(ring + kStageBytesTotal + ((sizeof(Control) + 127) & ~(size_t)127));
 
     if (blockIdx.x == 0 && threadIdx.x < (unsigned)P.L) {
         P.split_done_next[threadIdx.x] = 0u;

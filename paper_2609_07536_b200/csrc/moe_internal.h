@@ -58,6 +58,8 @@ struct alignas(64) FusedParams {
     int32_t num_kb, last_ksteps;
     int32_t drain_help;                 // compute CTAs serve communication tiles once their GEMM tiles are done
     int32_t co_warps;                   // co-resident communication warps per compute CTA (0..2)
+    int32_t pair_stages;                // operand stages of the CTA-pair kernel: 6, or 7 when the aux region of shared memory is
+                                        // free during the GEMM (256-bit epilogue stores, no co-resident warp)
     int32_t epi_warps;                  // epilogue warps of a compute CTA: 12 (warps 4-15), or 16 (warps 4-19) when no
                                         // co-resident warp is asked for and the epilogue needs no staging buffer
     int32_t tile_order;                 // 0: split-major tile sequence (the paper's); 1: m-tile-major across splits
