@@ -10,7 +10,7 @@
 //   warps 0, 2  TMA producers (one thread each): warp 0 the gathered rows (128 x 64 k), warp 2 the
 //               expert's 128 gate rows and 128 up rows of W1 for the same columns (two boxes that form
 //               one 256-row B operand), into four 48 KB stages, 128B swizzle;
-//   warp 1      one thread issues tcgen05.mma (M = 128, N = 256, K = 16, bf16 -> fp32): accumulator
+//   warp 1      issues tcgen05.mma (converged warp, elected lane; M = 128, N = 256, K = 16, bf16 -> fp32): accumulator
 //               columns 0..127 are the gate projection, 128..255 the up projection of the same outputs;
 //               two accumulator buffers in TMEM;
 //   warps 4-15  epilogue: tcgen05.ld of 32 gate and the matching 32 up columns, silu(g) * u in fp32,

@@ -13,14 +13,16 @@
 // Compute CTA (warp-specialised; tile_m x tile_n with tile_m in {64, 128}):
 //   warps 0, 2  TMA producers (one thread each): warp 0 the x_routed tile (128 rows x 64 k), warp 2 the
 //               W2 tile (tile_n rows x 64 k) of every k-block, into a ring of 128B-swizzled stages;
-//   warp 1      MMA issuer (one thread): tcgen05.mma (M = 128, N = tile_n, K = 16, bf16 -> fp32) into one
-//               of two TMEM accumulator buffers; tcgen05.commit frees stages / publishes the tile;
+//   warp 1      MMA issuer (the warp runs the loop converged, an elected lane issues; all operands warp-uniform):
+//               tcgen05.mma (M = 128, N = tile_n, K = 16, bf16 -> fp32) into one of two TMEM accumulator
+//               buffers; tcgen05.commit frees stages / publishes the tile;
 //   warps 4-15  epilogue: tcgen05.ld -> bf16 -> Y (three column groups x four TMEM lane quarters; warps 16-19
 //               are a fourth column group when the launch carries no co-resident communication warp);
 //   warp 3      publisher (one thread): once the epilogue warps have stored a tile, release fence, then the
 //               tile's readiness flag and the split counter (one fence for all tiles stored by then).
 // Compute CTA pair (256 x 256 tiles): the same roles in both CTAs of a cluster of two; one
-//   tcgen05.mma.cta_group::2 spans both SMs, each CTA loads only its own operand halves.
+//   tcgen05.mma.cta_group::2 spans both SMs, each CTA loads only its own operand halves; six operand
+//   stages, seven when the aux region of shared memory is free while the GEMM runs.
 // Y is token-major: the epilogue scatters each accumulator row to its (token, slot, shard) place, so
 //   that the k_tot * TP partial rows of one (token, split, column slab) form one contiguous block.
 // Communication CTA (12 independent warps): a warp fetches such a block with one bulk asynchronous
@@ -65,7 +67,7 @@ enum {
     kTlWaitTmem = 7, kTlMmaCycles = 8, kTlComputeEnd = 9, kTlCtaEnd = 10, kTlEpiWait = 11, kTlEpiWork = 12,
     kTlProducerWait = 13, kTlCommUnits = 14, kTlCommWaitNs = 15, kTlCoWarp = 16,  // 8 slots per co-resident warp (16..31)
     kTlPubWait = 32, kTlPubFence = 33, kTlEpiPubWait = 34,
-    kTlStageLate = 35   // pair tiles: k-blocks whose operand stage was not complete when the MMA thread first looked
+    kTlStageLate = 35   // pair tiles: k-blocks whose operand stage was not complete when the MMA issuer first looked
 };
 #if MOE_TIMELINE
 __device__ __forceinline__ void tl_put(const FusedParams &P, int slot, unsigned long long v)
