@@ -206,6 +206,29 @@ def test_pair_slots():
     assert plan.comm_ctas % 2 == 0           # an odd C never beats the even one below it by the model
 
 
+def test_a_family_closed_by_its_lower_bound_is_never_picked_but_a_forced_w_is_honoured():
+    # Section III-E (legal set from a one-time characterisation): for the CTA-pair tiles the library hands out
+    # co_min_waves = INT32_MAX, i.e. the co-resident family is not offered; a forced w bypasses the bound.
+    shape = B.make_shape(16384, 2048, 1408, 66, 8, 2, 2, 2)
+    occ = B.moe_occupancy(256, 256, 128, 1024, 1, 1, 2)
+    rho = B.moe_rho(14.96, 704, 256, 256, 2, 17, 1024, B.MOE_RHO_LOCAL)
+    rho.comm_warps_per_cta, rho.n_sat_warps, rho.comm_quanta_per_tile = 12, 1030, 128
+    rho.co_beta, rho.co_gamma, rho.co_order = 0.0125, 2.2, 0.02
+    tiles = [8] * 64 + [32] * 2
+    picks = {}
+    for waves in (24, 2 ** 31 - 1):
+        lim = B.moe_sm_limits(148, 74, 0, 0, 3, 1, 2, -1, 8, B.MOE_DEP_SPLIT, waves)
+        plan = B.plan_partition(tiles, occ, lim, shape, rho)
+        _same(plan, _oracle_plan(tiles, shape, occ, lim, rho))
+        picks[waves] = plan
+    assert picks[24].co_warps > 0                      # offered, the model takes it on this workload
+    assert picks[2 ** 31 - 1].co_warps == 0            # closed: only (C, 0) candidates are left
+    lim = B.moe_sm_limits(148, 74, 0, 0, 3, 1, 2, 2, 8, B.MOE_DEP_SPLIT, 2 ** 31 - 1)
+    plan = B.plan_partition(tiles, occ, lim, shape, rho)
+    _same(plan, _oracle_plan(tiles, shape, occ, lim, rho))
+    assert plan.co_warps == 2
+
+
 def test_drain_help_model():
     # the extension: after the last compute wave every SM serves communication tiles
     shape = B.make_shape(16384, 2048, 1408, 66, 8, 2, 2, 4)
