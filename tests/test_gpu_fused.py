@@ -237,6 +237,9 @@ def test_dispatch_by_shape():
         tm, tn = sel(w)
         occ, lim, rho = B.moe_query_occupancy(h, tm, tn)
         assert (occ.tile_m, occ.tile_n) == (tm, tn) and occ.comp_slot_sms == (2 if tm == 256 else 1)
+        # the co-resident family is offered for the one-CTA tiles (from 24 compute waves on), not for the CTA-pair
+        # tiles, where a co-resident warp would cost the seventh operand stage
+        assert lim.co_warps_max == 2 and lim.co_min_waves == (2 ** 31 - 1 if tm == 256 else 24)
 
 
 def test_pair_tiles_against_oracle():
