@@ -964,7 +964,14 @@ def main():
         torch.cuda.empty_cache()
         # ---- the other named workloads, briefly (a second or two each): fused time and roofline fractions
         if args.workload == "dsv2lite" and not args.tile and not args.T and not args.L:
-            extra["other_configs"] = [quick_config(h, wl.CONFIGS[n], device, peaks) for n in ("granite3moe", "qwen15moe")]
+            # the other two shapes of the task, each with the tile family the library's dispatch picks for it
+            from dataclasses import replace as _replace
+            others = []
+            for n in ("granite3moe", "qwen15moe"):
+                wo = wl.CONFIGS[n]
+                tm, tn = B.moe_select_tile(h, B.make_shape(wo.T, wo.H, wo.I, wo.E_tot, wo.k_tot, wo.TP, wo.EP, wo.L))
+                others.append(quick_config(h, _replace(wo, tile_m=tm, tile_n=tn), device, peaks))
+            extra["other_configs"] = others
         # ---- the up-stream stage (next row of the scope table), reported beside the headline, not in it
         g1res = time_gemm1(h, dw, torch, cpu_rows=0 if args.no_cpu_baseline else 4096)
         g1res["frac_of_bf16_peak"] = g1res["tflops"] / peaks["bf16_tflops"]

@@ -231,7 +231,7 @@ int32_t moe_query_occupancy(moe_handle *h, int32_t tile_m, int32_t tile_n,
 /* Kernel dispatch by shape (Section III-E, first paragraph: a conventional dispatch layer selects the GEMM2
  * kernel; the resource manager then reads that kernel's tile shape and residency).  Chooses the GEMM tile
  * family for `shape`: the widest n-tile the split width ceil(H/L) holds (256, 128 or 64), and 256-row
- * CTA-pair tiles when the experts hold at least 1536 routed rows on average (T * k_tot / E_tot), 128-row
+ * CTA-pair tiles when the experts hold at least 192 routed rows on average (T * k_tot / E_tot), 128-row
  * single-CTA tiles below (small and decode-sized token counts: less row padding, every SM its own tile).
  * The result is a valid (tile_m, tile_n) for every other call.  [host] */
 int32_t moe_select_tile(moe_handle *h, const moe_shape *shape, int32_t *tile_m, int32_t *tile_n);

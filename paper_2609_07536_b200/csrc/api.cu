@@ -39,7 +39,7 @@ inline size_t align16(size_t x) { return (x + 15) & ~(size_t)15; }
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 
-constexpr int64_t kPairTileMinRowsPerExpert = 1536;  // mean routed rows per expert from which 256-row pair tiles pay
+constexpr int64_t kPairTileMinRowsPerExpert = 192;   // mean routed rows per expert from which 256-row pair tiles pay
 constexpr int kSplitCounterWords = 64;  // 2 parities x MOE_MAX_L split counters (32-bit), then 2 x MOE_MAX_L work queues (64-bit), padded
 
 bool shape_ok(const moe_shape *s)
@@ -260,9 +260,10 @@ int32_t moe_select_tile(moe_handle *h, const moe_shape *s, int32_t *tile_m, int3
     // Conventional kernel dispatch (Section III-E: it runs before the resource manager and hands it the tile
     // shape and residency of the kernel it chose).  Widest n-tile the split holds; rows: the 256-row CTA-pair
     // tile moves a third less operand traffic per FLOP but pads every expert's last tile to 256 rows and needs
-    // two co-scheduled SMs, so it pays once an expert holds several such tiles on average (measured on the
-    // DeepSeek-V2-Lite shape, fused kernel, 128x256 against 256x256: 78 / 100 us at T = 16, 128 / 139 at 1024,
-    // 268 / 276 at 4096, 465 / 478 at 8192 (993 rows per expert), 889 / 880 at 16384 (1986 rows per expert)).
+    // two co-scheduled SMs, so it pays once an expert fills most of one such tile on average (measured on the
+    // DeepSeek-V2-Lite shape, fused kernel, 128x256 against 256x256: 78 / 100 us at T = 16, 128 / 132 at 1024
+    // (124 rows per expert), 172 / 160 at 2048 (248 rows), 257 / 243 at 4096, 466 / 423 at 8192, 885 / 791 at
+    // 16384; Qwen shape (546 rows per expert) 265 / 242, Granite shape (819 rows, K = 256) 134 / 131).
     const int64_t split_w = ceil_div(s->H, s->L);
     const int32_t tn = split_w >= 256 ? 256 : split_w >= 128 ? 128 : 64;
     const int64_t rows_per_expert = (int64_t)s->T * s->k_tot / s->E_tot;

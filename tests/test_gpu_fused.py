@@ -224,9 +224,9 @@ def test_decode_sized_token_counts_on_the_deepseek_shape(T):
 def test_dispatch_by_shape():
     h = G.handle()
     sel = lambda w: B.moe_select_tile(h, G.shape_of(w))
-    assert sel(wl.DSV2L) == (256, 256) and sel(replace(wl.DSV2L, T=32768)) == (256, 256)   # >= 1536 routed rows per expert
-    assert sel(replace(wl.DSV2L, T=8192)) == (128, 256) and sel(wl.QWEN) == (128, 256)     # 993 and 546 rows per expert
-    assert sel(replace(wl.DSV2L, T=1)) == (128, 256)
+    assert sel(wl.DSV2L) == (256, 256) and sel(replace(wl.DSV2L, T=2048)) == (256, 256)    # >= 192 routed rows per expert
+    assert sel(wl.QWEN) == (256, 256) and sel(wl.GRANITE) == (256, 256)                    # 546 and 819 rows per expert
+    assert sel(replace(wl.DSV2L, T=1024)) == (128, 256) and sel(replace(wl.DSV2L, T=1)) == (128, 256)   # 124 rows and fewer
     assert sel(replace(wl.DSV2L, L=8)) == (256, 256)                            # split width 256
     assert sel(replace(wl.DSV2L, L=4, H=512)) == (128, 128)                     # split width 128: no pair tile
     assert sel(wl.TINY) == (128, 256) and sel(replace(wl.TINY, H=64)) == (128, 64)
