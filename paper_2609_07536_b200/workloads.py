@@ -72,7 +72,7 @@ GRANITE = Workload("granite3moe", T=4096, H=1536, I=512, E=40, k=8, TP=2, EP=2,
                    tile_m=128, tile_n=256, L=1, routing="zipf", zipf_s=1.0,
                    target_r_expert=2.5, routing_seed=0, data_seed=1)
 QWEN = Workload("qwen15moe", T=8192, H=2048, I=1408, E=60, k=4, TP=2, EP=2,
-                tile_m=256, tile_n=256, L=2, routing="zipf", zipf_s=1.0,
+                tile_m=256, tile_n=256, L=1, routing="zipf", zipf_s=1.0,
                 target_r_expert=2.5, routing_seed=0, data_seed=1)
 DSV2L = Workload("dsv2lite", T=16384, H=2048, I=1408, E=64, k=6, n_shared=2, TP=2, EP=2,
                  tile_m=256, tile_n=256, L=2, routing="zipf", zipf_s=1.2,
